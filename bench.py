@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the CCA / CCGQA block on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path over one batch of seeded synthetic input: the forward
+of the block for the forward-only workloads (the 16k-context prefill headline), forward + backward
+for the training workloads.  Prints ONE JSON line (rank 0).  N > 1 runs N independent replicas of the
+same workload (the block has no exchange step), launched by torch.distributed.run.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+from paper_2510_04476_b200 import synth
+
+METRIC = "CCGQA block throughput at 16k context (algorithmic causal FLOPs / device time)"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAK_TFLOPS = 1590.0
+TRAIN_WORKLOADS = {"cfg2_small", "cfg4_train"}
+
+
+def flops_of(sh, backward: bool):
+    T = sh.B * sh.S
+    proj = 2 * T * sh.d_model * (sh.L_q + 2 * sh.L_k) + 2 * T * sh.L_q * sh.d_model
+    conv = 2 * T * (sh.L * sh.k_seq + sh.L * sh.head_dim * sh.k_ch)
+    attn = (2 if sh.causal else 4) * sh.B * sh.S * sh.S * sh.L_q
+    fwd = proj + conv + attn
+    total = fwd + (2 * (proj + conv) + 2.5 * attn if backward else 0)
+    return {"total": total, "fwd": fwd, "attn_fwd": attn, "proj": proj, "conv": conv}
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["bf16_tflops"]), "measured (cuBLAS bf16 burst)", d
+        except Exception:
+            pass
+    return FALLBACK_PEAK_TFLOPS, "fallback", {}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: str):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.06)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        clocks, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.lines:
+            if t0 is not None and not (t0 - 0.05 <= ts <= t1 + 0.1):
+                continue
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                clocks.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        clocks.sort()
+        med = clocks[len(clocks) // 2] if clocks else None
+        return {"sm_mhz": med, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(clocks)}
+
+
+def oracle_sample(sh, n_rows=256):
+    """The oracle, as it stands, on a bounded sample of the workload: projections and latent transforms
+    in full, the S^2 stage and the up-projection on n_rows sampled query positions per sequence."""
+    from oracle import cca_oracle as O
+    t = synth.make_inputs(sh, want_dout=False)
+    g = torch.Generator().manual_seed(123)
+    rows = sorted(set(int(r) for r in torch.randint(0, sh.S, (n_rows,), generator=g)))
+    cfg = O.OracleConfig(sh.d_model, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.k_seq, sh.k_ch, sh.causal, sh.flags,
+                         sh.rope_base)
+    t0 = time.perf_counter()
+    O.forward_rows(cfg, t, t["x"], rows)
+    dt = time.perf_counter() - t0
+    T = sh.B * sh.S
+    fl = 2 * T * sh.d_model * (sh.L_q + 2 * sh.L_k) + 2 * T * (sh.L * sh.k_seq + sh.L * sh.head_dim * sh.k_ch)
+    fl += sum(4 * sh.B * (r + 1 if sh.causal else sh.S) * sh.L_q for r in rows) + 2 * sh.B * len(rows) * sh.L_q * sh.d_model
+    return fl / dt / 1e12, dt, f"down-projections and latent transforms in full; attention and up-projection on {len(rows)} sampled query rows per sequence"
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    sh = synth.CONFIGS[args.workload]
+    vals = []
+    for _ in range(args.warmup):
+        pass                                   # the oracle has no warm-up state; keep the run short
+    t_all = time.perf_counter()
+    sample = ""
+    for _ in range(max(1, args.steps)):
+        v, dt, sample = oracle_sample(sh, n_rows=128)
+        vals.append((v, dt))
+        if time.perf_counter() - t_all > 150:
+            break
+    v = sum(x for x, _ in vals) / len(vals)
+    ms = 1e3 * sum(d for _, d in vals) / len(vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": len(vals),
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": sh.name, "B": sh.B, "S": sh.S, "d_model": sh.d_model, "n_q_heads": sh.n_q_heads,
+                   "n_kv_heads": sh.n_kv_heads, "head_dim": sh.head_dim, "note": "fp64 CPU oracle on a bounded sample"},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, rank, world, local_rank):
+    from paper_2510_04476_b200.binding import CCA
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    sh = synth.CONFIGS[args.workload]
+    backward = args.workload in TRAIN_WORKLOADS
+    t = synth.make_inputs(sh, want_dout=backward)
+    dev = {k: v.cuda(local_rank).contiguous() for k, v in t.items()}
+    cca = CCA.from_shape(sh, device=local_rank)
+    cca.set_impl(args.kernels)
+    act_bytes = sh.B * sh.S * sh.d_model * 2
+    ws = cca.alloc_workspace(sh.B, sh.S, True, extra=2 * act_bytes + 1024)
+    out = torch.empty_like(dev["x"])
+
+    def step():
+        cca.forward(dev, dev["x"], ws, out)
+        if backward:
+            return cca.backward(dev, dev["x"], dev["d_out"], ws)
+        return None
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in ev:
+        a.record(); b.record()
+    torch.cuda.synchronize()
+    vis = [v for v in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if v]
+    sampler = ClockSampler(vis[local_rank] if local_rank < len(vis) else str(local_rank))
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.15)
+    barrier()
+    l0 = cca.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0 = time.time()
+    e0.record()
+    for i in range(args.steps):
+        cca.set_attention_events(*ev[i])
+        step()
+    e1.record()
+    barrier()
+    w1 = time.time()
+    cca.set_attention_events(None, None)
+    launches = cca.launch_count() - l0
+    clocks = sampler.stop(w0, w1) if rank == 0 else None
+    ms_total = e0.elapsed_time(e1)
+    tm = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+    ms_step = float(tm.item()) / args.steps
+    status = cca.last_status()
+    fl = flops_of(sh, backward)
+    value = world * fl["total"] / (ms_step * 1e-3) / 1e12
+    attn_ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
+
+    # end to end through the C ABI with host buffers (forward workloads) / pinned copies (training)
+    xh = t["x"].pin_memory()
+    oh = torch.empty_like(t["x"]).pin_memory()
+    if backward:
+        dh_ = t["d_out"].pin_memory()
+        xd, dd = torch.empty_like(dev["x"]), torch.empty_like(dev["d_out"])
+
+    def e2e_step():
+        if not backward:
+            cca.forward_host(dev, xh, oh, ws)
+        else:
+            xd.copy_(xh, non_blocking=True)
+            dd.copy_(dh_, non_blocking=True)
+            cca.forward(dev, xd, ws, out)
+            d_x, _ = cca.backward(dev, xd, dd, ws)
+            oh.copy_(d_x, non_blocking=True)
+            torch.cuda.synchronize()
+
+    e2e_step()
+    barrier()
+    n_e2e = min(args.steps, 10)
+    t0 = time.perf_counter()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()
+    for _ in range(n_e2e):
+        e2e_step()
+    g1.record()
+    barrier()
+    e2e_ms = torch.tensor([g0.elapsed_time(g1) / n_e2e], device="cuda", dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+    e2e_val = world * fl["total"] / (float(e2e_ms.item()) * 1e-3) / 1e12
+    h2d = act_bytes * (2 if backward else 1)
+    d2h = act_bytes
+
+    peak, peak_kind, _ = measured_peak()
+    attn_tflops = fl["attn_fwd"] / (attn_ms * 1e-3) / 1e12
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": sh.name, "step": "forward+backward" if backward else "forward", "B": sh.B, "S": sh.S,
+                   "d_model": sh.d_model, "n_q_heads": sh.n_q_heads, "n_kv_heads": sh.n_kv_heads,
+                   "head_dim": sh.head_dim, "k_seq": sh.k_seq, "k_ch": sh.k_ch, "causal": sh.causal,
+                   "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
+                   "l2": "no flush: each step streams x, out and the latents (>= 0.4 GB), more than the 126 MB L2",
+                   "kernels": "tcgen05+simt" if args.kernels else "simt"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": float(e2e_ms.item())},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "latent attention forward", "achieved": attn_tflops, "peak": peak,
+                     "unit": "TFLOP/s", "frac": attn_tflops / peak, "peak_kind": peak_kind,
+                     "frac_of_nominal_2250": attn_tflops / NOMINAL_BF16_TFLOPS, "ms_per_launch": attn_ms,
+                     "flops_per_launch": fl["attn_fwd"], "traffic": None},
+        "pct_of_nominal_bf16_peak": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
+        "device_status": status,
+    }
+    if rank == 0 and world == 1 and not args.no_mha and not backward:
+        line["mha_same_shape"] = mha_compare(sh, args, ms_step, attn_ms, local_rank)
+    if rank == 0 and world == 1 and not args.no_cpu:
+        v, dt, sample = oracle_sample(sh)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                                "sample": sample, "seconds": dt}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    cca.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def mha_compare(sh, args, cca_ms, cca_attn_ms, local_rank):
+    """Same kernels configured as plain multi-head attention of equal d_model (no compression, no
+    latent transforms): reproduces the paper's speed-up ratio on this machine."""
+    from paper_2510_04476_b200.binding import CCA
+    m = synth.mha_like(sh)
+    t = synth.make_inputs(m, want_dout=False)
+    dev = {k: v.cuda(local_rank).contiguous() for k, v in t.items()}
+    cca = CCA.from_shape(m, device=local_rank)
+    cca.set_impl(args.kernels)
+    ws = cca.alloc_workspace(m.B, m.S, False)
+    out = torch.empty_like(dev["x"])
+    n = min(args.steps, 5)
+    for _ in range(2):
+        cca.forward(dev, dev["x"], ws, out)
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    for a, b in ev:
+        a.record(); b.record()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(n):
+        cca.set_attention_events(*ev[i])
+        cca.forward(dev, dev["x"], ws, out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / n
+    attn = sum(a.elapsed_time(b) for a, b in ev) / n
+    cca.close()
+    return {"config": f"{m.n_q_heads} heads x {m.head_dim}, C=1, transforms off", "block_ms": ms, "attention_ms": attn,
+            "block_speedup_of_ccgqa": ms / cca_ms, "attention_speedup_of_ccgqa": attn / cca_attn_ms}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3_prefill16k", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--kernels", type=int, default=1, help="0 = SIMT kernels only, 1 = tcgen05 kernels where available")
+    ap.add_argument("--no-mha", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,173 @@
+/*
+ * cca.h -- C ABI of the B200 (sm_100a) Compressed Convolutional Attention block.
+ *
+ * One block = down-projection of x to latent q/k/v, the latent transforms on q and k
+ * (two causal convolutions, q-k-mean, L2 norm with key temperature, RoPE), value-shift,
+ * causal softmax attention with grouped kv heads inside the latent, up-projection; and the
+ * matching backward.  The method is the paper's Section 2.2 (Eq. 7-11) and Listing A.1.
+ *
+ * Conventions
+ *   - Every pointer named "device" is CUDA device memory on the handle's device, owned by the
+ *     caller.  The library allocates nothing on the device except a 64-byte status word per
+ *     handle; cca_forward / cca_backward never allocate, never synchronise, never fall back to
+ *     the CPU.  All work is enqueued on the caller's stream.
+ *   - Activations are row-major [B, S, width] (the paper's listing is [S, B, width]; sequences
+ *     are independent so the result is the same).  bf16 = 16-bit brain float, raw bits.
+ *   - Linear weights are [out, in] row-major, like torch.nn.Linear.
+ *   - Every function returns a cca_status code; nothing throws, aborts or traps.
+ */
+#ifndef CCA_H_
+#define CCA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CCA_OK = 0,
+  CCA_ERR_INVALID_ARG = 1,         /* null pointer, non-positive size, inconsistent config   */
+  CCA_ERR_UNSUPPORTED = 2,         /* shape outside kernel coverage, or device is not sm_100 */
+  CCA_ERR_ALIGNMENT = 3,           /* a device pointer is not 16-byte aligned                */
+  CCA_ERR_WORKSPACE_TOO_SMALL = 4,
+  CCA_ERR_CUDA = 5,                /* a CUDA call failed; see cca_last_cuda_error            */
+  CCA_ERR_DEVICE_TIMEOUT = 6       /* a bounded device-side wait expired (cca_last_status)   */
+} cca_status;
+
+/* Optional stages (rows of the paper's ablation tables; all on = the method of Eq. 7-11). */
+enum {
+  CCA_CONV1 = 1,     /* conv1_seq: depth-wise causal conv over the sequence, Eq. 8          */
+  CCA_CONV2 = 2,     /* conv2_seq+ch: head-wise grouped causal conv, Eq. 8                  */
+  CCA_QK_MEAN = 4,   /* q-k-mean, Eq. 9                                                     */
+  CCA_V_SHIFT = 8,   /* value-shift, Eq. 10 (off: both value halves read x_t)               */
+  CCA_QK_NORM = 16,  /* L2 norm * sqrt(d_h), keys also * exp(temp), Eq. 11                  */
+  CCA_ROPE = 32,     /* rotary embedding on the normalised latents, Eq. 11                  */
+  CCA_ALL_STAGES = 63
+};
+
+/* The paper's parameters (notation table). */
+typedef struct {
+  int32_t d_model;      /* E                                                                */
+  int32_t n_q_heads;    /* h_q;  L_q = h_q * head_dim = E / C1                              */
+  int32_t n_kv_heads;   /* h_k;  L_k = h_k * head_dim = E / C2;  h_q % h_k == 0, L_k even   */
+  int32_t head_dim;     /* d_h, latent per-head size: 32, 64 or 128                         */
+  int32_t compression;  /* C = C1; checked: E == C * h_q * d_h                              */
+  int32_t k_seq;        /* taps of conv1_seq (1..4)                                         */
+  int32_t k_ch;         /* taps of conv2_seq+ch (1..4)                                      */
+  int32_t causal;       /* attention mask only; the convs and value-shift are always causal */
+  uint32_t flags;       /* CCA_* stage bits                                                 */
+  float rope_base;      /* RoPE base, e.g. 10000                                            */
+} cca_config;
+
+/* Parameters, all device pointers.  q rows of w_qk come first, then k rows (Listing A.1). */
+typedef struct {
+  const void* w_qk;     /* bf16 [L_q + L_k, E]   packed q/k down-projection, Eq. 7          */
+  const void* w_v1;     /* bf16 [L_k/2, E]       value projection of x_t, Eq. 10            */
+  const void* w_v2;     /* bf16 [L_k/2, E]       value projection of x_{t-1}, Eq. 10        */
+  const void* w_o;      /* bf16 [E, L_q]         up-projection, Eq. 11                      */
+  const void* conv0_w;  /* bf16 [L, k_seq]       depth-wise taps, last tap = current token  */
+  const void* conv1_w;  /* bf16 [L, d_h, k_ch]   (out channel, in channel in head, tap)     */
+  const float* temp;    /* fp32 [h_k]            log of the key temperature beta            */
+} cca_weights;
+
+/* Parameter gradients, fp32 device buffers of the parameters' shapes; overwritten. */
+typedef struct {
+  float* d_w_qk;
+  float* d_w_v1;
+  float* d_w_v2;
+  float* d_w_o;
+  float* d_conv0_w;
+  float* d_conv1_w;
+  float* d_temp;
+} cca_weight_grads;
+
+/* Shape and indexing metadata (integers only).  Offsets are bytes into the workspace. */
+typedef struct {
+  int64_t L_q, L_k, g;              /* latent widths and query heads per kv head            */
+  int64_t total_padding;            /* k_seq + k_ch - 2 tokens of causal history (listing)  */
+  int64_t v_shift_split;            /* first channel of the value latent fed by x_{t-1}     */
+  int64_t q_to_kv_head[64];         /* q head i reads kv head floor(i / g); -1 beyond h_q   */
+  int64_t conv_params;              /* L*k_seq + L*d_h*k_ch                                 */
+  int64_t params;                   /* 2E^2/C1 + 2E^2/C2 + conv (comparison table)          */
+  int64_t kv_cache_elems;           /* 2*B*S*E/C2                                           */
+  int64_t fwd_flops;                /* (1/C1+1/C2)*4BSE^2 + 4BES^2/C1 + conv                */
+  int64_t fwd_flops_causal;         /* same with the S^2 term halved                        */
+  int64_t decode_flops;             /* (1/C1+1/C2)*4BE^2 + 4BES/C1 + conv                   */
+  /* saved activations (written by cca_forward, read by cca_backward) */
+  int64_t off_qk0, off_q, off_k, off_v, off_o, off_lse, off_rope;
+  int64_t saved_bytes;              /* forward-only workspace size                          */
+  int64_t total_bytes;              /* forward + backward workspace size                    */
+} cca_layout;
+
+typedef struct cca_handle cca_handle;
+
+/* Validate the configuration for `device`, create a handle.  Paper: Eq. 7-11 parameters.
+ * Errors: INVALID_ARG (null, E != C*h_q*d_h, h_q % h_k, odd L_k, bad kernel sizes),
+ * UNSUPPORTED (head_dim not in {32,64,128}, h_q > 64, device not compute capability 10.x),
+ * CUDA.  device = -1 makes a host-only handle: cca_describe and cca_workspace_size work, every
+ * compute entry point returns INVALID_ARG. */
+int cca_init(const cca_config* cfg, int device, cca_handle** out);
+int cca_destroy(cca_handle* h);
+
+/* Fill `out` for batch B and sequence length S.  Pure host arithmetic; follows the CCGQA row
+ * of the paper's comparison table and the padding / grouping / concat rules of Listing A.1. */
+int cca_describe(const cca_handle* h, int64_t B, int64_t S, cca_layout* out);
+
+/* Bytes of caller-owned device workspace needed (need_backward != 0 adds backward scratch). */
+int cca_workspace_size(const cca_handle* h, int64_t B, int64_t S, int need_backward, size_t* bytes);
+
+/* Forward of the whole block, Eq. 7-11: out = W_o [ softmax(q k^T / sqrt(d_h)) v ]_heads.
+ *   x   device bf16 [B,S,E] (read), out device bf16 [B,S,E] (written).
+ *   workspace: device, 256-byte aligned, >= cca_workspace_size(..., need_backward).  On return
+ *   (stream order) it holds qk0, q, k, v, o, lse at the cca_layout offsets; keep it untouched
+ *   until cca_backward if gradients are wanted.
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE_TOO_SMALL, CUDA. */
+int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out,
+                void* workspace, size_t workspace_bytes, int64_t B, int64_t S, void* cuda_stream);
+
+/* Backward of the block: given d_out = dLoss/d out (device bf16 [B,S,E]) and the workspace
+ * left by cca_forward for the same x and weights, writes d_x (device bf16 [B,S,E]) and every
+ * field of `grads` (fp32, overwritten).  The paper prints no backward; this is the exact
+ * adjoint of Eq. 7-11.  Errors as cca_forward. */
+int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void* d_out,
+                 void* workspace, size_t workspace_bytes, void* d_x,
+                 const cca_weight_grads* grads, int64_t B, int64_t S, void* cuda_stream);
+
+/* Same block, host buffers: copies x (host, ideally pinned) to a staging area inside the
+ * workspace, runs cca_forward, copies out back to `out_host`, and synchronises the stream.
+ * workspace must be >= cca_workspace_size(...) + 2*B*S*E*2 bytes. */
+int cca_forward_host(cca_handle* h, const cca_weights* w, const void* x_host, void* out_host,
+                     void* workspace, size_t workspace_bytes, int64_t B, int64_t S,
+                     void* cuda_stream);
+
+/* Attention stage alone (Eq. 11, third line) on latents already in the workspace layout:
+ * q [B,S,h_q,d_h], k, v [B,S,h_k,d_h] bf16 device -> o bf16 [B,S,h_q,d_h], lse fp32 [B,h_q,S]. */
+int cca_attention_forward(cca_handle* h, const void* q, const void* k, const void* v, void* o,
+                          float* lse, int64_t B, int64_t S, void* cuda_stream);
+
+/* Select kernel implementations: 0 = plain SIMT kernels, 1 = tcgen05/TMA kernels where they
+ * exist (default).  Returns the previous value. */
+int cca_set_impl(cca_handle* h, int impl);
+
+/* Profiling hook: two cudaEvent_t (or null to clear) that every later attention stage records on the
+ * caller's stream immediately before and after its kernel. */
+int cca_set_attention_events(cca_handle* h, void* ev_begin, void* ev_end);
+
+/* Number of kernel launches the library has enqueued through this handle so far. */
+int64_t cca_launch_count(const cca_handle* h);
+
+/* After the caller has synchronised the stream: copies the device status word.  0 = no error;
+ * otherwise the code written by a kernel whose bounded wait expired.  Returns
+ * CCA_ERR_DEVICE_TIMEOUT if it is non-zero. */
+int cca_last_status(cca_handle* h, int* device_status);
+
+/* Last CUDA runtime error code seen by this handle, and its string. */
+int cca_last_cuda_error(const cca_handle* h);
+const char* cca_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CCA_H_ */

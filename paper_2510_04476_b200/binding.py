@@ -1,0 +1,266 @@
+"""Thin ctypes binding over libcca.so: argument marshalling only.
+
+Every step of the block runs inside the library's CUDA kernels; torch is used here for device
+memory and streams.  There is no CPU fallback: if the library cannot be loaded, or a call fails,
+an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import torch
+
+from . import build as _build
+
+_LIB = None
+
+
+class CcaError(RuntimeError):
+    pass
+
+
+class cca_config(C.Structure):
+    _fields_ = [("d_model", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("compression", C.c_int32), ("k_seq", C.c_int32), ("k_ch", C.c_int32),
+                ("causal", C.c_int32), ("flags", C.c_uint32), ("rope_base", C.c_float)]
+
+
+class cca_weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("w_qk", "w_v1", "w_v2", "w_o", "conv0_w", "conv1_w", "temp")]
+
+
+class cca_weight_grads(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("d_w_qk", "d_w_v1", "d_w_v2", "d_w_o", "d_conv0_w", "d_conv1_w", "d_temp")]
+
+
+class cca_layout(C.Structure):
+    _fields_ = [("L_q", C.c_int64), ("L_k", C.c_int64), ("g", C.c_int64), ("total_padding", C.c_int64),
+                ("v_shift_split", C.c_int64), ("q_to_kv_head", C.c_int64 * 64), ("conv_params", C.c_int64),
+                ("params", C.c_int64), ("kv_cache_elems", C.c_int64), ("fwd_flops", C.c_int64),
+                ("fwd_flops_causal", C.c_int64), ("decode_flops", C.c_int64),
+                ("off_qk0", C.c_int64), ("off_q", C.c_int64), ("off_k", C.c_int64), ("off_v", C.c_int64),
+                ("off_o", C.c_int64), ("off_lse", C.c_int64), ("off_rope", C.c_int64),
+                ("saved_bytes", C.c_int64), ("total_bytes", C.c_int64)]
+
+
+# name -> (restype, argtypes); also the list of symbols the header declares
+SYMBOLS = {
+    "cca_init": (C.c_int, [C.POINTER(cca_config), C.c_int, C.POINTER(C.c_void_p)]),
+    "cca_destroy": (C.c_int, [C.c_void_p]),
+    "cca_describe": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.POINTER(cca_layout)]),
+    "cca_workspace_size": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int, C.POINTER(C.c_size_t)]),
+    "cca_forward": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                              C.c_int64, C.c_int64, C.c_void_p]),
+    "cca_backward": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                               C.c_void_p, C.POINTER(cca_weight_grads), C.c_int64, C.c_int64, C.c_void_p]),
+    "cca_forward_host": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.c_void_p,
+                                   C.c_size_t, C.c_int64, C.c_int64, C.c_void_p]),
+    "cca_attention_forward": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_int64, C.c_int64, C.c_void_p]),
+    "cca_set_impl": (C.c_int, [C.c_void_p, C.c_int]),
+    "cca_set_attention_events": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cca_launch_count": (C.c_int64, [C.c_void_p]),
+    "cca_last_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int)]),
+    "cca_last_cuda_error": (C.c_int, [C.c_void_p]),
+    "cca_status_string": (C.c_char_p, [C.c_int]),
+}
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load_library(build_if_missing: bool = True) -> C.CDLL:
+    """Load libcca.so (building it first if it is missing or stale).  Raises if that fails."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = _build.build() if build_if_missing else _build.LIB
+    if not os.path.exists(path):
+        raise CcaError(f"{path} is missing: build the CUDA library first (python -m paper_2510_04476_b200.build)")
+    lib = C.CDLL(path)
+    for name, (res, args) in SYMBOLS.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _LIB = lib
+    return lib
+
+
+def _check(lib, code: int, handle=None, what: str = ""):
+    if code != 0:
+        msg = lib.cca_status_string(code).decode()
+        extra = ""
+        if handle is not None and code == 5:
+            extra = f" (cudaError {lib.cca_last_cuda_error(handle)})"
+        raise CcaError(f"{what}: {msg}{extra}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+class CCA:
+    """One configured block on one device.  Methods mirror the C entry points."""
+
+    def __init__(self, d_model, n_q_heads, n_kv_heads, head_dim, k_seq=2, k_ch=2, causal=1, flags=63,
+                 rope_base=10000.0, device=0, compression=None):
+        self.lib = load_library()
+        if compression is None:
+            compression = d_model // max(1, n_q_heads * head_dim)
+        self.cfg = cca_config(d_model, n_q_heads, n_kv_heads, head_dim, compression, k_seq, k_ch, causal, flags,
+                              rope_base)
+        self.device = torch.device("cuda", device)
+        self.handle = C.c_void_p()
+        _check(self.lib, self.lib.cca_init(C.byref(self.cfg), device, C.byref(self.handle)), None, "cca_init")
+
+    @classmethod
+    def from_shape(cls, sh, device=0) -> "CCA":
+        return cls(sh.d_model, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.k_seq, sh.k_ch, sh.causal, sh.flags,
+                   sh.rope_base, device)
+
+    def close(self):
+        if getattr(self, "handle", None) is not None and self.handle.value:
+            self.lib.cca_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- metadata -------------------------------------------------------------------------
+    def describe(self, B: int, S: int) -> Dict[str, object]:
+        lay = cca_layout()
+        _check(self.lib, self.lib.cca_describe(self.handle, B, S, C.byref(lay)), self.handle, "cca_describe")
+        out = {}
+        for name, _ in cca_layout._fields_:
+            val = getattr(lay, name)
+            out[name] = list(val) if name == "q_to_kv_head" else int(val)
+        return out
+
+    def workspace_size(self, B: int, S: int, need_backward: bool = True) -> int:
+        n = C.c_size_t()
+        _check(self.lib, self.lib.cca_workspace_size(self.handle, B, S, int(need_backward), C.byref(n)), self.handle,
+               "cca_workspace_size")
+        return int(n.value)
+
+    def alloc_workspace(self, B: int, S: int, need_backward: bool = True, extra: int = 0) -> torch.Tensor:
+        return torch.empty(self.workspace_size(B, S, need_backward) + extra + 256, dtype=torch.uint8,
+                           device=self.device)
+
+    @staticmethod
+    def _ws_ptr(ws: torch.Tensor):
+        p = ws.data_ptr()
+        a = (p + 255) // 256 * 256
+        return C.c_void_p(a), ws.numel() - (a - p)
+
+    def set_impl(self, impl: int) -> int:
+        return self.lib.cca_set_impl(self.handle, impl)
+
+    def set_attention_events(self, begin: Optional[torch.cuda.Event], end: Optional[torch.cuda.Event]):
+        """Events (created with enable_timing=True) recorded around the attention kernel; None clears."""
+        for e in (begin, end):
+            if e is not None and e.cuda_event == 0:
+                e.record(torch.cuda.current_stream(self.device))      # forces creation of the handle
+        b = C.c_void_p(begin.cuda_event) if begin is not None else None
+        e = C.c_void_p(end.cuda_event) if end is not None else None
+        _check(self.lib, self.lib.cca_set_attention_events(self.handle, b, e), self.handle, "set_attention_events")
+
+    def launch_count(self) -> int:
+        return int(self.lib.cca_launch_count(self.handle))
+
+    def last_status(self) -> int:
+        s = C.c_int()
+        self.lib.cca_last_status(self.handle, C.byref(s))
+        return int(s.value)
+
+    # ---- compute --------------------------------------------------------------------------
+    def _weights(self, w: Dict[str, torch.Tensor]) -> cca_weights:
+        cw = cca_weights()
+        for n in ("w_qk", "w_v1", "w_v2", "w_o", "conv0_w", "conv1_w", "temp"):
+            t = w.get(n)
+            if t is not None:
+                assert t.is_cuda and t.is_contiguous(), n
+                assert t.dtype == (torch.float32 if n == "temp" else torch.bfloat16), n
+            setattr(cw, n, t.data_ptr() if t is not None else None)
+        return cw
+
+    def forward(self, w, x: torch.Tensor, workspace: torch.Tensor, out: Optional[torch.Tensor] = None):
+        B, S, E = x.shape
+        assert x.is_cuda and x.is_contiguous() and x.dtype == torch.bfloat16
+        if out is None:
+            out = torch.empty_like(x)
+        cw = self._weights(w)
+        wp, wn = self._ws_ptr(workspace)
+        st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+        _check(self.lib, self.lib.cca_forward(self.handle, C.byref(cw), _ptr(x), _ptr(out), wp, wn, B, S, st),
+               self.handle, "cca_forward")
+        return out
+
+    def forward_host(self, w, x_host: torch.Tensor, out_host: torch.Tensor, workspace: torch.Tensor):
+        B, S, E = x_host.shape
+        assert not x_host.is_cuda and not out_host.is_cuda
+        cw = self._weights(w)
+        wp, wn = self._ws_ptr(workspace)
+        st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+        _check(self.lib, self.lib.cca_forward_host(self.handle, C.byref(cw), _ptr(x_host), _ptr(out_host), wp, wn,
+                                                   B, S, st), self.handle, "cca_forward_host")
+        return out_host
+
+    def backward(self, w, x: torch.Tensor, d_out: torch.Tensor, workspace: torch.Tensor):
+        """Returns (d_x bf16, dict of fp32 parameter gradients)."""
+        B, S, E = x.shape
+        assert d_out.is_cuda and d_out.is_contiguous() and d_out.dtype == torch.bfloat16
+        d_x = torch.empty_like(x)
+        grads = {}
+        cg = cca_weight_grads()
+        for n in ("w_qk", "w_v1", "w_v2", "w_o", "conv0_w", "conv1_w", "temp"):
+            shape = w[n].shape
+            grads["d_" + n] = torch.empty(shape, dtype=torch.float32, device=self.device)
+            setattr(cg, "d_" + n, grads["d_" + n].data_ptr())
+        cw = self._weights(w)
+        wp, wn = self._ws_ptr(workspace)
+        st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+        _check(self.lib, self.lib.cca_backward(self.handle, C.byref(cw), _ptr(x), _ptr(d_out), wp, wn, _ptr(d_x),
+                                               C.byref(cg), B, S, st), self.handle, "cca_backward")
+        return d_x, grads
+
+    def attention_forward(self, q, k, v, o=None, lse=None):
+        B, S, hq, dh = q.shape
+        if o is None:
+            o = torch.empty_like(q)
+        if lse is None:
+            lse = torch.empty(B, hq, S, dtype=torch.float32, device=q.device)
+        st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+        _check(self.lib, self.lib.cca_attention_forward(self.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse),
+                                                        B, S, st), self.handle, "cca_attention_forward")
+        return o, lse
+
+    def saved(self, workspace: torch.Tensor, B: int, S: int) -> Dict[str, torch.Tensor]:
+        """Views of the activations cca_forward left in the workspace (for tests)."""
+        lay = self.describe(B, S)
+        wp, _ = self._ws_ptr(workspace)
+        base = wp.value - workspace.data_ptr()
+        cfg = self.cfg
+        hq, hk, dh = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+        Lq, Lk = hq * dh, hk * dh
+
+        def view(off, shape, dtype):
+            n = 1
+            for s in shape:
+                n *= s
+            nbytes = n * torch.empty((), dtype=dtype).element_size()
+            return workspace[base + off: base + off + nbytes].view(dtype).view(*shape)
+
+        return {
+            "qk0": view(lay["off_qk0"], (B, S, Lq + Lk), torch.bfloat16),
+            "q": view(lay["off_q"], (B, S, hq, dh), torch.bfloat16),
+            "k": view(lay["off_k"], (B, S, hk, dh), torch.bfloat16),
+            "v": view(lay["off_v"], (B, S, hk, dh), torch.bfloat16),
+            "o": view(lay["off_o"], (B, S, hq, dh), torch.bfloat16),
+            "lse": view(lay["off_lse"], (B, hq, S), torch.float32),
+        }

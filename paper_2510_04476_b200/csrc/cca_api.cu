@@ -1,0 +1,430 @@
+// C ABI of the CCA library: handle, validation, metadata, workspace layout, forward / backward drivers.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "../../include/cca.h"
+#include "common.cuh"
+#include "tc_kernels.cuh"
+
+struct cca_handle {
+  cca_config cfg;
+  int device;
+  int impl;               // 0 = SIMT only, 1 = tensor-core kernels where available
+  int sm_count;
+  int* d_status;          // device status word (64 bytes)
+  int last_cuda;
+  long long launches;
+  TcState* tc;            // tensor-map cache etc. (may be null if unavailable)
+  cudaEvent_t ev_attn_begin, ev_attn_end;   // optional, recorded around the attention kernel
+};
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+  size_t qk0, q, k, v, o, lse, rope, saved_end;
+  size_t d_o, delta, dq, dk, dv, dlat, w_all, total_end;
+};
+
+Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
+  Layout l;
+  const size_t T = (size_t)B * S;
+  const size_t Lq = (size_t)c.n_q_heads * c.head_dim, Lk = (size_t)c.n_kv_heads * c.head_dim, L = Lq + Lk;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  l.qk0 = take(T * L * 2);
+  l.q = take(T * Lq * 2);
+  l.k = take(T * Lk * 2);
+  l.v = take(T * Lk * 2);
+  l.o = take(T * Lq * 2);
+  l.lse = take((size_t)B * c.n_q_heads * S * 4);
+  l.rope = take((size_t)S * (c.head_dim / 2) * 8);
+  l.saved_end = off;
+  l.d_o = take(T * Lq * 2);
+  l.delta = take((size_t)B * c.n_q_heads * S * 4);
+  l.dq = take(T * Lq * 4);
+  l.dk = take(T * Lk * 4);
+  l.dv = take(T * Lk * 4);
+  l.dlat = take(T * (L + Lk) * 2);
+  l.w_all = take((L + Lk) * (size_t)c.d_model * 2);
+  l.total_end = off;
+  return l;
+}
+
+CcaDims make_dims(const cca_config& c, int64_t B, int64_t S) {
+  CcaDims d;
+  d.B = (int)B; d.S = (int)S; d.E = c.d_model;
+  d.hq = c.n_q_heads; d.hk = c.n_kv_heads; d.dh = c.head_dim; d.g = c.n_q_heads / c.n_kv_heads;
+  d.Lq = d.hq * d.dh; d.Lk = d.hk * d.dh; d.L = d.Lq + d.Lk;
+  d.k_seq = c.k_seq; d.k_ch = c.k_ch; d.causal = c.causal; d.flags = c.flags; d.rope_base = c.rope_base;
+  return d;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int check_sizes(const cca_handle* h, int64_t B, int64_t S, bool need_device = false) {
+  if (!h || B < 1 || S < 1) return CCA_ERR_INVALID_ARG;
+  if (need_device && h->device < 0) return CCA_ERR_INVALID_ARG;
+  if (B * S > (int64_t)1 << 30 || S > (int64_t)1 << 24) return CCA_ERR_UNSUPPORTED;
+  return CCA_OK;
+}
+
+#define CU(call)                                   \
+  do {                                             \
+    cudaError_t e_ = (call);                       \
+    if (e_ != cudaSuccess) {                       \
+      h->last_cuda = (int)e_;                      \
+      return CCA_ERR_CUDA;                         \
+    }                                              \
+  } while (0)
+
+GemmOperand kmajor(const void* p, long long ld) { return GemmOperand{(const bf16*)p, ld, 1}; }
+GemmOperand mmajor(const void* p, long long ld) { return GemmOperand{(const bf16*)p, 1, ld}; }
+
+// One contraction: tensor-core kernel if it is enabled and covers the case, else the SIMT kernel.
+int run_gemm(cca_handle* h, const GemmArgs& g, cudaStream_t st) {
+  if (h->impl >= 1 && h->tc) {
+    int r = tc_gemm(h->tc, g, h->d_status, st);
+    if (r == 0) { h->launches++; return CCA_OK; }
+    if (r < 0) { h->last_cuda = -r; return CCA_ERR_CUDA; }
+  }
+  CU(launch_gemm_simt(g, st));
+  h->launches++;
+  return CCA_OK;
+}
+
+int run_attention_fwd(cca_handle* h, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o,
+                      float* lse, cudaStream_t st) {
+  if (h->ev_attn_begin) CU(cudaEventRecord(h->ev_attn_begin, st));
+  bool done = false;
+  if (h->impl >= 1 && h->tc) {
+    int r = tc_attn_fwd(h->tc, d, q, k, v, o, lse, h->d_status, st);
+    if (r == 0) done = true;
+    if (r < 0) { h->last_cuda = -r; return CCA_ERR_CUDA; }
+  }
+  if (!done) CU(launch_attn_fwd_simt(d, q, k, v, o, lse, st));
+  h->launches++;
+  if (h->ev_attn_end) CU(cudaEventRecord(h->ev_attn_end, st));
+  return CCA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* cca_status_string(int s) {
+  switch (s) {
+    case CCA_OK: return "ok";
+    case CCA_ERR_INVALID_ARG: return "invalid argument";
+    case CCA_ERR_UNSUPPORTED: return "unsupported shape or device";
+    case CCA_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+    case CCA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case CCA_ERR_CUDA: return "CUDA error";
+    case CCA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+static int validate_config(const cca_config* c) {
+  if (!c) return CCA_ERR_INVALID_ARG;
+  if (c->d_model < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->head_dim < 1 || c->compression < 1)
+    return CCA_ERR_INVALID_ARG;
+  if ((int64_t)c->compression * c->n_q_heads * c->head_dim != c->d_model) return CCA_ERR_INVALID_ARG;
+  if (c->n_q_heads % c->n_kv_heads != 0) return CCA_ERR_INVALID_ARG;
+  if (((int64_t)c->n_kv_heads * c->head_dim) % 2 != 0) return CCA_ERR_INVALID_ARG;
+  if (c->k_seq < 1 || c->k_ch < 1) return CCA_ERR_INVALID_ARG;
+  if (c->flags & ~(uint32_t)CCA_ALL_STAGES) return CCA_ERR_INVALID_ARG;
+  if ((c->flags & CCA_ROPE) && !(c->rope_base > 0.f)) return CCA_ERR_INVALID_ARG;
+  if (c->k_seq > 4 || c->k_ch > 4) return CCA_ERR_UNSUPPORTED;
+  if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return CCA_ERR_UNSUPPORTED;
+  if (c->n_q_heads > 64) return CCA_ERR_UNSUPPORTED;
+  if (c->d_model % 8 != 0) return CCA_ERR_UNSUPPORTED;
+  return CCA_OK;
+}
+
+int cca_init(const cca_config* cfg, int device, cca_handle** out) {
+  if (!out) return CCA_ERR_INVALID_ARG;
+  *out = nullptr;
+  int v = validate_config(cfg);
+  if (v != CCA_OK) return v;
+  cudaDeviceProp prop;
+  prop.multiProcessorCount = 0;
+  if (device >= 0) {
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device >= ndev) return CCA_ERR_CUDA;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return CCA_ERR_CUDA;
+    if (prop.major != 10) return CCA_ERR_UNSUPPORTED;
+    if (cudaSetDevice(device) != cudaSuccess) return CCA_ERR_CUDA;
+  } else if (device != -1) {
+    return CCA_ERR_INVALID_ARG;
+  }
+  cca_handle* h = new (std::nothrow) cca_handle();
+  if (!h) return CCA_ERR_INVALID_ARG;
+  h->cfg = *cfg;
+  h->device = device;
+  h->impl = 1;
+  h->sm_count = prop.multiProcessorCount;
+  h->last_cuda = 0;
+  h->launches = 0;
+  h->d_status = nullptr;
+  h->tc = nullptr;
+  h->ev_attn_begin = h->ev_attn_end = nullptr;
+  if (device >= 0) {
+    if (cudaMalloc(&h->d_status, 64) != cudaSuccess || cudaMemset(h->d_status, 0, 64) != cudaSuccess) {
+      if (h->d_status) cudaFree(h->d_status);
+      delete h;
+      return CCA_ERR_CUDA;
+    }
+    h->tc = tc_create(h->sm_count);
+  }
+  *out = h;
+  return CCA_OK;
+}
+
+int cca_destroy(cca_handle* h) {
+  if (!h) return CCA_ERR_INVALID_ARG;
+  if (h->tc) tc_destroy(h->tc);
+  if (h->d_status) cudaFree(h->d_status);
+  delete h;
+  return CCA_OK;
+}
+
+int cca_set_impl(cca_handle* h, int impl) {
+  if (!h) return -1;
+  int old = h->impl;
+  h->impl = impl;
+  return old;
+}
+
+int cca_set_attention_events(cca_handle* h, void* ev_begin, void* ev_end) {
+  if (!h) return CCA_ERR_INVALID_ARG;
+  h->ev_attn_begin = (cudaEvent_t)ev_begin;
+  h->ev_attn_end = (cudaEvent_t)ev_end;
+  return CCA_OK;
+}
+
+int64_t cca_launch_count(const cca_handle* h) { return h ? h->launches : -1; }
+int cca_last_cuda_error(const cca_handle* h) { return h ? h->last_cuda : -1; }
+
+int cca_last_status(cca_handle* h, int* device_status) {
+  if (!h || !device_status || h->device < 0) return CCA_ERR_INVALID_ARG;
+  int host[16];
+  CU(cudaMemcpy(host, h->d_status, 64, cudaMemcpyDeviceToHost));
+  *device_status = host[0];
+  if (host[0] != 0) {
+    cudaMemset(h->d_status, 0, 64);
+    return CCA_ERR_DEVICE_TIMEOUT;
+  }
+  return CCA_OK;
+}
+
+int cca_describe(const cca_handle* h, int64_t B, int64_t S, cca_layout* out) {
+  int r = check_sizes(h, B, S);
+  if (r != CCA_OK) return r;
+  if (!out) return CCA_ERR_INVALID_ARG;
+  const cca_config& c = h->cfg;
+  memset(out, 0, sizeof(*out));
+  const int64_t E = c.d_model, dh = c.head_dim;
+  const int64_t Lq = (int64_t)c.n_q_heads * dh, Lk = (int64_t)c.n_kv_heads * dh, L = Lq + Lk, T = B * S;
+  out->L_q = Lq;
+  out->L_k = Lk;
+  out->g = c.n_q_heads / c.n_kv_heads;
+  out->total_padding = c.k_seq + c.k_ch - 2;
+  out->v_shift_split = Lk / 2;
+  for (int i = 0; i < 64; ++i) out->q_to_kv_head[i] = i < c.n_q_heads ? i / out->g : -1;
+  out->conv_params = L * c.k_seq + L * dh * c.k_ch;
+  out->params = E * Lq + 2 * E * Lk + Lq * E + out->conv_params;
+  out->kv_cache_elems = 2 * B * S * Lk;
+  const int64_t proj = 2 * T * E * (Lq + 2 * Lk) + 2 * T * Lq * E;
+  out->fwd_flops = proj + 4 * B * S * S * Lq + 2 * T * out->conv_params;
+  out->fwd_flops_causal = proj + 2 * B * S * S * Lq + 2 * T * out->conv_params;
+  out->decode_flops = 2 * B * E * (Lq + 2 * Lk) + 2 * B * Lq * E + 4 * B * S * Lq + 2 * B * out->conv_params;
+  Layout l = make_layout(c, B, S);
+  out->off_qk0 = (int64_t)l.qk0; out->off_q = (int64_t)l.q; out->off_k = (int64_t)l.k; out->off_v = (int64_t)l.v;
+  out->off_o = (int64_t)l.o; out->off_lse = (int64_t)l.lse; out->off_rope = (int64_t)l.rope;
+  out->saved_bytes = (int64_t)l.saved_end;
+  out->total_bytes = (int64_t)l.total_end;
+  return CCA_OK;
+}
+
+int cca_workspace_size(const cca_handle* h, int64_t B, int64_t S, int need_backward, size_t* bytes) {
+  int r = check_sizes(h, B, S);
+  if (r != CCA_OK) return r;
+  if (!bytes) return CCA_ERR_INVALID_ARG;
+  Layout l = make_layout(h->cfg, B, S);
+  *bytes = need_backward ? l.total_end : l.saved_end;
+  return CCA_OK;
+}
+
+int cca_attention_forward(cca_handle* h, const void* q, const void* k, const void* v, void* o, float* lse, int64_t B,
+                          int64_t S, void* cuda_stream) {
+  int r = check_sizes(h, B, S, true);
+  if (r != CCA_OK) return r;
+  if (!q || !k || !v || !o || !lse) return CCA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return CCA_ERR_ALIGNMENT;
+  CU(cudaSetDevice(h->device));
+  CcaDims d = make_dims(h->cfg, B, S);
+  return run_attention_fwd(h, d, (const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)o, lse,
+                           (cudaStream_t)cuda_stream);
+}
+
+int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, void* workspace,
+                size_t workspace_bytes, int64_t B, int64_t S, void* cuda_stream) {
+  int r = check_sizes(h, B, S, true);
+  if (r != CCA_OK) return r;
+  if (!w || !x || !out || !workspace) return CCA_ERR_INVALID_ARG;
+  if (!w->w_qk || !w->w_v1 || !w->w_v2 || !w->w_o) return CCA_ERR_INVALID_ARG;
+  const cca_config& c = h->cfg;
+  if ((c.flags & CCA_CONV1) && !w->conv0_w) return CCA_ERR_INVALID_ARG;
+  if ((c.flags & CCA_CONV2) && !w->conv1_w) return CCA_ERR_INVALID_ARG;
+  if ((c.flags & CCA_QK_NORM) && !w->temp) return CCA_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(out) || !aligned16(w->w_qk) || !aligned16(w->w_v1) || !aligned16(w->w_v2) ||
+      !aligned16(w->w_o) || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CCA_ERR_ALIGNMENT;
+  Layout l = make_layout(c, B, S);
+  if (workspace_bytes < l.saved_end) return CCA_ERR_WORKSPACE_TOO_SMALL;
+  CU(cudaSetDevice(h->device));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CcaDims d = make_dims(c, B, S);
+  const int T = d.B * d.S;
+  char* ws = (char*)workspace;
+  bf16* qk0 = (bf16*)(ws + l.qk0);
+  bf16* q = (bf16*)(ws + l.q);
+  bf16* k = (bf16*)(ws + l.k);
+  bf16* v = (bf16*)(ws + l.v);
+  bf16* o = (bf16*)(ws + l.o);
+  float* lse = (float*)(ws + l.lse);
+  float2* rope = (float2*)(ws + l.rope);
+
+  if (c.flags & CCA_ROPE) {
+    CU(launch_rope_table(rope, d.S, d.dh, c.rope_base, st));
+    h->launches++;
+  }
+  // Eq. 7: packed q/k down-projection
+  GemmArgs g{};
+  g.A = kmajor(x, d.E); g.B = kmajor(w->w_qk, d.E);
+  g.M = T; g.N = d.L; g.K = d.E; g.a_row_off = 0; g.seq_len = d.S;
+  g.out_bf16 = qk0; g.out_f32 = nullptr; g.ldc = d.L;
+  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  // Eq. 10: value halves from x_t and x_{t-1}
+  g.B = kmajor(w->w_v1, d.E); g.N = d.Lk / 2; g.out_bf16 = v; g.ldc = d.Lk;
+  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  g.B = kmajor(w->w_v2, d.E); g.out_bf16 = v + d.Lk / 2;
+  g.a_row_off = (c.flags & CCA_V_SHIFT) ? -1 : 0;
+  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  // Eq. 8, 9, 11: convs, q-k-mean, norm, temperature, RoPE
+  CU(launch_transform_fwd(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k, st));
+  h->launches++;
+  // Eq. 11: attention in the latent
+  if ((r = run_attention_fwd(h, d, q, k, v, o, lse, st)) != CCA_OK) return r;
+  // Eq. 11: up-projection
+  g = GemmArgs{};
+  g.A = kmajor(o, d.Lq); g.B = kmajor(w->w_o, d.Lq);
+  g.M = T; g.N = d.E; g.K = d.Lq; g.a_row_off = 0; g.seq_len = d.S;
+  g.out_bf16 = (bf16*)out; g.ldc = d.E;
+  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  return CCA_OK;
+}
+
+int cca_forward_host(cca_handle* h, const cca_weights* w, const void* x_host, void* out_host, void* workspace,
+                     size_t workspace_bytes, int64_t B, int64_t S, void* cuda_stream) {
+  int r = check_sizes(h, B, S, true);
+  if (r != CCA_OK) return r;
+  if (!x_host || !out_host || !workspace) return CCA_ERR_INVALID_ARG;
+  Layout l = make_layout(h->cfg, B, S);
+  const size_t act = align_up((size_t)B * S * h->cfg.d_model * 2, 256);
+  if (workspace_bytes < l.total_end + 2 * act) return CCA_ERR_WORKSPACE_TOO_SMALL;
+  CU(cudaSetDevice(h->device));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  char* xs = (char*)workspace + l.total_end;
+  char* os = xs + act;
+  CU(cudaMemcpyAsync(xs, x_host, (size_t)B * S * h->cfg.d_model * 2, cudaMemcpyHostToDevice, st));
+  r = cca_forward(h, w, xs, os, workspace, l.total_end, B, S, cuda_stream);
+  if (r != CCA_OK) return r;
+  CU(cudaMemcpyAsync(out_host, os, (size_t)B * S * h->cfg.d_model * 2, cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  return CCA_OK;
+}
+
+int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void* d_out, void* workspace,
+                 size_t workspace_bytes, void* d_x, const cca_weight_grads* gr, int64_t B, int64_t S,
+                 void* cuda_stream) {
+  int r = check_sizes(h, B, S, true);
+  if (r != CCA_OK) return r;
+  if (!w || !x || !d_out || !workspace || !d_x || !gr) return CCA_ERR_INVALID_ARG;
+  if (!w->w_qk || !w->w_v1 || !w->w_v2 || !w->w_o) return CCA_ERR_INVALID_ARG;
+  if (!gr->d_w_qk || !gr->d_w_v1 || !gr->d_w_v2 || !gr->d_w_o || !gr->d_conv0_w || !gr->d_conv1_w || !gr->d_temp)
+    return CCA_ERR_INVALID_ARG;
+  const cca_config& c = h->cfg;
+  if (!aligned16(x) || !aligned16(d_out) || !aligned16(d_x) || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CCA_ERR_ALIGNMENT;
+  Layout l = make_layout(c, B, S);
+  if (workspace_bytes < l.total_end) return CCA_ERR_WORKSPACE_TOO_SMALL;
+  CU(cudaSetDevice(h->device));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CcaDims d = make_dims(c, B, S);
+  const int T = d.B * d.S;
+  char* ws = (char*)workspace;
+  const bf16* qk0 = (const bf16*)(ws + l.qk0);
+  const bf16* q = (const bf16*)(ws + l.q);
+  const bf16* k = (const bf16*)(ws + l.k);
+  const bf16* v = (const bf16*)(ws + l.v);
+  const bf16* o = (const bf16*)(ws + l.o);
+  const float* lse = (const float*)(ws + l.lse);
+  const float2* rope = (const float2*)(ws + l.rope);
+  bf16* d_o = (bf16*)(ws + l.d_o);
+  float* delta = (float*)(ws + l.delta);
+  float* dq = (float*)(ws + l.dq);
+  float* dk = (float*)(ws + l.dk);
+  float* dv = (float*)(ws + l.dv);
+  bf16* dlat = (bf16*)(ws + l.dlat);
+  bf16* w_all = (bf16*)(ws + l.w_all);
+  const long long ldl = d.L + d.Lk;
+
+  CU(cudaMemsetAsync(gr->d_conv0_w, 0, (size_t)d.L * c.k_seq * 4, st));
+  CU(cudaMemsetAsync(gr->d_conv1_w, 0, (size_t)d.L * d.dh * c.k_ch * 4, st));
+  CU(cudaMemsetAsync(gr->d_temp, 0, (size_t)d.hk * 4, st));
+  // up-projection adjoint: d_o = d_out W_o ; d_W_o = d_out^T o
+  GemmArgs g{};
+  g.A = kmajor(d_out, d.E); g.B = mmajor(w->w_o, d.Lq);
+  g.M = T; g.N = d.Lq; g.K = d.E; g.seq_len = d.S; g.out_bf16 = d_o; g.ldc = d.Lq;
+  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  g = GemmArgs{};
+  g.A = mmajor(d_out, d.E); g.B = mmajor(o, d.Lq);
+  g.M = d.E; g.N = d.Lq; g.K = T; g.seq_len = d.S; g.out_f32 = gr->d_w_o; g.ldc = d.Lq;
+  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  // attention adjoint
+  CU(launch_attn_bwd_simt(d, q, k, v, o, d_o, lse, delta, dq, dk, dv, st));
+  h->launches += 3;
+  // latent-transform adjoints
+  CU(launch_transform_bwd_norm(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, dq, dk,
+                               gr->d_temp, st));
+  CU(launch_transform_bwd_conv(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, dq, dk, dlat, ldl,
+                               gr->d_conv0_w, st));
+  CU(launch_transform_bwd_w1(d, qk0, (const bf16*)w->conv0_w, dq, dk, gr->d_conv1_w, st));
+  CU(launch_pack_dv(d, dv, dlat, ldl, st));
+  h->launches += 4;
+  // down-projection adjoints: parameter gradients
+  g = GemmArgs{};
+  g.A = mmajor(dlat, ldl); g.B = mmajor(x, d.E);
+  g.M = d.L; g.N = d.E; g.K = T; g.seq_len = d.S; g.out_f32 = gr->d_w_qk; g.ldc = d.E;
+  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  g.A = mmajor(dlat + d.L, ldl); g.M = d.Lk / 2; g.out_f32 = gr->d_w_v1;
+  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  g.A = mmajor(dlat + d.L + d.Lk / 2, ldl); g.out_f32 = gr->d_w_v2;
+  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  // input gradient: d_x = [d_qk0, d_v1, d_v2 moved one token earlier] [W_qk; W_v1; W_v2]
+  CU(cudaMemcpyAsync(w_all, w->w_qk, (size_t)d.L * d.E * 2, cudaMemcpyDeviceToDevice, st));
+  CU(cudaMemcpyAsync(w_all + (size_t)d.L * d.E, w->w_v1, (size_t)(d.Lk / 2) * d.E * 2, cudaMemcpyDeviceToDevice, st));
+  CU(cudaMemcpyAsync(w_all + (size_t)(d.L + d.Lk / 2) * d.E, w->w_v2, (size_t)(d.Lk / 2) * d.E * 2,
+                     cudaMemcpyDeviceToDevice, st));
+  g = GemmArgs{};
+  g.A = kmajor(dlat, ldl); g.B = mmajor(w_all, d.E);
+  g.M = T; g.N = d.E; g.K = (int)ldl; g.seq_len = d.S; g.out_bf16 = (bf16*)d_x; g.ldc = d.E;
+  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  return CCA_OK;
+}
+
+}  // extern "C"

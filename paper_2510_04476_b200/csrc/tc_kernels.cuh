@@ -1,0 +1,13 @@
+// Tensor-core (tcgen05 / TMEM / TMA) kernels of the CCA library: host-side interface.
+// Each tc_* launcher returns 0 if it enqueued the work, 1 if the case is outside its coverage
+// (the caller then uses the SIMT kernel), or -cudaError on a CUDA failure.
+#pragma once
+#include "common.cuh"
+
+struct TcState;
+
+TcState* tc_create(int sm_count);
+void tc_destroy(TcState* s);
+int tc_gemm(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st);
+int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* lse,
+                int* d_status, cudaStream_t st);

@@ -1,0 +1,531 @@
+// Latent transforms on q and k between the down-projection and the attention (Eq. 8, 9, 11):
+// conv1_seq, conv2_seq+ch, q-k-mean, L2 norm * sqrt(d_h) (* exp(temp) for keys), RoPE;
+// and their adjoints.  One thread block works on (a run of 32-token tiles, one head, one sequence).
+// Thread layout: 256 threads = (256/DH) token groups x DH channels; a thread owns one channel of
+// TT/(256/DH) consecutive tokens of the tile.
+#include "common.cuh"
+
+namespace {
+
+constexpr int TT = 32;             // tokens per tile
+constexpr int TILES_PER_BLOCK = 4; // tiles a block walks through with one load of the conv2 weights
+constexpr int MAXK = 4;            // largest conv kernel size
+
+enum : unsigned { F_CONV1 = 1, F_CONV2 = 2, F_QK_MEAN = 4, F_V_SHIFT = 8, F_QK_NORM = 16, F_ROPE = 32 };
+
+template <int DH>
+struct Lay {
+  static constexpr int NG = 256 / DH;        // token groups
+  static constexpr int TPT = TT / NG;        // tokens per thread
+  static constexpr int WLD = DH + 2;         // bf16 row stride of the staged conv2 weights
+  static constexpr int YLD = DH + 1;         // fp32 row stride of token-major tiles
+  static constexpr int YROWS = TT + 2 * (MAXK - 1);
+};
+
+CCA_DEVINL float ldbf(const bf16* p) { return __bfloat162float(*p); }
+
+// conv1_seq output (or the raw latent if the stage is off) of channel `ch` at token t of sequence b.
+CCA_DEVINL float y1_at(const CcaDims& d, const bf16* qk0, const bf16* w0, int b, int t, int ch) {
+  if (t < 0 || t >= d.S) return 0.f;
+  const bf16* col = qk0 + (long long)b * d.S * d.L + ch;
+  if (!(d.flags & F_CONV1)) return ldbf(col + (long long)t * d.L);
+  float acc = 0.f;
+  for (int j = 0; j < d.k_seq; ++j) {
+    int ts = t - (d.k_seq - 1) + j;
+    if (ts >= 0) acc = fmaf(ldbf(w0 + ch * d.k_seq + j), ldbf(col + (long long)ts * d.L), acc);
+  }
+  return acc;
+}
+
+// Stage the conv2 weights of head h as ws[(i*k_ch + j)][o]  (forward) or ws[(o*k_ch + j)][i] (adjoint).
+template <int DH, bool kAdjoint>
+CCA_DEVINL void stage_w1(const CcaDims& d, const bf16* w1, int h, bf16* ws) {
+  const int per_o = DH * d.k_ch;
+  const bf16* src = w1 + (long long)h * DH * per_o;
+  for (int f = threadIdx.x; f < DH * per_o; f += 256) {
+    int o = f / per_o, rem = f - o * per_o;       // rem = i*k_ch + j
+    if (!kAdjoint) ws[rem * Lay<DH>::WLD + o] = src[f];
+    else {
+      int i = rem / d.k_ch, j = rem - i * d.k_ch;
+      ws[(o * d.k_ch + j) * Lay<DH>::WLD + i] = src[f];
+    }
+  }
+}
+
+// y1s[r][c], r in [0, rows): conv1 output of head h's channels at token t_first + r.
+template <int DH>
+CCA_DEVINL void fill_y1(const CcaDims& d, const bf16* qk0, const bf16* w0, int b, int h, int t_first, int rows,
+                        float* y1s) {
+  for (int f = threadIdx.x; f < rows * DH; f += 256) {
+    int r = f / DH, c = f - r * DH;
+    y1s[r * Lay<DH>::YLD + c] = y1_at(d, qk0, w0, b, t_first + r, h * DH + c);
+  }
+}
+
+// Pre-norm latent (conv2 output + q-k-mean term) of channel o for this thread's tokens.
+// y1s row r holds token t0 - (k_ch-1) + r.
+template <int DH>
+CCA_DEVINL void hat_tile(const CcaDims& d, const bf16* qk0, const bf16* ws, const float* y1s, int b, int h, int t0,
+                         float (&acc)[Lay<DH>::TPT]) {
+  constexpr int TPT = Lay<DH>::TPT;
+  const int o = threadIdx.x % DH, tg = threadIdx.x / DH;
+  const int kc = (d.flags & F_CONV2) ? d.k_ch : 1;
+#pragma unroll
+  for (int n = 0; n < TPT; ++n) acc[n] = 0.f;
+  if (d.flags & F_CONV2) {
+    for (int i = 0; i < DH; ++i) {
+      for (int j = 0; j < kc; ++j) {
+        float w = __bfloat162float(ws[(i * kc + j) * Lay<DH>::WLD + o]);
+        const float* yp = y1s + (tg * TPT + j) * Lay<DH>::YLD + i;
+#pragma unroll
+        for (int n = 0; n < TPT; ++n) acc[n] = fmaf(w, yp[n * Lay<DH>::YLD], acc[n]);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int n = 0; n < TPT; ++n) acc[n] = y1s[(tg * TPT + n + (d.k_ch - 1)) * Lay<DH>::YLD + o];
+  }
+  if (d.flags & F_QK_MEAN) {
+    const bf16* base = qk0 + (long long)b * d.S * d.L;
+#pragma unroll
+    for (int n = 0; n < TPT; ++n) {
+      int t = t0 + tg * TPT + n;
+      if (t >= d.S) continue;
+      const bf16* row = base + (long long)t * d.L;
+      if (h < d.hq) {
+        acc[n] += 0.5f * (ldbf(row + h * DH + o) + ldbf(row + d.Lq + (h / d.g) * DH + o));
+      } else {
+        int jk = h - d.hq;
+        float sq = 0.f;
+        for (int i = 0; i < d.g; ++i) sq += ldbf(row + (jk * d.g + i) * DH + o);
+        acc[n] += 0.5f * ldbf(row + d.Lq + jk * DH + o) + (0.5f / d.g) * sq;
+      }
+    }
+  }
+}
+
+// Sum over the DH channels of each of this thread's tokens (all threads of the group get the result).
+template <int DH>
+CCA_DEVINL void reduce_channels(float (&v)[Lay<DH>::TPT], float* red /*[NG][DH/32][TPT]*/) {
+  constexpr int TPT = Lay<DH>::TPT, NW = DH / 32;
+  const int o = threadIdx.x % DH, tg = threadIdx.x / DH, wi = o / 32;
+#pragma unroll
+  for (int n = 0; n < TPT; ++n) {
+    float s = v[n];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    v[n] = s;
+  }
+  if (NW > 1) {
+    __syncthreads();
+    if ((o & 31) == 0)
+#pragma unroll
+      for (int n = 0; n < TPT; ++n) red[(tg * NW + wi) * TPT + n] = v[n];
+    __syncthreads();
+#pragma unroll
+    for (int n = 0; n < TPT; ++n) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) s += red[(tg * NW + w) * TPT + n];
+      v[n] = s;
+    }
+  }
+}
+
+template <int DH>
+constexpr size_t smem_bytes() {
+  return (size_t)DH * MAXK * Lay<DH>::WLD * sizeof(bf16) + (size_t)Lay<DH>::YROWS * Lay<DH>::YLD * sizeof(float) +
+         (size_t)(TT + 2 * (MAXK - 1)) * Lay<DH>::YLD * sizeof(float) + 256 * sizeof(float);
+}
+
+template <int DH>
+struct Smem {
+  bf16* ws;
+  float* y1s;
+  float* outs;
+  float* red;
+  __device__ explicit Smem(unsigned char* base) {
+    ws = reinterpret_cast<bf16*>(base);
+    y1s = reinterpret_cast<float*>(base + (size_t)DH * MAXK * Lay<DH>::WLD * sizeof(bf16));
+    outs = y1s + Lay<DH>::YROWS * Lay<DH>::YLD;
+    red = outs + (TT + 2 * (MAXK - 1)) * Lay<DH>::YLD;
+  }
+};
+
+// ------------------------------------------------------------------------------------------
+// forward
+// ------------------------------------------------------------------------------------------
+template <int DH>
+__global__ void __launch_bounds__(256) transform_fwd_kernel(CcaDims d, const bf16* __restrict__ qk0,
+                                                            const bf16* __restrict__ w0, const bf16* __restrict__ w1,
+                                                            const float* __restrict__ temp,
+                                                            const float2* __restrict__ rope_tab, bf16* __restrict__ q,
+                                                            bf16* __restrict__ k) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Smem<DH> sm(smem_raw);
+  constexpr int TPT = Lay<DH>::TPT, YLD = Lay<DH>::YLD;
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int o = threadIdx.x % DH, tg = threadIdx.x / DH;
+  if (d.flags & F_CONV2) stage_w1<DH, false>(d, w1, h, sm.ws);
+  const float scale = (d.flags & F_QK_NORM) ? sqrtf((float)DH) * (h >= d.hq ? __expf(temp[h - d.hq]) : 1.f) : 1.f;
+  for (int tile = 0; tile < TILES_PER_BLOCK; ++tile) {
+    const int t0 = (blockIdx.x * TILES_PER_BLOCK + tile) * TT;
+    if (t0 >= d.S) break;
+    __syncthreads();
+    fill_y1<DH>(d, qk0, w0, b, h, t0 - (d.k_ch - 1), TT + d.k_ch - 1, sm.y1s);
+    __syncthreads();
+    float acc[TPT];
+    hat_tile<DH>(d, qk0, sm.ws, sm.y1s, b, h, t0, acc);
+    if (d.flags & F_QK_NORM) {
+      float ss[TPT];
+#pragma unroll
+      for (int n = 0; n < TPT; ++n) ss[n] = acc[n] * acc[n];
+      reduce_channels<DH>(ss, sm.red);
+#pragma unroll
+      for (int n = 0; n < TPT; ++n) acc[n] *= scale * rsqrtf(ss[n]);
+    }
+#pragma unroll
+    for (int n = 0; n < TPT; ++n) sm.outs[(tg * TPT + n) * YLD + o] = acc[n];
+    __syncthreads();
+#pragma unroll
+    for (int n = 0; n < TPT; ++n) {
+      int tl = tg * TPT + n, t = t0 + tl;
+      if (t >= d.S) continue;
+      float val = acc[n];
+      if (d.flags & F_ROPE) {
+        constexpr int HALF = DH / 2;
+        int c = o < HALF ? o : o - HALF;
+        float2 cs = rope_tab[(long long)t * HALF + c];
+        float other = sm.outs[tl * YLD + (o < HALF ? o + HALF : o - HALF)];
+        val = o < HALF ? acc[n] * cs.x - other * cs.y : acc[n] * cs.x + other * cs.y;
+      }
+      long long row = (long long)b * d.S + t;
+      if (h < d.hq) q[row * d.Lq + h * DH + o] = __float2bfloat16(val);
+      else k[row * d.Lk + (h - d.hq) * DH + o] = __float2bfloat16(val);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// backward, part 1: RoPE adjoint, norm adjoint, d_temp.  In place on dq / dk (fp32).
+// ------------------------------------------------------------------------------------------
+template <int DH>
+__global__ void __launch_bounds__(256) transform_bwd_norm_kernel(CcaDims d, const bf16* __restrict__ qk0,
+                                                                 const bf16* __restrict__ w0,
+                                                                 const bf16* __restrict__ w1,
+                                                                 const float* __restrict__ temp,
+                                                                 const float2* __restrict__ rope_tab, float* dq,
+                                                                 float* dk, float* d_temp) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Smem<DH> sm(smem_raw);
+  constexpr int TPT = Lay<DH>::TPT, YLD = Lay<DH>::YLD, HALF = DH / 2;
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int o = threadIdx.x % DH, tg = threadIdx.x / DH;
+  const bool is_q = h < d.hq;
+  float* grad = is_q ? dq : dk;
+  const int ld = is_q ? d.Lq : d.Lk;
+  const int col = (is_q ? h : h - d.hq) * DH + o;
+  if (d.flags & F_CONV2) stage_w1<DH, false>(d, w1, h, sm.ws);
+  const float scale = sqrtf((float)DH) * (is_q ? 1.f : __expf(temp[h - d.hq]));
+  float dtemp_local = 0.f;
+  for (int tile = 0; tile < TILES_PER_BLOCK; ++tile) {
+    const int t0 = (blockIdx.x * TILES_PER_BLOCK + tile) * TT;
+    if (t0 >= d.S) break;
+    __syncthreads();
+    // incoming gradient tile -> outs
+#pragma unroll
+    for (int n = 0; n < TPT; ++n) {
+      int tl = tg * TPT + n, t = t0 + tl;
+      sm.outs[tl * YLD + o] = t < d.S ? grad[((long long)b * d.S + t) * ld + col] : 0.f;
+    }
+    if (d.flags & F_QK_NORM) fill_y1<DH>(d, qk0, w0, b, h, t0 - (d.k_ch - 1), TT + d.k_ch - 1, sm.y1s);
+    __syncthreads();
+    float dy[TPT];
+#pragma unroll
+    for (int n = 0; n < TPT; ++n) {
+      int tl = tg * TPT + n, t = t0 + tl;
+      float own = sm.outs[tl * YLD + o];
+      if ((d.flags & F_ROPE) && t < d.S) {
+        int c = o < HALF ? o : o - HALF;
+        float2 cs = rope_tab[(long long)t * HALF + c];
+        float other = sm.outs[tl * YLD + (o < HALF ? o + HALF : o - HALF)];
+        // rotation by the negated angle
+        own = o < HALF ? own * cs.x + other * cs.y : own * cs.x - other * cs.y;
+      }
+      dy[n] = own;
+    }
+    if (d.flags & F_QK_NORM) {
+      float xh[TPT], ss[TPT], dot[TPT];
+      hat_tile<DH>(d, qk0, sm.ws, sm.y1s, b, h, t0, xh);
+#pragma unroll
+      for (int n = 0; n < TPT; ++n) {
+        ss[n] = xh[n] * xh[n];
+        dot[n] = xh[n] * dy[n];
+      }
+      reduce_channels<DH>(ss, sm.red);
+      reduce_channels<DH>(dot, sm.red);
+#pragma unroll
+      for (int n = 0; n < TPT; ++n) {
+        int t = t0 + tg * TPT + n;
+        if (t >= d.S) { dy[n] = 0.f; continue; }
+        float inv = rsqrtf(ss[n]);                 // 1/|x|
+        float ndot = dot[n] * inv;                 // n . dy
+        if (!is_q && o == 0) dtemp_local += scale * ndot;
+        dy[n] = scale * inv * (dy[n] - xh[n] * inv * ndot);
+      }
+    }
+#pragma unroll
+    for (int n = 0; n < TPT; ++n) {
+      int t = t0 + tg * TPT + n;
+      if (t < d.S) grad[((long long)b * d.S + t) * ld + col] = dy[n];
+    }
+  }
+  if (!is_q && o == 0 && (d.flags & F_QK_NORM)) atomicAdd(d_temp + (h - d.hq), dtemp_local);
+}
+
+// ------------------------------------------------------------------------------------------
+// backward, part 2: q-k-mean adjoint, conv2 adjoint, conv1 adjoint -> gradient of the packed
+// latent qk0 (bf16), and the gradient of the depth-wise taps.
+// ------------------------------------------------------------------------------------------
+CCA_DEVINL float dhat_at(const CcaDims& d, const float* dqh, const float* dkh, int b, int t, int h, int o) {
+  if (t < 0 || t >= d.S) return 0.f;
+  long long row = (long long)b * d.S + t;
+  return h < d.hq ? dqh[row * d.Lq + h * d.dh + o] : dkh[row * d.Lk + (h - d.hq) * d.dh + o];
+}
+
+template <int DH>
+__global__ void __launch_bounds__(256) transform_bwd_conv_kernel(CcaDims d, const bf16* __restrict__ qk0,
+                                                                 const bf16* __restrict__ w0,
+                                                                 const bf16* __restrict__ w1,
+                                                                 const float* __restrict__ dqh,
+                                                                 const float* __restrict__ dkh, bf16* __restrict__ dlat,
+                                                                 long long ld_dlat, float* d_w0) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Smem<DH> sm(smem_raw);
+  constexpr int TPT = Lay<DH>::TPT, YLD = Lay<DH>::YLD, NG = Lay<DH>::NG;
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int i = threadIdx.x % DH, tg = threadIdx.x / DH;   // this thread's channel (input side of conv2)
+  const int ch = h * DH + i;
+  const int kc = (d.flags & F_CONV2) ? d.k_ch : 1;
+  const int ks = (d.flags & F_CONV1) ? d.k_seq : 1;
+  if (d.flags & F_CONV2) stage_w1<DH, true>(d, w1, h, sm.ws);
+  float w0r[MAXK];
+  for (int j = 0; j < MAXK; ++j) w0r[j] = (j < d.k_seq) ? ldbf(w0 + ch * d.k_seq + j) : 0.f;
+  float dw0[MAXK] = {0.f, 0.f, 0.f, 0.f};
+  float* dy2s = sm.y1s;    // [TT + (kc-1) + (ks-1)][YLD]: dy2 at tokens t0 + r
+  float* dy1s = sm.outs;   // [TT + (ks-1)][YLD]:          dy1 at tokens t0 + r
+  for (int tile = 0; tile < TILES_PER_BLOCK; ++tile) {
+    const int t0 = (blockIdx.x * TILES_PER_BLOCK + tile) * TT;
+    if (t0 >= d.S) break;
+    __syncthreads();
+    const int rows2 = TT + (kc - 1) + (ks - 1), rows1 = TT + (ks - 1);
+    for (int f = threadIdx.x; f < rows2 * DH; f += 256) {
+      int r = f / DH, c = f - r * DH;
+      dy2s[r * YLD + c] = dhat_at(d, dqh, dkh, b, t0 + r, h, c);
+    }
+    __syncthreads();
+    // conv2 adjoint: dy1[t'][i] = sum_{o,j} w1[o][i][j] dy2[t' + (kc-1) - j][o]
+    for (int r = tg; r < rows1; r += NG) {
+      float a = 0.f;
+      if (d.flags & F_CONV2) {
+        for (int o = 0; o < DH; ++o)
+          for (int j = 0; j < kc; ++j)
+            a = fmaf(__bfloat162float(sm.ws[(o * kc + j) * Lay<DH>::WLD + i]), dy2s[(r + (kc - 1) - j) * YLD + o], a);
+      } else {
+        a = dy2s[r * YLD + i];
+      }
+      dy1s[r * YLD + i] = (t0 + r < d.S) ? a : 0.f;
+    }
+    __syncthreads();
+    // conv1 adjoint + q-k-mean adjoint for this thread's tokens
+#pragma unroll
+    for (int n = 0; n < TPT; ++n) {
+      int tl = tg * TPT + n, t = t0 + tl;
+      if (t >= d.S) continue;
+      float gq;
+      if (d.flags & F_CONV1) {
+        gq = 0.f;
+        for (int j = 0; j < ks; ++j) gq = fmaf(w0r[j], dy1s[(tl + (ks - 1) - j) * YLD + i], gq);
+        // taps' gradient: dw0[j] += dy1[t] * qk0[t - (ks-1) + j]
+        float dy1_t = dy1s[tl * YLD + i];
+        for (int j = 0; j < ks; ++j) {
+          int ts = t - (ks - 1) + j;
+          if (ts >= 0) dw0[j] = fmaf(dy1_t, ldbf(qk0 + ((long long)b * d.S + ts) * d.L + ch), dw0[j]);
+        }
+      } else {
+        gq = dy1s[tl * YLD + i];
+      }
+      if (d.flags & F_QK_MEAN) {
+        if (h < d.hq) {
+          gq += 0.5f * (dhat_at(d, dqh, dkh, b, t, h, i) + dhat_at(d, dqh, dkh, b, t, d.hq + h / d.g, i) / d.g);
+        } else {
+          int jk = h - d.hq;
+          float s = dhat_at(d, dqh, dkh, b, t, h, i);
+          for (int m = 0; m < d.g; ++m) s += dhat_at(d, dqh, dkh, b, t, jk * d.g + m, i);
+          gq += 0.5f * s;
+        }
+      }
+      dlat[((long long)b * d.S + t) * ld_dlat + ch] = __float2bfloat16(gq);
+    }
+  }
+  if (d.flags & F_CONV1)
+    for (int j = 0; j < d.k_seq; ++j) atomicAdd(d_w0 + ch * d.k_seq + j, dw0[j]);
+}
+
+// ------------------------------------------------------------------------------------------
+// backward, part 3: gradient of the conv2 weights,
+//   d_w1[h,o,i,j] = sum_{b,t} dy2[t,h,o] * y1[t-(k_ch-1)+j, h, i].
+// Block = (token chunk, head, sequence); thread tile RO x RI outputs of the d_h x d_h block per tap.
+// ------------------------------------------------------------------------------------------
+template <int DH>
+__global__ void __launch_bounds__(256) transform_bwd_w1_kernel(CcaDims d, const bf16* __restrict__ qk0,
+                                                               const bf16* __restrict__ w0,
+                                                               const float* __restrict__ dqh,
+                                                               const float* __restrict__ dkh, float* d_w1,
+                                                               int chunk_tokens) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Smem<DH> sm(smem_raw);
+  constexpr int YLD = Lay<DH>::YLD;
+  constexpr int R = DH / 16;                // 16 x 16 threads, R x R outputs each
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int to = threadIdx.x / 16, ti = threadIdx.x % 16;
+  float* dy2s = sm.outs;   // [TT][YLD]
+  float* y1s = sm.y1s;     // [TT + k_ch - 1][YLD], row r = token t0 - (k_ch-1) + r
+  const int c_begin = blockIdx.x * chunk_tokens, c_end = min(d.S, c_begin + chunk_tokens);
+  for (int j = 0; j < d.k_ch; ++j) {
+    float acc[R][R];
+#pragma unroll
+    for (int a = 0; a < R; ++a)
+#pragma unroll
+      for (int c = 0; c < R; ++c) acc[a][c] = 0.f;
+    for (int t0 = c_begin; t0 < c_end; t0 += TT) {
+      __syncthreads();
+      for (int f = threadIdx.x; f < TT * DH; f += 256) {
+        int r = f / DH, c = f - r * DH;
+        dy2s[r * YLD + c] = (t0 + r < c_end) ? dhat_at(d, dqh, dkh, b, t0 + r, h, c) : 0.f;
+      }
+      fill_y1<DH>(d, qk0, w0, b, h, t0 - (d.k_ch - 1), TT + d.k_ch - 1, y1s);
+      __syncthreads();
+      for (int r = 0; r < TT; ++r) {
+        float dv[R], yv[R];
+#pragma unroll
+        for (int a = 0; a < R; ++a) dv[a] = dy2s[r * YLD + to + 16 * a];
+#pragma unroll
+        for (int c = 0; c < R; ++c) yv[c] = y1s[(r + j) * YLD + ti + 16 * c];
+#pragma unroll
+        for (int a = 0; a < R; ++a)
+#pragma unroll
+          for (int c = 0; c < R; ++c) acc[a][c] = fmaf(dv[a], yv[c], acc[a][c]);
+      }
+    }
+#pragma unroll
+    for (int a = 0; a < R; ++a)
+#pragma unroll
+      for (int c = 0; c < R; ++c) {
+        int o = to + 16 * a, i = ti + 16 * c;
+        atomicAdd(d_w1 + ((long long)(h * DH + o) * DH + i) * d.k_ch + j, acc[a][c]);
+      }
+  }
+}
+
+__global__ void rope_table_kernel(float2* tab, int S, int half, double log2_base) {
+  long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)S * half) return;
+  int t = (int)(idx / half), c = (int)(idx % half);
+  double theta = exp2(-(double)c / (double)half * log2_base);   // base^(-2c/d_h)
+  double s, co;
+  sincos((double)t * theta, &s, &co);
+  tab[idx] = make_float2((float)co, (float)s);
+}
+
+__global__ void pack_dv_kernel(CcaDims d, const float* __restrict__ dv, bf16* __restrict__ dlat, long long ld) {
+  long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  long long total = (long long)d.B * d.S * d.Lk;
+  if (idx >= total) return;
+  int c = (int)(idx % d.Lk);
+  long long row = idx / d.Lk;
+  int t = (int)(row % d.S);
+  float val;
+  if (c < d.Lk / 2 || !(d.flags & F_V_SHIFT)) val = dv[idx];
+  else val = (t + 1 < d.S) ? dv[(row + 1) * d.Lk + c] : 0.f;
+  dlat[row * ld + d.L + c] = __float2bfloat16(val);
+}
+
+template <typename K>
+cudaError_t set_smem(K kern, size_t bytes) {
+  return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+}  // namespace
+
+#define DISPATCH_DH(dh, ...)                                    \
+  switch (dh) {                                                 \
+    case 32: { constexpr int DH = 32; __VA_ARGS__; break; }     \
+    case 64: { constexpr int DH = 64; __VA_ARGS__; break; }     \
+    case 128: { constexpr int DH = 128; __VA_ARGS__; break; }   \
+    default: return cudaErrorInvalidValue;                      \
+  }
+
+cudaError_t launch_rope_table(float2* tab, int S, int dh, float base, cudaStream_t st) {
+  long long n = (long long)S * (dh / 2);
+  rope_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(tab, S, dh / 2, log2((double)base));
+  return cudaGetLastError();
+}
+
+static dim3 tile_grid(const CcaDims& d) {
+  return dim3((d.S + TT * TILES_PER_BLOCK - 1) / (TT * TILES_PER_BLOCK), d.hq + d.hk, d.B);
+}
+
+cudaError_t launch_transform_fwd(const CcaDims& d, const bf16* qk0, const bf16* w0, const bf16* w1, const float* temp,
+                                 const float2* rope_tab, bf16* q, bf16* k, cudaStream_t st) {
+  DISPATCH_DH(d.dh, {
+    cudaError_t e = set_smem(transform_fwd_kernel<DH>, smem_bytes<DH>());
+    if (e != cudaSuccess) return e;
+    transform_fwd_kernel<DH><<<tile_grid(d), 256, smem_bytes<DH>(), st>>>(d, qk0, w0, w1, temp, rope_tab, q, k);
+  });
+  return cudaGetLastError();
+}
+
+cudaError_t launch_transform_bwd_norm(const CcaDims& d, const bf16* qk0, const bf16* w0, const bf16* w1,
+                                      const float* temp, const float2* rope_tab, float* dq, float* dk, float* d_temp,
+                                      cudaStream_t st) {
+  if (!(d.flags & (F_QK_NORM | F_ROPE))) return cudaSuccess;
+  DISPATCH_DH(d.dh, {
+    cudaError_t e = set_smem(transform_bwd_norm_kernel<DH>, smem_bytes<DH>());
+    if (e != cudaSuccess) return e;
+    transform_bwd_norm_kernel<DH><<<tile_grid(d), 256, smem_bytes<DH>(), st>>>(d, qk0, w0, w1, temp, rope_tab, dq, dk,
+                                                                              d_temp);
+  });
+  return cudaGetLastError();
+}
+
+cudaError_t launch_transform_bwd_conv(const CcaDims& d, const bf16* qk0, const bf16* w0, const bf16* w1,
+                                      const float* dqh, const float* dkh, bf16* dlat, long long ld_dlat, float* d_w0,
+                                      cudaStream_t st) {
+  DISPATCH_DH(d.dh, {
+    cudaError_t e = set_smem(transform_bwd_conv_kernel<DH>, smem_bytes<DH>());
+    if (e != cudaSuccess) return e;
+    transform_bwd_conv_kernel<DH><<<tile_grid(d), 256, smem_bytes<DH>(), st>>>(d, qk0, w0, w1, dqh, dkh, dlat, ld_dlat,
+                                                                              d_w0);
+  });
+  return cudaGetLastError();
+}
+
+cudaError_t launch_transform_bwd_w1(const CcaDims& d, const bf16* qk0, const bf16* w0, const float* dqh,
+                                    const float* dkh, float* d_w1, cudaStream_t st) {
+  if (!(d.flags & F_CONV2)) return cudaSuccess;
+  const int chunk = 512;
+  dim3 grid((d.S + chunk - 1) / chunk, d.hq + d.hk, d.B);
+  DISPATCH_DH(d.dh, {
+    cudaError_t e = set_smem(transform_bwd_w1_kernel<DH>, smem_bytes<DH>());
+    if (e != cudaSuccess) return e;
+    transform_bwd_w1_kernel<DH><<<grid, 256, smem_bytes<DH>(), st>>>(d, qk0, w0, dqh, dkh, d_w1, chunk);
+  });
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pack_dv(const CcaDims& d, const float* dv, bf16* dlat, long long ld_dlat, cudaStream_t st) {
+  long long total = (long long)d.B * d.S * d.Lk;
+  pack_dv_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(d, dv, dlat, ld_dlat);
+  return cudaGetLastError();
+}

@@ -1,0 +1,171 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 oracle, element by element,
+on the same seeded inputs.  Outputs, saved activations, the input gradient and every parameter
+gradient are compared with max |err| <= 1e-2 + 1e-2 |ref| (see tests/util.py for the parameter-
+gradient scaling of the absolute term)."""
+import math
+
+import pytest
+import torch
+
+from oracle import cca_oracle as O
+from paper_2510_04476_b200 import synth
+from tests.util import PARAM_NAMES, check_close, oracle_cfg, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def _cca(sh):
+    from paper_2510_04476_b200.binding import CCA
+    return CCA.from_shape(sh)
+
+
+def run_case(sh, impl, backward=True, scale_w=1.0, check_saved=True):
+    t = synth.make_inputs(sh)
+    if scale_w != 1.0:
+        for n in ("w_qk", "w_v1", "w_v2"):
+            t[n] = (t[n].float() * scale_w).to(torch.bfloat16)
+    cfg = oracle_cfg(sh)
+    out_ref, I = O.forward(cfg, t, t["x"])
+    dev = to_device(t)
+    cca = _cca(sh)
+    cca.set_impl(impl)
+    ws = cca.alloc_workspace(sh.B, sh.S, True)
+    out = cca.forward(dev, dev["x"], ws)
+    torch.cuda.synchronize()
+    assert cca.last_status() == 0
+    if check_saved:
+        sv = cca.saved(ws, sh.B, sh.S)
+        for n in ("qk0", "v", "q", "k", "o"):
+            check_close(n, sv[n].reshape(I[n].shape) if n != "qk0" else sv[n], I[n])
+        check_close("lse", sv["lse"], I["lse"])
+    check_close("out", out, out_ref)
+    if backward:
+        G = O.backward(cfg, t, I, t["d_out"])
+        d_x, grads = cca.backward(dev, dev["x"], dev["d_out"], ws)
+        torch.cuda.synchronize()
+        assert cca.last_status() == 0
+        check_close("d_x", d_x, G["d_x"])
+        for n in PARAM_NAMES:
+            check_close("d_" + n, grads["d_" + n], G["d_" + n], scale_abs=True)
+    cca.close()
+
+
+def S_(name, B, S, E, hq, hk, dh, **kw):
+    return synth.Shape(name, B, S, E, hq, hk, dh, seed=kw.pop("seed", 7), **kw)
+
+
+SMALL = [
+    S_("dh32_ragged", 2, 100, 256, 4, 4, 32),
+    S_("dh64_gqa4", 1, 257, 512, 4, 1, 64),
+    S_("dh128_gqa2", 1, 130, 1024, 4, 2, 128),
+    S_("one_token", 3, 1, 256, 4, 2, 32),
+    S_("shorter_than_halo", 2, 2, 256, 4, 2, 32, k_seq=4, k_ch=4),
+    S_("k3_k4", 1, 77, 256, 2, 2, 64, k_seq=3, k_ch=4),
+    S_("k1_k1", 1, 65, 256, 2, 1, 64, k_seq=1, k_ch=1),
+    S_("non_causal", 2, 96, 256, 4, 2, 32, causal=0),
+    S_("no_qk_mean", 1, 70, 256, 4, 2, 32, flags=63 & ~4),
+    S_("no_v_shift", 1, 70, 256, 4, 2, 32, flags=63 & ~8),
+    S_("no_convs", 1, 70, 256, 4, 2, 32, flags=63 & ~3),
+    S_("conv1_only_no_rope", 1, 70, 256, 4, 2, 32, flags=1 | 16),
+    S_("three_tiles", 1, 300, 512, 8, 2, 64),
+]
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("sh", SMALL, ids=lambda s: s.name)
+def test_small_cases_forward_backward(sh, impl):
+    run_case(sh, impl)
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_plain_mha_configuration(impl):
+    """C = 1, every latent transform off: the in-house MHA configuration of the same kernels."""
+    sh = S_("mha", 2, 150, 256, 4, 4, 64, flags=0)
+    run_case(sh, impl, scale_w=6.0)
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_cfg1_tiny(impl):
+    run_case(synth.CONFIGS["cfg1_tiny"], impl)
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_cfg2_small_forward_backward(impl):
+    run_case(synth.CONFIGS["cfg2_small"], impl)
+
+
+def test_cfg4_train_forward_backward():
+    run_case(synth.CONFIGS["cfg4_train"], 1)
+
+
+def sample_rows(S, n_random=48, tile=128, seed=0):
+    g = torch.Generator().manual_seed(seed)
+    rows = {0, 1, S - 1, S - 2}
+    for b in (tile, 2 * tile, S // 2, S - tile):
+        rows.update({b - 1, b, b + 1})
+    rows.update(int(r) for r in torch.randint(0, S, (n_random,), generator=g))
+    return sorted(r for r in rows if 0 <= r < S)
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_cfg3_prefill16k_sampled_rows(impl):
+    """Full-size headline shape in the launch configuration the benchmark times.  Latents are
+    compared in full; the S^2 stage on sampled query rows (each row is independent given K, V)."""
+    sh = synth.CONFIGS["cfg3_prefill16k"]
+    t = synth.make_inputs(sh, want_dout=False)
+    rows = sample_rows(sh.S)
+    out_ref, o_ref, lse_ref, I = O.forward_rows(oracle_cfg(sh), t, t["x"], rows)
+    dev = to_device(t)
+    cca = _cca(sh)
+    cca.set_impl(impl)
+    ws = cca.alloc_workspace(sh.B, sh.S, False)
+    out = cca.forward(dev, dev["x"], ws)
+    torch.cuda.synchronize()
+    assert cca.last_status() == 0
+    sv = cca.saved(ws, sh.B, sh.S)
+    for n in ("v", "q", "k"):
+        check_close(n, sv[n], I[n])
+    check_close("o_rows", sv["o"][:, rows], o_ref)
+    check_close("lse_rows", sv["lse"][:, :, rows], lse_ref)
+    check_close("out_rows", out[:, rows], out_ref)
+    # properties that hold at any size: finite everywhere, |o| bounded by max |v| per kv head
+    assert torch.isfinite(out.float()).all()
+    vmax = sv["v"].float().abs().amax(dim=(0, 1, 3))
+    omax = sv["o"].float().abs().amax(dim=(0, 1, 3)).reshape(sh.n_kv_heads, -1).amax(dim=1)
+    assert (omax <= vmax * 1.01 + 1e-3).all()
+    cca.close()
+
+
+@pytest.mark.parametrize("S,C", [(1024, 8), (4096, 2)])
+def test_sweep_points_forward_backward(S, C):
+    sh = synth.sweep_shape(S, C)
+    sh = sh.replace(B=min(sh.B, 2))      # the oracle's share of the batch; sequences are independent
+    run_case(sh, 1)
+
+
+def test_run_to_run_determinism_of_forward():
+    sh = synth.CONFIGS["cfg2_small"]
+    t = to_device(synth.make_inputs(sh))
+    cca = _cca(sh)
+    ws = cca.alloc_workspace(sh.B, sh.S, True)
+    a = cca.forward(t, t["x"], ws).clone()
+    b = cca.forward(t, t["x"], ws).clone()
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+    cca.close()
+
+
+def test_bad_arguments_are_rejected_not_run():
+    from paper_2510_04476_b200.binding import CcaError
+    sh = synth.CONFIGS["cfg1_tiny"]
+    t = to_device(synth.make_inputs(sh))
+    cca = _cca(sh)
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(CcaError, match="workspace too small"):
+        cca.forward(t, t["x"], small)
+    ws = cca.alloc_workspace(sh.B, sh.S, True)
+    bad = dict(t)
+    bad["w_qk"] = None
+    with pytest.raises(CcaError, match="invalid argument"):
+        cca.forward(bad, t["x"], ws)
+    cca.close()
