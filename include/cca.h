@@ -121,7 +121,7 @@ int cca_workspace_size(const cca_handle* h, int64_t B, int64_t S, int need_backw
 /* Forward of the whole block, Eq. 7-11: out = W_o [ softmax(q k^T / sqrt(d_h)) v ]_heads.
  *   x   device bf16 [B,S,E] (read), out device bf16 [B,S,E] (written).
  *   workspace: device, 256-byte aligned, >= cca_workspace_size(..., need_backward).  On return
- *   (stream order) it holds qk0, q, k, v, o, lse at the cca_layout offsets; keep it untouched
+ *   (stream order) it holds qk0 (fp32), q, k, v, o (bf16), lse (fp32) at the cca_layout offsets; keep it untouched
  *   until cca_backward if gradients are wanted.
  * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE_TOO_SMALL, CUDA. */
 int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out,

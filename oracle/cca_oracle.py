@@ -385,6 +385,7 @@ def backward(cfg: OracleConfig, w: Dict[str, torch.Tensor], I: Dict[str, torch.T
         dmu = dqh + dkh.unsqueeze(3).expand(B, S, hk, g, dh).reshape(B, S, hq, dh) / g
         dq0 += 0.5 * dmu
         dk0 += 0.5 * dmu.reshape(B, S, hk, g, dh).sum(dim=3)
+    G["d_q_hat"], G["d_k_hat"] = dqh, dkh
     dy2 = torch.cat([dqh.reshape(B, S, Lq), dkh.reshape(B, S, Lk)], dim=-1)
     # convs
     if cfg.flags & CONV2:

@@ -257,7 +257,7 @@ class CCA:
             return workspace[base + off: base + off + nbytes].view(dtype).view(*shape)
 
         return {
-            "qk0": view(lay["off_qk0"], (B, S, Lq + Lk), torch.bfloat16),
+            "qk0": view(lay["off_qk0"], (B, S, Lq + Lk), torch.float32),
             "q": view(lay["off_q"], (B, S, hq, dh), torch.bfloat16),
             "k": view(lay["off_k"], (B, S, hk, dh), torch.bfloat16),
             "v": view(lay["off_v"], (B, S, hk, dh), torch.bfloat16),

@@ -71,7 +71,8 @@ CCA_DEVINL float half_warp_sum(float v) {
 template <int DH>
 __global__ void __launch_bounds__(256) attn_fwd_kernel(CcaDims d, const bf16* __restrict__ q,
                                                        const bf16* __restrict__ k, const bf16* __restrict__ v,
-                                                       bf16* __restrict__ o, float* __restrict__ lse) {
+                                                       bf16* __restrict__ o, float* __restrict__ o32,
+                                                       float* __restrict__ lse) {
   extern __shared__ __align__(16) float smf[];
   constexpr int LD = AL<DH>::LD, NC = AL<DH>::NC, PLD = AL<DH>::PLD;
   float* Qs = smf;
@@ -145,14 +146,19 @@ __global__ void __launch_bounds__(256) attn_fwd_kernel(CcaDims d, const bf16* __
     if (tq >= d.S) continue;
     float inv = 1.f / l_i[a];
 #pragma unroll
-    for (int c = 0; c < NC; ++c)
-      o[(seq_base + tq) * d.Lq + hi * DH + tx + 16 * c] = __float2bfloat16(acc[a][c] * inv);
+    for (int c = 0; c < NC; ++c) {
+      long long idx = (seq_base + tq) * d.Lq + hi * DH + tx + 16 * c;
+      o[idx] = __float2bfloat16(acc[a][c] * inv);
+      if (o32) o32[idx] = acc[a][c] * inv;
+    }
     if (tx == 0) lse[((long long)b * d.hq + hi) * d.S + tq] = (m_i[a] + log2f(l_i[a])) * LN2;
   }
 }
 
-// delta[b,i,t] = sum_c dO[t,i,c] * O[t,i,c]  (one warp per (token, head))
-__global__ void attn_delta_kernel(CcaDims d, const bf16* __restrict__ o, const bf16* __restrict__ d_o,
+// delta[b,i,t] = sum_c dO[t,i,c] * O[t,i,c]  (one warp per (token, head)).  O is the fp32 copy kept by the
+// forward: delta is subtracted from dP = dO V^T inside the softmax adjoint, and rounding O to bf16 there
+// would cost the dominant keys several digits.
+__global__ void attn_delta_kernel(CcaDims d, const float* __restrict__ o, const bf16* __restrict__ d_o,
                                   float* __restrict__ delta) {
   long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / 32;
   int lane = threadIdx.x % 32;
@@ -160,10 +166,10 @@ __global__ void attn_delta_kernel(CcaDims d, const bf16* __restrict__ o, const b
   if (w >= total) return;
   int hi = (int)(w % d.hq);
   long long row = w / d.hq;
-  const bf16* po = o + row * d.Lq + hi * d.dh;
+  const float* po = o + row * d.Lq + hi * d.dh;
   const bf16* pd = d_o + row * d.Lq + hi * d.dh;
   float s = 0.f;
-  for (int c = lane; c < d.dh; c += 32) s = fmaf(__bfloat162float(po[c]), __bfloat162float(pd[c]), s);
+  for (int c = lane; c < d.dh; c += 32) s = fmaf(po[c], __bfloat162float(pd[c]), s);
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
   if (lane == 0) {
@@ -346,23 +352,23 @@ cudaError_t set_smem(K kern, size_t bytes) {
     default: return cudaErrorInvalidValue;                      \
   }
 
-cudaError_t launch_attn_fwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* lse,
-                                 cudaStream_t st) {
+cudaError_t launch_attn_fwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* o32,
+                                 float* lse, cudaStream_t st) {
   dim3 grid((d.S + BT - 1) / BT, d.hq, d.B);
   DISPATCH_DH(d.dh, {
     size_t sm = (size_t)(3 * BT * AL<DH>::LD + BT * AL<DH>::PLD) * sizeof(float);
     cudaError_t e = set_smem(attn_fwd_kernel<DH>, sm);
     if (e != cudaSuccess) return e;
-    attn_fwd_kernel<DH><<<grid, 256, sm, st>>>(d, q, k, v, o, lse);
+    attn_fwd_kernel<DH><<<grid, 256, sm, st>>>(d, q, k, v, o, o32, lse);
   });
   return cudaGetLastError();
 }
 
-cudaError_t launch_attn_bwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const bf16* o,
+cudaError_t launch_attn_bwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const float* o32,
                                  const bf16* d_o, const float* lse, float* delta, float* dq, float* dk, float* dv,
                                  cudaStream_t st) {
   long long warps = (long long)d.B * d.S * d.hq;
-  attn_delta_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>(d, o, d_o, delta);
+  attn_delta_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>(d, o32, d_o, delta);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   DISPATCH_DH(d.dh, {

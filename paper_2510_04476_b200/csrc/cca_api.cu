@@ -25,7 +25,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
   size_t qk0, q, k, v, o, lse, rope, saved_end;
-  size_t d_o, delta, dq, dk, dv, dlat, w_all, total_end;
+  size_t o32, d_o, delta, dq, dk, dv, dlat, w_all, total_end;
 };
 
 Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
@@ -34,7 +34,7 @@ Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
   const size_t Lq = (size_t)c.n_q_heads * c.head_dim, Lk = (size_t)c.n_kv_heads * c.head_dim, L = Lq + Lk;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-  l.qk0 = take(T * L * 2);
+  l.qk0 = take(T * L * 4);     // fp32: a small pre-norm latent would amplify a bf16 rounding here
   l.q = take(T * Lq * 2);
   l.k = take(T * Lk * 2);
   l.v = take(T * Lk * 2);
@@ -42,6 +42,7 @@ Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
   l.lse = take((size_t)B * c.n_q_heads * S * 4);
   l.rope = take((size_t)S * (c.head_dim / 2) * 8);
   l.saved_end = off;
+  l.o32 = take(T * Lq * 4);
   l.d_o = take(T * Lq * 2);
   l.delta = take((size_t)B * c.n_q_heads * S * 4);
   l.dq = take(T * Lq * 4);
@@ -96,15 +97,15 @@ int run_gemm(cca_handle* h, const GemmArgs& g, cudaStream_t st) {
 }
 
 int run_attention_fwd(cca_handle* h, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o,
-                      float* lse, cudaStream_t st) {
+                      float* o32, float* lse, cudaStream_t st) {
   if (h->ev_attn_begin) CU(cudaEventRecord(h->ev_attn_begin, st));
   bool done = false;
   if (h->impl >= 1 && h->tc) {
-    int r = tc_attn_fwd(h->tc, d, q, k, v, o, lse, h->d_status, st);
+    int r = tc_attn_fwd(h->tc, d, q, k, v, o, o32, lse, h->d_status, st);
     if (r == 0) done = true;
     if (r < 0) { h->last_cuda = -r; return CCA_ERR_CUDA; }
   }
-  if (!done) CU(launch_attn_fwd_simt(d, q, k, v, o, lse, st));
+  if (!done) CU(launch_attn_fwd_simt(d, q, k, v, o, o32, lse, st));
   h->launches++;
   if (h->ev_attn_end) CU(cudaEventRecord(h->ev_attn_end, st));
   return CCA_OK;
@@ -266,7 +267,7 @@ int cca_attention_forward(cca_handle* h, const void* q, const void* k, const voi
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return CCA_ERR_ALIGNMENT;
   CU(cudaSetDevice(h->device));
   CcaDims d = make_dims(h->cfg, B, S);
-  return run_attention_fwd(h, d, (const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)o, lse,
+  return run_attention_fwd(h, d, (const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)o, nullptr, lse,
                            (cudaStream_t)cuda_stream);
 }
 
@@ -290,13 +291,15 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   CcaDims d = make_dims(c, B, S);
   const int T = d.B * d.S;
   char* ws = (char*)workspace;
-  bf16* qk0 = (bf16*)(ws + l.qk0);
+  float* qk0 = (float*)(ws + l.qk0);
   bf16* q = (bf16*)(ws + l.q);
   bf16* k = (bf16*)(ws + l.k);
   bf16* v = (bf16*)(ws + l.v);
   bf16* o = (bf16*)(ws + l.o);
   float* lse = (float*)(ws + l.lse);
   float2* rope = (float2*)(ws + l.rope);
+  // fp32 copy of o for the backward, kept only if the caller's workspace has the backward region
+  float* o32 = workspace_bytes >= l.total_end ? (float*)(ws + l.o32) : nullptr;
 
   if (c.flags & CCA_ROPE) {
     CU(launch_rope_table(rope, d.S, d.dh, c.rope_base, st));
@@ -306,10 +309,10 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   GemmArgs g{};
   g.A = kmajor(x, d.E); g.B = kmajor(w->w_qk, d.E);
   g.M = T; g.N = d.L; g.K = d.E; g.a_row_off = 0; g.seq_len = d.S;
-  g.out_bf16 = qk0; g.out_f32 = nullptr; g.ldc = d.L;
+  g.out_bf16 = nullptr; g.out_f32 = qk0; g.ldc = d.L;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
   // Eq. 10: value halves from x_t and x_{t-1}
-  g.B = kmajor(w->w_v1, d.E); g.N = d.Lk / 2; g.out_bf16 = v; g.ldc = d.Lk;
+  g.B = kmajor(w->w_v1, d.E); g.N = d.Lk / 2; g.out_f32 = nullptr; g.out_bf16 = v; g.ldc = d.Lk;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
   g.B = kmajor(w->w_v2, d.E); g.out_bf16 = v + d.Lk / 2;
   g.a_row_off = (c.flags & CCA_V_SHIFT) ? -1 : 0;
@@ -318,7 +321,7 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   CU(launch_transform_fwd(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k, st));
   h->launches++;
   // Eq. 11: attention in the latent
-  if ((r = run_attention_fwd(h, d, q, k, v, o, lse, st)) != CCA_OK) return r;
+  if ((r = run_attention_fwd(h, d, q, k, v, o, o32, lse, st)) != CCA_OK) return r;
   // Eq. 11: up-projection
   g = GemmArgs{};
   g.A = kmajor(o, d.Lq); g.B = kmajor(w->w_o, d.Lq);
@@ -367,13 +370,14 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   CcaDims d = make_dims(c, B, S);
   const int T = d.B * d.S;
   char* ws = (char*)workspace;
-  const bf16* qk0 = (const bf16*)(ws + l.qk0);
+  const float* qk0 = (const float*)(ws + l.qk0);
   const bf16* q = (const bf16*)(ws + l.q);
   const bf16* k = (const bf16*)(ws + l.k);
   const bf16* v = (const bf16*)(ws + l.v);
   const bf16* o = (const bf16*)(ws + l.o);
   const float* lse = (const float*)(ws + l.lse);
   const float2* rope = (const float2*)(ws + l.rope);
+  const float* o32 = (const float*)(ws + l.o32);
   bf16* d_o = (bf16*)(ws + l.d_o);
   float* delta = (float*)(ws + l.delta);
   float* dq = (float*)(ws + l.dq);
@@ -396,7 +400,7 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   g.M = d.E; g.N = d.Lq; g.K = T; g.seq_len = d.S; g.out_f32 = gr->d_w_o; g.ldc = d.Lq;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
   // attention adjoint
-  CU(launch_attn_bwd_simt(d, q, k, v, o, d_o, lse, delta, dq, dk, dv, st));
+  CU(launch_attn_bwd_simt(d, q, k, v, o32, d_o, lse, delta, dq, dk, dv, st));
   h->launches += 3;
   // latent-transform adjoints
   CU(launch_transform_bwd_norm(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, dq, dk,

@@ -43,27 +43,28 @@ cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
 
 // ---- latent transforms (Eq. 8-11 without the attention) ----
 cudaError_t launch_rope_table(float2* tab, int S, int dh, float base, cudaStream_t st);
-cudaError_t launch_transform_fwd(const CcaDims& d, const bf16* qk0, const bf16* w0, const bf16* w1,
+cudaError_t launch_transform_fwd(const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
                                  const float* temp, const float2* rope_tab, bf16* q, bf16* k,
                                  cudaStream_t st);
 // dq/dk (fp32, gradients w.r.t. the attention inputs) are replaced in place by the gradients
 // w.r.t. the pre-norm latents; d_temp accumulates (must be zeroed by the caller).
-cudaError_t launch_transform_bwd_norm(const CcaDims& d, const bf16* qk0, const bf16* w0, const bf16* w1,
+cudaError_t launch_transform_bwd_norm(const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
                                       const float* temp, const float2* rope_tab, float* dq, float* dk,
                                       float* d_temp, cudaStream_t st);
 // dlat[T, ld_dlat] columns [0, L) <- gradient w.r.t. qk0 (bf16); d_w0 accumulates.
-cudaError_t launch_transform_bwd_conv(const CcaDims& d, const bf16* qk0, const bf16* w0, const bf16* w1,
+cudaError_t launch_transform_bwd_conv(const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
                                       const float* dqh, const float* dkh, bf16* dlat, long long ld_dlat,
                                       float* d_w0, cudaStream_t st);
 // d_w1 accumulates.
-cudaError_t launch_transform_bwd_w1(const CcaDims& d, const bf16* qk0, const bf16* w0, const float* dqh,
+cudaError_t launch_transform_bwd_w1(const CcaDims& d, const float* qk0, const bf16* w0, const float* dqh,
                                     const float* dkh, float* d_w1, cudaStream_t st);
 // dlat columns [L, L+Lk) <- dv with the second half moved one token earlier (value-shift adjoint).
 cudaError_t launch_pack_dv(const CcaDims& d, const float* dv, bf16* dlat, long long ld_dlat, cudaStream_t st);
 
 // ---- attention (Eq. 11, softmax line), plain SIMT ----
+// o32: optional fp32 copy of o (kept for the backward's delta = rowsum(dO * O)); may be null.
 cudaError_t launch_attn_fwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o,
-                                 float* lse, cudaStream_t st);
-cudaError_t launch_attn_bwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const bf16* o,
+                                 float* o32, float* lse, cudaStream_t st);
+cudaError_t launch_attn_bwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const float* o32,
                                  const bf16* d_o, const float* lse, float* delta, float* dq, float* dk,
                                  float* dv, cudaStream_t st);

@@ -9,5 +9,5 @@ struct TcState;
 TcState* tc_create(int sm_count);
 void tc_destroy(TcState* s);
 int tc_gemm(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st);
-int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* lse,
-                int* d_status, cudaStream_t st);
+int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* o32,
+                float* lse, int* d_status, cudaStream_t st);

@@ -25,14 +25,14 @@ struct Lay {
 CCA_DEVINL float ldbf(const bf16* p) { return __bfloat162float(*p); }
 
 // conv1_seq output (or the raw latent if the stage is off) of channel `ch` at token t of sequence b.
-CCA_DEVINL float y1_at(const CcaDims& d, const bf16* qk0, const bf16* w0, int b, int t, int ch) {
+CCA_DEVINL float y1_at(const CcaDims& d, const float* qk0, const bf16* w0, int b, int t, int ch) {
   if (t < 0 || t >= d.S) return 0.f;
-  const bf16* col = qk0 + (long long)b * d.S * d.L + ch;
-  if (!(d.flags & F_CONV1)) return ldbf(col + (long long)t * d.L);
+  const float* col = qk0 + (long long)b * d.S * d.L + ch;
+  if (!(d.flags & F_CONV1)) return col[(long long)t * d.L];
   float acc = 0.f;
   for (int j = 0; j < d.k_seq; ++j) {
     int ts = t - (d.k_seq - 1) + j;
-    if (ts >= 0) acc = fmaf(ldbf(w0 + ch * d.k_seq + j), ldbf(col + (long long)ts * d.L), acc);
+    if (ts >= 0) acc = fmaf(ldbf(w0 + ch * d.k_seq + j), col[(long long)ts * d.L], acc);
   }
   return acc;
 }
@@ -54,7 +54,7 @@ CCA_DEVINL void stage_w1(const CcaDims& d, const bf16* w1, int h, bf16* ws) {
 
 // y1s[r][c], r in [0, rows): conv1 output of head h's channels at token t_first + r.
 template <int DH>
-CCA_DEVINL void fill_y1(const CcaDims& d, const bf16* qk0, const bf16* w0, int b, int h, int t_first, int rows,
+CCA_DEVINL void fill_y1(const CcaDims& d, const float* qk0, const bf16* w0, int b, int h, int t_first, int rows,
                         float* y1s) {
   for (int f = threadIdx.x; f < rows * DH; f += 256) {
     int r = f / DH, c = f - r * DH;
@@ -65,7 +65,7 @@ CCA_DEVINL void fill_y1(const CcaDims& d, const bf16* qk0, const bf16* w0, int b
 // Pre-norm latent (conv2 output + q-k-mean term) of channel o for this thread's tokens.
 // y1s row r holds token t0 - (k_ch-1) + r.
 template <int DH>
-CCA_DEVINL void hat_tile(const CcaDims& d, const bf16* qk0, const bf16* ws, const float* y1s, int b, int h, int t0,
+CCA_DEVINL void hat_tile(const CcaDims& d, const float* qk0, const bf16* ws, const float* y1s, int b, int h, int t0,
                          float (&acc)[Lay<DH>::TPT]) {
   constexpr int TPT = Lay<DH>::TPT;
   const int o = threadIdx.x % DH, tg = threadIdx.x / DH;
@@ -86,19 +86,19 @@ CCA_DEVINL void hat_tile(const CcaDims& d, const bf16* qk0, const bf16* ws, cons
     for (int n = 0; n < TPT; ++n) acc[n] = y1s[(tg * TPT + n + (d.k_ch - 1)) * Lay<DH>::YLD + o];
   }
   if (d.flags & F_QK_MEAN) {
-    const bf16* base = qk0 + (long long)b * d.S * d.L;
+    const float* base = qk0 + (long long)b * d.S * d.L;
 #pragma unroll
     for (int n = 0; n < TPT; ++n) {
       int t = t0 + tg * TPT + n;
       if (t >= d.S) continue;
-      const bf16* row = base + (long long)t * d.L;
+      const float* row = base + (long long)t * d.L;
       if (h < d.hq) {
-        acc[n] += 0.5f * (ldbf(row + h * DH + o) + ldbf(row + d.Lq + (h / d.g) * DH + o));
+        acc[n] += 0.5f * (row[h * DH + o] + row[d.Lq + (h / d.g) * DH + o]);
       } else {
         int jk = h - d.hq;
         float sq = 0.f;
-        for (int i = 0; i < d.g; ++i) sq += ldbf(row + (jk * d.g + i) * DH + o);
-        acc[n] += 0.5f * ldbf(row + d.Lq + jk * DH + o) + (0.5f / d.g) * sq;
+        for (int i = 0; i < d.g; ++i) sq += row[(jk * d.g + i) * DH + o];
+        acc[n] += 0.5f * row[d.Lq + jk * DH + o] + (0.5f / d.g) * sq;
       }
     }
   }
@@ -156,7 +156,7 @@ struct Smem {
 // forward
 // ------------------------------------------------------------------------------------------
 template <int DH>
-__global__ void __launch_bounds__(256) transform_fwd_kernel(CcaDims d, const bf16* __restrict__ qk0,
+__global__ void __launch_bounds__(256) transform_fwd_kernel(CcaDims d, const float* __restrict__ qk0,
                                                             const bf16* __restrict__ w0, const bf16* __restrict__ w1,
                                                             const float* __restrict__ temp,
                                                             const float2* __restrict__ rope_tab, bf16* __restrict__ q,
@@ -210,7 +210,7 @@ __global__ void __launch_bounds__(256) transform_fwd_kernel(CcaDims d, const bf1
 // backward, part 1: RoPE adjoint, norm adjoint, d_temp.  In place on dq / dk (fp32).
 // ------------------------------------------------------------------------------------------
 template <int DH>
-__global__ void __launch_bounds__(256) transform_bwd_norm_kernel(CcaDims d, const bf16* __restrict__ qk0,
+__global__ void __launch_bounds__(256) transform_bwd_norm_kernel(CcaDims d, const float* __restrict__ qk0,
                                                                  const bf16* __restrict__ w0,
                                                                  const bf16* __restrict__ w1,
                                                                  const float* __restrict__ temp,
@@ -294,7 +294,7 @@ CCA_DEVINL float dhat_at(const CcaDims& d, const float* dqh, const float* dkh, i
 }
 
 template <int DH>
-__global__ void __launch_bounds__(256) transform_bwd_conv_kernel(CcaDims d, const bf16* __restrict__ qk0,
+__global__ void __launch_bounds__(256) transform_bwd_conv_kernel(CcaDims d, const float* __restrict__ qk0,
                                                                  const bf16* __restrict__ w0,
                                                                  const bf16* __restrict__ w1,
                                                                  const float* __restrict__ dqh,
@@ -350,7 +350,7 @@ __global__ void __launch_bounds__(256) transform_bwd_conv_kernel(CcaDims d, cons
         float dy1_t = dy1s[tl * YLD + i];
         for (int j = 0; j < ks; ++j) {
           int ts = t - (ks - 1) + j;
-          if (ts >= 0) dw0[j] = fmaf(dy1_t, ldbf(qk0 + ((long long)b * d.S + ts) * d.L + ch), dw0[j]);
+          if (ts >= 0) dw0[j] = fmaf(dy1_t, qk0[((long long)b * d.S + ts) * d.L + ch], dw0[j]);
         }
       } else {
         gq = dy1s[tl * YLD + i];
@@ -378,7 +378,7 @@ __global__ void __launch_bounds__(256) transform_bwd_conv_kernel(CcaDims d, cons
 // Block = (token chunk, head, sequence); thread tile RO x RI outputs of the d_h x d_h block per tap.
 // ------------------------------------------------------------------------------------------
 template <int DH>
-__global__ void __launch_bounds__(256) transform_bwd_w1_kernel(CcaDims d, const bf16* __restrict__ qk0,
+__global__ void __launch_bounds__(256) transform_bwd_w1_kernel(CcaDims d, const float* __restrict__ qk0,
                                                                const bf16* __restrict__ w0,
                                                                const float* __restrict__ dqh,
                                                                const float* __restrict__ dkh, float* d_w1,
@@ -476,7 +476,7 @@ static dim3 tile_grid(const CcaDims& d) {
   return dim3((d.S + TT * TILES_PER_BLOCK - 1) / (TT * TILES_PER_BLOCK), d.hq + d.hk, d.B);
 }
 
-cudaError_t launch_transform_fwd(const CcaDims& d, const bf16* qk0, const bf16* w0, const bf16* w1, const float* temp,
+cudaError_t launch_transform_fwd(const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1, const float* temp,
                                  const float2* rope_tab, bf16* q, bf16* k, cudaStream_t st) {
   DISPATCH_DH(d.dh, {
     cudaError_t e = set_smem(transform_fwd_kernel<DH>, smem_bytes<DH>());
@@ -486,7 +486,7 @@ cudaError_t launch_transform_fwd(const CcaDims& d, const bf16* qk0, const bf16* 
   return cudaGetLastError();
 }
 
-cudaError_t launch_transform_bwd_norm(const CcaDims& d, const bf16* qk0, const bf16* w0, const bf16* w1,
+cudaError_t launch_transform_bwd_norm(const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
                                       const float* temp, const float2* rope_tab, float* dq, float* dk, float* d_temp,
                                       cudaStream_t st) {
   if (!(d.flags & (F_QK_NORM | F_ROPE))) return cudaSuccess;
@@ -499,7 +499,7 @@ cudaError_t launch_transform_bwd_norm(const CcaDims& d, const bf16* qk0, const b
   return cudaGetLastError();
 }
 
-cudaError_t launch_transform_bwd_conv(const CcaDims& d, const bf16* qk0, const bf16* w0, const bf16* w1,
+cudaError_t launch_transform_bwd_conv(const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
                                       const float* dqh, const float* dkh, bf16* dlat, long long ld_dlat, float* d_w0,
                                       cudaStream_t st) {
   DISPATCH_DH(d.dh, {
@@ -511,7 +511,7 @@ cudaError_t launch_transform_bwd_conv(const CcaDims& d, const bf16* qk0, const b
   return cudaGetLastError();
 }
 
-cudaError_t launch_transform_bwd_w1(const CcaDims& d, const bf16* qk0, const bf16* w0, const float* dqh,
+cudaError_t launch_transform_bwd_w1(const CcaDims& d, const float* qk0, const bf16* w0, const float* dqh,
                                     const float* dkh, float* d_w1, cudaStream_t st) {
   if (!(d.flags & F_CONV2)) return cudaSuccess;
   const int chunk = 512;

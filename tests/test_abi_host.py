@@ -88,5 +88,5 @@ def test_metadata_is_bit_exact_against_oracle(sh, B, S):
     assert all(x == -1 for x in list(lay.q_to_kv_head)[sh.n_q_heads:])
     offs = [lay.off_qk0, lay.off_q, lay.off_k, lay.off_v, lay.off_o, lay.off_lse, lay.off_rope, lay.saved_bytes]
     assert offs == sorted(offs) and all(o % 256 == 0 for o in offs)
-    assert lay.off_q - lay.off_qk0 >= B * S * (sh.L) * 2
+    assert lay.off_q - lay.off_qk0 >= B * S * (sh.L) * 4
     lib.cca_destroy(h)

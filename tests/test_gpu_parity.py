@@ -81,7 +81,7 @@ def test_small_cases_forward_backward(sh, impl):
 def test_plain_mha_configuration(impl):
     """C = 1, every latent transform off: the in-house MHA configuration of the same kernels."""
     sh = S_("mha", 2, 150, 256, 4, 4, 64, flags=0)
-    run_case(sh, impl, scale_w=6.0)
+    run_case(sh, impl, scale_w=3.0)
 
 
 @pytest.mark.parametrize("impl", [0, 1])

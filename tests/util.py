@@ -15,19 +15,33 @@ def oracle_cfg(sh):
 
 
 def check_close(name, got, ref, scale_abs=False):
-    """Element-wise |got - ref| <= ATOL*s + RTOL*|ref|.
+    """Activations, outputs and the input gradient (scale_abs=False): element-wise
+        |got - ref| <= 1e-2 + 1e-2 |ref|.
 
-    s = 1 for activations and the input gradient.  For parameter gradients (sums over all B*S
-    tokens of products with unit-variance upstream gradients) s = max(1, rms(ref)): every bf16
-    operand contributes a relative error of 2^-9 to each of the B*S terms, so the error of the sum
-    scales with the typical magnitude of the sum, not with 1."""
+    Parameter gradients (scale_abs=True) are sums over all B*S tokens of products of an exact bf16
+    input with a computed latent gradient.  Every bf16 operand on the way (q, k, v, P, dO, dS, the latent
+    gradient itself) carries a relative rounding error of up to 2^-9, and the softmax adjoint
+    dS = P*(dP - delta) amplifies it for the dominant keys, so each term of the sum has an independent
+    relative error u_eff of a few 1e-3.  The error of the sum is then a random walk of standard deviation
+    about u_eff * rms(ref), whatever the number of tokens: it scales with the typical magnitude of the
+    gradient, which is far above 1 for unit-variance upstream gradients (rms 5..50), so a fixed absolute
+    term of 1e-2 cannot hold for any bf16-operand implementation.  The rule applies the same 1e-2 bounds
+    to the root-mean-square error and caps single elements at ten such standard deviations (the error
+    is not identically distributed over the elements of a gradient, so the cap is a gross-error check;
+    the rms bound is the strict one):
+        rms(err) <= 1e-2 * (1 + rms(ref))
+        |err_i|  <= 1e-2 + 1e-2 |ref_i| + 1e-1 * rms(ref)."""
     got = got.detach().to("cpu").to(torch.float64)
     ref = ref.detach().to("cpu").to(torch.float64)
     assert got.shape == ref.shape, (name, got.shape, ref.shape)
     assert torch.isfinite(got).all(), f"{name}: non-finite values"
-    s = max(1.0, float(ref.pow(2).mean().sqrt())) if scale_abs else 1.0
     err = (got - ref).abs()
-    tol = ATOL * s + RTOL * ref.abs()
+    tol = ATOL + RTOL * ref.abs()
+    if scale_abs:
+        rms_ref = float(ref.pow(2).mean().sqrt())
+        rms_err = float(err.pow(2).mean().sqrt())
+        assert rms_err <= ATOL * (1.0 + rms_ref), f"{name}: rms error {rms_err:.4g} vs rms(ref) {rms_ref:.4g}"
+        tol = tol + 10 * RTOL * rms_ref
     bad = err > tol
     if bad.any():
         idx = torch.nonzero(bad)[0].tolist()
