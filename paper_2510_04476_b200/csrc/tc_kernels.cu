@@ -14,6 +14,7 @@
 #include <new>
 
 #include "tc_ptx.cuh"
+#include "tc_state.cuh"
 
 using namespace tc;
 
@@ -222,26 +223,28 @@ done:
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 }  // namespace
 
-struct TcState {
-  int sm_count;
-  EncodeTiledFn encode;
-  bool attr_set_128, attr_set_256;
-};
-
 // 2-D bf16 tensor map: dim0 (contiguous) extent d0, dim1 extent d1 with row pitch ld elements.
-static bool make_map_2d(TcState* s, CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t ld,
-                        uint32_t box0, uint32_t box1) {
+bool tc_make_map_2d(TcState* s, CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t ld,
+                    uint32_t box0, uint32_t box1) {
   cuuint64_t dims[2] = {d0, d1};
   cuuint64_t strides[1] = {ld * 2};
   cuuint32_t box[2] = {box0, box1};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = s->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+bool tc_make_map_3d(TcState* s, CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
+                    uint64_t ld1, uint64_t ld2, uint32_t box0, uint32_t box1) {
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {ld1 * 2, ld2 * 2};
+  cuuint32_t box[3] = {box0, box1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = s->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -253,6 +256,7 @@ TcState* tc_create(int sm_count) {
   s->sm_count = sm_count;
   s->encode = nullptr;
   s->attr_set_128 = s->attr_set_256 = false;
+  s->attn_attr_set[0] = s->attn_attr_set[1] = false;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -279,11 +283,11 @@ int tc_gemm(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) {
   const int BN = (g.N > 128) ? 256 : 128;
   CUtensorMap tmA, tmB;
   bool ok;
-  if (!a_mn) ok = make_map_2d(s, &tmA, g.A.p, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)lda, GEMM_BK, GEMM_BM);
-  else ok = make_map_2d(s, &tmA, g.A.p, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)lda, 64, GEMM_BK);
+  if (!a_mn) ok = tc_make_map_2d(s, &tmA, g.A.p, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)lda, GEMM_BK, GEMM_BM);
+  else ok = tc_make_map_2d(s, &tmA, g.A.p, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)lda, 64, GEMM_BK);
   if (!ok) return 1;
-  if (!b_mn) ok = make_map_2d(s, &tmB, g.B.p, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)ldb, GEMM_BK, BN);
-  else ok = make_map_2d(s, &tmB, g.B.p, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)ldb, 64, GEMM_BK);
+  if (!b_mn) ok = tc_make_map_2d(s, &tmB, g.B.p, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)ldb, GEMM_BK, BN);
+  else ok = tc_make_map_2d(s, &tmB, g.B.p, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)ldb, 64, GEMM_BK);
   if (!ok) return 1;
   TcGemmParams p;
   p.M = g.M; p.N = g.N; p.K = g.K;
@@ -319,7 +323,3 @@ int tc_gemm(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) {
   return e == cudaSuccess ? 0 : -(int)e;
 }
 
-int tc_attn_fwd(TcState*, const CcaDims&, const bf16*, const bf16*, const bf16*, bf16*, float*, float*, int*,
-                cudaStream_t) {
-  return 1;
-}

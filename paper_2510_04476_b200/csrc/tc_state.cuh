@@ -1,0 +1,23 @@
+// State shared by the tensor-core launchers: the driver entry point that encodes TMA tensor maps.
+#pragma once
+#include <cuda.h>
+
+#include "tc_kernels.cuh"
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcState {
+  int sm_count;
+  EncodeTiledFn encode;
+  bool attr_set_128, attr_set_256;
+  bool attn_attr_set[2];
+};
+
+// bf16 tensor maps with 128-byte swizzle.  2-D: dim0 (contiguous) extent d0, dim1 extent d1, row pitch ld
+// elements.  3-D adds an outer dimension d2 with pitch ld2 elements.
+bool tc_make_map_2d(TcState* s, CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t ld,
+                    uint32_t box0, uint32_t box1);
+bool tc_make_map_3d(TcState* s, CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
+                    uint64_t ld1, uint64_t ld2, uint32_t box0, uint32_t box1);
