@@ -318,8 +318,17 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   g.a_row_off = (c.flags & CCA_V_SHIFT) ? -1 : 0;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
   // Eq. 8, 9, 11: convs, q-k-mean, norm, temperature, RoPE
-  CU(launch_transform_fwd(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k, st));
-  h->launches++;
+  {
+    bool done = false;
+    if (h->impl >= 1 && h->tc) {
+      int tr = tc_transform_fwd(h->tc, d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k,
+                                h->d_status, st);
+      if (tr == 0) done = true;
+      if (tr < 0) { h->last_cuda = -tr; return CCA_ERR_CUDA; }
+    }
+    if (!done) CU(launch_transform_fwd(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k, st));
+    h->launches++;
+  }
   // Eq. 11: attention in the latent
   if ((r = run_attention_fwd(h, d, q, k, v, o, o32, lse, st)) != CCA_OK) return r;
   // Eq. 11: up-projection
