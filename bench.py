@@ -108,22 +108,34 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(clocks)}
 
 
-def oracle_sample(sh, n_rows=256):
-    """The oracle, as it stands, on a bounded sample of the workload: projections and latent transforms
-    in full, the S^2 stage and the up-projection on n_rows sampled query positions per sequence."""
+def oracle_sample(sh, n_rows=4096, backward=False):
+    """The oracle, as it stands, on a bounded sample of the workload.  Forward workloads: projections and
+    latent transforms in full, the S^2 stage and the up-projection on n_rows sampled query positions per
+    sequence (every position if n_rows >= S).  Training workloads: the whole forward and backward."""
     from oracle import cca_oracle as O
-    t = synth.make_inputs(sh, want_dout=False)
-    g = torch.Generator().manual_seed(123)
-    rows = sorted(set(int(r) for r in torch.randint(0, sh.S, (n_rows,), generator=g)))
+    t = synth.make_inputs(sh, want_dout=backward)
     cfg = O.OracleConfig(sh.d_model, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.k_seq, sh.k_ch, sh.causal, sh.flags,
                          sh.rope_base)
+    if backward:
+        t0 = time.perf_counter()
+        _, I = O.forward(cfg, t, t["x"])
+        O.backward(cfg, t, I, t["d_out"])
+        dt = time.perf_counter() - t0
+        return flops_of(sh, True)["total"] / dt / 1e12, dt, "whole workload: forward and backward of every sequence"
+    g = torch.Generator().manual_seed(123)
+    if n_rows >= sh.S:
+        rows = list(range(sh.S))
+    else:
+        rows = sorted(set(int(r) for r in torch.randint(0, sh.S, (n_rows,), generator=g)))
     t0 = time.perf_counter()
     O.forward_rows(cfg, t, t["x"], rows)
     dt = time.perf_counter() - t0
     T = sh.B * sh.S
     fl = 2 * T * sh.d_model * (sh.L_q + 2 * sh.L_k) + 2 * T * (sh.L * sh.k_seq + sh.L * sh.head_dim * sh.k_ch)
-    fl += sum(4 * sh.B * (r + 1 if sh.causal else sh.S) * sh.L_q for r in rows) + 2 * sh.B * len(rows) * sh.L_q * sh.d_model
-    return fl / dt / 1e12, dt, f"down-projections and latent transforms in full; attention and up-projection on {len(rows)} sampled query rows per sequence"
+    fl += sum((2 if sh.causal else 4) * sh.B * (2 * (r + 1) if sh.causal else sh.S) * sh.L_q for r in rows)
+    fl += 2 * sh.B * len(rows) * sh.L_q * sh.d_model
+    return fl / dt / 1e12, dt, (f"down-projections and latent transforms in full; attention and up-projection on "
+                                f"{len(rows)} of {sh.S} query rows per sequence")
 
 
 def run_reference(args, rank, world):
@@ -136,7 +148,7 @@ def run_reference(args, rank, world):
     t_all = time.perf_counter()
     sample = ""
     for _ in range(max(1, args.steps)):
-        v, dt, sample = oracle_sample(sh, n_rows=128)
+        v, dt, sample = oracle_sample(sh, n_rows=512, backward=False)
         vals.append((v, dt))
         if time.perf_counter() - t_all > 150:
             break
@@ -172,7 +184,7 @@ def run_ours(args, rank, world, local_rank):
     cca = CCA.from_shape(sh, device=local_rank)
     cca.set_impl(args.kernels)
     act_bytes = sh.B * sh.S * sh.d_model * 2
-    ws = cca.alloc_workspace(sh.B, sh.S, True, extra=2 * act_bytes + 1024)
+    ws = cca.alloc_workspace(sh.B, sh.S, backward, extra=2 * act_bytes + 1024)
     out = torch.empty_like(dev["x"])
 
     def step():
@@ -283,7 +295,7 @@ def run_ours(args, rank, world, local_rank):
     if rank == 0 and world == 1 and not args.no_mha and not backward:
         line["mha_same_shape"] = mha_compare(sh, args, ms_step, attn_ms, local_rank)
     if rank == 0 and world == 1 and not args.no_cpu:
-        v, dt, sample = oracle_sample(sh)
+        v, dt, sample = oracle_sample(sh, backward=backward)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                                 "sample": sample, "seconds": dt}
     if rank == 0:

@@ -137,7 +137,8 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
 
 /* Same block, host buffers: copies x (host, ideally pinned) to a staging area inside the
  * workspace, runs cca_forward, copies out back to `out_host`, and synchronises the stream.
- * workspace must be >= cca_workspace_size(...) + 2*B*S*E*2 bytes. */
+ * workspace must be >= cca_workspace_size(h, B, S, 0, ..) + 2 * round_up(B*S*E*2, 256) bytes; nothing is kept
+ * for a backward. */
 int cca_forward_host(cca_handle* h, const cca_weights* w, const void* x_host, void* out_host,
                      void* workspace, size_t workspace_bytes, int64_t B, int64_t S,
                      void* cuda_stream);

@@ -347,13 +347,13 @@ int cca_forward_host(cca_handle* h, const cca_weights* w, const void* x_host, vo
   if (!x_host || !out_host || !workspace) return CCA_ERR_INVALID_ARG;
   Layout l = make_layout(h->cfg, B, S);
   const size_t act = align_up((size_t)B * S * h->cfg.d_model * 2, 256);
-  if (workspace_bytes < l.total_end + 2 * act) return CCA_ERR_WORKSPACE_TOO_SMALL;
+  if (workspace_bytes < l.saved_end + 2 * act) return CCA_ERR_WORKSPACE_TOO_SMALL;
   CU(cudaSetDevice(h->device));
   cudaStream_t st = (cudaStream_t)cuda_stream;
-  char* xs = (char*)workspace + l.total_end;
+  char* xs = (char*)workspace + l.saved_end;
   char* os = xs + act;
   CU(cudaMemcpyAsync(xs, x_host, (size_t)B * S * h->cfg.d_model * 2, cudaMemcpyHostToDevice, st));
-  r = cca_forward(h, w, xs, os, workspace, l.total_end, B, S, cuda_stream);
+  r = cca_forward(h, w, xs, os, workspace, l.saved_end, B, S, cuda_stream);
   if (r != CCA_OK) return r;
   CU(cudaMemcpyAsync(out_host, os, (size_t)B * S * h->cfg.d_model * 2, cudaMemcpyDeviceToHost, st));
   CU(cudaStreamSynchronize(st));
