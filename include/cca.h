@@ -33,7 +33,8 @@ typedef enum {
   CCA_ERR_ALIGNMENT = 3,           /* a device pointer is not 16-byte aligned                */
   CCA_ERR_WORKSPACE_TOO_SMALL = 4,
   CCA_ERR_CUDA = 5,                /* a CUDA call failed; see cca_last_cuda_error            */
-  CCA_ERR_DEVICE_TIMEOUT = 6       /* a bounded device-side wait expired (cca_last_status)   */
+  CCA_ERR_DEVICE_TIMEOUT = 6,      /* a bounded device-side wait expired (cca_last_status)   */
+  CCA_ERR_STATIC_WORKSPACE_EXCEEDED = 7  /* cca_forward_static: B, S need more than the built-in scratch */
 } cca_status;
 
 /* Optional stages (rows of the paper's ablation tables; all on = the method of Eq. 7-11). */
@@ -142,6 +143,32 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
 int cca_forward_host(cca_handle* h, const cca_weights* w, const void* x_host, void* out_host,
                      void* workspace, size_t workspace_bytes, int64_t B, int64_t S,
                      void* cuda_stream);
+
+/* Forward for callers that cannot allocate device memory.  (The paper has no counterpart: this is a
+ * deployment variant of cca_forward, same arithmetic, same kernels.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a serving process whose device memory
+ * was handed in full to another allocator at start-up, a plug-in that is only lent a stream and its
+ * input/output buffers, a latency-critical loop that must not take the device-wide synchronisation an
+ * allocation implies.  Such a caller has nowhere to get the workspace cca_forward asks for.  Here the
+ * workspace is a fixed array of CCA_STATIC_WORKSPACE_BYTES inside the library's device image, so the
+ * caller passes only x, out and the weights.  The function calls no cudaMalloc / cudaFree and no
+ * allocating library routine.
+ *
+ *   - Limit: cca_workspace_size(h, B, S, 0, &n) must give n <= CCA_STATIC_WORKSPACE_BYTES, otherwise
+ *     CCA_ERR_STATIC_WORKSPACE_EXCEEDED is returned and nothing is enqueued.  (32 MiB holds, for
+ *     example, 4096 tokens of an 8 x 64 / 2 x 64 latent, or 2048 tokens of a 16 x 64 / 4 x 64 one.)
+ *   - Cost: every GPU on which the library is loaded holds those bytes until the process exits.
+ *   - The first call on a device looks up the array's device address (once, under a lock, with that
+ *     device current).  Make that first call before any stream capture begins.
+ *   - One array per device, shared by every handle and every call, holding whatever the last call
+ *     left.  The forward overwrites each region before reading it, so nothing is cleared.  Two calls
+ *     whose kernels can overlap on the GPU (different streams without an ordering between them) race
+ *     on it: order them.  No activations are kept for cca_backward.
+ * x, out: device bf16 [B,S,E] as in cca_forward.  Errors: as cca_forward, plus the one above. */
+#define CCA_STATIC_WORKSPACE_BYTES (32u << 20)
+int cca_forward_static(cca_handle* h, const cca_weights* w, const void* x, void* out, int64_t B, int64_t S,
+                       void* cuda_stream);
 
 /* Attention stage alone (Eq. 11, third line) on latents already in the workspace layout:
  * q [B,S,h_q,d_h], k, v [B,S,h_k,d_h] bf16 device -> o bf16 [B,S,h_q,d_h], lse fp32 [B,h_q,S]. */

@@ -57,6 +57,8 @@ SYMBOLS = {
                                C.c_void_p, C.POINTER(cca_weight_grads), C.c_int64, C.c_int64, C.c_void_p]),
     "cca_forward_host": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_size_t, C.c_int64, C.c_int64, C.c_void_p]),
+    "cca_forward_static": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
+                                     C.c_void_p]),
     "cca_attention_forward": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_int64, C.c_int64, C.c_void_p]),
     "cca_set_impl": (C.c_int, [C.c_void_p, C.c_int]),
@@ -210,6 +212,18 @@ class CCA:
         _check(self.lib, self.lib.cca_forward_host(self.handle, C.byref(cw), _ptr(x_host), _ptr(out_host), wp, wn,
                                                    B, S, st), self.handle, "cca_forward_host")
         return out_host
+
+    def forward_static(self, w, x: torch.Tensor, out: torch.Tensor):
+        """cca_forward_static: the forward with the library's built-in scratch; `out` is caller-provided and
+        nothing is allocated on the way (not here either)."""
+        B, S, E = x.shape
+        assert x.is_cuda and x.is_contiguous() and x.dtype == torch.bfloat16
+        assert out.is_cuda and out.is_contiguous() and out.dtype == torch.bfloat16 and out.shape == x.shape
+        cw = self._weights(w)
+        st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+        _check(self.lib, self.lib.cca_forward_static(self.handle, C.byref(cw), _ptr(x), _ptr(out), B, S, st),
+               self.handle, "cca_forward_static")
+        return out
 
     def backward(self, w, x: torch.Tensor, d_out: torch.Tensor, workspace: torch.Tensor):
         """Returns (d_x bf16, dict of fp32 parameter gradients)."""

@@ -1,6 +1,7 @@
 // C ABI of the CCA library: handle, validation, metadata, workspace layout, forward / backward drivers.
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "../../include/cca.h"
@@ -124,6 +125,7 @@ const char* cca_status_string(int s) {
     case CCA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case CCA_ERR_CUDA: return "CUDA error";
     case CCA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case CCA_ERR_STATIC_WORKSPACE_EXCEEDED: return "problem needs more than the built-in static workspace";
     default: return "unknown status";
   }
 }
@@ -438,6 +440,43 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   g.M = T; g.N = d.E; g.K = (int)ldl; g.seq_len = d.S; g.out_bf16 = (bf16*)d_x; g.ldc = d.E;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
   return CCA_OK;
+}
+
+// ---- forward without any caller-provided or allocated workspace ---------------------------------
+// The scratch of cca_forward_static: one array in the library's device image.  Every GPU that loads the
+// library reserves these bytes until the process exits.  In host code `g_static_ws` is only a handle for
+// cudaGetSymbolAddress, never a pointer a kernel may be given.
+static __device__ __align__(256) unsigned char g_static_ws[CCA_STATIC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxStaticDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxStaticDevices];     // device address of g_static_ws on each device, once resolved
+}  // namespace
+
+int cca_forward_static(cca_handle* h, const cca_weights* w, const void* x, void* out, int64_t B, int64_t S,
+                       void* cuda_stream) {
+  int r = check_sizes(h, B, S, true);
+  if (r != CCA_OK) return r;
+  if (h->device >= kMaxStaticDevices) return CCA_ERR_UNSUPPORTED;
+  Layout l = make_layout(h->cfg, B, S);
+  if (l.saved_end > (size_t)CCA_STATIC_WORKSPACE_BYTES) return CCA_ERR_STATIC_WORKSPACE_EXCEEDED;
+  CU(cudaSetDevice(h->device));
+  void* ws = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[h->device]) {
+      // set-up, once per device, with that device current: resolve the array's address on this device
+      void* p = nullptr;
+      CU(cudaGetSymbolAddress(&p, g_static_ws));
+      if (!p || (reinterpret_cast<uintptr_t>(p) & 255)) return CCA_ERR_ALIGNMENT;
+      g_static_ptr[h->device] = p;
+    }
+    ws = g_static_ptr[h->device];
+  }
+  // Every region of the forward workspace is written in full before it is read, so the previous call's
+  // contents need no clearing.  Passing exactly the forward-only size keeps the fp32 copy of o off.
+  return cca_forward(h, w, x, out, ws, l.saved_end, B, S, cuda_stream);
 }
 
 }  // extern "C"
