@@ -98,11 +98,11 @@ int run_gemm(cca_handle* h, const GemmArgs& g, cudaStream_t st) {
 }
 
 int run_attention_fwd(cca_handle* h, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o,
-                      float* o32, float* lse, cudaStream_t st) {
+                      float* o32, float* lse, const float* temp, cudaStream_t st) {
   if (h->ev_attn_begin) CU(cudaEventRecord(h->ev_attn_begin, st));
   bool done = false;
   if (h->impl >= 1 && h->tc) {
-    int r = tc_attn_fwd(h->tc, d, q, k, v, o, o32, lse, h->d_status, st);
+    int r = tc_attn_fwd(h->tc, d, q, k, v, o, o32, lse, temp, h->d_status, st);
     if (r == 0) done = true;
     if (r < 0) { h->last_cuda = -r; return CCA_ERR_CUDA; }
   }
@@ -269,7 +269,8 @@ int cca_attention_forward(cca_handle* h, const void* q, const void* k, const voi
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return CCA_ERR_ALIGNMENT;
   CU(cudaSetDevice(h->device));
   CcaDims d = make_dims(h->cfg, B, S);
-  return run_attention_fwd(h, d, (const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)o, nullptr, lse,
+  // q and k come from the caller: nothing is known about their norms
+  return run_attention_fwd(h, d, (const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)o, nullptr, lse, nullptr,
                            (cudaStream_t)cuda_stream);
 }
 
@@ -332,7 +333,9 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
     h->launches++;
   }
   // Eq. 11: attention in the latent
-  if ((r = run_attention_fwd(h, d, q, k, v, o, o32, lse, st)) != CCA_OK) return r;
+  // with the norm stage on, the logits are bounded by sqrt(d_h) exp(temp): the kernel may use that as the row maximum
+  if ((r = run_attention_fwd(h, d, q, k, v, o, o32, lse, (c.flags & CCA_QK_NORM) ? w->temp : nullptr, st)) != CCA_OK)
+    return r;
   // Eq. 11: up-projection
   g = GemmArgs{};
   g.A = kmajor(o, d.Lq); g.B = kmajor(w->w_o, d.Lq);

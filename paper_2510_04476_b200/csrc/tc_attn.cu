@@ -3,16 +3,23 @@
 // 128-row tiles that ping-pong: while the softmax warps of one tile work on S = Q K^T, the tensor core
 // runs the other tile's MMAs.
 //
-//   warps 0-3  : softmax + epilogue of query tile 0 (thread = query row = TMEM lane)
-//   warps 4-7  : softmax + epilogue of query tile 1
-//   warp  8    : TMA loader (Q tiles once, then a 2-stage ring of K and of V tiles)
-//   warp  9    : TMEM owner and MMA issuer
+//   warps 0-7  : softmax + epilogue of query tile 0: warps 0-3 take score columns 0-63 of a KV tile,
+//                warps 4-7 columns 64-127 (thread = query row = TMEM lane; two threads per row keep four
+//                warps per scheduler busy, which the latency of the per-element chain needs)
+//   warps 8-15 : the same for query tile 1
+//   warp  16   : TMA loader (Q tiles once, then a 2-stage ring of K and of V tiles)
+//   warp  17   : TMEM owner and MMA issuer
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+DH) O1 [384,384+DH).  The bf16 probabilities P
-// overwrite the first 64 columns of their S tile and feed the P V MMA directly from TMEM.
-// Softmax is online with a lazy rescale: the running row maximum only moves (and O is only rescaled)
-// when it grows by more than 2^8; with normalised q, k the logits are bounded by sqrt(d_h) * beta, so
-// after the first tile this never happens.
+// overwrite columns [0,32) and [64,96) of their S tile and feed the P V MMA directly from TMEM.
+// Softmax: with L2-normalised q and k (Eq. 11) every logit is bounded by sqrt(d_h) * beta, so that bound
+// serves as a fixed row maximum: no max pass, no rescale of O (the kernel falls back to the online form,
+// with a lazy rescale when the running maximum grows by more than 2^8, if the latents are not normalised
+// or the bound is too loose for fp32).  One score costs 4 d_h tensor FLOPs and one exponential; at
+// d_h = 128 the tensor pipe and the 16-per-clock transcendental unit would need the same time, so a
+// fixed share of the exponentials is evaluated on the FMA pipe instead (round to integer + cubic for
+// 2^f, |f| <= 1/2, relative error 7.5e-5, well under the bf16 rounding of P), two at a time with the
+// packed f32x2 instructions.
 #include "tc_kernels.cuh"
 #include "tc_ptx.cuh"
 #include "tc_state.cuh"
@@ -21,7 +28,9 @@ using namespace tc;
 
 namespace {
 
-constexpr int AT_THREADS = 320;
+constexpr int AT_SOFTMAX_WARPS = 16;                 // 2 query tiles x 2 column halves x 4 lane quarters
+constexpr int AT_TMA_WARP = AT_SOFTMAX_WARPS, AT_MMA_WARP = AT_SOFTMAX_WARPS + 1;
+constexpr int AT_THREADS = 32 * (AT_SOFTMAX_WARPS + 2);
 constexpr int BQ = 128, BKV = 128, KV_STAGES = 2;
 constexpr float LOG2E_F = 1.4426950408889634f;
 constexpr float LN2_F = 0.6931471805599453f;
@@ -34,6 +43,7 @@ struct AttnParams {
   float* lse;
   int n_blocks;       // 256-row blocks per sequence
   int* status;
+  const float* temp;  // log key temperature per kv head if q, k are L2-normalised (Eq. 11), else null
 };
 
 template <int DH>
@@ -44,7 +54,8 @@ struct AttnSmem {
   static constexpr int V_OFF = K_OFF + KV_STAGES * TILE_BYTES;
   static constexpr int BAR_OFF = V_OFF + KV_STAGES * TILE_BYTES;
   // at least 120 KB so that two CTAs (each wanting all 512 TMEM columns) never share an SM
-  static constexpr int TOTAL = (BAR_OFF + 512 + 1024) > 122880 ? (BAR_OFF + 512 + 1024) : 122880;
+  static constexpr int XCH_OFF = BAR_OFF + 512;              // float [2 tiles][2 halves][128 rows]: max / sum exchange
+  static constexpr int TOTAL = (XCH_OFF + 2048 + 1024) > 122880 ? (XCH_OFF + 2048 + 1024) : 122880;
 };
 
 TC_DEVINL void fail(volatile int* abort_flag, int* status, int code) {
@@ -62,7 +73,81 @@ TC_DEVINL uint64_t kmajor_desc(uint32_t tile_addr, int kk) {
 // kk-th 16-key slice; 64-channel chunks are one box (16384 B) apart.
 TC_DEVINL uint64_t v_desc(uint32_t tile_addr, int kk) { return smem_desc_sw128(tile_addr + kk * 2048, 16384, 1024); }
 
-template <int DH>
+
+// ---- packed fp32 pairs (one 64-bit register = two floats) ----
+TC_DEVINL uint64_t pack2u(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+TC_DEVINL uint64_t pack2f(float lo, float hi) { return pack2u(__float_as_uint(lo), __float_as_uint(hi)); }
+TC_DEVINL void unpack2u(uint64_t v, uint32_t& lo, uint32_t& hi) { asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v)); }
+TC_DEVINL uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+TC_DEVINL uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+TC_DEVINL float ex2f(float x) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+// 2^x for a pair, x in [-120, 8], on the FMA and integer pipes: n = round(x) from the magic-number add,
+// f = x - n in [-1/2, 1/2], 2^f by a cubic (minimax in relative error), then n is added to the exponent.
+TC_DEVINL uint64_t exp2_poly2(uint64_t x) {
+  const uint64_t magic = pack2f(12582912.f, 12582912.f), neg_magic = pack2f(-12582912.f, -12582912.f);
+  const uint64_t neg1 = pack2f(-1.f, -1.f);
+  const uint64_t c3 = pack2f(0.0551716685f, 0.0551716685f), c2 = pack2f(0.242611125f, 0.242611125f);
+  const uint64_t c1 = pack2f(0.693260968f, 0.693260968f), c0 = pack2f(0.999928057f, 0.999928057f);
+  const uint64_t t = add2(x, magic);
+  const uint64_t n = add2(t, neg_magic);
+  const uint64_t f = fma2(n, neg1, x);
+  uint64_t pl = fma2(c3, f, c2);
+  pl = fma2(pl, f, c1);
+  pl = fma2(pl, f, c0);
+  uint32_t t0, t1, p0, p1;
+  unpack2u(t, t0, t1);
+  unpack2u(pl, p0, p1);
+  return pack2u(p0 + (t0 << 23), p1 + (t1 << 23));
+}
+// Exponentials of 8 consecutive scores (already in registers) -> 4 packed bf16 pairs; adds the rounded
+// values to the two running partial sums in `sum2`.  POLY of the 4 pairs go through the
+// polynomial.  CLAMP: x may be far below the smallest exponent (online mode); then it is clamped first.
+template <int POLY, bool CLAMP>
+TC_DEVINL void exp8(const uint32_t* v, uint64_t scale2, uint64_t negm2, uint64_t& sum2, uint32_t* out) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint64_t x = fma2(pack2u(v[2 * i], v[2 * i + 1]), scale2, negm2);
+    uint64_t e;
+    if (i < POLY) {
+      if (CLAMP) {
+        uint32_t a, b;
+        unpack2u(x, a, b);
+        x = pack2f(fmaxf(__uint_as_float(a), -120.f), fmaxf(__uint_as_float(b), -120.f));
+      }
+      e = exp2_poly2(x);
+    } else {
+      uint32_t a, b;
+      unpack2u(x, a, b);
+      e = pack2f(ex2f(__uint_as_float(a)), ex2f(__uint_as_float(b)));
+    }
+    // The row sum is taken over the bf16-rounded probabilities, the values the P V product really uses, so
+    // that the weights of a row sum to one whatever the rounding did (with a fixed maximum even the
+    // largest probability of a row is rounded).
+    uint32_t a, b;
+    unpack2u(e, a, b);
+    const uint32_t w = pack_bf16(__uint_as_float(a), __uint_as_float(b));
+    out[i] = w;
+    sum2 = add2(sum2, pack2u(w << 16, w & 0xffff0000u));
+  }
+}
+
+template <int DH, int POLY>
 __global__ void __launch_bounds__(AT_THREADS, 1)
 tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, AttnParams p) {
@@ -107,7 +192,7 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       mbar_init(&v_full[i], 1);
       mbar_init(&v_empty[i], 1);
       mbar_init(&s_full[i], 1);
-      mbar_init(&p_full[i], 128);
+      mbar_init(&p_full[i], 256);
       mbar_init(&o_done[i], 1);
     }
     *abort_flag = 0;
@@ -116,7 +201,7 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmV);
   }
-  if (warp == 9) {
+  if (warp == AT_MMA_WARP) {
     tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
   }
@@ -125,7 +210,7 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 8) {
+  if (warp == AT_TMA_WARP) {
     // ---------------------------------------------------------------- TMA loader
     if (lane == 0) {
 #pragma unroll
@@ -152,146 +237,205 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           tma_load_3d(smem + SM::V_OFF + st * SM::TILE_BYTES + c * 16384, &tmV, hj * DH + c * 64, j * BKV, b, &v_full[st]);
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == AT_MMA_WARP) {
     // ---------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    // The whole warp runs the loop (so the address arithmetic stays warp-uniform and cheap); one elected lane
+    // issues the MMAs and the commits.
+    {
+      const bool leader = elect_one();
       const uint32_t idesc_s = idesc_bf16(BKV, 0, 0);
       const uint32_t idesc_o = idesc_bf16(DH, 0, 1);
-      const uint32_t q_addr = smem_u32(smem + SM::Q_OFF), k_addr = smem_u32(smem + SM::K_OFF),
-                     v_addr = smem_u32(smem + SM::V_OFF);
+      // descriptor words: low = address >> 4 | leading offset << 16, high = stride offset, version, swizzle
+      const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
+      const uint32_t q_lo = (smem_u32(smem + SM::Q_OFF) >> 4) | (1u << 16);
+      const uint32_t k_lo = (smem_u32(smem + SM::K_OFF) >> 4) | (1u << 16);
+      const uint32_t v_lo = (smem_u32(smem + SM::V_OFF) >> 4) | ((16384u >> 4) << 16);   // 64-channel chunks 16 KB apart
+      constexpr uint32_t TILE16 = SM::TILE_BYTES >> 4;
+      auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+      };
       auto issue_s = [&](int s, int j) {      // S_s = Q_s K_j^T
-        const uint32_t qa = q_addr + s * SM::TILE_BYTES, ka = k_addr + (j & 1) * SM::TILE_BYTES;
+        const uint32_t qa = q_lo + s * TILE16, ka = k_lo + (j & 1) * TILE16;
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < DH / 16; ++kk)
-          mma_ss(tmem_base + s * 128, kmajor_desc<DH>(qa, kk), kmajor_desc<DH>(ka, kk), idesc_s, kk != 0);
+          for (int kk = 0; kk < DH / 16; ++kk) {
+            const uint32_t off = (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+            mma_ss_w(tmem_base + s * 128, qa + off, desc_hi, ka + off, desc_hi, idesc_s, kk != 0);
+          }
+        }
       };
       auto issue_pv = [&](int s, int j) {     // O_s (+)= P_s V_j
-        const uint32_t va = v_addr + (j & 1) * SM::TILE_BYTES;
+        const uint32_t va = v_lo + (j & 1) * TILE16;
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < BKV / 16; ++kk)
-          mma_ts(tmem_base + 256 + s * 128, tmem_base + s * 128 + kk * 8, v_desc(va, kk), idesc_o, (j | kk) != 0);
+          for (int kk = 0; kk < BKV / 16; ++kk)
+            mma_ts_w(tmem_base + 256 + s * 128, tmem_base + s * 128 + (kk >> 2) * 64 + (kk & 3) * 8, va + kk * (2048 >> 4),
+                     desc_hi, idesc_o, (j | kk) != 0);
+        }
+      };
+      auto commit = [&](uint64_t* bar) {
+        if (leader) mma_commit(bar);
       };
       // prologue: first S tile of each query tile
       if (n_max > 0) {
-        if (!mbar_wait(&k_full[0], 0, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+        if (!wait_all(&k_full[0], 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
         tc_fence_after();
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
           if (n_s[s] == 0) continue;
-          if (!mbar_wait(&q_full[s], 0, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+          if (!wait_all(&q_full[s], 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
           tc_fence_after();
           issue_s(s, 0);
-          mma_commit(&s_full[s]);
+          commit(&s_full[s]);
         }
       }
       for (int j = 0; j < n_max; ++j) {
         const int st = j & 1;
         const uint32_t ph = (j >> 1) & 1;
         // all S(j) were issued before this point: release K_j when they complete
-        mma_commit(&k_empty[st]);
+        commit(&k_empty[st]);
         bool k_next_ready = false;
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
           if (j >= n_s[s]) continue;
-          if (!mbar_wait(&p_full[s], j & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
-          if (!mbar_wait(&v_full[st], ph, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+          if (!wait_all(&p_full[s], j & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+          if (!wait_all(&v_full[st], ph)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
           tc_fence_after();
           issue_pv(s, j);
           if (j + 1 < n_s[s]) {
             if (!k_next_ready) {
-              if (!mbar_wait(&k_full[(j + 1) & 1], ((j + 1) >> 1) & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+              if (!wait_all(&k_full[(j + 1) & 1], ((j + 1) >> 1) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
               tc_fence_after();
               k_next_ready = true;
             }
             issue_s(s, j + 1);
-            mma_commit(&s_full[s]);
+            commit(&s_full[s]);
           } else {
-            mma_commit(&o_done[s]);
+            commit(&o_done[s]);
           }
         }
-        mma_commit(&v_empty[st]);
+        commit(&v_empty[st]);
       }
     }
   } else {
     // ---------------------------------------------------------------- softmax + epilogue
-    const int s = warp >> 2;                         // query tile of this warpgroup
+    const int s = warp >> 3;                         // query tile of this warp
+    const int part = (warp >> 2) & 1;                // which 64 score columns of each KV tile
     const int row = threadIdx.x & 127;
     const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t s_tmem = tmem_base + lane_sel + s * 128;
+    const uint32_t s_tmem = tmem_base + lane_sel + s * 128;          // S tile; P goes to its first 64 columns
     const uint32_t o_tmem = tmem_base + lane_sel + 256 + s * 128;
+    float* xch = reinterpret_cast<float*>(smem + SM::XCH_OFF) + s * 256;   // [2 halves][128 rows]
+    const int bar_id = 1 + s;                        // named barrier of the 256 threads of this tile
     const int m0 = blk * 256 + s * BQ;
     const int tq = m0 + row;
     const float c_scale = rsqrtf((float)DH) * LOG2E_F;
-    float m_run = -INFINITY, l_run = 0.f;
+    // Fixed maximum: |q| = sqrt(d_h), |k| = sqrt(d_h) beta, so the scaled logit (log2 units) is at most
+    // sqrt(d_h) beta log2(e); 1 % covers the bf16 rounding of q and k.  Used while 2^(-2 bound) is a normal
+    // fp32 number with room to spare.
+    float m_fixed = 0.f;
+    bool fixed = false;
+    if (p.temp != nullptr) {
+      m_fixed = sqrtf((float)DH) * __expf(p.temp[hj]) * LOG2E_F * 1.01f;
+      fixed = m_fixed <= 56.f;
+    }
+    const uint64_t scale2 = pack2f(c_scale, c_scale);
+    float m_run = fixed ? m_fixed : -INFINITY, l_run = 0.f;
     for (int j = 0; j < n_s[s]; ++j) {
       if (!mbar_wait(&s_full[s], j & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
       tc_fence_after();
-      uint32_t v[128];
-      tmem_ld32(s_tmem + 0, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-      tmem_ld32(s_tmem + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
-      tmem_ld32(s_tmem + 64, *reinterpret_cast<uint32_t(*)[32]>(&v[64]));
-      tmem_ld32(s_tmem + 96, *reinterpret_cast<uint32_t(*)[32]>(&v[96]));
-      tmem_ld_wait();
-      const int k0 = j * BKV;
-      const bool need_mask = (p.causal && k0 + BKV - 1 > m0) || (k0 + BKV > p.S);
-      if (need_mask) {
-        const int lim = p.causal ? min(tq, p.S - 1) : p.S - 1;     // last visible key
-#pragma unroll
-        for (int c = 0; c < 128; ++c)
-          if (k0 + c > lim) v[c] = 0xff800000u;                    // -inf
-      }
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(v[c]));
-      mx *= c_scale;
+      const int k0 = j * BKV + part * 64;            // first key of this thread's columns
+      const bool need_mask = (p.causal && j * BKV + BKV - 1 > m0) || (j * BKV + BKV > p.S);
+      const int lim = p.causal ? min(tq, p.S - 1) : p.S - 1;       // last visible key
       float m_use = m_run;
-      const bool grow = mx > m_run + RESCALE_THRESHOLD;           // also true on the first tile
-      if (grow) m_use = mx;
-      if (m_use == -INFINITY) m_use = 0.f;
-      if (j > 0 && __any_sync(0xffffffffu, grow)) {
-        // rescale the running output of this warp's 32 rows (rare)
-        const float alpha = grow ? exp2f(m_run - m_use) : 1.f;
-        l_run *= alpha;
-#pragma unroll 1
-        for (int c = 0; c < DH / 32; ++c) {
-          uint32_t t[32];
-          tmem_ld32(o_tmem + c * 32, t);
+      if (!fixed) {
+        // first pass over this thread's 64 scores for the row maximum (they are read again below)
+        float mx = -INFINITY;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t v[32];
+          tmem_ld32(s_tmem + part * 64 + hf * 32, v);
           tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) t[i] = __float_as_uint(__uint_as_float(t[i]) * alpha);
-          tmem_st32(o_tmem + c * 32, t);
+          for (int c = 0; c < 32; ++c)
+            if (!need_mask || k0 + hf * 32 + c <= lim) mx = fmaxf(mx, __uint_as_float(v[c]));
         }
-        tmem_st_wait();
-      }
-      m_run = m_use;
-      float sum = 0.f;
-      uint32_t pk[64];
+        // the other half of the row is another thread's: exchange through shared memory
+        xch[part * 128 + row] = mx;
+        asm volatile("bar.sync %0, 256;" ::"r"(bar_id) : "memory");
+        mx = fmaxf(mx, xch[(part ^ 1) * 128 + row]) * c_scale;
+        asm volatile("bar.sync %0, 256;" ::"r"(bar_id) : "memory");
+        const bool grow = mx > m_run + RESCALE_THRESHOLD;           // also true on the first tile
+        if (grow) m_use = mx;
+        if (m_use == -INFINITY) m_use = 0.f;
+        if (j > 0 && __any_sync(0xffffffffu, grow)) {
+          // rescale this thread's half of the running output (rare)
+          const float alpha = grow ? exp2f(m_run - m_use) : 1.f;
+          l_run *= alpha;
+#pragma unroll 1
+          for (int c = 0; c < DH / 64; ++c) {
+            uint32_t t[32];
+            tmem_ld32(o_tmem + part * (DH / 2) + c * 32, t);
+            tmem_ld_wait();
 #pragma unroll
-      for (int c = 0; c < 64; ++c) {
-        const float p0 = exp2f(fmaf(__uint_as_float(v[2 * c]), c_scale, -m_use));
-        const float p1 = exp2f(fmaf(__uint_as_float(v[2 * c + 1]), c_scale, -m_use));
-        sum += p0 + p1;
-        pk[c] = pack_bf16(p0, p1);
+            for (int i = 0; i < 32; ++i) t[i] = __float_as_uint(__uint_as_float(t[i]) * alpha);
+            tmem_st32(o_tmem + part * (DH / 2) + c * 32, t);
+          }
+          tmem_st_wait();
+        }
+        m_run = m_use;
       }
-      l_run += sum;
-      tmem_st32(s_tmem + 0, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
-      tmem_st32(s_tmem + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+      const uint64_t negm2 = pack2f(-m_use, -m_use);
+      uint64_t sum2 = pack2f(0.f, 0.f);
+      // 32 scores at a time.  The bf16 pairs of P go over the S columns the same thread has already read:
+      // part p reads S columns [64p, 64p+64) and writes P into storage columns [64p, 64p+32), so P of a
+      // KV tile sits in two separate 32-column pieces (the P V MMAs address them piece by piece).
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t v[32], pk[16];
+        tmem_ld32(s_tmem + part * 64 + hf * 32, v);
+        tmem_ld_wait();
+        if (need_mask) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c)
+            if (k0 + hf * 32 + c > lim) v[c] = 0xff800000u;        // -inf
+#pragma unroll
+          for (int c = 0; c < 4; ++c) exp8<0, false>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
+        } else if (fixed) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) exp8<POLY, false>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) exp8<POLY, true>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
+        }
+        tmem_st16(s_tmem + part * 64 + hf * 16, pk);
+      }
+      {
+        uint32_t a, b;
+        unpack2u(sum2, a, b);
+        l_run += __uint_as_float(a) + __uint_as_float(b);
+      }
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(&p_full[s]);
     }
     if (n_s[s] > 0) {
+      // total of the two halves of the row
+      xch[part * 128 + row] = l_run;
+      asm volatile("bar.sync %0, 256;" ::"r"(bar_id) : "memory");
+      l_run += xch[(part ^ 1) * 128 + row];
       if (!mbar_wait(&o_done[s], 0, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
       tc_fence_after();
       const float inv_l = 1.f / l_run;
       const long long row_g = (long long)b * p.S + tq;
 #pragma unroll 1
-      for (int c = 0; c < DH / 32; ++c) {
+      for (int c = 0; c < DH / 64; ++c) {
         uint32_t t[32];
-        tmem_ld32(o_tmem + c * 32, t);
+        const int col = part * (DH / 2) + c * 32;
+        tmem_ld32(o_tmem + col, t);
         tmem_ld_wait();
         if (tq < p.S) {
-          bf16* dst = p.o + row_g * p.Lq + hi * DH + c * 32;
+          bf16* dst = p.o + row_g * p.Lq + hi * DH + col;
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             uint4 w;
@@ -302,7 +446,7 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             reinterpret_cast<uint4*>(dst)[i] = w;
           }
           if (p.o32) {
-            float* d32 = p.o32 + row_g * p.Lq + hi * DH + c * 32;
+            float* d32 = p.o32 + row_g * p.Lq + hi * DH + col;
 #pragma unroll
             for (int i = 0; i < 8; ++i)
               reinterpret_cast<float4*>(d32)[i] =
@@ -311,7 +455,7 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           }
         }
       }
-      if (tq < p.S) p.lse[((long long)b * p.hq + hi) * p.S + tq] = (m_run + log2f(l_run)) * LN2_F;
+      if (part == 0 && tq < p.S) p.lse[((long long)b * p.hq + hi) * p.S + tq] = (m_run + log2f(l_run)) * LN2_F;
     }
   }
 done:
@@ -323,7 +467,7 @@ done:
     while (clock64() - t0 < 2000000) {}
     __syncthreads();
   }
-  if (warp == 9) {
+  if (warp == AT_MMA_WARP) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
@@ -331,8 +475,25 @@ done:
 
 }  // namespace
 
+namespace {
+template <int DH, int POLY>
+int launch_attn(TcState* s, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnParams& p,
+                unsigned grid, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(tc_attn_fwd_kernel<DH, POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         AttnSmem<DH>::TOTAL);
+    if (e != cudaSuccess) return -(int)e;
+    attr_set = true;
+  }
+  tc_attn_fwd_kernel<DH, POLY><<<grid, AT_THREADS, AttnSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, p);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? 0 : -(int)e;
+}
+}  // namespace
+
 int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* o32,
-                float* lse, int* d_status, cudaStream_t st) {
+                float* lse, const float* temp, int* d_status, cudaStream_t st) {
   if (!s || !s->encode) return 1;
   if (d.dh != 64 && d.dh != 128) return 1;
   if (d.Lq % 8 || d.Lk % 8) return 1;
@@ -350,22 +511,16 @@ int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, cons
   p.status = d_status;
   const long long grid = (long long)p.n_blocks * d.B * d.hq;
   if (grid > 0x7fffffffLL) return 1;
-  cudaError_t e;
+  p.temp = (s->attn_poly & 8) ? nullptr : temp;
+  const int poly = s->attn_poly & 7;
   if (d.dh == 128) {
-    if (!s->attn_attr_set[1]) {
-      e = cudaFuncSetAttribute(tc_attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::TOTAL);
-      if (e != cudaSuccess) return -(int)e;
-      s->attn_attr_set[1] = true;
-    }
-    tc_attn_fwd_kernel<128><<<(unsigned)grid, AT_THREADS, AttnSmem<128>::TOTAL, st>>>(tmQ, tmK, tmV, p);
-  } else {
-    if (!s->attn_attr_set[0]) {
-      e = cudaFuncSetAttribute(tc_attn_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::TOTAL);
-      if (e != cudaSuccess) return -(int)e;
-      s->attn_attr_set[0] = true;
-    }
-    tc_attn_fwd_kernel<64><<<(unsigned)grid, AT_THREADS, AttnSmem<64>::TOTAL, st>>>(tmQ, tmK, tmV, p);
+    if (poly == 0) return launch_attn<128, 0>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
+    if (poly == 1) return launch_attn<128, 1>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
+    if (poly == 3) return launch_attn<128, 3>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
+    return launch_attn<128, 2>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
   }
-  e = cudaGetLastError();
-  return e == cudaSuccess ? 0 : -(int)e;
+  if (poly == 0) return launch_attn<64, 0>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
+  if (poly == 1) return launch_attn<64, 1>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
+  if (poly == 3) return launch_attn<64, 3>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
+  return launch_attn<64, 2>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
 }

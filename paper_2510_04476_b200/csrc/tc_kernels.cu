@@ -11,6 +11,7 @@
 #include "tc_kernels.cuh"
 
 #include <cstdio>
+#include <cstdlib>
 #include <new>
 
 #include "tc_ptx.cuh"
@@ -257,6 +258,8 @@ TcState* tc_create(int sm_count) {
   s->encode = nullptr;
   s->attr_set_128 = s->attr_set_256 = false;
   s->attn_attr_set[0] = s->attn_attr_set[1] = false;
+  s->attn_poly = 1;
+  if (const char* e = getenv("CCA_ATTN_POLY")) s->attn_poly = atoi(e);
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||

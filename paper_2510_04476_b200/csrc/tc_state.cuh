@@ -13,6 +13,7 @@ struct TcState {
   EncodeTiledFn encode;
   bool attr_set_128, attr_set_256;
   bool attn_attr_set[2];
+  int attn_poly;          // of every 4 score pairs, how many take the polynomial exp2 (0..3)
 };
 
 // bf16 tensor maps with 128-byte swizzle.  2-D: dim0 (contiguous) extent d0, dim1 extent d1, row pitch ld
