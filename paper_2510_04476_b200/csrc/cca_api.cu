@@ -414,8 +414,18 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   g.M = d.E; g.N = d.Lq; g.K = T; g.seq_len = d.S; g.out_f32 = gr->d_w_o; g.ldc = d.Lq;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
   // attention adjoint
-  CU(launch_attn_bwd_simt(d, q, k, v, o32, d_o, lse, delta, dq, dk, dv, st));
-  h->launches += 3;
+  CU(launch_attn_delta(d, o32, d_o, delta, st));
+  h->launches++;
+  {
+    bool done = false;
+    if (h->impl >= 1 && h->tc) {
+      int tr = tc_attn_bwd(h->tc, d, q, k, v, d_o, lse, delta, dq, dk, dv, h->d_status, st);
+      if (tr == 0) done = true;
+      if (tr < 0) { h->last_cuda = -tr; return CCA_ERR_CUDA; }
+    }
+    if (!done) CU(launch_attn_bwd_simt(d, q, k, v, o32, d_o, lse, delta, dq, dk, dv, st));
+    h->launches += 2;
+  }
   // latent-transform adjoints
   CU(launch_transform_bwd_norm(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, dq, dk,
                                gr->d_temp, st));

@@ -65,6 +65,9 @@ cudaError_t launch_pack_dv(const CcaDims& d, const float* dv, bf16* dlat, long l
 // o32: optional fp32 copy of o (kept for the backward's delta = rowsum(dO * O)); may be null.
 cudaError_t launch_attn_fwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o,
                                  float* o32, float* lse, cudaStream_t st);
+// delta[b,i,t] = sum_c dO[t,i,c] * O[t,i,c] from the fp32 copy of o.
+cudaError_t launch_attn_delta(const CcaDims& d, const float* o32, const bf16* d_o, float* delta, cudaStream_t st);
+// dq, dk, dv from a delta that launch_attn_delta has filled.
 cudaError_t launch_attn_bwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const float* o32,
                                  const bf16* d_o, const float* lse, float* delta, float* dq, float* dk,
                                  float* dv, cudaStream_t st);

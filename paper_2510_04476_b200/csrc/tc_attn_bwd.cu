@@ -1,0 +1,550 @@
+// Tensor-core kernels, part 4: adjoint of the softmax attention of Eq. 11 (the paper prints no backward;
+// this is the exact adjoint).  With P = softmax(Q K^T / sqrt(d_h)) recomputed from the saved log-sum-exp,
+// dP = dO V^T, delta = rowsum(dO o O) and dS = P o (dP - delta):
+//     dV = P^T dO,   dK = dS^T Q / sqrt(d_h),   dQ = dS K / sqrt(d_h),
+// dK and dV summed over the g query heads that share a kv head.  Two kernels, no atomics:
+//
+//   tc_attn_bwd_dq_kernel   one CTA = 128 query rows of one (sequence, query head), loops over KV tiles.
+//                           TMEM: S (two buffers), dP, dQ accumulator; thread = query row.
+//   tc_attn_bwd_dkv_kernel  one CTA = 128 keys of one (sequence, kv head), loops over the g query heads and
+//                           their query tiles.  It works on the transposed tiles S^T = K Q^T and
+//                           dP^T = V dO^T (thread = key), so that P^T and dS^T are the TMEM A operands of
+//                           dV += P^T dO and dK += dS^T Q and both accumulators stay in TMEM.
+//
+// Both: warps 0-7 compute (two column halves x four TMEM lane quarters), warp 8 TMA loads, warp 9 issues
+// the MMAs (warp-uniform loop, one elected lane).  P and dS are bf16 MMA operands, everything else fp32.
+#include "tc_kernels.cuh"
+#include "tc_ptx.cuh"
+#include "tc_state.cuh"
+
+using namespace tc;
+
+namespace {
+
+constexpr int BW_THREADS = 320, BW_TMA_WARP = 8, BW_MMA_WARP = 9;
+constexpr float LOG2E_F = 1.4426950408889634f;
+
+struct BwdParams {
+  int B, S, hq, hk, g, Lq, Lk, causal;
+  const float* lse;     // [B, hq, S] natural-log sum of exponentials from the forward
+  const float* delta;   // [B, hq, S]
+  float* dq;            // [B*S, Lq]
+  float* dk;            // [B*S, Lk]
+  float* dv;            // [B*S, Lk]
+  int n_tiles;          // 128-row tiles per sequence
+  int* status;
+};
+
+template <int DH>
+struct BwdSmem {
+  static constexpr int TILE = 128 * DH * 2;
+  static constexpr int FIX_OFF = 0;                    // two tiles loaded once
+  static constexpr int RING_OFF = 2 * TILE;            // two rings of two tiles
+  static constexpr int BAR_OFF = 6 * TILE;
+  static constexpr int STAT_OFF = BAR_OFF + 256;       // float [2 buffers][2][128]
+  // at least 120 KB so that two CTAs (each wanting all 512 TMEM columns) never share an SM
+  static constexpr int TOTAL = (STAT_OFF + 2048 + 1024) > 122880 ? (STAT_OFF + 2048 + 1024) : 122880;
+};
+
+TC_DEVINL void fail(volatile int* abort_flag, int* status, int code) {
+  *abort_flag = 1;
+  atomicCAS(status, 0, code);
+}
+TC_DEVINL float ex2f(float x) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+
+// descriptor low words (address >> 4 | leading offset << 16) and the common high word
+TC_DEVINL uint32_t lo_kmajor(uint32_t addr) { return (addr >> 4) | (1u << 16); }
+TC_DEVINL uint32_t lo_mnmajor(uint32_t addr) { return (addr >> 4) | ((16384u >> 4) << 16); }
+
+// C[128 x 128] = A[128 x DH] B[128 x DH]^T, both operands K-major tiles in shared memory
+template <int DH>
+TC_DEVINL void mma_kk(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi) {
+  const uint32_t idesc = idesc_bf16(128, 0, 0);
+#pragma unroll
+  for (int kk = 0; kk < DH / 16; ++kk) {
+    const uint32_t off = (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+    mma_ss_w(d_tmem, a_lo + off, hi, b_lo + off, hi, idesc, kk != 0);
+  }
+}
+// C[128 x DH] (+)= A[128 x 128] B, A = bf16 pairs in TMEM (pieces at columns [0,32) and [64,96) of a_tmem),
+// B = a [128 rows][DH] tile in shared memory read along its rows (MN-major)
+template <int DH>
+TC_DEVINL void mma_tm(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t accumulate) {
+  const uint32_t idesc = idesc_bf16(DH, 0, 1);
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk)
+    mma_ts_w(d_tmem, a_tmem + (kk >> 2) * 64 + (kk & 3) * 8, b_lo + kk * (2048 >> 4), hi, idesc, (accumulate | kk) != 0);
+}
+
+template <int DH>
+TC_DEVINL void tma_tile(unsigned char* dst, const CUtensorMap* map, int c0, int row, int b, uint64_t* bar) {
+#pragma unroll
+  for (int c = 0; c < DH / 64; ++c) tma_load_3d(dst + c * 16384, map, c0 + c * 64, row, b, bar);
+}
+
+// ------------------------------------------------------------------------------------------ dQ
+template <int DH>
+__global__ void __launch_bounds__(BW_THREADS, 1)
+tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                      const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO, BwdParams p) {
+  using SM = BwdSmem<DH>;
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  unsigned char* sQ = smem + SM::FIX_OFF;
+  unsigned char* sDO = sQ + SM::TILE;
+  unsigned char* sK = smem + SM::RING_OFF;            // [2]
+  unsigned char* sV = sK + 2 * SM::TILE;              // [2]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFF);
+  uint64_t* qdo_full = bars;          // Q and dO tiles loaded
+  uint64_t* k_full = bars + 1;        // [2]
+  uint64_t* k_empty = bars + 3;       // [2]
+  uint64_t* v_full = bars + 5;        // [2]
+  uint64_t* v_empty = bars + 7;       // [2]
+  uint64_t* s_full = bars + 9;        // [2] MMA -> compute: S buffer ready
+  uint64_t* dp_full = bars + 11;      // MMA -> compute: dP ready
+  uint64_t* ds_full = bars + 12;      // compute -> MMA: dS written, dP consumed (256 arrivals)
+  uint64_t* dq_done = bars + 13;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // heavy (late) query tiles first
+  const int per_tile = p.B * p.hq;
+  const int tile = p.n_tiles - 1 - (int)(blockIdx.x / per_tile);
+  const int rem = blockIdx.x % per_tile;
+  const int b = rem / p.hq, hi = rem % p.hq, hj = hi / p.g;
+  const int m0 = tile * 128;
+  const int n_kv = p.causal ? tile + 1 : p.n_tiles;
+
+  if (threadIdx.x == 0) {
+    mbar_init(qdo_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&k_full[i], 1);
+      mbar_init(&k_empty[i], 1);
+      mbar_init(&v_full[i], 1);
+      mbar_init(&v_empty[i], 1);
+      mbar_init(&s_full[i], 1);
+    }
+    mbar_init(dp_full, 1);
+    mbar_init(ds_full, 256);
+    mbar_init(dq_done, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmQ);
+    prefetch_tmap(&tmK);
+    prefetch_tmap(&tmV);
+    prefetch_tmap(&tmDO);
+  }
+  if (warp == BW_MMA_WARP) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // TMEM columns: S0 [0,128) S1 [128,256) dP [256,384) dQ [384,384+DH)
+
+  if (warp == BW_TMA_WARP) {
+    if (lane == 0) {
+      mbar_expect_tx(qdo_full, 2 * SM::TILE);
+      tma_tile<DH>(sQ, &tmQ, hi * DH, m0, b, qdo_full);
+      tma_tile<DH>(sDO, &tmDO, hi * DH, m0, b, qdo_full);
+      for (int j = 0; j < n_kv; ++j) {
+        const int st = j & 1;
+        const uint32_t ph = (j >> 1) & 1;
+        if (!mbar_wait(&k_empty[st], ph ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
+        mbar_expect_tx(&k_full[st], SM::TILE);
+        tma_tile<DH>(sK + st * SM::TILE, &tmK, hj * DH, j * 128, b, &k_full[st]);
+        if (!mbar_wait(&v_empty[st], ph ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
+        mbar_expect_tx(&v_full[st], SM::TILE);
+        tma_tile<DH>(sV + st * SM::TILE, &tmV, hj * DH, j * 128, b, &v_full[st]);
+      }
+    }
+  } else if (warp == BW_MMA_WARP) {
+    const bool leader = elect_one();
+    const uint32_t hi_w = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
+    const uint32_t q_lo = lo_kmajor(smem_u32(sQ)), do_lo = lo_kmajor(smem_u32(sDO));
+    const uint32_t k_lo = lo_kmajor(smem_u32(sK)), v_lo = lo_kmajor(smem_u32(sV)), k_mn = lo_mnmajor(smem_u32(sK));
+    constexpr uint32_t TILE16 = SM::TILE >> 4;
+    auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+    };
+    if (!wait_all(qdo_full, 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+    if (!wait_all(&k_full[0], 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+    tc_fence_after();
+    if (leader) {
+      mma_kk<DH>(tmem_base, q_lo, k_lo, hi_w);                         // S(0) = Q K_0^T
+      mma_commit(&s_full[0]);
+    }
+    if (!wait_all(&v_full[0], 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+    tc_fence_after();
+    if (leader) {
+      mma_kk<DH>(tmem_base + 256, do_lo, v_lo, hi_w);                  // dP(0) = dO V_0^T
+      mma_commit(dp_full);
+      mma_commit(&v_empty[0]);
+    }
+    for (int j = 0; j < n_kv; ++j) {
+      const int st = j & 1, nx = (j + 1) & 1;
+      const uint32_t nph = ((j + 1) >> 1) & 1;
+      if (j + 1 < n_kv) {
+        // S(j+1) into the other buffer; the dQ MMA that read dS(j-1) from it was issued earlier (in order)
+        if (!wait_all(&k_full[nx], nph)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+        tc_fence_after();
+        if (leader) {
+          mma_kk<DH>(tmem_base + nx * 128, q_lo, k_lo + nx * TILE16, hi_w);
+          mma_commit(&s_full[nx]);
+        }
+      }
+      if (!wait_all(ds_full, j & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+      tc_fence_after();
+      if (j + 1 < n_kv) {
+        if (!wait_all(&v_full[nx], nph)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+        tc_fence_after();
+        if (leader) {
+          mma_kk<DH>(tmem_base + 256, do_lo, v_lo + nx * TILE16, hi_w);
+          mma_commit(dp_full);
+          mma_commit(&v_empty[nx]);
+        }
+      }
+      if (leader) {
+        mma_tm<DH>(tmem_base + 384, tmem_base + st * 128, k_mn + st * TILE16, hi_w, j != 0);   // dQ += dS(j) K_j
+        mma_commit(&k_empty[st]);
+      }
+    }
+    if (leader) mma_commit(dq_done);
+  } else {
+    // ------------------------------------------------------------------ compute, thread = query row
+    const int part = (warp >> 2) & 1;
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+    const int tq = m0 + row;
+    const float c_scale = rsqrtf((float)DH) * LOG2E_F;
+    const long long stat_idx = ((long long)b * p.hq + hi) * p.S + tq;
+    const float l2 = tq < p.S ? p.lse[stat_idx] * LOG2E_F : INFINITY;     // rows past the end: P = 0
+    const float dl = tq < p.S ? p.delta[stat_idx] : 0.f;
+    for (int j = 0; j < n_kv; ++j) {
+      const uint32_t s_t = tmem_base + lane_sel + (j & 1) * 128 + part * 64;
+      const uint32_t dp_t = tmem_base + lane_sel + 256 + part * 64;
+      if (!mbar_wait(&s_full[j & 1], (j >> 1) & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+      if (!mbar_wait(dp_full, j & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+      tc_fence_after();
+      const int k0 = j * 128 + part * 64;
+      const bool need_mask = (p.causal && j * 128 + 127 > m0) || (j * 128 + 128 > p.S);
+      const int lim = p.causal ? min(tq, p.S - 1) : p.S - 1;
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t sv[32], dv[32], pk[16];
+        tmem_ld32(s_t + hf * 32, sv);
+        tmem_ld32(dp_t + hf * 32, dv);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          float p0 = ex2f(fmaf(__uint_as_float(sv[2 * c]), c_scale, -l2));
+          float p1 = ex2f(fmaf(__uint_as_float(sv[2 * c + 1]), c_scale, -l2));
+          if (need_mask) {
+            if (k0 + hf * 32 + 2 * c > lim) p0 = 0.f;
+            if (k0 + hf * 32 + 2 * c + 1 > lim) p1 = 0.f;
+          }
+          pk[c] = pack_bf16(p0 * (__uint_as_float(dv[2 * c]) - dl), p1 * (__uint_as_float(dv[2 * c + 1]) - dl));
+        }
+        tmem_st16(s_t + hf * 16, pk);                 // dS over columns this thread has read
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(ds_full);
+    }
+    if (!mbar_wait(dq_done, 0, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
+    tc_fence_after();
+    {
+      const float scale = rsqrtf((float)DH);
+#pragma unroll 1
+      for (int c = 0; c < DH / 64; ++c) {
+        uint32_t t[32];
+        const int col = part * (DH / 2) + c * 32;
+        tmem_ld32(tmem_base + lane_sel + 384 + col, t);
+        tmem_ld_wait();
+        if (tq < p.S) {
+          float* dst = p.dq + ((long long)b * p.S + tq) * p.Lq + hi * DH + col;
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            reinterpret_cast<float4*>(dst)[i] =
+                make_float4(__uint_as_float(t[4 * i]) * scale, __uint_as_float(t[4 * i + 1]) * scale,
+                            __uint_as_float(t[4 * i + 2]) * scale, __uint_as_float(t[4 * i + 3]) * scale);
+        }
+      }
+    }
+  }
+done:
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000) {}
+    __syncthreads();
+  }
+  if (warp == BW_MMA_WARP) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ------------------------------------------------------------------------------------------ dK, dV
+template <int DH>
+__global__ void __launch_bounds__(BW_THREADS, 1)
+tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                       const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO, BwdParams p) {
+  using SM = BwdSmem<DH>;
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  unsigned char* sK = smem + SM::FIX_OFF;
+  unsigned char* sV = sK + SM::TILE;
+  unsigned char* sQ = smem + SM::RING_OFF;            // [2]
+  unsigned char* sDO = sQ + 2 * SM::TILE;             // [2]
+  float* stat = reinterpret_cast<float*>(smem + SM::STAT_OFF);   // [2 buffers][lse2 | delta][128 queries]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFF);
+  uint64_t* kv_full = bars;
+  uint64_t* qdo_full = bars + 1;      // [2]
+  uint64_t* qdo_empty = bars + 3;     // [2]
+  uint64_t* sdp_full = bars + 5;      // MMA -> compute: S^T and dP^T ready
+  uint64_t* pds_full = bars + 6;      // compute -> MMA: P^T and dS^T written (256 arrivals)
+  uint64_t* acc_done = bars + 7;
+  uint64_t* stat_ready = bars + 8;    // compute threads: column statistics of the tile are in shared memory
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 9);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // heavy (early) key tiles first
+  const int per_tile = p.B * p.hk;
+  const int tile = (int)(blockIdx.x / per_tile);
+  const int rem = blockIdx.x % per_tile;
+  const int b = rem / p.hk, hj = rem % p.hk;
+  const int n0 = tile * 128;
+  const int i0 = p.causal ? tile : 0;                  // first query tile that sees these keys
+  const int n_q = p.n_tiles - i0;
+  const int n_it = n_q * p.g;                          // iteration it = (gi, i): gi = it / n_q, i = i0 + it % n_q
+
+  if (threadIdx.x == 0) {
+    mbar_init(kv_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&qdo_full[i], 1);
+      mbar_init(&qdo_empty[i], 1);
+    }
+    mbar_init(sdp_full, 1);
+    mbar_init(pds_full, 256);
+    mbar_init(acc_done, 1);
+    mbar_init(stat_ready, 256);
+    *abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmQ);
+    prefetch_tmap(&tmK);
+    prefetch_tmap(&tmV);
+    prefetch_tmap(&tmDO);
+  }
+  if (warp == BW_MMA_WARP) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // TMEM columns: S^T [0,128) dP^T [128,256) dV [256,256+DH) dK [384,384+DH)
+
+  if (warp == BW_TMA_WARP) {
+    if (lane == 0) {
+      mbar_expect_tx(kv_full, 2 * SM::TILE);
+      tma_tile<DH>(sK, &tmK, hj * DH, n0, b, kv_full);
+      tma_tile<DH>(sV, &tmV, hj * DH, n0, b, kv_full);
+      for (int it = 0; it < n_it; ++it) {
+        const int st = it & 1;
+        const uint32_t ph = (it >> 1) & 1;
+        const int hi = hj * p.g + it / n_q, m0 = (i0 + it % n_q) * 128;
+        if (!mbar_wait(&qdo_empty[st], ph ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
+        mbar_expect_tx(&qdo_full[st], 2 * SM::TILE);
+        tma_tile<DH>(sQ + st * SM::TILE, &tmQ, hi * DH, m0, b, &qdo_full[st]);
+        tma_tile<DH>(sDO + st * SM::TILE, &tmDO, hi * DH, m0, b, &qdo_full[st]);
+      }
+    }
+  } else if (warp == BW_MMA_WARP) {
+    const bool leader = elect_one();
+    const uint32_t hi_w = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
+    const uint32_t k_lo = lo_kmajor(smem_u32(sK)), v_lo = lo_kmajor(smem_u32(sV));
+    const uint32_t q_lo = lo_kmajor(smem_u32(sQ)), do_lo = lo_kmajor(smem_u32(sDO));
+    const uint32_t q_mn = lo_mnmajor(smem_u32(sQ)), do_mn = lo_mnmajor(smem_u32(sDO));
+    constexpr uint32_t TILE16 = SM::TILE >> 4;
+    auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+    };
+    if (!wait_all(kv_full, 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+    for (int it = 0; it < n_it; ++it) {
+      const int st = it & 1;
+      if (!wait_all(&qdo_full[st], (it >> 1) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+      tc_fence_after();
+      if (leader) {
+        // the MMAs that read P^T / dS^T of the previous tile from these columns were issued before (in order)
+        mma_kk<DH>(tmem_base, k_lo, q_lo + st * TILE16, hi_w);               // S^T = K Q^T
+        mma_kk<DH>(tmem_base + 128, v_lo, do_lo + st * TILE16, hi_w);        // dP^T = V dO^T
+        mma_commit(sdp_full);
+      }
+      if (!wait_all(pds_full, it & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+      tc_fence_after();
+      if (leader) {
+        mma_tm<DH>(tmem_base + 256, tmem_base, do_mn + st * TILE16, hi_w, it != 0);        // dV += P^T dO
+        mma_tm<DH>(tmem_base + 384, tmem_base + 128, q_mn + st * TILE16, hi_w, it != 0);   // dK += dS^T Q
+        mma_commit(&qdo_empty[st]);
+      }
+    }
+    if (leader) mma_commit(acc_done);
+  } else {
+    // ------------------------------------------------------------------ compute, thread = key
+    const int part = (warp >> 2) & 1;
+    const int row = (warp & 3) * 32 + lane;
+    const int ct = threadIdx.x;                        // 0..255
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+    const int tk = n0 + row;
+    const float c_scale = rsqrtf((float)DH) * LOG2E_F;
+    // column statistics of a query tile: thread ct < 128 fetches lse * log2(e) of query ct, the others delta;
+    // queries past the end of the sequence get lse = +inf, so their P is 0
+    auto fetch_stat = [&](int it) -> float {
+      const int hi = hj * p.g + it / n_q, m0 = (i0 + it % n_q) * 128;
+      const int tq = m0 + (ct & 127);
+      const long long idx = ((long long)b * p.hq + hi) * p.S + tq;
+      if (ct < 128) return tq < p.S ? p.lse[idx] * LOG2E_F : INFINITY;
+      return tq < p.S ? p.delta[idx] : 0.f;
+    };
+    float next_stat = n_it > 0 ? fetch_stat(0) : 0.f;
+    for (int it = 0; it < n_it; ++it) {
+      const int sb = it & 1;
+      stat[sb * 256 + ct] = next_stat;                 // buffer sb was last read two tiles ago
+      if (it + 1 < n_it) next_stat = fetch_stat(it + 1);
+      mbar_arrive(stat_ready);
+      if (!mbar_wait(stat_ready, it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+      const int m0 = (i0 + it % n_q) * 128;
+      const bool diag = p.causal && m0 == n0;
+      if (!mbar_wait(sdp_full, it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+      tc_fence_after();
+      const uint32_t s_t = tmem_base + lane_sel + part * 64;
+      const uint32_t dp_t = tmem_base + lane_sel + 128 + part * 64;
+      const float4* l2v = reinterpret_cast<const float4*>(stat + sb * 256 + part * 64);
+      const float4* dlv = reinterpret_cast<const float4*>(stat + sb * 256 + 128 + part * 64);
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t sv[32], dv[32], pk[16], dk_[16];
+        tmem_ld32(s_t + hf * 32, sv);
+        tmem_ld32(dp_t + hf * 32, dv);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const float4 l2 = l2v[hf * 8 + c], dl = dlv[hf * 8 + c];
+          float pr[4];
+          pr[0] = ex2f(fmaf(__uint_as_float(sv[4 * c + 0]), c_scale, -l2.x));
+          pr[1] = ex2f(fmaf(__uint_as_float(sv[4 * c + 1]), c_scale, -l2.y));
+          pr[2] = ex2f(fmaf(__uint_as_float(sv[4 * c + 2]), c_scale, -l2.z));
+          pr[3] = ex2f(fmaf(__uint_as_float(sv[4 * c + 3]), c_scale, -l2.w));
+          if (diag) {
+            const int q0 = m0 + part * 64 + hf * 32 + 4 * c;      // query of pr[0]
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              if (tk > q0 + e) pr[e] = 0.f;
+          }
+          pk[2 * c] = pack_bf16(pr[0], pr[1]);
+          pk[2 * c + 1] = pack_bf16(pr[2], pr[3]);
+          dk_[2 * c] = pack_bf16(pr[0] * (__uint_as_float(dv[4 * c + 0]) - dl.x), pr[1] * (__uint_as_float(dv[4 * c + 1]) - dl.y));
+          dk_[2 * c + 1] = pack_bf16(pr[2] * (__uint_as_float(dv[4 * c + 2]) - dl.z), pr[3] * (__uint_as_float(dv[4 * c + 3]) - dl.w));
+        }
+        tmem_st16(s_t + hf * 16, pk);                  // P^T over S^T columns this thread has read
+        tmem_st16(dp_t + hf * 16, dk_);                // dS^T over dP^T columns this thread has read
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(pds_full);
+    }
+    if (!mbar_wait(acc_done, 0, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
+    tc_fence_after();
+    {
+      const float scale = rsqrtf((float)DH);
+#pragma unroll 1
+      for (int c = 0; c < DH / 64; ++c) {
+        uint32_t t[32], u[32];
+        const int col = part * (DH / 2) + c * 32;
+        tmem_ld32(tmem_base + lane_sel + 256 + col, t);
+        tmem_ld32(tmem_base + lane_sel + 384 + col, u);
+        tmem_ld_wait();
+        if (tk < p.S) {
+          const long long off = ((long long)b * p.S + tk) * p.Lk + hj * DH + col;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            reinterpret_cast<float4*>(p.dv + off)[i] = make_float4(__uint_as_float(t[4 * i]), __uint_as_float(t[4 * i + 1]),
+                                                                    __uint_as_float(t[4 * i + 2]), __uint_as_float(t[4 * i + 3]));
+            reinterpret_cast<float4*>(p.dk + off)[i] =
+                make_float4(__uint_as_float(u[4 * i]) * scale, __uint_as_float(u[4 * i + 1]) * scale,
+                            __uint_as_float(u[4 * i + 2]) * scale, __uint_as_float(u[4 * i + 3]) * scale);
+          }
+        }
+      }
+    }
+  }
+done:
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000) {}
+    __syncthreads();
+  }
+  if (warp == BW_MMA_WARP) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+template <int DH>
+int launch_bwd(TcState* s, const CcaDims& d, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
+               const CUtensorMap& tmDO, const BwdParams& p, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(tc_attn_bwd_dq_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<DH>::TOTAL);
+    if (e != cudaSuccess) return -(int)e;
+    e = cudaFuncSetAttribute(tc_attn_bwd_dkv_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<DH>::TOTAL);
+    if (e != cudaSuccess) return -(int)e;
+    attr_set = true;
+  }
+  const long long g_kv = (long long)p.n_tiles * d.B * d.hk, g_q = (long long)p.n_tiles * d.B * d.hq;
+  if (g_q > 0x7fffffffLL) return 1;
+  tc_attn_bwd_dkv_kernel<DH><<<(unsigned)g_kv, BW_THREADS, BwdSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, tmDO, p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return -(int)e;
+  tc_attn_bwd_dq_kernel<DH><<<(unsigned)g_q, BW_THREADS, BwdSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, tmDO, p);
+  e = cudaGetLastError();
+  return e == cudaSuccess ? 0 : -(int)e;
+}
+
+}  // namespace
+
+// delta must already hold rowsum(dO o O).  Returns 0 if both kernels were enqueued (2 launches).
+int tc_attn_bwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                const float* lse, const float* delta, float* dq, float* dk, float* dv, int* d_status, cudaStream_t st) {
+  if (!s || !s->encode) return 1;
+  if (d.dh != 64 && d.dh != 128) return 1;
+  if (d.Lq % 8 || d.Lk % 8) return 1;
+  CUtensorMap tmQ, tmK, tmV, tmDO;
+  const uint64_t S = (uint64_t)d.S, B = (uint64_t)d.B, Lq = (uint64_t)d.Lq, Lk = (uint64_t)d.Lk;
+  if (!tc_make_map_3d(s, &tmQ, q, Lq, S, B, Lq, S * Lq, 64, 128)) return 1;
+  if (!tc_make_map_3d(s, &tmDO, d_o, Lq, S, B, Lq, S * Lq, 64, 128)) return 1;
+  if (!tc_make_map_3d(s, &tmK, k, Lk, S, B, Lk, S * Lk, 64, 128)) return 1;
+  if (!tc_make_map_3d(s, &tmV, v, Lk, S, B, Lk, S * Lk, 64, 128)) return 1;
+  BwdParams p;
+  p.B = d.B; p.S = d.S; p.hq = d.hq; p.hk = d.hk; p.g = d.g; p.Lq = d.Lq; p.Lk = d.Lk; p.causal = d.causal;
+  p.lse = lse; p.delta = delta; p.dq = dq; p.dk = dk; p.dv = dv;
+  p.n_tiles = (d.S + 127) / 128;
+  p.status = d_status;
+  if (d.dh == 128) return launch_bwd<128>(s, d, tmQ, tmK, tmV, tmDO, p, st);
+  return launch_bwd<64>(s, d, tmQ, tmK, tmV, tmDO, p, st);
+}

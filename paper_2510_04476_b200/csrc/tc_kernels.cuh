@@ -11,5 +11,8 @@ void tc_destroy(TcState* s);
 int tc_gemm(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st);
 int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* o32,
                 float* lse, const float* temp, int* d_status, cudaStream_t st);
+// Attention adjoint (dq, dk, dv in fp32) from q, k, v, d_o, the forward's lse and delta = rowsum(dO o O).
+int tc_attn_bwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                const float* lse, const float* delta, float* dq, float* dk, float* dv, int* d_status, cudaStream_t st);
 int tc_transform_fwd(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
                      const float* temp, const float2* rope, bf16* q, bf16* k, int* d_status, cudaStream_t st);
