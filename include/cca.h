@@ -100,6 +100,7 @@ typedef struct {
   int64_t off_qk0, off_q, off_k, off_v, off_o, off_lse, off_rope;
   int64_t saved_bytes;              /* forward-only workspace size                          */
   int64_t total_bytes;              /* forward + backward workspace size                    */
+  int64_t off_rnorm;                /* fp32 [B*S, h_q+h_k]: norm scale sqrt(d_h)[*beta]/|x| kept for the backward */
 } cca_layout;
 
 typedef struct cca_handle cca_handle;
@@ -122,7 +123,7 @@ int cca_workspace_size(const cca_handle* h, int64_t B, int64_t S, int need_backw
 /* Forward of the whole block, Eq. 7-11: out = W_o [ softmax(q k^T / sqrt(d_h)) v ]_heads.
  *   x   device bf16 [B,S,E] (read), out device bf16 [B,S,E] (written).
  *   workspace: device, 256-byte aligned, >= cca_workspace_size(..., need_backward).  On return
- *   (stream order) it holds qk0 (fp32), q, k, v, o (bf16), lse (fp32) at the cca_layout offsets; keep it untouched
+ *   (stream order) it holds qk0 (fp32), q, k, v, o (bf16), lse and the norm scales (fp32) at the cca_layout offsets; keep it untouched
  *   until cca_backward if gradients are wanted.
  * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE_TOO_SMALL, CUDA. */
 int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out,

@@ -42,7 +42,7 @@ class cca_layout(C.Structure):
                 ("fwd_flops_causal", C.c_int64), ("decode_flops", C.c_int64),
                 ("off_qk0", C.c_int64), ("off_q", C.c_int64), ("off_k", C.c_int64), ("off_v", C.c_int64),
                 ("off_o", C.c_int64), ("off_lse", C.c_int64), ("off_rope", C.c_int64),
-                ("saved_bytes", C.c_int64), ("total_bytes", C.c_int64)]
+                ("saved_bytes", C.c_int64), ("total_bytes", C.c_int64), ("off_rnorm", C.c_int64)]
 
 
 # name -> (restype, argtypes); also the list of symbols the header declares

@@ -25,7 +25,7 @@ namespace {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
-  size_t qk0, q, k, v, o, lse, rope, saved_end;
+  size_t qk0, q, k, v, o, lse, rope, rnorm, saved_end;
   size_t o32, d_o, delta, dq, dk, dv, dlat, w_all, total_end;
 };
 
@@ -42,6 +42,7 @@ Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
   l.o = take(T * Lq * 2);
   l.lse = take((size_t)B * c.n_q_heads * S * 4);
   l.rope = take((size_t)S * (c.head_dim / 2) * 8);
+  l.rnorm = take(T * (size_t)(c.n_q_heads + c.n_kv_heads) * 4);   // norm scale of every (token, head)
   l.saved_end = off;
   l.o32 = take(T * Lq * 4);
   l.d_o = take(T * Lq * 2);
@@ -247,6 +248,7 @@ int cca_describe(const cca_handle* h, int64_t B, int64_t S, cca_layout* out) {
   Layout l = make_layout(c, B, S);
   out->off_qk0 = (int64_t)l.qk0; out->off_q = (int64_t)l.q; out->off_k = (int64_t)l.k; out->off_v = (int64_t)l.v;
   out->off_o = (int64_t)l.o; out->off_lse = (int64_t)l.lse; out->off_rope = (int64_t)l.rope;
+  out->off_rnorm = (int64_t)l.rnorm;
   out->saved_bytes = (int64_t)l.saved_end;
   out->total_bytes = (int64_t)l.total_end;
   return CCA_OK;
@@ -301,6 +303,7 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   bf16* o = (bf16*)(ws + l.o);
   float* lse = (float*)(ws + l.lse);
   float2* rope = (float2*)(ws + l.rope);
+  float* rnorm = (float*)(ws + l.rnorm);
   // fp32 copy of o for the backward, kept only if the caller's workspace has the backward region
   float* o32 = workspace_bytes >= l.total_end ? (float*)(ws + l.o32) : nullptr;
 
@@ -325,11 +328,12 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
     bool done = false;
     if (h->impl >= 1 && h->tc) {
       int tr = tc_transform_fwd(h->tc, d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k,
-                                h->d_status, st);
+                                rnorm, h->d_status, st);
       if (tr == 0) done = true;
       if (tr < 0) { h->last_cuda = -tr; return CCA_ERR_CUDA; }
     }
-    if (!done) CU(launch_transform_fwd(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k, st));
+    if (!done)
+      CU(launch_transform_fwd(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k, rnorm, st));
     h->launches++;
   }
   // Eq. 11: attention in the latent
@@ -391,6 +395,7 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   const bf16* o = (const bf16*)(ws + l.o);
   const float* lse = (const float*)(ws + l.lse);
   const float2* rope = (const float2*)(ws + l.rope);
+  const float* rnorm = (const float*)(ws + l.rnorm);
   const float* o32 = (const float*)(ws + l.o32);
   bf16* d_o = (bf16*)(ws + l.d_o);
   float* delta = (float*)(ws + l.delta);
@@ -427,8 +432,7 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
     h->launches += 2;
   }
   // latent-transform adjoints
-  CU(launch_transform_bwd_norm(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, dq, dk,
-                               gr->d_temp, st));
+  CU(launch_transform_bwd_norm(d, q, k, rnorm, w->temp, rope, dq, dk, gr->d_temp, st));
   CU(launch_transform_bwd_conv(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, dq, dk, dlat, ldl,
                                gr->d_conv0_w, st));
   CU(launch_transform_bwd_w1(d, qk0, (const bf16*)w->conv0_w, dq, dk, gr->d_conv1_w, st));

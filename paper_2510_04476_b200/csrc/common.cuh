@@ -44,11 +44,12 @@ cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
 // ---- latent transforms (Eq. 8-11 without the attention) ----
 cudaError_t launch_rope_table(float2* tab, int S, int dh, float base, cudaStream_t st);
 cudaError_t launch_transform_fwd(const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
-                                 const float* temp, const float2* rope_tab, bf16* q, bf16* k,
+                                 const float* temp, const float2* rope_tab, bf16* q, bf16* k, float* rnorm,
                                  cudaStream_t st);
+// rnorm[token, head] = sqrt(d_h) [* exp(temp)] / |pre-norm latent|, written by the forward.
 // dq/dk (fp32, gradients w.r.t. the attention inputs) are replaced in place by the gradients
 // w.r.t. the pre-norm latents; d_temp accumulates (must be zeroed by the caller).
-cudaError_t launch_transform_bwd_norm(const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
+cudaError_t launch_transform_bwd_norm(const CcaDims& d, const bf16* q, const bf16* k, const float* rnorm,
                                       const float* temp, const float2* rope_tab, float* dq, float* dk,
                                       float* d_temp, cudaStream_t st);
 // dlat[T, ld_dlat] columns [0, L) <- gradient w.r.t. qk0 (bf16); d_w0 accumulates.

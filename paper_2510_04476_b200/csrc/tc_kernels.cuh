@@ -15,4 +15,5 @@ int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, cons
 int tc_attn_bwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                 const float* lse, const float* delta, float* dq, float* dk, float* dv, int* d_status, cudaStream_t st);
 int tc_transform_fwd(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
-                     const float* temp, const float2* rope, bf16* q, bf16* k, int* d_status, cudaStream_t st);
+                     const float* temp, const float2* rope, bf16* q, bf16* k, float* rnorm, int* d_status,
+                     cudaStream_t st);

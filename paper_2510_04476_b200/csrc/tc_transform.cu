@@ -61,6 +61,7 @@ struct TrParams {
   const float2* rope;
   bf16* q;
   bf16* k;
+  float* rnorm;         // [B*S, hq+hk] norm scale kept for the backward
   int* status;
   int n_tiles;          // 128-token tiles per sequence
   int units_per_head;   // B * n_tiles
@@ -370,6 +371,7 @@ __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const T
           for (int i = 0; i < 32; ++i) ss = fmaf(__uint_as_float(r[i]), __uint_as_float(r[i]), ss);
         }
         sc = sqrtf((float)DH) * (is_q ? 1.f : __expf(p.temp[hj])) * rsqrtf(ss);
+        if (valid) p.rnorm[((long long)b * d.S + t) * (d.hq + d.hk) + h] = sc;
       }
       const long long tok = (long long)b * d.S + (valid ? t : 0);
       bf16* dst = is_q ? p.q + tok * d.Lq + h * DH : p.k + tok * d.Lk + hj * DH;
@@ -455,7 +457,7 @@ done:
 
 template <int DH, int KC>
 int launch_tr(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1, const float* temp,
-              const float2* rope, bf16* q, bf16* k, int* status, cudaStream_t st) {
+              const float2* rope, bf16* q, bf16* k, float* rnorm, int* status, cudaStream_t st) {
   static bool attr_done = false;
   using SM = TrSmem<DH, KC>;
   if (!attr_done) {
@@ -464,7 +466,7 @@ int launch_tr(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, co
     attr_done = true;
   }
   TrParams p;
-  p.d = d; p.qk0 = qk0; p.w0 = w0; p.w1 = w1; p.temp = temp; p.rope = rope; p.q = q; p.k = k; p.status = status;
+  p.d = d; p.qk0 = qk0; p.w0 = w0; p.w1 = w1; p.temp = temp; p.rope = rope; p.q = q; p.k = k; p.rnorm = rnorm; p.status = status;
   p.n_tiles = (d.S + 127) / 128;
   const long long uph = (long long)d.B * p.n_tiles, total = uph * (d.hq + d.hk);
   if (total > 0x7fffffffLL) return 1;
@@ -481,21 +483,22 @@ int launch_tr(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, co
 }  // namespace
 
 int tc_transform_fwd(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
-                     const float* temp, const float2* rope, bf16* q, bf16* k, int* d_status, cudaStream_t st) {
+                     const float* temp, const float2* rope, bf16* q, bf16* k, float* rnorm, int* d_status,
+                     cudaStream_t st) {
   if (!s || s->sm_count < 1) return 1;
   if (!(d.flags & F_CONV2)) return 1;                 // no contraction to run: the SIMT kernel is the right tool
   if (d.L % 4 || d.Lq % 8 || d.Lk % 8) return 1;
   if ((reinterpret_cast<uintptr_t>(w1) & 15) || (reinterpret_cast<uintptr_t>(qk0) & 15)) return 1;
   if (d.dh == 128) {
-    if (d.k_ch == 1) return launch_tr<128, 1>(s, d, qk0, w0, w1, temp, rope, q, k, d_status, st);
-    if (d.k_ch == 2) return launch_tr<128, 2>(s, d, qk0, w0, w1, temp, rope, q, k, d_status, st);
+    if (d.k_ch == 1) return launch_tr<128, 1>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
+    if (d.k_ch == 2) return launch_tr<128, 2>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
     return 1;
   }
   if (d.dh == 64) {
-    if (d.k_ch == 1) return launch_tr<64, 1>(s, d, qk0, w0, w1, temp, rope, q, k, d_status, st);
-    if (d.k_ch == 2) return launch_tr<64, 2>(s, d, qk0, w0, w1, temp, rope, q, k, d_status, st);
-    if (d.k_ch == 3) return launch_tr<64, 3>(s, d, qk0, w0, w1, temp, rope, q, k, d_status, st);
-    if (d.k_ch == 4) return launch_tr<64, 4>(s, d, qk0, w0, w1, temp, rope, q, k, d_status, st);
+    if (d.k_ch == 1) return launch_tr<64, 1>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
+    if (d.k_ch == 2) return launch_tr<64, 2>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
+    if (d.k_ch == 3) return launch_tr<64, 3>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
+    if (d.k_ch == 4) return launch_tr<64, 4>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
   }
   return 1;
 }

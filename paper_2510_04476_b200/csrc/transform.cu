@@ -160,7 +160,7 @@ __global__ void __launch_bounds__(256) transform_fwd_kernel(CcaDims d, const flo
                                                             const bf16* __restrict__ w0, const bf16* __restrict__ w1,
                                                             const float* __restrict__ temp,
                                                             const float2* __restrict__ rope_tab, bf16* __restrict__ q,
-                                                            bf16* __restrict__ k) {
+                                                            bf16* __restrict__ k, float* __restrict__ rnorm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem<DH> sm(smem_raw);
   constexpr int TPT = Lay<DH>::TPT, YLD = Lay<DH>::YLD;
@@ -182,7 +182,12 @@ __global__ void __launch_bounds__(256) transform_fwd_kernel(CcaDims d, const flo
       for (int n = 0; n < TPT; ++n) ss[n] = acc[n] * acc[n];
       reduce_channels<DH>(ss, sm.red);
 #pragma unroll
-      for (int n = 0; n < TPT; ++n) acc[n] *= scale * rsqrtf(ss[n]);
+      for (int n = 0; n < TPT; ++n) {
+        const float sc = scale * rsqrtf(ss[n]);
+        acc[n] *= sc;
+        const int t = t0 + tg * TPT + n;
+        if (o == 0 && t < d.S) rnorm[((long long)b * d.S + t) * (d.hq + d.hk) + h] = sc;
+      }
     }
 #pragma unroll
     for (int n = 0; n < TPT; ++n) sm.outs[(tg * TPT + n) * YLD + o] = acc[n];
@@ -208,79 +213,74 @@ __global__ void __launch_bounds__(256) transform_fwd_kernel(CcaDims d, const flo
 
 // ------------------------------------------------------------------------------------------
 // backward, part 1: RoPE adjoint, norm adjoint, d_temp.  In place on dq / dk (fp32).
+// One warp per (token, head); lane l owns channels l, l+32, ... so that the rotation pairs
+// (c, c + d_h/2) sit in one lane and every access is a run of 32 consecutive elements.
+//   x = pre-norm latent, y = r x with r = sqrt(d_h)[beta]/|x| (kept by the forward), q = RoPE(y):
+//   dy = RoPE^T(dq);  dx = r (dy - y (y . dy) / |y|^2),  |y|^2 = d_h [beta^2];  d_temp = sum y . dy.
+// y is taken from the stored bf16 q / k (rotated back), r in fp32: the 1/|x| amplification is exact,
+// the projection direction carries the bf16 rounding of q.
 // ------------------------------------------------------------------------------------------
 template <int DH>
-__global__ void __launch_bounds__(256) transform_bwd_norm_kernel(CcaDims d, const float* __restrict__ qk0,
-                                                                 const bf16* __restrict__ w0,
-                                                                 const bf16* __restrict__ w1,
+__global__ void __launch_bounds__(256) transform_bwd_norm_kernel(CcaDims d, const bf16* __restrict__ q,
+                                                                 const bf16* __restrict__ k,
+                                                                 const float* __restrict__ rnorm,
                                                                  const float* __restrict__ temp,
                                                                  const float2* __restrict__ rope_tab, float* dq,
                                                                  float* dk, float* d_temp) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  Smem<DH> sm(smem_raw);
-  constexpr int TPT = Lay<DH>::TPT, YLD = Lay<DH>::YLD, HALF = DH / 2;
-  const int h = blockIdx.y, b = blockIdx.z;
-  const int o = threadIdx.x % DH, tg = threadIdx.x / DH;
+  constexpr int HALF = DH / 2, NP = HALF / 32 > 0 ? HALF / 32 : 1;     // rotation pairs per lane
+  const int H = d.hq + d.hk;
+  const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / 32;
+  const int lane = threadIdx.x % 32;
+  const long long total = (long long)d.B * d.S * H;
+  if (w >= total) return;
+  const int h = (int)(w % H);
+  const long long row = w / H;
+  const int t = (int)(row % d.S);
   const bool is_q = h < d.hq;
-  float* grad = is_q ? dq : dk;
-  const int ld = is_q ? d.Lq : d.Lk;
-  const int col = (is_q ? h : h - d.hq) * DH + o;
-  if (d.flags & F_CONV2) stage_w1<DH, false>(d, w1, h, sm.ws);
-  const float scale = sqrtf((float)DH) * (is_q ? 1.f : __expf(temp[h - d.hq]));
-  float dtemp_local = 0.f;
-  for (int tile = 0; tile < TILES_PER_BLOCK; ++tile) {
-    const int t0 = (blockIdx.x * TILES_PER_BLOCK + tile) * TT;
-    if (t0 >= d.S) break;
-    __syncthreads();
-    // incoming gradient tile -> outs
+  const int hj = is_q ? h : h - d.hq;
+  float* g = (is_q ? dq + row * d.Lq : dk + row * d.Lk) + hj * DH;
+  const bf16* y = (is_q ? q + row * d.Lq : k + row * d.Lk) + hj * DH;
+  const bool act = lane < HALF;                   // d_h = 32: only 16 pairs
+  float ga[NP], gb[NP], ya[NP], yb[NP];
 #pragma unroll
-    for (int n = 0; n < TPT; ++n) {
-      int tl = tg * TPT + n, t = t0 + tl;
-      sm.outs[tl * YLD + o] = t < d.S ? grad[((long long)b * d.S + t) * ld + col] : 0.f;
-    }
-    if (d.flags & F_QK_NORM) fill_y1<DH>(d, qk0, w0, b, h, t0 - (d.k_ch - 1), TT + d.k_ch - 1, sm.y1s);
-    __syncthreads();
-    float dy[TPT];
-#pragma unroll
-    for (int n = 0; n < TPT; ++n) {
-      int tl = tg * TPT + n, t = t0 + tl;
-      float own = sm.outs[tl * YLD + o];
-      if ((d.flags & F_ROPE) && t < d.S) {
-        int c = o < HALF ? o : o - HALF;
-        float2 cs = rope_tab[(long long)t * HALF + c];
-        float other = sm.outs[tl * YLD + (o < HALF ? o + HALF : o - HALF)];
-        // rotation by the negated angle
-        own = o < HALF ? own * cs.x + other * cs.y : own * cs.x - other * cs.y;
-      }
-      dy[n] = own;
-    }
-    if (d.flags & F_QK_NORM) {
-      float xh[TPT], ss[TPT], dot[TPT];
-      hat_tile<DH>(d, qk0, sm.ws, sm.y1s, b, h, t0, xh);
-#pragma unroll
-      for (int n = 0; n < TPT; ++n) {
-        ss[n] = xh[n] * xh[n];
-        dot[n] = xh[n] * dy[n];
-      }
-      reduce_channels<DH>(ss, sm.red);
-      reduce_channels<DH>(dot, sm.red);
-#pragma unroll
-      for (int n = 0; n < TPT; ++n) {
-        int t = t0 + tg * TPT + n;
-        if (t >= d.S) { dy[n] = 0.f; continue; }
-        float inv = rsqrtf(ss[n]);                 // 1/|x|
-        float ndot = dot[n] * inv;                 // n . dy
-        if (!is_q && o == 0) dtemp_local += scale * ndot;
-        dy[n] = scale * inv * (dy[n] - xh[n] * inv * ndot);
-      }
-    }
-#pragma unroll
-    for (int n = 0; n < TPT; ++n) {
-      int t = t0 + tg * TPT + n;
-      if (t < d.S) grad[((long long)b * d.S + t) * ld + col] = dy[n];
+  for (int i = 0; i < NP; ++i) {
+    const int c = lane + 32 * i;
+    ga[i] = act ? g[c] : 0.f;
+    gb[i] = act ? g[c + HALF] : 0.f;
+    ya[i] = act ? __bfloat162float(y[c]) : 0.f;
+    yb[i] = act ? __bfloat162float(y[c + HALF]) : 0.f;
+    if ((d.flags & F_ROPE) && act) {
+      const float2 cs = rope_tab[(long long)t * HALF + c];
+      // rotation by the negated angle
+      const float a0 = ga[i] * cs.x + gb[i] * cs.y, b0 = gb[i] * cs.x - ga[i] * cs.y;
+      ga[i] = a0; gb[i] = b0;
+      const float a1 = ya[i] * cs.x + yb[i] * cs.y, b1 = yb[i] * cs.x - ya[i] * cs.y;
+      ya[i] = a1; yb[i] = b1;
     }
   }
-  if (!is_q && o == 0 && (d.flags & F_QK_NORM)) atomicAdd(d_temp + (h - d.hq), dtemp_local);
+  if (d.flags & F_QK_NORM) {
+    float dot = 0.f;
+#pragma unroll
+    for (int i = 0; i < NP; ++i) dot = fmaf(ya[i], ga[i], fmaf(yb[i], gb[i], dot));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    const float beta = is_q ? 1.f : __expf(temp[hj]);
+    const float r = rnorm[row * H + h];
+    const float proj = dot / ((float)DH * beta * beta);
+    if (!is_q && lane == 0) atomicAdd(d_temp + hj, dot);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      ga[i] = r * (ga[i] - ya[i] * proj);
+      gb[i] = r * (gb[i] - yb[i] * proj);
+    }
+  }
+  if (act) {
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      g[lane + 32 * i] = ga[i];
+      g[lane + 32 * i + HALF] = gb[i];
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -477,24 +477,23 @@ static dim3 tile_grid(const CcaDims& d) {
 }
 
 cudaError_t launch_transform_fwd(const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1, const float* temp,
-                                 const float2* rope_tab, bf16* q, bf16* k, cudaStream_t st) {
+                                 const float2* rope_tab, bf16* q, bf16* k, float* rnorm, cudaStream_t st) {
   DISPATCH_DH(d.dh, {
     cudaError_t e = set_smem(transform_fwd_kernel<DH>, smem_bytes<DH>());
     if (e != cudaSuccess) return e;
-    transform_fwd_kernel<DH><<<tile_grid(d), 256, smem_bytes<DH>(), st>>>(d, qk0, w0, w1, temp, rope_tab, q, k);
+    transform_fwd_kernel<DH><<<tile_grid(d), 256, smem_bytes<DH>(), st>>>(d, qk0, w0, w1, temp, rope_tab, q, k, rnorm);
   });
   return cudaGetLastError();
 }
 
-cudaError_t launch_transform_bwd_norm(const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
+cudaError_t launch_transform_bwd_norm(const CcaDims& d, const bf16* q, const bf16* k, const float* rnorm,
                                       const float* temp, const float2* rope_tab, float* dq, float* dk, float* d_temp,
                                       cudaStream_t st) {
   if (!(d.flags & (F_QK_NORM | F_ROPE))) return cudaSuccess;
+  const long long warps = (long long)d.B * d.S * (d.hq + d.hk);
+  const unsigned grid = (unsigned)((warps * 32 + 255) / 256);
   DISPATCH_DH(d.dh, {
-    cudaError_t e = set_smem(transform_bwd_norm_kernel<DH>, smem_bytes<DH>());
-    if (e != cudaSuccess) return e;
-    transform_bwd_norm_kernel<DH><<<tile_grid(d), 256, smem_bytes<DH>(), st>>>(d, qk0, w0, w1, temp, rope_tab, dq, dk,
-                                                                              d_temp);
+    transform_bwd_norm_kernel<DH><<<grid, 256, 0, st>>>(d, q, k, rnorm, temp, rope_tab, dq, dk, d_temp);
   });
   return cudaGetLastError();
 }
