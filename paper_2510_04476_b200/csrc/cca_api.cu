@@ -26,7 +26,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
   size_t qk0, q, k, v, o, lse, rope, rnorm, saved_end;
-  size_t o32, d_o, delta, dq, dk, dv, dlat, w_all, total_end;
+  size_t o32, d_o, delta, dq, dk, dv, dlat, w_all, dy1, total_end;
 };
 
 Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
@@ -52,6 +52,7 @@ Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
   l.dv = take(T * Lk * 4);
   l.dlat = take(T * (L + Lk) * 2);
   l.w_all = take((L + Lk) * (size_t)c.d_model * 2);
+  l.dy1 = take(T * L * 4);
   l.total_end = off;
   return l;
 }
@@ -433,9 +434,24 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   }
   // latent-transform adjoints
   CU(launch_transform_bwd_norm(d, q, k, rnorm, w->temp, rope, dq, dk, gr->d_temp, st));
-  CU(launch_transform_bwd_conv(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, dq, dk, dlat, ldl,
-                               gr->d_conv0_w, st));
-  CU(launch_transform_bwd_w1(d, qk0, (const bf16*)w->conv0_w, dq, dk, gr->d_conv1_w, st));
+  {
+    bool done = false;
+    if (h->impl >= 1 && h->tc) {
+      float* dy1 = (float*)(ws + l.dy1);
+      int tr = tc_transform_bwd(h->tc, d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, dq, dk, dy1,
+                                gr->d_conv1_w, h->d_status, st);
+      if (tr < 0) { h->last_cuda = -tr; return CCA_ERR_CUDA; }
+      if (tr == 0) {
+        CU(launch_conv1_adjoint(d, dy1, dq, dk, qk0, (const bf16*)w->conv0_w, dlat, ldl, gr->d_conv0_w, st));
+        done = true;
+      }
+    }
+    if (!done) {
+      CU(launch_transform_bwd_conv(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, dq, dk, dlat, ldl,
+                                   gr->d_conv0_w, st));
+      CU(launch_transform_bwd_w1(d, qk0, (const bf16*)w->conv0_w, dq, dk, gr->d_conv1_w, st));
+    }
+  }
   CU(launch_pack_dv(d, dv, dlat, ldl, st));
   h->launches += 4;
   // down-projection adjoints: parameter gradients

@@ -56,6 +56,9 @@ cudaError_t launch_transform_bwd_norm(const CcaDims& d, const bf16* q, const bf1
 cudaError_t launch_transform_bwd_conv(const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
                                       const float* dqh, const float* dkh, bf16* dlat, long long ld_dlat,
                                       float* d_w0, cudaStream_t st);
+// Same result as launch_transform_bwd_conv when dy1 [T, L] (fp32) already holds the conv2 adjoint of d_hat.
+cudaError_t launch_conv1_adjoint(const CcaDims& d, const float* dy1, const float* dqh, const float* dkh, const float* qk0,
+                                 const bf16* w0, bf16* dlat, long long ld_dlat, float* d_w0, cudaStream_t st);
 // d_w1 accumulates.
 cudaError_t launch_transform_bwd_w1(const CcaDims& d, const float* qk0, const bf16* w0, const float* dqh,
                                     const float* dkh, float* d_w1, cudaStream_t st);

@@ -428,6 +428,68 @@ __global__ void __launch_bounds__(256) transform_bwd_w1_kernel(CcaDims d, const 
   }
 }
 
+// conv1 adjoint + q-k-mean adjoint + gradient of the depth-wise taps, given dy1 = gradient w.r.t. conv1's output:
+//   d_qk0[t][c]  = sum_j w0[c][j] dy1[t + (ks-1) - j][c]  +  (direct q-k-mean terms of d_hat)
+//   d_w0[c][j]  += sum_t dy1[t][c] qk0[t - (ks-1) + j][c]
+// One thread per channel (coalesced over channels), walking CONV1_TOK consecutive tokens with sliding windows.
+constexpr int CONV1_TOK = 64;
+template <int KS>
+__global__ void __launch_bounds__(128) conv1_adjoint_kernel(CcaDims d, const float* __restrict__ dy1,
+                                                            const float* __restrict__ dqh, const float* __restrict__ dkh,
+                                                            const float* __restrict__ qk0, const bf16* __restrict__ w0,
+                                                            bf16* __restrict__ dlat, long long ld, float* d_w0) {
+  const int c = blockIdx.x * 128 + threadIdx.x;
+  if (c >= d.L) return;
+  const int b = blockIdx.z;
+  const int t_begin = blockIdx.y * CONV1_TOK, t_end = min(d.S, t_begin + CONV1_TOK);
+  const bool conv1 = (d.flags & F_CONV1) != 0;         // off: KS = 1 with unit weight
+  float w[KS], dw[KS], win[KS], qwin[KS];
+#pragma unroll
+  for (int j = 0; j < KS; ++j) {
+    w[j] = conv1 ? ldbf(w0 + c * KS + j) : 1.f;
+    dw[j] = 0.f;
+  }
+  const long long seq = (long long)b * d.S;
+  auto dy_at = [&](int t) { return t < d.S ? dy1[(seq + t) * d.L + c] : 0.f; };
+  auto q_at = [&](int t) { return t >= 0 ? qk0[(seq + t) * d.L + c] : 0.f; };
+  // win[m] = dy1[t + m], qwin[m] = qk0[t - (KS-1) + m]
+#pragma unroll
+  for (int m = 0; m < KS; ++m) {
+    win[m] = dy_at(t_begin + m);
+    qwin[m] = q_at(t_begin - (KS - 1) + m);
+  }
+  const bool is_q = c < d.Lq;
+  const int cj = is_q ? c : c - d.Lq, hh = cj / d.dh, o = cj % d.dh;
+  for (int t = t_begin; t < t_end; ++t) {
+    float gq = 0.f;
+#pragma unroll
+    for (int j = 0; j < KS; ++j) gq = fmaf(w[j], win[KS - 1 - j], gq);
+#pragma unroll
+    for (int j = 0; j < KS; ++j) dw[j] = fmaf(win[0], qwin[j], dw[j]);
+    if (d.flags & F_QK_MEAN) {
+      const long long row = seq + t;
+      if (is_q) {
+        gq += 0.5f * (dqh[row * d.Lq + c] + dkh[row * d.Lk + (hh / d.g) * d.dh + o] / d.g);
+      } else {
+        float sg = dkh[row * d.Lk + cj];
+        for (int m = 0; m < d.g; ++m) sg += dqh[row * d.Lq + (hh * d.g + m) * d.dh + o];
+        gq += 0.5f * sg;
+      }
+    }
+    dlat[(seq + t) * ld + c] = __float2bfloat16(gq);
+#pragma unroll
+    for (int m = 0; m < KS - 1; ++m) {
+      win[m] = win[m + 1];
+      qwin[m] = qwin[m + 1];
+    }
+    win[KS - 1] = dy_at(t + KS);
+    qwin[KS - 1] = q_at(t + 1);
+  }
+  if (conv1)
+#pragma unroll
+    for (int j = 0; j < KS; ++j) atomicAdd(d_w0 + c * KS + j, dw[j]);
+}
+
 __global__ void rope_table_kernel(float2* tab, int S, int half, double log2_base) {
   long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (long long)S * half) return;
@@ -526,5 +588,16 @@ cudaError_t launch_transform_bwd_w1(const CcaDims& d, const float* qk0, const bf
 cudaError_t launch_pack_dv(const CcaDims& d, const float* dv, bf16* dlat, long long ld_dlat, cudaStream_t st) {
   long long total = (long long)d.B * d.S * d.Lk;
   pack_dv_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(d, dv, dlat, ld_dlat);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_conv1_adjoint(const CcaDims& d, const float* dy1, const float* dqh, const float* dkh, const float* qk0,
+                                 const bf16* w0, bf16* dlat, long long ld_dlat, float* d_w0, cudaStream_t st) {
+  dim3 grid((d.L + 127) / 128, (d.S + CONV1_TOK - 1) / CONV1_TOK, d.B);
+  const int ks = (d.flags & F_CONV1) ? d.k_seq : 1;
+  if (ks == 1) conv1_adjoint_kernel<1><<<grid, 128, 0, st>>>(d, dy1, dqh, dkh, qk0, w0, dlat, ld_dlat, d_w0);
+  else if (ks == 2) conv1_adjoint_kernel<2><<<grid, 128, 0, st>>>(d, dy1, dqh, dkh, qk0, w0, dlat, ld_dlat, d_w0);
+  else if (ks == 3) conv1_adjoint_kernel<3><<<grid, 128, 0, st>>>(d, dy1, dqh, dkh, qk0, w0, dlat, ld_dlat, d_w0);
+  else conv1_adjoint_kernel<4><<<grid, 128, 0, st>>>(d, dy1, dqh, dkh, qk0, w0, dlat, ld_dlat, d_w0);
   return cudaGetLastError();
 }
