@@ -31,6 +31,7 @@ struct TcGemmParams {
   float* out_f32;
   long long ldc;
   int tiles_m, tiles_n, num_kb;
+  int splits, kb_per_split;   // split-K: work item = (tile, split); partial sums are added atomically (fp32 output)
   int a_mn, b_mn;
   int vec_ok;            // rows of C are 16-byte aligned: vector stores allowed
   int* status;
@@ -64,7 +65,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int num_tiles = p.tiles_m * p.tiles_n;
+  const int num_tiles = p.tiles_m * p.tiles_n * p.splits;      // work items
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < GEMM_STAGES; ++s) {
@@ -94,8 +95,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int stage = 0;
       uint32_t phase = 0;
       for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
-        const int m0 = (tile / p.tiles_n) * GEMM_BM, n0 = (tile % p.tiles_n) * BN;
-        for (int kb = 0; kb < p.num_kb; ++kb) {
+        const int sp = tile % p.splits, mn = tile / p.splits;
+        const int m0 = (mn / p.tiles_n) * GEMM_BM, n0 = (mn % p.tiles_n) * BN;
+        const int kb_end = min(p.num_kb, (sp + 1) * p.kb_per_split);
+        for (int kb = sp * p.kb_per_split; kb < kb_end; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
           unsigned char* sa = smem + stage * SM::STAGE_BYTES;
           unsigned char* sb = sa + SM::A_BYTES;
@@ -129,7 +132,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!mbar_wait(&acc_empty[as], aphase ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + as * BN;
-        for (int kb = 0; kb < p.num_kb; ++kb) {
+        const int sp = tile % p.splits;
+        const int kb_begin = sp * p.kb_per_split, kb_end = min(p.num_kb, kb_begin + p.kb_per_split);
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * SM::STAGE_BYTES);
@@ -138,7 +143,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int k = 0; k < GEMM_BK / 16; ++k) {
             const uint64_t da = p.a_mn ? smem_desc_sw128(sa + k * 2048, 8192, 1024) : smem_desc_sw128(sa + k * 32, 16, 1024);
             const uint64_t db = p.b_mn ? smem_desc_sw128(sb + k * 2048, 8192, 1024) : smem_desc_sw128(sb + k * 32, 16, 1024);
-            mma_ss(d_tmem, da, db, idesc, (kb | k) != 0);
+            mma_ss(d_tmem, da, db, idesc, ((kb - kb_begin) | k) != 0);
           }
           mma_commit(&empty_bar[stage]);
           if (++stage == GEMM_STAGES) { stage = 0; phase ^= 1; }
@@ -152,7 +157,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
       const int as = it & 1;
       const uint32_t aphase = (it >> 1) & 1;
-      const int m0 = (tile / p.tiles_n) * GEMM_BM, n0 = (tile % p.tiles_n) * BN;
+      const int mn = tile / p.splits;
+      const int m0 = (mn / p.tiles_n) * GEMM_BM, n0 = (mn % p.tiles_n) * BN;
       if (!mbar_wait(&acc_full[as], aphase, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
       tc_fence_after();
       const int m = m0 + q * 32 + lane;
@@ -191,7 +197,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           } else {
             float* dst = p.out_f32 + (long long)m * p.ldc + n;
-            if (p.vec_ok && n + 32 <= p.N) {
+            if (p.splits > 1) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (n + i < p.N) atomicAdd(dst + i, __uint_as_float(r[i]));
+            } else if (p.vec_ok && n + 32 <= p.N) {
 #pragma unroll
               for (int i = 0; i < 8; ++i)
                 reinterpret_cast<uint4*>(dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
@@ -299,12 +309,28 @@ int tc_gemm(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) {
   p.tiles_m = (g.M + GEMM_BM - 1) / GEMM_BM;
   p.tiles_n = (g.N + BN - 1) / BN;
   p.num_kb = (g.K + GEMM_BK - 1) / GEMM_BK;
+  // split-K when the output has too few tiles to fill the machine and the reduction is long (weight gradients)
+  p.splits = 1;
+  {
+    const int mn_tiles = p.tiles_m * p.tiles_n;
+    if (g.out_f32 && g.ldc == g.N && g.a_row_off == 0 && mn_tiles * 2 <= s->sm_count && p.num_kb >= 16) {
+      int sp = s->sm_count / mn_tiles;
+      if (sp > p.num_kb / 8) sp = p.num_kb / 8;
+      if (sp > 1) p.splits = sp;
+    }
+  }
+  p.kb_per_split = (p.num_kb + p.splits - 1) / p.splits;
+  p.splits = (p.num_kb + p.kb_per_split - 1) / p.kb_per_split;     // no empty split
+  if (p.splits > 1) {
+    cudaError_t me = cudaMemsetAsync(g.out_f32, 0, (size_t)g.M * g.N * sizeof(float), st);
+    if (me != cudaSuccess) return -(int)me;
+  }
   p.a_mn = a_mn; p.b_mn = b_mn;
   const void* outp = g.out_bf16 ? (const void*)g.out_bf16 : (const void*)g.out_f32;
   const int esz = g.out_bf16 ? 2 : 4;
   p.vec_ok = ((reinterpret_cast<uintptr_t>(outp) & 15) == 0) && ((g.ldc * esz) % 16 == 0);
   p.status = d_status;
-  const int tiles = p.tiles_m * p.tiles_n;
+  const int tiles = p.tiles_m * p.tiles_n * p.splits;
   const int grid = tiles < s->sm_count ? tiles : s->sm_count;
   cudaError_t e;
   if (BN == 256) {
