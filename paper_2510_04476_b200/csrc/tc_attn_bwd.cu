@@ -9,9 +9,11 @@
 //   tc_attn_bwd_dkv_kernel  one CTA = 128 keys of one (sequence, kv head), loops over the g query heads and
 //                           their query tiles.  It works on the transposed tiles S^T = K Q^T and
 //                           dP^T = V dO^T (thread = key), so that P^T and dS^T are the TMEM A operands of
-//                           dV += P^T dO and dK += dS^T Q and both accumulators stay in TMEM.
+//                           dV += P^T dO and dK += dS^T Q and both accumulators stay in TMEM.  A query tile is
+//                           handled as two 64-query sub-tiles in alternating TMEM buffers, so the MMAs of one
+//                           overlap the exponentials of the other.
 //
-// Both: warps 0-7 compute (two column halves x four TMEM lane quarters), warp 8 TMA loads, warp 9 issues
+// Both: warps 0-15 compute (four column groups x four TMEM lane quarters), warp 16 TMA loads, warp 17 issues
 // the MMAs (warp-uniform loop, one elected lane).  P and dS are bf16 MMA operands, everything else fp32.
 #include "tc_kernels.cuh"
 #include "tc_ptx.cuh"
@@ -21,7 +23,9 @@ using namespace tc;
 
 namespace {
 
-constexpr int BW_THREADS = 320, BW_TMA_WARP = 8, BW_MMA_WARP = 9;
+constexpr int BW_COMPUTE_WARPS = 16;       // four warps per scheduler: the per-element chains are latency-bound
+constexpr int BW_TMA_WARP = BW_COMPUTE_WARPS, BW_MMA_WARP = BW_COMPUTE_WARPS + 1;
+constexpr int BW_THREADS = 32 * (BW_COMPUTE_WARPS + 2);
 constexpr float LOG2E_F = 1.4426950408889634f;
 
 struct BwdParams {
@@ -41,9 +45,9 @@ struct BwdSmem {
   static constexpr int FIX_OFF = 0;                    // two tiles loaded once
   static constexpr int RING_OFF = 2 * TILE;            // two rings of two tiles
   static constexpr int BAR_OFF = 6 * TILE;
-  static constexpr int STAT_OFF = BAR_OFF + 256;       // float [2 buffers][2][128]
+  static constexpr int STAT_OFF = BAR_OFF + 256;       // float [2 groups][2 buffers][2][128]
   // at least 120 KB so that two CTAs (each wanting all 512 TMEM columns) never share an SM
-  static constexpr int TOTAL = (STAT_OFF + 2048 + 1024) > 122880 ? (STAT_OFF + 2048 + 1024) : 122880;
+  static constexpr int TOTAL = (STAT_OFF + 4096 + 1024) > 122880 ? (STAT_OFF + 4096 + 1024) : 122880;
 };
 
 TC_DEVINL void fail(volatile int* abort_flag, int* status, int code) {
@@ -70,14 +74,14 @@ TC_DEVINL void mma_kk(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi
     mma_ss_w(d_tmem, a_lo + off, hi, b_lo + off, hi, idesc, kk != 0);
   }
 }
-// C[128 x DH] (+)= A[128 x 128] B, A = bf16 pairs in TMEM (pieces at columns [0,32) and [64,96) of a_tmem),
+// C[128 x DH] (+)= A[128 x 128] B, A = bf16 pairs in TMEM (32 keys in 16 columns at every 32nd column of a_tmem),
 // B = a [128 rows][DH] tile in shared memory read along its rows (MN-major)
 template <int DH>
 TC_DEVINL void mma_tm(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t accumulate) {
   const uint32_t idesc = idesc_bf16(DH, 0, 1);
 #pragma unroll
   for (int kk = 0; kk < 8; ++kk)
-    mma_ts_w(d_tmem, a_tmem + (kk >> 2) * 64 + (kk & 3) * 8, b_lo + kk * (2048 >> 4), hi, idesc, (accumulate | kk) != 0);
+    mma_ts_w(d_tmem, a_tmem + (kk >> 1) * 32 + (kk & 1) * 8, b_lo + kk * (2048 >> 4), hi, idesc, (accumulate | kk) != 0);
 }
 
 template <int DH>
@@ -106,7 +110,7 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint64_t* v_empty = bars + 7;       // [2]
   uint64_t* s_full = bars + 9;        // [2] MMA -> compute: S buffer ready
   uint64_t* dp_full = bars + 11;      // MMA -> compute: dP ready
-  uint64_t* ds_full = bars + 12;      // compute -> MMA: dS written, dP consumed (256 arrivals)
+  uint64_t* ds_full = bars + 12;      // compute -> MMA: dS written, dP consumed (all compute threads)
   uint64_t* dq_done = bars + 13;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -130,7 +134,7 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mbar_init(&s_full[i], 1);
     }
     mbar_init(dp_full, 1);
-    mbar_init(ds_full, 256);
+    mbar_init(ds_full, 32 * BW_COMPUTE_WARPS);
     mbar_init(dq_done, 1);
     *abort_flag = 0;
     fence_barrier_init();
@@ -219,7 +223,7 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     if (leader) mma_commit(dq_done);
   } else {
     // ------------------------------------------------------------------ compute, thread = query row
-    const int part = (warp >> 2) & 1;
+    const int part = warp >> 2;                        // which 32 keys of each KV tile
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
     const int tq = m0 + row;
@@ -228,31 +232,32 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const float l2 = tq < p.S ? p.lse[stat_idx] * LOG2E_F : INFINITY;     // rows past the end: P = 0
     const float dl = tq < p.S ? p.delta[stat_idx] : 0.f;
     for (int j = 0; j < n_kv; ++j) {
-      const uint32_t s_t = tmem_base + lane_sel + (j & 1) * 128 + part * 64;
-      const uint32_t dp_t = tmem_base + lane_sel + 256 + part * 64;
+      const uint32_t s_t = tmem_base + lane_sel + (j & 1) * 128 + part * 32;
+      const uint32_t dp_t = tmem_base + lane_sel + 256 + part * 32;
       if (!mbar_wait(&s_full[j & 1], (j >> 1) & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
       if (!mbar_wait(dp_full, j & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
       tc_fence_after();
-      const int k0 = j * 128 + part * 64;
+      const int k0 = j * 128 + part * 32;
       const bool need_mask = (p.causal && j * 128 + 127 > m0) || (j * 128 + 128 > p.S);
       const int lim = p.causal ? min(tq, p.S - 1) : p.S - 1;
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
-        uint32_t sv[32], dv[32], pk[16];
-        tmem_ld32(s_t + hf * 32, sv);
-        tmem_ld32(dp_t + hf * 32, dv);
+        uint32_t sv[16], dv[16], pk[8];
+        tmem_ld16(s_t + hf * 16, sv);
+        tmem_ld16(dp_t + hf * 16, dv);
         tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
+        for (int c = 0; c < 8; ++c) {
           float p0 = ex2f(fmaf(__uint_as_float(sv[2 * c]), c_scale, -l2));
           float p1 = ex2f(fmaf(__uint_as_float(sv[2 * c + 1]), c_scale, -l2));
           if (need_mask) {
-            if (k0 + hf * 32 + 2 * c > lim) p0 = 0.f;
-            if (k0 + hf * 32 + 2 * c + 1 > lim) p1 = 0.f;
+            if (k0 + hf * 16 + 2 * c > lim) p0 = 0.f;
+            if (k0 + hf * 16 + 2 * c + 1 > lim) p1 = 0.f;
           }
           pk[c] = pack_bf16(p0 * (__uint_as_float(dv[2 * c]) - dl), p1 * (__uint_as_float(dv[2 * c + 1]) - dl));
         }
-        tmem_st16(s_t + hf * 16, pk);                 // dS over columns this thread has read
+        // dS (bf16 pairs) over columns this thread has read: keys 32 part + [0,32) -> columns 32 part + [0,16)
+        tmem_st8(s_t + hf * 8, pk);
       }
       tmem_st_wait();
       tc_fence_before();
@@ -264,14 +269,14 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       const float scale = rsqrtf((float)DH);
 #pragma unroll 1
       for (int c = 0; c < DH / 64; ++c) {
-        uint32_t t[32];
-        const int col = part * (DH / 2) + c * 32;
-        tmem_ld32(tmem_base + lane_sel + 384 + col, t);
+        uint32_t t[16];
+        const int col = part * (DH / 4) + c * 16;
+        tmem_ld16(tmem_base + lane_sel + 384 + col, t);
         tmem_ld_wait();
         if (tq < p.S) {
           float* dst = p.dq + ((long long)b * p.S + tq) * p.Lq + hi * DH + col;
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
+          for (int i = 0; i < 4; ++i)
             reinterpret_cast<float4*>(dst)[i] =
                 make_float4(__uint_as_float(t[4 * i]) * scale, __uint_as_float(t[4 * i + 1]) * scale,
                             __uint_as_float(t[4 * i + 2]) * scale, __uint_as_float(t[4 * i + 3]) * scale);
@@ -311,11 +316,11 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   uint64_t* kv_full = bars;
   uint64_t* qdo_full = bars + 1;      // [2]
   uint64_t* qdo_empty = bars + 3;     // [2]
-  uint64_t* sdp_full = bars + 5;      // MMA -> compute: S^T and dP^T ready
-  uint64_t* pds_full = bars + 6;      // compute -> MMA: P^T and dS^T written (256 arrivals)
-  uint64_t* acc_done = bars + 7;
-  uint64_t* stat_ready = bars + 8;    // compute threads: column statistics of the tile are in shared memory
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 9);
+  uint64_t* sdp_full = bars + 5;      // [2] MMA -> compute: S^T and dP^T of a 64-query sub-tile ready
+  uint64_t* pds_full = bars + 7;      // [2] compute group -> MMA: P^T and dS^T written (256 arrivals)
+  uint64_t* acc_done = bars + 9;
+  uint64_t* stat_ready = bars + 10;   // [2] per compute group: column statistics of the tile are in shared memory
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -335,10 +340,13 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       mbar_init(&qdo_full[i], 1);
       mbar_init(&qdo_empty[i], 1);
     }
-    mbar_init(sdp_full, 1);
-    mbar_init(pds_full, 256);
+    mbar_init(&sdp_full[0], 1);
+    mbar_init(&sdp_full[1], 1);
+    mbar_init(&pds_full[0], 256);
+    mbar_init(&pds_full[1], 256);
     mbar_init(acc_done, 1);
-    mbar_init(stat_ready, 256);
+    mbar_init(&stat_ready[0], 256);
+    mbar_init(&stat_ready[1], 256);
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmQ);
@@ -354,7 +362,8 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // TMEM columns: S^T [0,128) dP^T [128,256) dV [256,256+DH) dK [384,384+DH)
+  // TMEM columns: S^T two 64-query buffers [0,64) [64,128), dP^T likewise [128,192) [192,256),
+  // dV [256,256+DH), dK [384,384+DH)
 
   if (warp == BW_TMA_WARP) {
     if (lane == 0) {
@@ -372,43 +381,85 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
     }
   } else if (warp == BW_MMA_WARP) {
+    // Sub-tile = 64 queries; S^T / dP^T of sub-tile s live in TMEM buffer s & 1, so the MMAs of sub-tile s + 1
+    // run while the compute warps work on sub-tile s.
     const bool leader = elect_one();
     const uint32_t hi_w = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
     const uint32_t k_lo = lo_kmajor(smem_u32(sK)), v_lo = lo_kmajor(smem_u32(sV));
     const uint32_t q_lo = lo_kmajor(smem_u32(sQ)), do_lo = lo_kmajor(smem_u32(sDO));
     const uint32_t q_mn = lo_mnmajor(smem_u32(sQ)), do_mn = lo_mnmajor(smem_u32(sDO));
     constexpr uint32_t TILE16 = SM::TILE >> 4;
+    constexpr uint32_t HALF16 = (64 * 128) >> 4;       // 64 query rows further down a tile
+    const int n_sub = 2 * n_it;
     auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
       return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
     };
-    if (!wait_all(kv_full, 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
-    for (int it = 0; it < n_it; ++it) {
-      const int st = it & 1;
-      if (!wait_all(&qdo_full[st], (it >> 1) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
-      tc_fence_after();
+    auto issue_sdp = [&](int sub) {     // S^T = K Q^T and dP^T = V dO^T for 64 queries
+      const int it = sub >> 1, st = it & 1, hf = sub & 1, sb = sub & 1;
+      const uint32_t idesc = idesc_bf16(64, 0, 0);
+      const uint32_t qb = q_lo + st * TILE16 + hf * HALF16, ob = do_lo + st * TILE16 + hf * HALF16;
       if (leader) {
-        // the MMAs that read P^T / dS^T of the previous tile from these columns were issued before (in order)
-        mma_kk<DH>(tmem_base, k_lo, q_lo + st * TILE16, hi_w);               // S^T = K Q^T
-        mma_kk<DH>(tmem_base + 128, v_lo, do_lo + st * TILE16, hi_w);        // dP^T = V dO^T
-        mma_commit(sdp_full);
+#pragma unroll
+        for (int kk = 0; kk < DH / 16; ++kk) {
+          const uint32_t off = (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+          mma_ss_w(tmem_base + sb * 64, k_lo + off, hi_w, qb + off, hi_w, idesc, kk != 0);
+        }
+#pragma unroll
+        for (int kk = 0; kk < DH / 16; ++kk) {
+          const uint32_t off = (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+          mma_ss_w(tmem_base + 128 + sb * 64, v_lo + off, hi_w, ob + off, hi_w, idesc, kk != 0);
+        }
+        mma_commit(&sdp_full[sb]);
       }
-      if (!wait_all(pds_full, it & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
-      tc_fence_after();
+    };
+    auto issue_dvdk = [&](int sub) {    // dV += P^T dO, dK += dS^T Q over the sub-tile's 64 queries
+      const int it = sub >> 1, st = it & 1, hf = sub & 1, sb = sub & 1;
+      const uint32_t idesc = idesc_bf16(DH, 0, 1);
+      const uint32_t ob = do_mn + st * TILE16 + hf * HALF16, qb = q_mn + st * TILE16 + hf * HALF16;
       if (leader) {
-        mma_tm<DH>(tmem_base + 256, tmem_base, do_mn + st * TILE16, hi_w, it != 0);        // dV += P^T dO
-        mma_tm<DH>(tmem_base + 384, tmem_base + 128, q_mn + st * TILE16, hi_w, it != 0);   // dK += dS^T Q
-        mma_commit(&qdo_empty[st]);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          mma_ts_w(tmem_base + 256, tmem_base + sb * 64 + (kk >> 1) * 32 + (kk & 1) * 8, ob + kk * (2048 >> 4), hi_w, idesc,
+                   (sub | kk) != 0);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          mma_ts_w(tmem_base + 384, tmem_base + 128 + sb * 64 + (kk >> 1) * 32 + (kk & 1) * 8, qb + kk * (2048 >> 4), hi_w,
+                   idesc, (sub | kk) != 0);
+        if (hf == 1) mma_commit(&qdo_empty[st]);
+      }
+    };
+    if (!wait_all(kv_full, 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+    if (!wait_all(&qdo_full[0], 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+    tc_fence_after();
+    issue_sdp(0);
+    issue_sdp(1);
+    for (int sub = 0; sub < n_sub; ++sub) {
+      // sub-tile sub belongs to compute group sub & 1
+      if (!wait_all(&pds_full[sub & 1], (sub >> 1) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+      tc_fence_after();
+      issue_dvdk(sub);
+      if (sub + 2 < n_sub) {
+        const int nit = (sub + 2) >> 1;
+        if ((sub & 1) == 0) {
+          if (!wait_all(&qdo_full[nit & 1], (nit >> 1) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+          tc_fence_after();
+        }
+        issue_sdp(sub + 2);        // into the buffer whose P^T / dS^T the MMAs just issued are reading (in order)
       }
     }
     if (leader) mma_commit(acc_done);
   } else {
     // ------------------------------------------------------------------ compute, thread = key
-    const int part = (warp >> 2) & 1;
+    // Two groups of eight warps: group gsel works on the sub-tiles with (sub & 1) == gsel, i.e. on queries
+    // [64 gsel, 64 gsel + 64) of every query tile, in TMEM buffer gsel.
+    const int gsel = warp >> 3;
+    const int part = (warp >> 2) & 1;                  // which 32 of the sub-tile's 64 queries
     const int row = (warp & 3) * 32 + lane;
-    const int ct = threadIdx.x;                        // 0..255
+    const int ct = threadIdx.x & 255;                  // index inside the group
     const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
     const int tk = n0 + row;
     const float c_scale = rsqrtf((float)DH) * LOG2E_F;
+    float* gstat = stat + gsel * 512;                  // [2 buffers][lse2 | delta][128 queries] of this group
     // column statistics of a query tile: thread ct < 128 fetches lse * log2(e) of query ct, the others delta;
     // queries past the end of the sequence get lse = +inf, so their P is 0
     auto fetch_stat = [&](int it) -> float {
@@ -419,36 +470,37 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       return tq < p.S ? p.delta[idx] : 0.f;
     };
     float next_stat = n_it > 0 ? fetch_stat(0) : 0.f;
+    const uint32_t s_t = tmem_base + lane_sel + gsel * 64 + part * 32;
+    const uint32_t dp_t = tmem_base + lane_sel + 128 + gsel * 64 + part * 32;
+    const int qoff = gsel * 64 + part * 32;            // first query (within the tile) of this thread's columns
     for (int it = 0; it < n_it; ++it) {
-      const int sb = it & 1;
-      stat[sb * 256 + ct] = next_stat;                 // buffer sb was last read two tiles ago
+      const int stb = it & 1;
+      gstat[stb * 256 + ct] = next_stat;               // buffer stb was last read two tiles ago
       if (it + 1 < n_it) next_stat = fetch_stat(it + 1);
-      mbar_arrive(stat_ready);
-      if (!mbar_wait(stat_ready, it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+      mbar_arrive(&stat_ready[gsel]);
+      if (!mbar_wait(&stat_ready[gsel], it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
       const int m0 = (i0 + it % n_q) * 128;
       const bool diag = p.causal && m0 == n0;
-      if (!mbar_wait(sdp_full, it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+      if (!mbar_wait(&sdp_full[gsel], it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
       tc_fence_after();
-      const uint32_t s_t = tmem_base + lane_sel + part * 64;
-      const uint32_t dp_t = tmem_base + lane_sel + 128 + part * 64;
-      const float4* l2v = reinterpret_cast<const float4*>(stat + sb * 256 + part * 64);
-      const float4* dlv = reinterpret_cast<const float4*>(stat + sb * 256 + 128 + part * 64);
+      const float4* l2v = reinterpret_cast<const float4*>(gstat + stb * 256 + qoff);
+      const float4* dlv = reinterpret_cast<const float4*>(gstat + stb * 256 + 128 + qoff);
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
-        uint32_t sv[32], dv[32], pk[16], dk_[16];
-        tmem_ld32(s_t + hf * 32, sv);
-        tmem_ld32(dp_t + hf * 32, dv);
+        uint32_t sv[16], dv[16], pk[8], dk_[8];
+        tmem_ld16(s_t + hf * 16, sv);
+        tmem_ld16(dp_t + hf * 16, dv);
         tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const float4 l2 = l2v[hf * 8 + c], dl = dlv[hf * 8 + c];
+        for (int c = 0; c < 4; ++c) {
+          const float4 l2 = l2v[hf * 4 + c], dl = dlv[hf * 4 + c];
           float pr[4];
           pr[0] = ex2f(fmaf(__uint_as_float(sv[4 * c + 0]), c_scale, -l2.x));
           pr[1] = ex2f(fmaf(__uint_as_float(sv[4 * c + 1]), c_scale, -l2.y));
           pr[2] = ex2f(fmaf(__uint_as_float(sv[4 * c + 2]), c_scale, -l2.z));
           pr[3] = ex2f(fmaf(__uint_as_float(sv[4 * c + 3]), c_scale, -l2.w));
           if (diag) {
-            const int q0 = m0 + part * 64 + hf * 32 + 4 * c;      // query of pr[0]
+            const int q0 = m0 + qoff + hf * 16 + 4 * c;      // query of pr[0]
 #pragma unroll
             for (int e = 0; e < 4; ++e)
               if (tk > q0 + e) pr[e] = 0.f;
@@ -458,12 +510,12 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           dk_[2 * c] = pack_bf16(pr[0] * (__uint_as_float(dv[4 * c + 0]) - dl.x), pr[1] * (__uint_as_float(dv[4 * c + 1]) - dl.y));
           dk_[2 * c + 1] = pack_bf16(pr[2] * (__uint_as_float(dv[4 * c + 2]) - dl.z), pr[3] * (__uint_as_float(dv[4 * c + 3]) - dl.w));
         }
-        tmem_st16(s_t + hf * 16, pk);                  // P^T over S^T columns this thread has read
-        tmem_st16(dp_t + hf * 16, dk_);                // dS^T over dP^T columns this thread has read
+        tmem_st8(s_t + hf * 8, pk);                    // P^T over S^T columns this thread has read
+        tmem_st8(dp_t + hf * 8, dk_);                  // dS^T over dP^T columns this thread has read
       }
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(pds_full);
+      mbar_arrive(&pds_full[gsel]);
     }
     if (!mbar_wait(acc_done, 0, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
     tc_fence_after();
@@ -471,15 +523,15 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const float scale = rsqrtf((float)DH);
 #pragma unroll 1
       for (int c = 0; c < DH / 64; ++c) {
-        uint32_t t[32], u[32];
-        const int col = part * (DH / 2) + c * 32;
-        tmem_ld32(tmem_base + lane_sel + 256 + col, t);
-        tmem_ld32(tmem_base + lane_sel + 384 + col, u);
+        uint32_t t[16], u[16];
+        const int col = (gsel * 2 + part) * (DH / 4) + c * 16;
+        tmem_ld16(tmem_base + lane_sel + 256 + col, t);
+        tmem_ld16(tmem_base + lane_sel + 384 + col, u);
         tmem_ld_wait();
         if (tk < p.S) {
           const long long off = ((long long)b * p.S + tk) * p.Lk + hj * DH + col;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
+          for (int i = 0; i < 4; ++i) {
             reinterpret_cast<float4*>(p.dv + off)[i] = make_float4(__uint_as_float(t[4 * i]), __uint_as_float(t[4 * i + 1]),
                                                                     __uint_as_float(t[4 * i + 2]), __uint_as_float(t[4 * i + 3]));
             reinterpret_cast<float4*>(p.dk + off)[i] =
