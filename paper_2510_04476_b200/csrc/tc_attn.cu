@@ -74,47 +74,6 @@ TC_DEVINL uint64_t kmajor_desc(uint32_t tile_addr, int kk) {
 TC_DEVINL uint64_t v_desc(uint32_t tile_addr, int kk) { return smem_desc_sw128(tile_addr + kk * 2048, 16384, 1024); }
 
 
-// ---- packed fp32 pairs (one 64-bit register = two floats) ----
-TC_DEVINL uint64_t pack2u(uint32_t lo, uint32_t hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
-  return r;
-}
-TC_DEVINL uint64_t pack2f(float lo, float hi) { return pack2u(__float_as_uint(lo), __float_as_uint(hi)); }
-TC_DEVINL void unpack2u(uint64_t v, uint32_t& lo, uint32_t& hi) { asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v)); }
-TC_DEVINL uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t r;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-  return r;
-}
-TC_DEVINL uint64_t add2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-TC_DEVINL float ex2f(float x) {
-  float r;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-  return r;
-}
-// 2^x for a pair, x in [-120, 8], on the FMA and integer pipes: n = round(x) from the magic-number add,
-// f = x - n in [-1/2, 1/2], 2^f by a cubic (minimax in relative error), then n is added to the exponent.
-TC_DEVINL uint64_t exp2_poly2(uint64_t x) {
-  const uint64_t magic = pack2f(12582912.f, 12582912.f), neg_magic = pack2f(-12582912.f, -12582912.f);
-  const uint64_t neg1 = pack2f(-1.f, -1.f);
-  const uint64_t c3 = pack2f(0.0551716685f, 0.0551716685f), c2 = pack2f(0.242611125f, 0.242611125f);
-  const uint64_t c1 = pack2f(0.693260968f, 0.693260968f), c0 = pack2f(0.999928057f, 0.999928057f);
-  const uint64_t t = add2(x, magic);
-  const uint64_t n = add2(t, neg_magic);
-  const uint64_t f = fma2(n, neg1, x);
-  uint64_t pl = fma2(c3, f, c2);
-  pl = fma2(pl, f, c1);
-  pl = fma2(pl, f, c0);
-  uint32_t t0, t1, p0, p1;
-  unpack2u(t, t0, t1);
-  unpack2u(pl, p0, p1);
-  return pack2u(p0 + (t0 << 23), p1 + (t1 << 23));
-}
 // Exponentials of 8 consecutive scores (already in registers) -> 4 packed bf16 pairs; adds the rounded
 // values to the two running partial sums in `sum2`.  POLY of the 4 pairs go through the
 // polynomial.  CLAMP: x may be far below the smallest exponent (online mode); then it is clamped first.

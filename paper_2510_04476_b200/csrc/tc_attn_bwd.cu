@@ -54,10 +54,19 @@ TC_DEVINL void fail(volatile int* abort_flag, int* status, int code) {
   *abort_flag = 1;
   atomicCAS(status, 0, code);
 }
-TC_DEVINL float ex2f(float x) {
-  float r;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-  return r;
+
+// 2^x for a pair: on the FMA pipe (clamped to the polynomial's range) or on the transcendental unit
+template <bool POLY>
+TC_DEVINL uint64_t exp2_pair(uint64_t x) {
+  uint32_t a, b;
+  unpack2u(x, a, b);
+  if (POLY) return exp2_poly2(pack2f(fmaxf(__uint_as_float(a), -120.f), fmaxf(__uint_as_float(b), -120.f)));
+  return pack2f(ex2f(__uint_as_float(a)), ex2f(__uint_as_float(b)));
+}
+TC_DEVINL uint32_t cvt_bf16x2(uint64_t v) {
+  uint32_t a, b;
+  unpack2u(v, a, b);
+  return pack_bf16(__uint_as_float(a), __uint_as_float(b));
 }
 
 // descriptor low words (address >> 4 | leading offset << 16) and the common high word
@@ -91,7 +100,7 @@ TC_DEVINL void tma_tile(unsigned char* dst, const CUtensorMap* map, int c0, int 
 }
 
 // ------------------------------------------------------------------------------------------ dQ
-template <int DH>
+template <int DH, int POLY>
 __global__ void __launch_bounds__(BW_THREADS, 1)
 tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                       const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO, BwdParams p) {
@@ -231,6 +240,7 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const long long stat_idx = ((long long)b * p.hq + hi) * p.S + tq;
     const float l2 = tq < p.S ? p.lse[stat_idx] * LOG2E_F : INFINITY;     // rows past the end: P = 0
     const float dl = tq < p.S ? p.delta[stat_idx] : 0.f;
+    const uint64_t scale2 = pack2f(c_scale, c_scale), nl2 = pack2f(-l2, -l2), ndl2 = pack2f(-dl, -dl);
     for (int j = 0; j < n_kv; ++j) {
       const uint32_t s_t = tmem_base + lane_sel + (j & 1) * 128 + part * 32;
       const uint32_t dp_t = tmem_base + lane_sel + 256 + part * 32;
@@ -248,13 +258,16 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         tmem_ld_wait();
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-          float p0 = ex2f(fmaf(__uint_as_float(sv[2 * c]), c_scale, -l2));
-          float p1 = ex2f(fmaf(__uint_as_float(sv[2 * c + 1]), c_scale, -l2));
+          const uint64_t x = fma2(pack2u(sv[2 * c], sv[2 * c + 1]), scale2, nl2);
+          uint64_t e = (c & 3) < POLY ? exp2_pair<true>(x) : exp2_pair<false>(x);
           if (need_mask) {
-            if (k0 + hf * 16 + 2 * c > lim) p0 = 0.f;
-            if (k0 + hf * 16 + 2 * c + 1 > lim) p1 = 0.f;
+            uint32_t a, bb;
+            unpack2u(e, a, bb);
+            if (k0 + hf * 16 + 2 * c > lim) a = 0u;
+            if (k0 + hf * 16 + 2 * c + 1 > lim) bb = 0u;
+            e = pack2u(a, bb);
           }
-          pk[c] = pack_bf16(p0 * (__uint_as_float(dv[2 * c]) - dl), p1 * (__uint_as_float(dv[2 * c + 1]) - dl));
+          pk[c] = cvt_bf16x2(mul2(e, add2(pack2u(dv[2 * c], dv[2 * c + 1]), ndl2)));
         }
         // dS (bf16 pairs) over columns this thread has read: keys 32 part + [0,32) -> columns 32 part + [0,16)
         tmem_st8(s_t + hf * 8, pk);
@@ -300,7 +313,7 @@ done:
 }
 
 // ------------------------------------------------------------------------------------------ dK, dV
-template <int DH>
+template <int DH, int POLY>
 __global__ void __launch_bounds__(BW_THREADS, 1)
 tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO, BwdParams p) {
@@ -460,16 +473,17 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const int tk = n0 + row;
     const float c_scale = rsqrtf((float)DH) * LOG2E_F;
     float* gstat = stat + gsel * 512;                  // [2 buffers][lse2 | delta][128 queries] of this group
-    // column statistics of a query tile: thread ct < 128 fetches lse * log2(e) of query ct, the others delta;
-    // queries past the end of the sequence get lse = +inf, so their P is 0
+    // column statistics of a query tile, negated: thread ct < 128 fetches -lse * log2(e) of query ct, the others
+    // -delta; queries past the end of the sequence get -inf, so their P is 0
     auto fetch_stat = [&](int it) -> float {
       const int hi = hj * p.g + it / n_q, m0 = (i0 + it % n_q) * 128;
       const int tq = m0 + (ct & 127);
       const long long idx = ((long long)b * p.hq + hi) * p.S + tq;
-      if (ct < 128) return tq < p.S ? p.lse[idx] * LOG2E_F : INFINITY;
-      return tq < p.S ? p.delta[idx] : 0.f;
+      if (ct < 128) return tq < p.S ? -p.lse[idx] * LOG2E_F : -INFINITY;
+      return tq < p.S ? -p.delta[idx] : 0.f;
     };
     float next_stat = n_it > 0 ? fetch_stat(0) : 0.f;
+    const uint64_t scale2 = pack2f(c_scale, c_scale);
     const uint32_t s_t = tmem_base + lane_sel + gsel * 64 + part * 32;
     const uint32_t dp_t = tmem_base + lane_sel + 128 + gsel * 64 + part * 32;
     const int qoff = gsel * 64 + part * 32;            // first query (within the tile) of this thread's columns
@@ -483,8 +497,8 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const bool diag = p.causal && m0 == n0;
       if (!mbar_wait(&sdp_full[gsel], it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
       tc_fence_after();
-      const float4* l2v = reinterpret_cast<const float4*>(gstat + stb * 256 + qoff);
-      const float4* dlv = reinterpret_cast<const float4*>(gstat + stb * 256 + 128 + qoff);
+      const ulonglong2* nlv = reinterpret_cast<const ulonglong2*>(gstat + stb * 256 + qoff);        // pairs of -lse2
+      const ulonglong2* ndv = reinterpret_cast<const ulonglong2*>(gstat + stb * 256 + 128 + qoff);  // pairs of -delta
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
         uint32_t sv[16], dv[16], pk[8], dk_[8];
@@ -493,22 +507,27 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tmem_ld_wait();
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          const float4 l2 = l2v[hf * 4 + c], dl = dlv[hf * 4 + c];
-          float pr[4];
-          pr[0] = ex2f(fmaf(__uint_as_float(sv[4 * c + 0]), c_scale, -l2.x));
-          pr[1] = ex2f(fmaf(__uint_as_float(sv[4 * c + 1]), c_scale, -l2.y));
-          pr[2] = ex2f(fmaf(__uint_as_float(sv[4 * c + 2]), c_scale, -l2.z));
-          pr[3] = ex2f(fmaf(__uint_as_float(sv[4 * c + 3]), c_scale, -l2.w));
+          const ulonglong2 nl = nlv[hf * 4 + c], nd = ndv[hf * 4 + c];
+          uint64_t e0 = fma2(pack2u(sv[4 * c + 0], sv[4 * c + 1]), scale2, nl.x);
+          uint64_t e1 = fma2(pack2u(sv[4 * c + 2], sv[4 * c + 3]), scale2, nl.y);
+          e0 = (2 * c & 3) < POLY ? exp2_pair<true>(e0) : exp2_pair<false>(e0);
+          e1 = ((2 * c + 1) & 3) < POLY ? exp2_pair<true>(e1) : exp2_pair<false>(e1);
           if (diag) {
-            const int q0 = m0 + qoff + hf * 16 + 4 * c;      // query of pr[0]
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-              if (tk > q0 + e) pr[e] = 0.f;
+            const int q0 = m0 + qoff + hf * 16 + 4 * c;      // query of the first of the four
+            uint32_t a0, a1, a2, a3;
+            unpack2u(e0, a0, a1);
+            unpack2u(e1, a2, a3);
+            if (tk > q0) a0 = 0u;
+            if (tk > q0 + 1) a1 = 0u;
+            if (tk > q0 + 2) a2 = 0u;
+            if (tk > q0 + 3) a3 = 0u;
+            e0 = pack2u(a0, a1);
+            e1 = pack2u(a2, a3);
           }
-          pk[2 * c] = pack_bf16(pr[0], pr[1]);
-          pk[2 * c + 1] = pack_bf16(pr[2], pr[3]);
-          dk_[2 * c] = pack_bf16(pr[0] * (__uint_as_float(dv[4 * c + 0]) - dl.x), pr[1] * (__uint_as_float(dv[4 * c + 1]) - dl.y));
-          dk_[2 * c + 1] = pack_bf16(pr[2] * (__uint_as_float(dv[4 * c + 2]) - dl.z), pr[3] * (__uint_as_float(dv[4 * c + 3]) - dl.w));
+          pk[2 * c] = cvt_bf16x2(e0);
+          pk[2 * c + 1] = cvt_bf16x2(e1);
+          dk_[2 * c] = cvt_bf16x2(mul2(e0, add2(pack2u(dv[4 * c + 0], dv[4 * c + 1]), nd.x)));
+          dk_[2 * c + 1] = cvt_bf16x2(mul2(e1, add2(pack2u(dv[4 * c + 2], dv[4 * c + 3]), nd.y)));
         }
         tmem_st8(s_t + hf * 8, pk);                    // P^T over S^T columns this thread has read
         tmem_st8(dp_t + hf * 8, dk_);                  // dS^T over dP^T columns this thread has read
@@ -557,23 +576,23 @@ done:
   }
 }
 
-template <int DH>
+template <int DH, int POLY>
 int launch_bwd(TcState* s, const CcaDims& d, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                const CUtensorMap& tmDO, const BwdParams& p, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tc_attn_bwd_dq_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<DH>::TOTAL);
+    cudaError_t e = cudaFuncSetAttribute(tc_attn_bwd_dq_kernel<DH, POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<DH>::TOTAL);
     if (e != cudaSuccess) return -(int)e;
-    e = cudaFuncSetAttribute(tc_attn_bwd_dkv_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<DH>::TOTAL);
+    e = cudaFuncSetAttribute(tc_attn_bwd_dkv_kernel<DH, POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<DH>::TOTAL);
     if (e != cudaSuccess) return -(int)e;
     attr_set = true;
   }
   const long long g_kv = (long long)p.n_tiles * d.B * d.hk, g_q = (long long)p.n_tiles * d.B * d.hq;
   if (g_q > 0x7fffffffLL) return 1;
-  tc_attn_bwd_dkv_kernel<DH><<<(unsigned)g_kv, BW_THREADS, BwdSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, tmDO, p);
+  tc_attn_bwd_dkv_kernel<DH, POLY><<<(unsigned)g_kv, BW_THREADS, BwdSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, tmDO, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return -(int)e;
-  tc_attn_bwd_dq_kernel<DH><<<(unsigned)g_q, BW_THREADS, BwdSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, tmDO, p);
+  tc_attn_bwd_dq_kernel<DH, POLY><<<(unsigned)g_q, BW_THREADS, BwdSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, tmDO, p);
   e = cudaGetLastError();
   return e == cudaSuccess ? 0 : -(int)e;
 }
@@ -597,6 +616,13 @@ int tc_attn_bwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, cons
   p.lse = lse; p.delta = delta; p.dq = dq; p.dk = dk; p.dv = dv;
   p.n_tiles = (d.S + 127) / 128;
   p.status = d_status;
-  if (d.dh == 128) return launch_bwd<128>(s, d, tmQ, tmK, tmV, tmDO, p, st);
-  return launch_bwd<64>(s, d, tmQ, tmK, tmV, tmDO, p, st);
+  const int poly = s->attn_poly_bwd;
+  if (d.dh == 128) {
+    if (poly == 0) return launch_bwd<128, 0>(s, d, tmQ, tmK, tmV, tmDO, p, st);
+    if (poly == 2) return launch_bwd<128, 2>(s, d, tmQ, tmK, tmV, tmDO, p, st);
+    return launch_bwd<128, 1>(s, d, tmQ, tmK, tmV, tmDO, p, st);
+  }
+  if (poly == 0) return launch_bwd<64, 0>(s, d, tmQ, tmK, tmV, tmDO, p, st);
+  if (poly == 2) return launch_bwd<64, 2>(s, d, tmQ, tmK, tmV, tmDO, p, st);
+  return launch_bwd<64, 1>(s, d, tmQ, tmK, tmV, tmDO, p, st);
 }

@@ -13,6 +13,7 @@ struct TcState {
   EncodeTiledFn encode;
   bool attr_set_128, attr_set_256;
   bool attn_attr_set[2];
+  int attn_poly_bwd;      // the same share in the backward kernels
   int attn_poly;          // of every 4 score pairs, how many take the polynomial exp2 (0..3)
 };
 
