@@ -155,25 +155,36 @@ __global__ void __launch_bounds__(256) attn_fwd_kernel(CcaDims d, const bf16* __
   }
 }
 
-// delta[b,i,t] = sum_c dO[t,i,c] * O[t,i,c]  (one warp per (token, head)).  O is the fp32 copy kept by the
-// forward: delta is subtracted from dP = dO V^T inside the softmax adjoint, and rounding O to bf16 there
-// would cost the dominant keys several digits.
-__global__ void attn_delta_kernel(CcaDims d, const float* __restrict__ o, const bf16* __restrict__ d_o,
-                                  float* __restrict__ delta) {
-  long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / 32;
-  int lane = threadIdx.x % 32;
-  long long total = (long long)d.B * d.S * d.hq;
-  if (w >= total) return;
-  int hi = (int)(w % d.hq);
-  long long row = w / d.hq;
-  const float* po = o + row * d.Lq + hi * d.dh;
-  const bf16* pd = d_o + row * d.Lq + hi * d.dh;
+// delta[b,i,t] = sum_c dO[t,i,c] * O[t,i,c].  O is the fp32 copy kept by the forward: delta is subtracted from
+// dP = dO V^T inside the softmax adjoint, and rounding O to bf16 there would cost the dominant keys several
+// digits.  A group of d_h/8 lanes owns one (token, head): 8 channels per lane, 128-bit loads.
+template <int DH>
+__global__ void __launch_bounds__(256) attn_delta_kernel(CcaDims d, const float* __restrict__ o,
+                                                         const bf16* __restrict__ d_o, float* __restrict__ delta) {
+  constexpr int TPR = DH / 8;                       // lanes per row
+  const long long gt = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long w = gt / TPR;
+  const int sub = (int)(gt % TPR);
+  const long long total = (long long)d.B * d.S * d.hq;
   float s = 0.f;
-  for (int c = lane; c < d.dh; c += 32) s = fmaf(po[c], __bfloat162float(pd[c]), s);
+  const bool act = w < total;
+  int hi = 0;
+  long long row = 0;
+  if (act) {
+    hi = (int)(w % d.hq);
+    row = w / d.hq;
+    const float4* po = reinterpret_cast<const float4*>(o + row * d.Lq + hi * DH + sub * 8);
+    const uint4 dv = *reinterpret_cast<const uint4*>(d_o + row * d.Lq + hi * DH + sub * 8);
+    const float4 a = po[0], c = po[1];
+    const __nv_bfloat162* db = reinterpret_cast<const __nv_bfloat162*>(&dv);
+    const float2 d0 = __bfloat1622float2(db[0]), d1 = __bfloat1622float2(db[1]), d2 = __bfloat1622float2(db[2]),
+                 d3 = __bfloat1622float2(db[3]);
+    s = a.x * d0.x + a.y * d0.y + a.z * d1.x + a.w * d1.y + c.x * d2.x + c.y * d2.y + c.z * d3.x + c.w * d3.y;
+  }
 #pragma unroll
-  for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-  if (lane == 0) {
-    int b = (int)(row / d.S), t = (int)(row % d.S);
+  for (int off = TPR / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+  if (act && sub == 0) {
+    const int b = (int)(row / d.S), t = (int)(row % d.S);
     delta[((long long)b * d.hq + hi) * d.S + t] = s;
   }
 }
@@ -365,8 +376,11 @@ cudaError_t launch_attn_fwd_simt(const CcaDims& d, const bf16* q, const bf16* k,
 }
 
 cudaError_t launch_attn_delta(const CcaDims& d, const float* o32, const bf16* d_o, float* delta, cudaStream_t st) {
-  long long warps = (long long)d.B * d.S * d.hq;
-  attn_delta_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>(d, o32, d_o, delta);
+  const long long rows = (long long)d.B * d.S * d.hq;
+  DISPATCH_DH(d.dh, {
+    const long long threads = rows * (DH / 8);
+    attn_delta_kernel<DH><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(d, o32, d_o, delta);
+  });
   return cudaGetLastError();
 }
 

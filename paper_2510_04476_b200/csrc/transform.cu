@@ -213,8 +213,8 @@ __global__ void __launch_bounds__(256) transform_fwd_kernel(CcaDims d, const flo
 
 // ------------------------------------------------------------------------------------------
 // backward, part 1: RoPE adjoint, norm adjoint, d_temp.  In place on dq / dk (fp32).
-// One warp per (token, head); lane l owns channels l, l+32, ... so that the rotation pairs
-// (c, c + d_h/2) sit in one lane and every access is a run of 32 consecutive elements.
+// A group of d_h/8 lanes owns one (token, head); lane l of the group owns channels [4l, 4l+4) and their
+// rotation partners [4l + d_h/2, ...), so every access is a 64- or 128-bit vector.
 //   x = pre-norm latent, y = r x with r = sqrt(d_h)[beta]/|x| (kept by the forward), q = RoPE(y):
 //   dy = RoPE^T(dq);  dx = r (dy - y (y . dy) / |y|^2),  |y|^2 = d_h [beta^2];  d_temp = sum y . dy.
 // y is taken from the stored bf16 q / k (rotated back), r in fp32: the 1/|x| amplification is exact,
@@ -227,59 +227,66 @@ __global__ void __launch_bounds__(256) transform_bwd_norm_kernel(CcaDims d, cons
                                                                  const float* __restrict__ temp,
                                                                  const float2* __restrict__ rope_tab, float* dq,
                                                                  float* dk, float* d_temp) {
-  constexpr int HALF = DH / 2, NP = HALF / 32 > 0 ? HALF / 32 : 1;     // rotation pairs per lane
+  constexpr int HALF = DH / 2, TPR = HALF / 4;     // lanes per row
   const int H = d.hq + d.hk;
-  const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / 32;
-  const int lane = threadIdx.x % 32;
+  const long long gt = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long w = gt / TPR;
+  const int sub = (int)(gt % TPR);
   const long long total = (long long)d.B * d.S * H;
-  if (w >= total) return;
-  const int h = (int)(w % H);
-  const long long row = w / H;
+  const bool act = w < total;
+  const long long wc = act ? w : 0;
+  const int h = (int)(wc % H);
+  const long long row = wc / H;
   const int t = (int)(row % d.S);
   const bool is_q = h < d.hq;
   const int hj = is_q ? h : h - d.hq;
-  float* g = (is_q ? dq + row * d.Lq : dk + row * d.Lk) + hj * DH;
-  const bf16* y = (is_q ? q + row * d.Lq : k + row * d.Lk) + hj * DH;
-  const bool act = lane < HALF;                   // d_h = 32: only 16 pairs
-  float ga[NP], gb[NP], ya[NP], yb[NP];
+  float* g = (is_q ? dq + row * d.Lq : dk + row * d.Lk) + hj * DH + sub * 4;
+  const bf16* y = (is_q ? q + row * d.Lq : k + row * d.Lk) + hj * DH + sub * 4;
+  float ga[4], gb[4], ya[4], yb[4];
+  {
+    const float4 va = *reinterpret_cast<const float4*>(g), vb = *reinterpret_cast<const float4*>(g + HALF);
+    ga[0] = va.x; ga[1] = va.y; ga[2] = va.z; ga[3] = va.w;
+    gb[0] = vb.x; gb[1] = vb.y; gb[2] = vb.z; gb[3] = vb.w;
+    const uint2 ua = *reinterpret_cast<const uint2*>(y), ub = *reinterpret_cast<const uint2*>(y + HALF);
+    const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&ua);
+    const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&ub);
+    const float2 a0 = __bfloat1622float2(pa[0]), a1 = __bfloat1622float2(pa[1]);
+    const float2 b0 = __bfloat1622float2(pb[0]), b1 = __bfloat1622float2(pb[1]);
+    ya[0] = a0.x; ya[1] = a0.y; ya[2] = a1.x; ya[3] = a1.y;
+    yb[0] = b0.x; yb[1] = b0.y; yb[2] = b1.x; yb[3] = b1.y;
+  }
+  if (d.flags & F_ROPE) {
+    const float4* tab = reinterpret_cast<const float4*>(rope_tab + (long long)t * HALF + sub * 4);
+    const float4 c01 = tab[0], c23 = tab[1];
+    const float cs[4] = {c01.x, c01.z, c23.x, c23.z}, sn[4] = {c01.y, c01.w, c23.y, c23.w};
 #pragma unroll
-  for (int i = 0; i < NP; ++i) {
-    const int c = lane + 32 * i;
-    ga[i] = act ? g[c] : 0.f;
-    gb[i] = act ? g[c + HALF] : 0.f;
-    ya[i] = act ? __bfloat162float(y[c]) : 0.f;
-    yb[i] = act ? __bfloat162float(y[c + HALF]) : 0.f;
-    if ((d.flags & F_ROPE) && act) {
-      const float2 cs = rope_tab[(long long)t * HALF + c];
+    for (int i = 0; i < 4; ++i) {
       // rotation by the negated angle
-      const float a0 = ga[i] * cs.x + gb[i] * cs.y, b0 = gb[i] * cs.x - ga[i] * cs.y;
+      const float a0 = ga[i] * cs[i] + gb[i] * sn[i], b0 = gb[i] * cs[i] - ga[i] * sn[i];
       ga[i] = a0; gb[i] = b0;
-      const float a1 = ya[i] * cs.x + yb[i] * cs.y, b1 = yb[i] * cs.x - ya[i] * cs.y;
+      const float a1 = ya[i] * cs[i] + yb[i] * sn[i], b1 = yb[i] * cs[i] - ya[i] * sn[i];
       ya[i] = a1; yb[i] = b1;
     }
   }
   if (d.flags & F_QK_NORM) {
     float dot = 0.f;
 #pragma unroll
-    for (int i = 0; i < NP; ++i) dot = fmaf(ya[i], ga[i], fmaf(yb[i], gb[i], dot));
+    for (int i = 0; i < 4; ++i) dot = fmaf(ya[i], ga[i], fmaf(yb[i], gb[i], dot));
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    for (int off = TPR / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
     const float beta = is_q ? 1.f : __expf(temp[hj]);
     const float r = rnorm[row * H + h];
     const float proj = dot / ((float)DH * beta * beta);
-    if (!is_q && lane == 0) atomicAdd(d_temp + hj, dot);
+    if (act && !is_q && sub == 0) atomicAdd(d_temp + hj, dot);
 #pragma unroll
-    for (int i = 0; i < NP; ++i) {
+    for (int i = 0; i < 4; ++i) {
       ga[i] = r * (ga[i] - ya[i] * proj);
       gb[i] = r * (gb[i] - yb[i] * proj);
     }
   }
   if (act) {
-#pragma unroll
-    for (int i = 0; i < NP; ++i) {
-      g[lane + 32 * i] = ga[i];
-      g[lane + 32 * i + HALF] = gb[i];
-    }
+    *reinterpret_cast<float4*>(g) = make_float4(ga[0], ga[1], ga[2], ga[3]);
+    *reinterpret_cast<float4*>(g + HALF) = make_float4(gb[0], gb[1], gb[2], gb[3]);
   }
 }
 
@@ -432,7 +439,7 @@ __global__ void __launch_bounds__(256) transform_bwd_w1_kernel(CcaDims d, const 
 //   d_qk0[t][c]  = sum_j w0[c][j] dy1[t + (ks-1) - j][c]  +  (direct q-k-mean terms of d_hat)
 //   d_w0[c][j]  += sum_t dy1[t][c] qk0[t - (ks-1) + j][c]
 // One thread per channel (coalesced over channels), walking CONV1_TOK consecutive tokens with sliding windows.
-constexpr int CONV1_TOK = 64;
+constexpr int CONV1_TOK = 32;
 template <int KS>
 __global__ void __launch_bounds__(128) conv1_adjoint_kernel(CcaDims d, const float* __restrict__ dy1,
                                                             const float* __restrict__ dqh, const float* __restrict__ dkh,
@@ -460,30 +467,46 @@ __global__ void __launch_bounds__(128) conv1_adjoint_kernel(CcaDims d, const flo
   }
   const bool is_q = c < d.Lq;
   const int cj = is_q ? c : c - d.Lq, hh = cj / d.dh, o = cj % d.dh;
-  for (int t = t_begin; t < t_end; ++t) {
-    float gq = 0.f;
+  const bool mean = (d.flags & F_QK_MEAN) != 0;
+  constexpr int U = 4;                               // tokens per batch: all loads of a batch are issued together
+  for (int tb = t_begin; tb < t_end; tb += U) {
+    float ndy[U], nq[U], dir[U];
 #pragma unroll
-    for (int j = 0; j < KS; ++j) gq = fmaf(w[j], win[KS - 1 - j], gq);
-#pragma unroll
-    for (int j = 0; j < KS; ++j) dw[j] = fmaf(win[0], qwin[j], dw[j]);
-    if (d.flags & F_QK_MEAN) {
-      const long long row = seq + t;
-      if (is_q) {
-        gq += 0.5f * (dqh[row * d.Lq + c] + dkh[row * d.Lk + (hh / d.g) * d.dh + o] / d.g);
-      } else {
-        float sg = dkh[row * d.Lk + cj];
-        for (int m = 0; m < d.g; ++m) sg += dqh[row * d.Lq + (hh * d.g + m) * d.dh + o];
-        gq += 0.5f * sg;
+    for (int u = 0; u < U; ++u) {
+      const int t = tb + u;
+      ndy[u] = dy_at(t + KS);
+      nq[u] = (t + 1 < d.S) ? q_at(t + 1) : 0.f;
+      dir[u] = 0.f;
+      if (mean && t < t_end) {
+        const long long row = seq + t;
+        if (is_q) {
+          dir[u] = 0.5f * (dqh[row * d.Lq + c] + dkh[row * d.Lk + (hh / d.g) * d.dh + o] / d.g);
+        } else {
+          float sg = dkh[row * d.Lk + cj];
+          for (int m = 0; m < d.g; ++m) sg += dqh[row * d.Lq + (hh * d.g + m) * d.dh + o];
+          dir[u] = 0.5f * sg;
+        }
       }
     }
-    dlat[(seq + t) * ld + c] = __float2bfloat16(gq);
 #pragma unroll
-    for (int m = 0; m < KS - 1; ++m) {
-      win[m] = win[m + 1];
-      qwin[m] = qwin[m + 1];
+    for (int u = 0; u < U; ++u) {
+      const int t = tb + u;
+      if (t < t_end) {
+        float gq = dir[u];
+#pragma unroll
+        for (int j = 0; j < KS; ++j) gq = fmaf(w[j], win[KS - 1 - j], gq);
+#pragma unroll
+        for (int j = 0; j < KS; ++j) dw[j] = fmaf(win[0], qwin[j], dw[j]);
+        dlat[(seq + t) * ld + c] = __float2bfloat16(gq);
+#pragma unroll
+        for (int m = 0; m < KS - 1; ++m) {
+          win[m] = win[m + 1];
+          qwin[m] = qwin[m + 1];
+        }
+        win[KS - 1] = ndy[u];
+        qwin[KS - 1] = nq[u];
+      }
     }
-    win[KS - 1] = dy_at(t + KS);
-    qwin[KS - 1] = q_at(t + 1);
   }
   if (conv1)
 #pragma unroll
@@ -552,10 +575,11 @@ cudaError_t launch_transform_bwd_norm(const CcaDims& d, const bf16* q, const bf1
                                       const float* temp, const float2* rope_tab, float* dq, float* dk, float* d_temp,
                                       cudaStream_t st) {
   if (!(d.flags & (F_QK_NORM | F_ROPE))) return cudaSuccess;
-  const long long warps = (long long)d.B * d.S * (d.hq + d.hk);
-  const unsigned grid = (unsigned)((warps * 32 + 255) / 256);
+  const long long rows = (long long)d.B * d.S * (d.hq + d.hk);
   DISPATCH_DH(d.dh, {
-    transform_bwd_norm_kernel<DH><<<grid, 256, 0, st>>>(d, q, k, rnorm, temp, rope_tab, dq, dk, d_temp);
+    const long long threads = rows * (DH / 8);
+    transform_bwd_norm_kernel<DH><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(d, q, k, rnorm, temp, rope_tab, dq,
+                                                                                     dk, d_temp);
   });
   return cudaGetLastError();
 }
