@@ -31,6 +31,9 @@ UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAK_TFLOPS = 1590.0
 TRAIN_WORKLOADS = {"cfg2_small", "cfg4_train"}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the attention-forward kernel as it stands, from
+# the full ncu capture summarised under profiles/ (set to None when the kernel changes until it is re-captured)
+ATTN_FWD_DRAM_BYTES = {"cfg3_prefill16k": 53.1e6}
 
 
 def flops_of(sh, backward: bool):
@@ -108,7 +111,7 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(clocks)}
 
 
-def oracle_sample(sh, n_rows=4096, backward=False):
+def oracle_sample(sh, n_rows=16384, backward=False):
     """The oracle, as it stands, on a bounded sample of the workload.  Forward workloads: projections and
     latent transforms in full, the S^2 stage and the up-projection on n_rows sampled query positions per
     sequence (every position if n_rows >= S).  Training workloads: the whole forward and backward."""
@@ -288,7 +291,8 @@ def run_ours(args, rank, world, local_rank):
         "roofline": {"bound": "tensor", "kernel": "latent attention forward", "achieved": attn_tflops, "peak": peak,
                      "unit": "TFLOP/s", "frac": attn_tflops / peak, "peak_kind": peak_kind,
                      "frac_of_nominal_2250": attn_tflops / NOMINAL_BF16_TFLOPS, "ms_per_launch": attn_ms,
-                     "flops_per_launch": fl["attn_fwd"], "traffic": None},
+                     "flops_per_launch": fl["attn_fwd"],
+                     "traffic": ATTN_FWD_DRAM_BYTES.get(sh.name) if args.kernels else None},
         "pct_of_nominal_bf16_peak": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
         "device_status": status,
     }
