@@ -181,7 +181,7 @@ def run_ours(args, rank, world, local_rank):
         dist = dist_mod
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     sh = synth.CONFIGS[args.workload]
-    backward = args.workload in TRAIN_WORKLOADS
+    backward = args.workload in TRAIN_WORKLOADS or args.backward
     t = synth.make_inputs(sh, want_dout=backward)
     dev = {k: v.cuda(local_rank).contiguous() for k, v in t.items()}
     cca = CCA.from_shape(sh, device=local_rank)
@@ -386,6 +386,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3_prefill16k", choices=sorted(synth.CONFIGS))
     ap.add_argument("--kernels", type=int, default=1, help="0 = SIMT kernels only, 1 = tcgen05 kernels where available")
+    ap.add_argument("--backward", action="store_true", help="time forward + backward on a forward-only workload too")
     ap.add_argument("--no-mha", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -121,35 +121,42 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      const uint32_t idesc = idesc_bf16(BN, p.a_mn, p.b_mn);
-      int stage = 0;
-      uint32_t phase = 0;
-      int it = 0;
-      for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
-        const int as = it & 1;
-        const uint32_t aphase = (it >> 1) & 1;
-        if (!mbar_wait(&acc_empty[as], aphase ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+    // The whole warp runs the loop so that the address arithmetic stays warp-uniform; one elected lane issues.
+    const bool leader = elect_one();
+    const uint32_t idesc = idesc_bf16(BN, p.a_mn, p.b_mn);
+    // descriptor words: high = stride offset 1024, version, 128-byte swizzle; low = address >> 4 | leading offset << 16
+    const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
+    const uint32_t a_lbo = p.a_mn ? ((8192u >> 4) << 16) : (1u << 16), b_lbo = p.b_mn ? ((8192u >> 4) << 16) : (1u << 16);
+    const uint32_t a_step = p.a_mn ? (2048u >> 4) : (32u >> 4), b_step = p.b_mn ? (2048u >> 4) : (32u >> 4);
+    const uint32_t smem_lo = smem_u32(smem) >> 4;
+    auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+    };
+    int stage = 0;
+    uint32_t phase = 0;
+    int it = 0;
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+      const int as = it & 1;
+      const uint32_t aphase = (it >> 1) & 1;
+      if (!wait_all(&acc_empty[as], aphase ^ 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + as * BN;
+      const int sp = tile % p.splits;
+      const int kb_begin = sp * p.kb_per_split, kb_end = min(p.num_kb, kb_begin + p.kb_per_split);
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
+        if (!wait_all(&full_bar[stage], phase)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + as * BN;
-        const int sp = tile % p.splits;
-        const int kb_begin = sp * p.kb_per_split, kb_end = min(p.num_kb, kb_begin + p.kb_per_split);
-        for (int kb = kb_begin; kb < kb_end; ++kb) {
-          if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
-          tc_fence_after();
-          const uint32_t sa = smem_u32(smem + stage * SM::STAGE_BYTES);
-          const uint32_t sb = sa + SM::A_BYTES;
+        const uint32_t sa = (smem_lo + stage * (SM::STAGE_BYTES >> 4)) | a_lbo;
+        const uint32_t sb = (smem_lo + stage * (SM::STAGE_BYTES >> 4) + (SM::A_BYTES >> 4)) | b_lbo;
+        if (leader) {
 #pragma unroll
-          for (int k = 0; k < GEMM_BK / 16; ++k) {
-            const uint64_t da = p.a_mn ? smem_desc_sw128(sa + k * 2048, 8192, 1024) : smem_desc_sw128(sa + k * 32, 16, 1024);
-            const uint64_t db = p.b_mn ? smem_desc_sw128(sb + k * 2048, 8192, 1024) : smem_desc_sw128(sb + k * 32, 16, 1024);
-            mma_ss(d_tmem, da, db, idesc, ((kb - kb_begin) | k) != 0);
-          }
+          for (int k = 0; k < GEMM_BK / 16; ++k)
+            mma_ss_w(d_tmem, sa + k * a_step, desc_hi, sb + k * b_step, desc_hi, idesc, ((kb - kb_begin) | k) != 0);
           mma_commit(&empty_bar[stage]);
-          if (++stage == GEMM_STAGES) { stage = 0; phase ^= 1; }
         }
-        mma_commit(&acc_full[as]);
+        if (++stage == GEMM_STAGES) { stage = 0; phase ^= 1; }
       }
+      if (leader) mma_commit(&acc_full[as]);
     }
   } else {
     const int q = warp & 3;                       // TMEM lane quarter this warp may access
