@@ -90,7 +90,8 @@ GemmOperand mmajor(const void* p, long long ld) { return GemmOperand{(const bf16
 // One contraction: tensor-core kernel if it is enabled and covers the case, else the SIMT kernel.
 int run_gemm(cca_handle* h, const GemmArgs& g, cudaStream_t st) {
   if (h->impl >= 1 && h->tc) {
-    int r = tc_gemm(h->tc, g, h->d_status, st);
+    int r = tc_gemm_pair(h->tc, g, h->d_status, st);
+    if (r == 1) r = tc_gemm(h->tc, g, h->d_status, st);
     if (r == 0) { h->launches++; return CCA_OK; }
     if (r < 0) { h->last_cuda = -r; return CCA_ERR_CUDA; }
   }

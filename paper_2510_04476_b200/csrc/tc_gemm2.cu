@@ -1,0 +1,325 @@
+// Tensor-core kernels, part 6: the large projection GEMMs on CTA pairs.
+//   C[M,N] = sum_k A(m,k) B(n,k), A K-major, B K-major or MN-major, bf16 operands, fp32 accumulate.
+// Two CTAs on neighbouring SMs (a cluster of 2) work on one 256 x 256 tile with tcgen05.mma.cta_group::2:
+// each CTA loads its own 128 rows of A and only HALF of the B tile (128 of the 256 output columns), the
+// tensor cores of both SMs read B from both shared memories.  Per k-block a CTA therefore pulls 32 KB
+// through the L2 instead of the 48 KB a stand-alone 128 x 256 tile needs, which is what limited that
+// kernel.  Loads use plain TMA (no multicast); only the MMA-completion signal is sent to both CTAs.
+//
+//   warp 0      : TMA producer, in both CTAs (transaction bytes are counted on the leader CTA's barrier)
+//   warp 1      : TMEM owner in both CTAs; in the leader CTA it issues the MMAs for the pair
+//   warps 2..5  : epilogue, each CTA drains its own 128 accumulator rows from its own TMEM
+#include <cstdio>
+
+#include "tc_kernels.cuh"
+#include "tc_ptx.cuh"
+#include "tc_state.cuh"
+
+using namespace tc;
+
+namespace {
+
+constexpr int G2_BM = 128;            // rows per CTA (256 per pair)
+constexpr int G2_BN = 256;
+constexpr int G2_BK = 64;
+constexpr int G2_STAGES = 6;
+constexpr int G2_THREADS = 192;
+
+struct G2Params {
+  int M, N, K;
+  bf16* out_bf16;
+  float* out_f32;
+  long long ldc;
+  int tiles_m, tiles_n, num_kb;     // tiles of 256 x 256
+  int b_mn;
+  int vec_ok;
+  int* status;
+};
+
+struct G2Smem {
+  static constexpr int A_BYTES = G2_BM * G2_BK * 2;          // 16 KB
+  static constexpr int B_BYTES = (G2_BN / 2) * G2_BK * 2;    // 16 KB: this CTA's half of the B tile
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int BAR_OFFSET = G2_STAGES * STAGE_BYTES;
+  static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;
+};
+
+TC_DEVINL void fail(volatile int* abort_flag, int* status, int code) {
+  *abort_flag = 1;
+  atomicCAS(status, 0, code);
+}
+TC_DEVINL uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+TC_DEVINL void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// 2-D TMA tile load of one CTA of a pair; the bytes are counted on the barrier at the same offset in the
+// pair's leader CTA (peer bit of the barrier address cleared)
+TC_DEVINL void tma_load_2d_pair(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar) & 0xFEFFFFFFu)
+      : "memory");
+}
+// D[tmem of both CTAs] (+)= A B over the pair: 256 x N x 16
+TC_DEVINL void mma2_ss_w(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                         uint32_t accumulate) {
+  const uint32_t z = 0;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\tsetp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, {%7, %7, %7, %7, %7, %7, %7, %7}, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(z)
+      : "memory");
+}
+// arrive on the barrier at this offset in both CTAs of the pair once all MMAs issued so far have completed
+TC_DEVINL void mma2_commit_both(uint64_t* bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"(mask)
+               : "memory");
+}
+// arrive on the barrier at this offset in CTA `rank` of the cluster
+TC_DEVINL void mbar_arrive_cta(uint64_t* bar, uint32_t rank) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(bar)), "r"(rank));
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+
+__global__ void __launch_bounds__(G2_THREADS, 1)
+tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, G2Params p) {
+  using SM = G2Smem;
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFFSET);   // used in the leader CTA
+  uint64_t* empty_bar = full_bar + G2_STAGES;                                 // one set per CTA
+  uint64_t* acc_full = empty_bar + G2_STAGES;                                 // [2], one set per CTA
+  uint64_t* acc_empty = acc_full + 2;                                         // [2], used in the leader CTA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int num_tiles = p.tiles_m * p.tiles_n;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < G2_STAGES; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&acc_full[s], 1);
+      mbar_init(&acc_empty[s], 8);          // four epilogue warps of each CTA
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmA);
+    prefetch_tmap(&tmB);
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                       // the peer's barriers exist before anything is sent to them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int tile = pair; tile < num_tiles; tile += n_pairs) {
+        const int m0 = (tile / p.tiles_n) * (2 * G2_BM) + (int)rank * G2_BM;
+        const int n0 = (tile % p.tiles_n) * G2_BN + (int)rank * (G2_BN / 2);
+        for (int kb = 0; kb < p.num_kb; ++kb) {
+          if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
+          unsigned char* sa = smem + stage * SM::STAGE_BYTES;
+          unsigned char* sb = sa + SM::A_BYTES;
+          if (rank == 0) mbar_expect_tx(&full_bar[stage], 2 * SM::STAGE_BYTES);
+          const int k0 = kb * G2_BK;
+          tma_load_2d_pair(sa, &tmA, k0, m0, &full_bar[stage]);
+          if (!p.b_mn) {
+            tma_load_2d_pair(sb, &tmB, k0, n0, &full_bar[stage]);
+          } else {
+            tma_load_2d_pair(sb, &tmB, n0, k0, &full_bar[stage]);
+            tma_load_2d_pair(sb + 8192, &tmB, n0 + 64, k0, &full_bar[stage]);
+          }
+          if (++stage == G2_STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (rank == 0) {
+      const bool leader = elect_one();
+      // M = 256 over the pair, N = 256
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.b_mn << 16) | ((uint32_t)(G2_BN >> 3) << 17) |
+                             ((uint32_t)(256 >> 4) << 24);
+      const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
+      const uint32_t a_lbo = 1u << 16, b_lbo = p.b_mn ? ((8192u >> 4) << 16) : (1u << 16);
+      const uint32_t a_step = 32u >> 4, b_step = p.b_mn ? (2048u >> 4) : (32u >> 4);
+      const uint32_t smem_lo = smem_u32(smem) >> 4;
+      auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+      };
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      for (int tile = pair; tile < num_tiles; tile += n_pairs, ++it) {
+        const int as = it & 1;
+        const uint32_t aphase = (it >> 1) & 1;
+        if (!wait_all(&acc_empty[as], aphase ^ 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + as * G2_BN;
+        for (int kb = 0; kb < p.num_kb; ++kb) {
+          if (!wait_all(&full_bar[stage], phase)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+          tc_fence_after();
+          const uint32_t sa = (smem_lo + stage * (SM::STAGE_BYTES >> 4)) | a_lbo;
+          const uint32_t sb = (smem_lo + stage * (SM::STAGE_BYTES >> 4) + (SM::A_BYTES >> 4)) | b_lbo;
+          if (leader) {
+#pragma unroll
+            for (int k = 0; k < G2_BK / 16; ++k)
+              mma2_ss_w(d_tmem, sa + k * a_step, desc_hi, sb + k * b_step, desc_hi, idesc, (kb | k) != 0);
+            mma2_commit_both(&empty_bar[stage]);
+          }
+          if (++stage == G2_STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (leader) mma2_commit_both(&acc_full[as]);
+      }
+    }
+  } else {
+    const int q = warp & 3;                       // TMEM lane quarter this warp may access
+    int it = 0;
+    for (int tile = pair; tile < num_tiles; tile += n_pairs, ++it) {
+      const int as = it & 1;
+      const uint32_t aphase = (it >> 1) & 1;
+      const int m0 = (tile / p.tiles_n) * (2 * G2_BM) + (int)rank * G2_BM, n0 = (tile % p.tiles_n) * G2_BN;
+      if (!mbar_wait(&acc_full[as], aphase, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
+      tc_fence_after();
+      const int m = m0 + q * 32 + lane;
+#pragma unroll 1
+      for (int c = 0; c < G2_BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + as * G2_BN + c * 32, r);
+        tmem_ld_wait();
+        const int n = n0 + c * 32;
+        if (m < p.M && n < p.N) {
+          if (p.out_bf16) {
+            bf16* dst = p.out_bf16 + (long long)m * p.ldc + n;
+            if (p.vec_ok && n + 32 <= p.N) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                uint4 v;
+                v.x = pack_bf16(__uint_as_float(r[8 * i + 0]), __uint_as_float(r[8 * i + 1]));
+                v.y = pack_bf16(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]));
+                v.z = pack_bf16(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]));
+                v.w = pack_bf16(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7]));
+                reinterpret_cast<uint4*>(dst)[i] = v;
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (n + i < p.N) dst[i] = __float2bfloat16(__uint_as_float(r[i]));
+            }
+          } else {
+            float* dst = p.out_f32 + (long long)m * p.ldc + n;
+            if (p.vec_ok && n + 32 <= p.N) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                reinterpret_cast<uint4*>(dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (n + i < p.N) dst[i] = __uint_as_float(r[i]);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cta(&acc_empty[as], 0);     // the leader CTA's barrier, from either CTA
+    }
+  }
+done:
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000) {}
+    __syncthreads();
+  }
+  // neither CTA may leave while the other can still read its shared memory or signal its barriers
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+}  // namespace
+
+// Returns 0 if enqueued, 1 if the case is outside this kernel's coverage, -cudaError on failure.
+int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) {
+  if (!s || !s->encode || !s->use_pairs) return 1;
+  if (g.A.cs != 1 || g.a_row_off != 0) return 1;                  // A K-major, no row shift
+  const int b_mn = g.B.cs != 1;
+  if (b_mn && g.B.rs != 1) return 1;
+  const long long lda = g.A.rs, ldb = b_mn ? g.B.cs : g.B.rs;
+  if (lda % 8 || ldb % 8) return 1;
+  if ((reinterpret_cast<uintptr_t>(g.A.p) & 15) || (reinterpret_cast<uintptr_t>(g.B.p) & 15)) return 1;
+  if (g.M < 512 || g.N < 256 || g.K < 64) return 1;
+  if (s->pair_clusters < 0) {
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, G2Smem::TOTAL);
+    if (e != cudaSuccess) return -(int)e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * s->sm_count, 1, 1);
+    cfg.blockDim = dim3(G2_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = G2Smem::TOTAL;
+    cudaLaunchAttribute at;
+    at.id = cudaLaunchAttributeClusterDimension;
+    at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+    cfg.attrs = &at; cfg.numAttrs = 1;
+    int n = 0;
+    e = cudaOccupancyMaxActiveClusters(&n, tc_gemm2_kernel, &cfg);
+    s->pair_clusters = (e == cudaSuccess) ? n : 0;
+    if (e != cudaSuccess) (void)cudaGetLastError();
+  }
+  if (s->pair_clusters < 8) return 1;
+  CUtensorMap tmA, tmB;
+  if (!tc_make_map_2d(s, &tmA, g.A.p, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)lda, G2_BK, G2_BM)) return 1;
+  bool ok;
+  if (!b_mn) ok = tc_make_map_2d(s, &tmB, g.B.p, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)ldb, G2_BK, G2_BN / 2);
+  else ok = tc_make_map_2d(s, &tmB, g.B.p, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)ldb, 64, G2_BK);
+  if (!ok) return 1;
+  G2Params p;
+  p.M = g.M; p.N = g.N; p.K = g.K;
+  p.out_bf16 = g.out_bf16; p.out_f32 = g.out_f32; p.ldc = g.ldc;
+  p.tiles_m = (g.M + 2 * G2_BM - 1) / (2 * G2_BM);
+  p.tiles_n = (g.N + G2_BN - 1) / G2_BN;
+  p.num_kb = (g.K + G2_BK - 1) / G2_BK;
+  p.b_mn = b_mn;
+  const void* outp = g.out_bf16 ? (const void*)g.out_bf16 : (const void*)g.out_f32;
+  const int esz = g.out_bf16 ? 2 : 4;
+  p.vec_ok = ((reinterpret_cast<uintptr_t>(outp) & 15) == 0) && ((g.ldc * esz) % 16 == 0);
+  p.status = d_status;
+  const int tiles = p.tiles_m * p.tiles_n;
+  const int pairs = tiles < s->pair_clusters ? tiles : s->pair_clusters;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  cfg.blockDim = dim3(G2_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = G2Smem::TOTAL;
+  cfg.stream = st;
+  cudaLaunchAttribute at;
+  at.id = cudaLaunchAttributeClusterDimension;
+  at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+  cfg.attrs = &at; cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm2_kernel, tmA, tmB, p);
+  return e == cudaSuccess ? 0 : -(int)e;
+}

@@ -274,6 +274,9 @@ TcState* tc_create(int sm_count) {
   s->sm_count = sm_count;
   s->encode = nullptr;
   s->attr_set_128 = s->attr_set_256 = false;
+  s->pair_clusters = -1;
+  s->use_pairs = 1;
+  if (const char* e = getenv("CCA_GEMM_PAIRS")) s->use_pairs = atoi(e);
   s->attn_attr_set[0] = s->attn_attr_set[1] = false;
   s->attn_poly = 1;
   if (const char* e = getenv("CCA_ATTN_POLY")) s->attn_poly = atoi(e);

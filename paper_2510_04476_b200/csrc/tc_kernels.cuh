@@ -9,6 +9,8 @@ struct TcState;
 TcState* tc_create(int sm_count);
 void tc_destroy(TcState* s);
 int tc_gemm(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st);
+// Same contraction on CTA pairs (256 x 256 tiles); covers large K-major-A cases only.
+int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st);
 int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* o32,
                 float* lse, const float* temp, int* d_status, cudaStream_t st);
 // Attention adjoint (dq, dk, dv in fp32) from q, k, v, d_o, the forward's lse and delta = rowsum(dO o O).

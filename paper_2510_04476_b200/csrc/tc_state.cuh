@@ -12,6 +12,8 @@ struct TcState {
   int sm_count;
   EncodeTiledFn encode;
   bool attr_set_128, attr_set_256;
+  int pair_clusters;      // co-resident CTA pairs of the pair GEMM (-1: not asked yet, 0: unavailable)
+  int use_pairs;          // 0 disables the pair GEMM
   bool attn_attr_set[2];
   int attn_poly_bwd;      // the same share in the backward kernels
   int attn_poly;          // of every 4 score pairs, how many take the polynomial exp2 (0..3)
