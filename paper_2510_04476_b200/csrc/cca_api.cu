@@ -25,8 +25,8 @@ namespace {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
-  size_t qk0, q, k, v, o, lse, rope, rnorm, saved_end;
-  size_t o32, d_o, delta, dq, dk, dv, dlat, w_all, dy1, total_end;
+  size_t qk0, q, k, v, o, lse, rope, rnorm, w_all, saved_end;
+  size_t o32, d_o, delta, dq, dk, dv, dlat, dy1, total_end;
 };
 
 Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
@@ -43,6 +43,7 @@ Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
   l.lse = take((size_t)B * c.n_q_heads * S * 4);
   l.rope = take((size_t)S * (c.head_dim / 2) * 8);
   l.rnorm = take(T * (size_t)(c.n_q_heads + c.n_kv_heads) * 4);   // norm scale of every (token, head)
+  l.w_all = take((L + Lk) * (size_t)c.d_model * 2);                // [W_qk; W_v1; W_v2] stacked
   l.saved_end = off;
   l.o32 = take(T * Lq * 4);
   l.d_o = take(T * Lq * 2);
@@ -51,7 +52,6 @@ Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
   l.dk = take(T * Lk * 4);
   l.dv = take(T * Lk * 4);
   l.dlat = take(T * (L + Lk) * 2);
-  l.w_all = take((L + Lk) * (size_t)c.d_model * 2);
   l.dy1 = take(T * L * 4);
   l.total_end = off;
   return l;
@@ -313,18 +313,38 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
     CU(launch_rope_table(rope, d.S, d.dh, c.rope_base, st));
     h->launches++;
   }
-  // Eq. 7: packed q/k down-projection
+  // the three down-projection weights stacked (also the B operand of the input gradient in the backward)
+  bf16* w_all = (bf16*)(ws + l.w_all);
+  CU(cudaMemcpyAsync(w_all, w->w_qk, (size_t)d.L * d.E * 2, cudaMemcpyDeviceToDevice, st));
+  CU(cudaMemcpyAsync(w_all + (size_t)d.L * d.E, w->w_v1, (size_t)(d.Lk / 2) * d.E * 2, cudaMemcpyDeviceToDevice, st));
+  CU(cudaMemcpyAsync(w_all + (size_t)(d.L + d.Lk / 2) * d.E, w->w_v2, (size_t)(d.Lk / 2) * d.E * 2,
+                     cudaMemcpyDeviceToDevice, st));
   GemmArgs g{};
-  g.A = kmajor(x, d.E); g.B = kmajor(w->w_qk, d.E);
-  g.M = T; g.N = d.L; g.K = d.E; g.a_row_off = 0; g.seq_len = d.S;
-  g.out_bf16 = nullptr; g.out_f32 = qk0; g.ldc = d.L;
-  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
-  // Eq. 10: value halves from x_t and x_{t-1}
-  g.B = kmajor(w->w_v1, d.E); g.N = d.Lk / 2; g.out_f32 = nullptr; g.out_bf16 = v; g.ldc = d.Lk;
-  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
-  g.B = kmajor(w->w_v2, d.E); g.out_bf16 = v + d.Lk / 2;
-  g.a_row_off = (c.flags & CCA_V_SHIFT) ? -1 : 0;
-  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  bool fused = false;
+  if (h->impl >= 1 && h->tc) {
+    // Eq. 7 and Eq. 10 in one contraction: [qk0 | v1 | v2] = x [W_qk; W_v1; W_v2]^T, the v2 columns stored one token later
+    g.A = kmajor(x, d.E); g.B = kmajor(w_all, d.E);
+    g.M = T; g.N = d.L + d.Lk; g.K = d.E; g.a_row_off = 0; g.seq_len = d.S;
+    g.out_bf16 = v; g.out_f32 = qk0; g.ldc = d.L;
+    g.split_L = d.L; g.split_Lk = d.Lk; g.split_shift = (c.flags & CCA_V_SHIFT) ? 1 : 0;
+    int pr = tc_gemm_pair(h->tc, g, h->d_status, st);
+    if (pr < 0) { h->last_cuda = -pr; return CCA_ERR_CUDA; }
+    if (pr == 0) { fused = true; h->launches++; }
+  }
+  if (!fused) {
+    // Eq. 7: packed q/k down-projection
+    g = GemmArgs{};
+    g.A = kmajor(x, d.E); g.B = kmajor(w->w_qk, d.E);
+    g.M = T; g.N = d.L; g.K = d.E; g.a_row_off = 0; g.seq_len = d.S;
+    g.out_bf16 = nullptr; g.out_f32 = qk0; g.ldc = d.L;
+    if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+    // Eq. 10: value halves from x_t and x_{t-1}
+    g.B = kmajor(w->w_v1, d.E); g.N = d.Lk / 2; g.out_f32 = nullptr; g.out_bf16 = v; g.ldc = d.Lk;
+    if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+    g.B = kmajor(w->w_v2, d.E); g.out_bf16 = v + d.Lk / 2;
+    g.a_row_off = (c.flags & CCA_V_SHIFT) ? -1 : 0;
+    if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  }
   // Eq. 8, 9, 11: convs, q-k-mean, norm, temperature, RoPE
   {
     bool done = false;
@@ -464,11 +484,7 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
   g.A = mmajor(dlat + d.L + d.Lk / 2, ldl); g.out_f32 = gr->d_w_v2;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
-  // input gradient: d_x = [d_qk0, d_v1, d_v2 moved one token earlier] [W_qk; W_v1; W_v2]
-  CU(cudaMemcpyAsync(w_all, w->w_qk, (size_t)d.L * d.E * 2, cudaMemcpyDeviceToDevice, st));
-  CU(cudaMemcpyAsync(w_all + (size_t)d.L * d.E, w->w_v1, (size_t)(d.Lk / 2) * d.E * 2, cudaMemcpyDeviceToDevice, st));
-  CU(cudaMemcpyAsync(w_all + (size_t)(d.L + d.Lk / 2) * d.E, w->w_v2, (size_t)(d.Lk / 2) * d.E * 2,
-                     cudaMemcpyDeviceToDevice, st));
+  // input gradient: d_x = [d_qk0, d_v1, d_v2 moved one token earlier] [W_qk; W_v1; W_v2] (stacked by the forward)
   g = GemmArgs{};
   g.A = kmajor(dlat, ldl); g.B = mmajor(w_all, d.E);
   g.M = T; g.N = d.E; g.K = (int)ldl; g.seq_len = d.S; g.out_bf16 = (bf16*)d_x; g.ldc = d.E;

@@ -30,6 +30,10 @@ struct GemmOperand {
 //   are grouped in sequences of seq_len); rows whose source falls outside the sequence count as
 //   zero.  This is how the value-shift reads x_{t-1}.
 //   out_bf16 / out_f32: exactly one is non-null; ldc is the row stride of C in elements.
+//   split_L > 0 selects the fused down-projection output instead (Eq. 7 and Eq. 10 in one contraction with the
+//   rows of W_qk, W_v1, W_v2 stacked): columns [0, split_L) go to out_f32 (row stride ldc), the next split_Lk/2
+//   columns to out_bf16 (row stride split_Lk) in the same row, the last split_Lk/2 columns to out_bf16 one row
+//   later in the same sequence if split_shift (value-shift: v2 of token t is W_v2 x_{t-1}; row 0 gets zeros).
 struct GemmArgs {
   GemmOperand A, B;
   int M, N, K;
@@ -37,6 +41,7 @@ struct GemmArgs {
   bf16* out_bf16;
   float* out_f32;
   long long ldc;
+  int split_L, split_Lk, split_shift;
 };
 
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);

@@ -20,9 +20,7 @@ using namespace tc;
 namespace {
 
 constexpr int G2_BM = 128;            // rows per CTA (256 per pair)
-constexpr int G2_BN = 256;
 constexpr int G2_BK = 64;
-constexpr int G2_STAGES = 6;
 constexpr int G2_THREADS = 192;
 
 struct G2Params {
@@ -33,14 +31,17 @@ struct G2Params {
   int tiles_m, tiles_n, num_kb;     // tiles of 256 x 256
   int b_mn;
   int vec_ok;
+  int split_L, split_Lk, split_shift, seq_len;   // fused down-projection output (see GemmArgs)
   int* status;
 };
 
+template <int BN>
 struct G2Smem {
   static constexpr int A_BYTES = G2_BM * G2_BK * 2;          // 16 KB
-  static constexpr int B_BYTES = (G2_BN / 2) * G2_BK * 2;    // 16 KB: this CTA's half of the B tile
+  static constexpr int B_BYTES = (BN / 2) * G2_BK * 2;       // this CTA's half of the B tile (16 or 12 KB)
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int BAR_OFFSET = G2_STAGES * STAGE_BYTES;
+  static constexpr int STAGES = BN == 256 ? 6 : 7;
+  static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
   static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;
 };
 
@@ -89,9 +90,11 @@ TC_DEVINL void mbar_arrive_cta(uint64_t* bar, uint32_t rank) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
 }
 
+template <int BN>
 __global__ void __launch_bounds__(G2_THREADS, 1)
 tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, G2Params p) {
-  using SM = G2Smem;
+  using SM = G2Smem<BN>;
+  constexpr int G2_BN = BN, G2_STAGES = SM::STAGES;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFFSET);   // used in the leader CTA
@@ -148,8 +151,8 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           if (!p.b_mn) {
             tma_load_2d_pair(sb, &tmB, k0, n0, &full_bar[stage]);
           } else {
-            tma_load_2d_pair(sb, &tmB, n0, k0, &full_bar[stage]);
-            tma_load_2d_pair(sb + 8192, &tmB, n0 + 64, k0, &full_bar[stage]);
+#pragma unroll
+            for (int c = 0; c < G2_BN / 128; ++c) tma_load_2d_pair(sb + c * 8192, &tmB, n0 + c * 64, k0, &full_bar[stage]);
           }
           if (++stage == G2_STAGES) { stage = 0; phase ^= 1; }
         }
@@ -209,7 +212,38 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + as * G2_BN + c * 32, r);
         tmem_ld_wait();
         const int n = n0 + c * 32;
-        if (m < p.M && n < p.N) {
+        if (p.split_L > 0) {
+          // fused down-projection: latent columns in fp32, value columns in bf16 (second half one token later)
+          if (m < p.M && n < p.N) {
+            if (n < p.split_L) {
+              float* dst = p.out_f32 + (long long)m * p.ldc + n;
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                reinterpret_cast<uint4*>(dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+            } else {
+              const int vc = n - p.split_L;
+              const bool late = p.split_shift && vc >= p.split_Lk / 2;
+              const int t = m % p.seq_len;
+              bf16* dst = p.out_bf16 + (long long)(m + (late ? 1 : 0)) * p.split_Lk + vc;
+              if (!late || t + 1 < p.seq_len) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  uint4 v;
+                  v.x = pack_bf16(__uint_as_float(r[8 * i + 0]), __uint_as_float(r[8 * i + 1]));
+                  v.y = pack_bf16(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]));
+                  v.z = pack_bf16(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]));
+                  v.w = pack_bf16(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7]));
+                  reinterpret_cast<uint4*>(dst)[i] = v;
+                }
+              }
+              if (late && t == 0) {                     // x_{-1} = 0
+                bf16* z = p.out_bf16 + (long long)m * p.split_Lk + vc;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(z)[i] = make_uint4(0u, 0u, 0u, 0u);
+              }
+            }
+          }
+        } else if (m < p.M && n < p.N) {
           if (p.out_bf16) {
             bf16* dst = p.out_bf16 + (long long)m * p.ldc + n;
             if (p.vec_ok && n + 32 <= p.N) {
@@ -263,6 +297,38 @@ done:
   }
 }
 
+template <int BN>
+int launch_pair(TcState* s, const GemmArgs& g, const G2Params& p0, bool b_mn, long long lda, long long ldb, cudaStream_t st) {
+  static bool attr_set = false;
+  using SM = G2Smem<BN>;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm2_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL);
+    if (e != cudaSuccess) return -(int)e;
+    attr_set = true;
+  }
+  CUtensorMap tmA, tmB;
+  if (!tc_make_map_2d(s, &tmA, g.A.p, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)lda, G2_BK, G2_BM)) return 1;
+  bool ok;
+  if (!b_mn) ok = tc_make_map_2d(s, &tmB, g.B.p, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)ldb, G2_BK, BN / 2);
+  else ok = tc_make_map_2d(s, &tmB, g.B.p, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)ldb, 64, G2_BK);
+  if (!ok) return 1;
+  G2Params p = p0;
+  p.tiles_n = (g.N + BN - 1) / BN;
+  const int tiles = p.tiles_m * p.tiles_n;
+  const int pairs = tiles < s->pair_clusters ? tiles : s->pair_clusters;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  cfg.blockDim = dim3(G2_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = SM::TOTAL;
+  cfg.stream = st;
+  cudaLaunchAttribute at;
+  at.id = cudaLaunchAttributeClusterDimension;
+  at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+  cfg.attrs = &at; cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm2_kernel<BN>, tmA, tmB, p);
+  return e == cudaSuccess ? 0 : -(int)e;
+}
+
 }  // namespace
 
 // Returns 0 if enqueued, 1 if the case is outside this kernel's coverage, -cudaError on failure.
@@ -275,51 +341,45 @@ int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) 
   if (lda % 8 || ldb % 8) return 1;
   if ((reinterpret_cast<uintptr_t>(g.A.p) & 15) || (reinterpret_cast<uintptr_t>(g.B.p) & 15)) return 1;
   if (g.M < 512 || g.N < 256 || g.K < 64) return 1;
+  if (g.split_L > 0) {
+    if (g.split_L % 32 || (g.split_Lk / 2) % 32 || g.N != g.split_L + g.split_Lk || g.ldc % 4 || g.split_Lk % 8) return 1;
+    if ((reinterpret_cast<uintptr_t>(g.out_f32) & 15) || (reinterpret_cast<uintptr_t>(g.out_bf16) & 15)) return 1;
+  }
   if (s->pair_clusters < 0) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, G2Smem::TOTAL);
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm2_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, G2Smem<256>::TOTAL);
     if (e != cudaSuccess) return -(int)e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * s->sm_count, 1, 1);
     cfg.blockDim = dim3(G2_THREADS, 1, 1);
-    cfg.dynamicSmemBytes = G2Smem::TOTAL;
+    cfg.dynamicSmemBytes = G2Smem<256>::TOTAL;
     cudaLaunchAttribute at;
     at.id = cudaLaunchAttributeClusterDimension;
     at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
     cfg.attrs = &at; cfg.numAttrs = 1;
     int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, tc_gemm2_kernel, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, tc_gemm2_kernel<256>, &cfg);
     s->pair_clusters = (e == cudaSuccess) ? n : 0;
     if (e != cudaSuccess) (void)cudaGetLastError();
   }
   if (s->pair_clusters < 8) return 1;
-  CUtensorMap tmA, tmB;
-  if (!tc_make_map_2d(s, &tmA, g.A.p, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)lda, G2_BK, G2_BM)) return 1;
-  bool ok;
-  if (!b_mn) ok = tc_make_map_2d(s, &tmB, g.B.p, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)ldb, G2_BK, G2_BN / 2);
-  else ok = tc_make_map_2d(s, &tmB, g.B.p, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)ldb, 64, G2_BK);
-  if (!ok) return 1;
   G2Params p;
   p.M = g.M; p.N = g.N; p.K = g.K;
   p.out_bf16 = g.out_bf16; p.out_f32 = g.out_f32; p.ldc = g.ldc;
   p.tiles_m = (g.M + 2 * G2_BM - 1) / (2 * G2_BM);
-  p.tiles_n = (g.N + G2_BN - 1) / G2_BN;
+  p.tiles_n = 0;
   p.num_kb = (g.K + G2_BK - 1) / G2_BK;
   p.b_mn = b_mn;
   const void* outp = g.out_bf16 ? (const void*)g.out_bf16 : (const void*)g.out_f32;
   const int esz = g.out_bf16 ? 2 : 4;
   p.vec_ok = ((reinterpret_cast<uintptr_t>(outp) & 15) == 0) && ((g.ldc * esz) % 16 == 0);
+  p.split_L = g.split_L; p.split_Lk = g.split_Lk; p.split_shift = g.split_shift; p.seq_len = g.seq_len > 0 ? g.seq_len : 1;
   p.status = d_status;
-  const int tiles = p.tiles_m * p.tiles_n;
-  const int pairs = tiles < s->pair_clusters ? tiles : s->pair_clusters;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2 * pairs, 1, 1);
-  cfg.blockDim = dim3(G2_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = G2Smem::TOTAL;
-  cfg.stream = st;
-  cudaLaunchAttribute at;
-  at.id = cudaLaunchAttributeClusterDimension;
-  at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
-  cfg.attrs = &at; cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm2_kernel, tmA, tmB, p);
-  return e == cudaSuccess ? 0 : -(int)e;
+  // tile width: fewer, fuller waves of CTA pairs win (time of a wave is proportional to the tile width)
+  auto cost = [&](int bn) {
+    const long long tiles = (long long)p.tiles_m * ((g.N + bn - 1) / bn);
+    return ((tiles + s->pair_clusters - 1) / s->pair_clusters) * bn;
+  };
+  // (an MN-major B half of 96 columns would not be a whole number of 64-column swizzle chunks)
+  if (!b_mn && cost(192) < cost(256)) return launch_pair<192>(s, g, p, b_mn, lda, ldb, st);
+  return launch_pair<256>(s, g, p, b_mn, lda, ldb, st);
 }
