@@ -3,7 +3,7 @@
 // Work unit = (one head, one sequence, 128 consecutive tokens).  A persistent CTA walks a contiguous
 // range of units (ordered head-major, so the head's weights are staged once per head) with three roles:
 //
-//   warps 4-11 producers: read the head's channels of the fp32 latent qk0 with coalesced 128-bit loads,
+//   warps 8-15 producers: read the head's channels of the fp32 latent qk0 with coalesced 128-bit loads,
 //              apply conv1_seq (depth-wise, fp32) and write, as bf16 in the 128-byte-swizzled K-major
 //              layout the tensor core reads, the k_ch row-shifted copies
 //                  A_j[rho] = y1[t0 + rho - (k_ch-1) + j]            (Eq. 8, operand of conv2)
@@ -14,7 +14,7 @@
 //              Once a unit's tiles are complete, the first producer thread issues
 //                  acc = sum_j A_j B_j^T + (A_hi + A_lo) I
 //              as tcgen05.mma into one of two TMEM accumulators (128 tokens x d_h, K = d_h * (k_ch + 2)).
-//   warps 0-3  epilogue, one token per thread (= one TMEM lane): L2 norm * sqrt(d_h) (* exp(temp)),
+//   warps 0-7  epilogue, two threads per token (= one TMEM lane), each with half of the rotation pairs: L2 norm * sqrt(d_h) (* exp(temp)),
 //              RoPE, bf16 store.  The norm and the rotation pairs (c, c + d_h/2) are local to the thread.
 //
 // The accumulator is double-buffered, so the epilogue of a unit overlaps the loads of the next one.
@@ -29,8 +29,9 @@ using namespace tc;
 namespace {
 
 constexpr int TR_PRODUCERS = 256;
-constexpr int TR_THREADS = 128 + TR_PRODUCERS;      // 12 warps: registers are granted per 4 warps
-constexpr int TR_MMA_WARP = 4;                      // its lane 0 also issues the MMAs of each unit
+constexpr int TR_EPILOGUE = 256;                    // two threads per token: each takes half of the rotation pairs
+constexpr int TR_THREADS = TR_EPILOGUE + TR_PRODUCERS;
+constexpr int TR_MMA_WARP = TR_EPILOGUE / 32;       // first producer warp: its lane 0 also issues the MMAs of each unit
 enum : unsigned { F_CONV1 = 1, F_CONV2 = 2, F_QK_MEAN = 4, F_QK_NORM = 16, F_ROPE = 32 };
 
 // byte offset of element (row, col) inside a K-major operand tile [rows][DH] stored as DH/64 boxes of
@@ -110,7 +111,7 @@ __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const T
     mbar_init(a_empty, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&acc_full[s], 1);
-      mbar_init(&acc_empty[s], 128);
+      mbar_init(&acc_empty[s], TR_EPILOGUE);
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -124,12 +125,12 @@ __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const T
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp >= 4) {
+  if (warp >= TR_MMA_WARP) {
     // ------------------------------------------------------------------ producers
     // Thread (cq, rg) owns 4 channels and the operand-tile rows [rg*RPG, (rg+1)*RPG).  Tile j row rho holds
     // y1 of token t0 + rho - (KC-1) + j, so the thread needs y1 at KC-1 tokens before its first row as well
     // (recomputed rather than exchanged), and conv1 needs k_seq-1 raw tokens before that.
-    const int pt = threadIdx.x - 128;
+    const int pt = threadIdx.x - TR_EPILOGUE;
     constexpr int CG = DH / 4;                   // channel quads per row
     constexpr int RG = TR_PRODUCERS / CG;        // row groups
     constexpr int RPG = 128 / RG;                // tile rows per thread
@@ -299,12 +300,13 @@ __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const T
       {
         using std::integral_constant;
         bool ok;
-        constexpr int C8 = RPG < 8 ? RPG : 8, C4 = RPG < 4 ? RPG : 4, C2 = RPG < 2 ? RPG : 2;
-        if (n_oth == 1) ok = run_rows(integral_constant<int, C8>{}, integral_constant<int, 1>{});
+        constexpr int C4 = RPG < 4 ? RPG : 4, C2 = RPG < 2 ? RPG : 2;
+        constexpr int C1 = 1;
+        if (n_oth == 1) ok = run_rows(integral_constant<int, C4>{}, integral_constant<int, 1>{});
         else if (n_oth == 2) ok = run_rows(integral_constant<int, C4>{}, integral_constant<int, 2>{});
-        else if (n_oth == 4) ok = run_rows(integral_constant<int, C4>{}, integral_constant<int, 4>{});
-        else if (n_oth == 8) ok = run_rows(integral_constant<int, C2>{}, integral_constant<int, 8>{});
-        else ok = run_rows(integral_constant<int, C4>{}, integral_constant<int, 0>{});
+        else if (n_oth == 4) ok = run_rows(integral_constant<int, C2>{}, integral_constant<int, 4>{});
+        else if (n_oth == 8) ok = run_rows(integral_constant<int, C1>{}, integral_constant<int, 8>{});
+        else ok = run_rows(integral_constant<int, C2>{}, integral_constant<int, 0>{});
         if (!ok) goto done;
       }
       fence_proxy_async();          // generic-proxy smem writes -> visible to the tensor core
@@ -335,8 +337,9 @@ __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const T
   } else {
     // ------------------------------------------------------------------ epilogue, thread = token
     constexpr int HALF = DH / 2;
-    const int rho = threadIdx.x;
-    const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+    constexpr int NCH = (HALF / 16) / 2;             // 16-pair chunks per thread
+    const int rho = threadIdx.x & 127, part = threadIdx.x >> 7;
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
     int it = 0;
     for (int u = u_begin; u < u_end; ++u, ++it) {
       const int h = u / p.units_per_head, rem = u % p.units_per_head;
@@ -350,11 +353,11 @@ __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const T
       // the wait so that the latency hides behind it.  The thread's own position is t0 + rho:
       // cos / sin of (t0 + rho) theta follow from the angle-addition formulas with (cos, sin)(rho * theta_c)
       // evaluated here (rho < 128, so the fast sine's argument stays small after one 2 pi reduction).
-      float4 cs0[HALF / 2];
+      float4 cs0[NCH * 8];
       if (d.flags & F_ROPE) {
-        const float4* tab0 = reinterpret_cast<const float4*>(p.rope + (long long)t0 * HALF);
+        const float4* tab0 = reinterpret_cast<const float4*>(p.rope + (long long)t0 * HALF) + part * NCH * 8;
 #pragma unroll
-        for (int i = 0; i < HALF / 2; ++i) cs0[i] = tab0[i];
+        for (int i = 0; i < NCH * 8; ++i) cs0[i] = tab0[i];
       }
       if (!mbar_wait(&acc_full[buf], (it >> 1) & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
       tc_fence_after();
@@ -371,13 +374,14 @@ __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const T
           for (int i = 0; i < 32; ++i) ss = fmaf(__uint_as_float(r[i]), __uint_as_float(r[i]), ss);
         }
         sc = sqrtf((float)DH) * (is_q ? 1.f : __expf(p.temp[hj])) * rsqrtf(ss);
-        if (valid) p.rnorm[((long long)b * d.S + t) * (d.hq + d.hk) + h] = sc;
+        if (valid && part == 0) p.rnorm[((long long)b * d.S + t) * (d.hq + d.hk) + h] = sc;
       }
       const long long tok = (long long)b * d.S + (valid ? t : 0);
       bf16* dst = is_q ? p.q + tok * d.Lq + h * DH : p.k + tok * d.Lk + hj * DH;
       const float rho_f = (float)rho;
 #pragma unroll
-      for (int c = 0; c < HALF / 16; ++c) {
+      for (int cl = 0; cl < NCH; ++cl) {
+        const int c = part * NCH + cl;                 // this thread's pairs: channels [16c, 16c+16) and + d_h/2
         uint32_t ra[16], rb[16];
         tmem_ld16(acc + c * 16, ra);
         tmem_ld16(acc + HALF + c * 16, rb);
@@ -388,7 +392,7 @@ __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const T
           for (int i = 0; i < 8; ++i) {
             float4 cs;                                                    // (cos, sin) x 2 channels at t0 + rho
             {
-              const float4 z = cs0[c * 8 + i];
+              const float4 z = cs0[cl * 8 + i];
               float sr, cr;
               float ang = rho_f * theta_s[c * 16 + 2 * i];
               float n = rintf(ang * 0.15915494309189535f);
