@@ -42,12 +42,23 @@ struct BwdParams {
 template <int DH>
 struct BwdSmem {
   static constexpr int TILE = 128 * DH * 2;
-  static constexpr int FIX_OFF = 0;                    // two tiles loaded once
-  static constexpr int RING_OFF = 2 * TILE;            // two rings of two tiles
-  static constexpr int BAR_OFF = 6 * TILE;
+  static constexpr int HALF_TILE = 64 * DH * 2;        // 64 queries of Q or dO
+  static constexpr int STAGES = DH == 128 ? 4 : 6;     // ring of (Q, dO) half-tile pairs (shared memory is full at 128)
+  static constexpr int FIX_OFF = 0;                    // K and V tiles, loaded once
+  static constexpr int RING_OFF = 2 * TILE;
+  static constexpr int BAR_OFF = RING_OFF + STAGES * 2 * HALF_TILE;
   static constexpr int STAT_OFF = BAR_OFF + 256;       // float [2 groups][2 buffers][2][128]
   // at least 120 KB so that two CTAs (each wanting all 512 TMEM columns) never share an SM
   static constexpr int TOTAL = (STAT_OFF + 4096 + 1024) > 122880 ? (STAT_OFF + 4096 + 1024) : 122880;
+};
+
+// dQ kernel: Q, dO, three K stages, two V stages
+template <int DH>
+struct DqSmem {
+  static constexpr int TILE = 128 * DH * 2;
+  static constexpr int K_STAGES = 3;
+  static constexpr int BAR_OFF = (4 + K_STAGES) * TILE;
+  static constexpr int TOTAL = (BAR_OFF + 256 + 1024) > 122880 ? (BAR_OFF + 256 + 1024) : 122880;
 };
 
 TC_DEVINL void fail(volatile int* abort_flag, int* status, int code) {
@@ -104,24 +115,25 @@ template <int DH, int POLY>
 __global__ void __launch_bounds__(BW_THREADS, 1)
 tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                       const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO, BwdParams p) {
-  using SM = BwdSmem<DH>;
+  using SM = DqSmem<DH>;
+  constexpr int KS = SM::K_STAGES;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-  unsigned char* sQ = smem + SM::FIX_OFF;
+  unsigned char* sQ = smem;
   unsigned char* sDO = sQ + SM::TILE;
-  unsigned char* sK = smem + SM::RING_OFF;            // [2]
-  unsigned char* sV = sK + 2 * SM::TILE;              // [2]
+  unsigned char* sK = sDO + SM::TILE;                 // [KS]: K_j lives from S(j) (issued a tile ahead) to dQ(j)
+  unsigned char* sV = sK + KS * SM::TILE;             // [2]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFF);
   uint64_t* qdo_full = bars;          // Q and dO tiles loaded
-  uint64_t* k_full = bars + 1;        // [2]
-  uint64_t* k_empty = bars + 3;       // [2]
-  uint64_t* v_full = bars + 5;        // [2]
-  uint64_t* v_empty = bars + 7;       // [2]
-  uint64_t* s_full = bars + 9;        // [2] MMA -> compute: S buffer ready
-  uint64_t* dp_full = bars + 11;      // MMA -> compute: dP ready
-  uint64_t* ds_full = bars + 12;      // compute -> MMA: dS written, dP consumed (all compute threads)
-  uint64_t* dq_done = bars + 13;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
+  uint64_t* k_full = bars + 1;        // [KS]
+  uint64_t* k_empty = bars + 4;       // [KS]
+  uint64_t* v_full = bars + 7;        // [2]
+  uint64_t* v_empty = bars + 9;       // [2]
+  uint64_t* s_full = bars + 11;       // [2] MMA -> compute: S buffer ready
+  uint64_t* dp_full = bars + 13;      // MMA -> compute: dP ready
+  uint64_t* ds_full = bars + 14;      // compute -> MMA: dS written, dP consumed (all compute threads)
+  uint64_t* dq_done = bars + 15;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -135,9 +147,11 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 
   if (threadIdx.x == 0) {
     mbar_init(qdo_full, 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < KS; ++i) {
       mbar_init(&k_full[i], 1);
       mbar_init(&k_empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(&v_full[i], 1);
       mbar_init(&v_empty[i], 1);
       mbar_init(&s_full[i], 1);
@@ -168,11 +182,11 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       tma_tile<DH>(sQ, &tmQ, hi * DH, m0, b, qdo_full);
       tma_tile<DH>(sDO, &tmDO, hi * DH, m0, b, qdo_full);
       for (int j = 0; j < n_kv; ++j) {
-        const int st = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
-        if (!mbar_wait(&k_empty[st], ph ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
-        mbar_expect_tx(&k_full[st], SM::TILE);
-        tma_tile<DH>(sK + st * SM::TILE, &tmK, hj * DH, j * 128, b, &k_full[st]);
+        const int st = j & 1, ks = j % KS;
+        const uint32_t ph = (j >> 1) & 1, kph = (j / KS) & 1;
+        if (!mbar_wait(&k_empty[ks], kph ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
+        mbar_expect_tx(&k_full[ks], SM::TILE);
+        tma_tile<DH>(sK + ks * SM::TILE, &tmK, hj * DH, j * 128, b, &k_full[ks]);
         if (!mbar_wait(&v_empty[st], ph ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
         mbar_expect_tx(&v_full[st], SM::TILE);
         tma_tile<DH>(sV + st * SM::TILE, &tmV, hj * DH, j * 128, b, &v_full[st]);
@@ -202,14 +216,14 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mma_commit(&v_empty[0]);
     }
     for (int j = 0; j < n_kv; ++j) {
-      const int st = j & 1, nx = (j + 1) & 1;
-      const uint32_t nph = ((j + 1) >> 1) & 1;
+      const int st = j & 1, nx = (j + 1) & 1, kst = j % KS, knx = (j + 1) % KS;
+      const uint32_t nph = ((j + 1) >> 1) & 1, knph = ((j + 1) / KS) & 1;
       if (j + 1 < n_kv) {
         // S(j+1) into the other buffer; the dQ MMA that read dS(j-1) from it was issued earlier (in order)
-        if (!wait_all(&k_full[nx], nph)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+        if (!wait_all(&k_full[knx], knph)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
         tc_fence_after();
         if (leader) {
-          mma_kk<DH>(tmem_base + nx * 128, q_lo, k_lo + nx * TILE16, hi_w);
+          mma_kk<DH>(tmem_base + nx * 128, q_lo, k_lo + knx * TILE16, hi_w);
           mma_commit(&s_full[nx]);
         }
       }
@@ -225,8 +239,8 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
       }
       if (leader) {
-        mma_tm<DH>(tmem_base + 384, tmem_base + st * 128, k_mn + st * TILE16, hi_w, j != 0);   // dQ += dS(j) K_j
-        mma_commit(&k_empty[st]);
+        mma_tm<DH>(tmem_base + 384, tmem_base + st * 128, k_mn + kst * TILE16, hi_w, j != 0);   // dQ += dS(j) K_j
+        mma_commit(&k_empty[kst]);
       }
     }
     if (leader) mma_commit(dq_done);
@@ -318,22 +332,22 @@ __global__ void __launch_bounds__(BW_THREADS, 1)
 tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO, BwdParams p) {
   using SM = BwdSmem<DH>;
+  constexpr int NST = SM::STAGES;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   unsigned char* sK = smem + SM::FIX_OFF;
   unsigned char* sV = sK + SM::TILE;
-  unsigned char* sQ = smem + SM::RING_OFF;            // [2]
-  unsigned char* sDO = sQ + 2 * SM::TILE;             // [2]
+  unsigned char* sRing = smem + SM::RING_OFF;         // [NST] stages of (Q half-tile, dO half-tile): 64 queries each
   float* stat = reinterpret_cast<float*>(smem + SM::STAT_OFF);   // [2 buffers][lse2 | delta][128 queries]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFF);
   uint64_t* kv_full = bars;
-  uint64_t* qdo_full = bars + 1;      // [2]
-  uint64_t* qdo_empty = bars + 3;     // [2]
-  uint64_t* sdp_full = bars + 5;      // [2] MMA -> compute: S^T and dP^T of a 64-query sub-tile ready
-  uint64_t* pds_full = bars + 7;      // [2] compute group -> MMA: P^T and dS^T written (256 arrivals)
-  uint64_t* acc_done = bars + 9;
-  uint64_t* stat_ready = bars + 10;   // [2] per compute group: column statistics of the tile are in shared memory
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
+  uint64_t* qdo_full = bars + 1;      // [NST]
+  uint64_t* qdo_empty = bars + 1 + NST;   // [NST]
+  uint64_t* sdp_full = bars + 1 + 2 * NST;   // [2] MMA -> compute: S^T and dP^T of a 64-query sub-tile ready
+  uint64_t* pds_full = sdp_full + 2;  // [2] compute group -> MMA: P^T and dS^T written (256 arrivals)
+  uint64_t* acc_done = pds_full + 2;
+  uint64_t* stat_ready = acc_done + 1;   // [2] per compute group: column statistics of the tile are in shared memory
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(stat_ready + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -349,7 +363,7 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
   if (threadIdx.x == 0) {
     mbar_init(kv_full, 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < NST; ++i) {
       mbar_init(&qdo_full[i], 1);
       mbar_init(&qdo_empty[i], 1);
     }
@@ -383,14 +397,18 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       mbar_expect_tx(kv_full, 2 * SM::TILE);
       tma_tile<DH>(sK, &tmK, hj * DH, n0, b, kv_full);
       tma_tile<DH>(sV, &tmV, hj * DH, n0, b, kv_full);
-      for (int it = 0; it < n_it; ++it) {
-        const int st = it & 1;
-        const uint32_t ph = (it >> 1) & 1;
-        const int hi = hj * p.g + it / n_q, m0 = (i0 + it % n_q) * 128;
+      for (int sub = 0; sub < 2 * n_it; ++sub) {
+        const int it = sub >> 1, st = sub % NST;
+        const uint32_t ph = (sub / NST) & 1;
+        const int hi = hj * p.g + it / n_q, m0 = (i0 + it % n_q) * 128 + (sub & 1) * 64;
         if (!mbar_wait(&qdo_empty[st], ph ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
-        mbar_expect_tx(&qdo_full[st], 2 * SM::TILE);
-        tma_tile<DH>(sQ + st * SM::TILE, &tmQ, hi * DH, m0, b, &qdo_full[st]);
-        tma_tile<DH>(sDO + st * SM::TILE, &tmDO, hi * DH, m0, b, &qdo_full[st]);
+        mbar_expect_tx(&qdo_full[st], 2 * SM::HALF_TILE);
+        unsigned char* dst = sRing + st * 2 * SM::HALF_TILE;
+#pragma unroll
+        for (int c = 0; c < DH / 64; ++c) {
+          tma_load_3d(dst + c * 8192, &tmQ, hi * DH + c * 64, m0, b, &qdo_full[st]);
+          tma_load_3d(dst + SM::HALF_TILE + c * 8192, &tmDO, hi * DH + c * 64, m0, b, &qdo_full[st]);
+        }
       }
     }
   } else if (warp == BW_MMA_WARP) {
@@ -399,36 +417,38 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const bool leader = elect_one();
     const uint32_t hi_w = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
     const uint32_t k_lo = lo_kmajor(smem_u32(sK)), v_lo = lo_kmajor(smem_u32(sV));
-    const uint32_t q_lo = lo_kmajor(smem_u32(sQ)), do_lo = lo_kmajor(smem_u32(sDO));
-    const uint32_t q_mn = lo_mnmajor(smem_u32(sQ)), do_mn = lo_mnmajor(smem_u32(sDO));
-    constexpr uint32_t TILE16 = SM::TILE >> 4;
-    constexpr uint32_t HALF16 = (64 * 128) >> 4;       // 64 query rows further down a tile
+    const uint32_t ring16 = smem_u32(sRing) >> 4;
+    constexpr uint32_t STAGE16 = (2 * SM::HALF_TILE) >> 4, HALF16 = SM::HALF_TILE >> 4;
     const int n_sub = 2 * n_it;
     auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
       return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
     };
+    // half-tiles are [64 rows][DH] as DH/64 boxes of 8 KB
     auto issue_sdp = [&](int sub) {     // S^T = K Q^T and dP^T = V dO^T for 64 queries
-      const int it = sub >> 1, st = it & 1, hf = sub & 1, sb = sub & 1;
+      const int sb = sub & 1;
       const uint32_t idesc = idesc_bf16(64, 0, 0);
-      const uint32_t qb = q_lo + st * TILE16 + hf * HALF16, ob = do_lo + st * TILE16 + hf * HALF16;
+      const uint32_t qb = (ring16 + (sub % NST) * STAGE16) | (1u << 16), ob = qb + HALF16;
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < DH / 16; ++kk) {
-          const uint32_t off = (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
-          mma_ss_w(tmem_base + sb * 64, k_lo + off, hi_w, qb + off, hi_w, idesc, kk != 0);
+          const uint32_t offk = (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+          const uint32_t offq = (uint32_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4);
+          mma_ss_w(tmem_base + sb * 64, k_lo + offk, hi_w, qb + offq, hi_w, idesc, kk != 0);
         }
 #pragma unroll
         for (int kk = 0; kk < DH / 16; ++kk) {
-          const uint32_t off = (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
-          mma_ss_w(tmem_base + 128 + sb * 64, v_lo + off, hi_w, ob + off, hi_w, idesc, kk != 0);
+          const uint32_t offk = (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+          const uint32_t offq = (uint32_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4);
+          mma_ss_w(tmem_base + 128 + sb * 64, v_lo + offk, hi_w, ob + offq, hi_w, idesc, kk != 0);
         }
         mma_commit(&sdp_full[sb]);
       }
     };
     auto issue_dvdk = [&](int sub) {    // dV += P^T dO, dK += dS^T Q over the sub-tile's 64 queries
-      const int it = sub >> 1, st = it & 1, hf = sub & 1, sb = sub & 1;
+      const int sb = sub & 1, st = sub % NST;
       const uint32_t idesc = idesc_bf16(DH, 0, 1);
-      const uint32_t ob = do_mn + st * TILE16 + hf * HALF16, qb = q_mn + st * TILE16 + hf * HALF16;
+      // read along the rows (N = d_h contiguous): 64-channel chunks are one 8 KB box apart
+      const uint32_t qb = (ring16 + st * STAGE16) | ((8192u >> 4) << 16), ob = qb + HALF16;
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)
@@ -438,26 +458,25 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         for (int kk = 0; kk < 4; ++kk)
           mma_ts_w(tmem_base + 384, tmem_base + 128 + sb * 64 + (kk >> 1) * 32 + (kk & 1) * 8, qb + kk * (2048 >> 4), hi_w,
                    idesc, (sub | kk) != 0);
-        if (hf == 1) mma_commit(&qdo_empty[st]);
+        mma_commit(&qdo_empty[st]);
       }
     };
     if (!wait_all(kv_full, 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
-    if (!wait_all(&qdo_full[0], 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
-    tc_fence_after();
-    issue_sdp(0);
-    issue_sdp(1);
+    for (int s0 = 0; s0 < 2 && s0 < n_sub; ++s0) {
+      if (!wait_all(&qdo_full[s0 % NST], (s0 / NST) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+      tc_fence_after();
+      issue_sdp(s0);
+    }
     for (int sub = 0; sub < n_sub; ++sub) {
       // sub-tile sub belongs to compute group sub & 1
       if (!wait_all(&pds_full[sub & 1], (sub >> 1) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
       tc_fence_after();
       issue_dvdk(sub);
       if (sub + 2 < n_sub) {
-        const int nit = (sub + 2) >> 1;
-        if ((sub & 1) == 0) {
-          if (!wait_all(&qdo_full[nit & 1], (nit >> 1) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
-          tc_fence_after();
-        }
-        issue_sdp(sub + 2);        // into the buffer whose P^T / dS^T the MMAs just issued are reading (in order)
+        const int nx = sub + 2;
+        if (!wait_all(&qdo_full[nx % NST], (nx / NST) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+        tc_fence_after();
+        issue_sdp(nx);             // into the buffer whose P^T / dS^T the MMAs just issued are reading (in order)
       }
     }
     if (leader) mma_commit(acc_done);
@@ -578,10 +597,11 @@ done:
 
 template <int DH, int POLY>
 int launch_bwd(TcState* s, const CcaDims& d, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
-               const CUtensorMap& tmDO, const BwdParams& p, cudaStream_t st) {
+               const CUtensorMap& tmDO, const CUtensorMap& tmQh, const CUtensorMap& tmDOh, const BwdParams& p,
+               cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tc_attn_bwd_dq_kernel<DH, POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<DH>::TOTAL);
+    cudaError_t e = cudaFuncSetAttribute(tc_attn_bwd_dq_kernel<DH, POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<DH>::TOTAL);
     if (e != cudaSuccess) return -(int)e;
     e = cudaFuncSetAttribute(tc_attn_bwd_dkv_kernel<DH, POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<DH>::TOTAL);
     if (e != cudaSuccess) return -(int)e;
@@ -589,10 +609,10 @@ int launch_bwd(TcState* s, const CcaDims& d, const CUtensorMap& tmQ, const CUten
   }
   const long long g_kv = (long long)p.n_tiles * d.B * d.hk, g_q = (long long)p.n_tiles * d.B * d.hq;
   if (g_q > 0x7fffffffLL) return 1;
-  tc_attn_bwd_dkv_kernel<DH, POLY><<<(unsigned)g_kv, BW_THREADS, BwdSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, tmDO, p);
+  tc_attn_bwd_dkv_kernel<DH, POLY><<<(unsigned)g_kv, BW_THREADS, BwdSmem<DH>::TOTAL, st>>>(tmQh, tmK, tmV, tmDOh, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return -(int)e;
-  tc_attn_bwd_dq_kernel<DH, POLY><<<(unsigned)g_q, BW_THREADS, BwdSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, tmDO, p);
+  tc_attn_bwd_dq_kernel<DH, POLY><<<(unsigned)g_q, BW_THREADS, DqSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, tmDO, p);
   e = cudaGetLastError();
   return e == cudaSuccess ? 0 : -(int)e;
 }
@@ -609,6 +629,9 @@ int tc_attn_bwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, cons
   const uint64_t S = (uint64_t)d.S, B = (uint64_t)d.B, Lq = (uint64_t)d.Lq, Lk = (uint64_t)d.Lk;
   if (!tc_make_map_3d(s, &tmQ, q, Lq, S, B, Lq, S * Lq, 64, 128)) return 1;
   if (!tc_make_map_3d(s, &tmDO, d_o, Lq, S, B, Lq, S * Lq, 64, 128)) return 1;
+  CUtensorMap tmQh, tmDOh;       // 64-row boxes for the dK/dV kernel's half-tiles
+  if (!tc_make_map_3d(s, &tmQh, q, Lq, S, B, Lq, S * Lq, 64, 64)) return 1;
+  if (!tc_make_map_3d(s, &tmDOh, d_o, Lq, S, B, Lq, S * Lq, 64, 64)) return 1;
   if (!tc_make_map_3d(s, &tmK, k, Lk, S, B, Lk, S * Lk, 64, 128)) return 1;
   if (!tc_make_map_3d(s, &tmV, v, Lk, S, B, Lk, S * Lk, 64, 128)) return 1;
   BwdParams p;
@@ -618,11 +641,11 @@ int tc_attn_bwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, cons
   p.status = d_status;
   const int poly = s->attn_poly_bwd;
   if (d.dh == 128) {
-    if (poly == 0) return launch_bwd<128, 0>(s, d, tmQ, tmK, tmV, tmDO, p, st);
-    if (poly == 2) return launch_bwd<128, 2>(s, d, tmQ, tmK, tmV, tmDO, p, st);
-    return launch_bwd<128, 1>(s, d, tmQ, tmK, tmV, tmDO, p, st);
+    if (poly == 0) return launch_bwd<128, 0>(s, d, tmQ, tmK, tmV, tmDO, tmQh, tmDOh, p, st);
+    if (poly == 2) return launch_bwd<128, 2>(s, d, tmQ, tmK, tmV, tmDO, tmQh, tmDOh, p, st);
+    return launch_bwd<128, 1>(s, d, tmQ, tmK, tmV, tmDO, tmQh, tmDOh, p, st);
   }
-  if (poly == 0) return launch_bwd<64, 0>(s, d, tmQ, tmK, tmV, tmDO, p, st);
-  if (poly == 2) return launch_bwd<64, 2>(s, d, tmQ, tmK, tmV, tmDO, p, st);
-  return launch_bwd<64, 1>(s, d, tmQ, tmK, tmV, tmDO, p, st);
+  if (poly == 0) return launch_bwd<64, 0>(s, d, tmQ, tmK, tmV, tmDO, tmQh, tmDOh, p, st);
+  if (poly == 2) return launch_bwd<64, 2>(s, d, tmQ, tmK, tmV, tmDO, tmQh, tmDOh, p, st);
+  return launch_bwd<64, 1>(s, d, tmQ, tmK, tmV, tmDO, tmQh, tmDOh, p, st);
 }
