@@ -7,7 +7,7 @@
 //                warps 4-7 columns 64-127 (thread = query row = TMEM lane; two threads per row keep four
 //                warps per scheduler busy, which the latency of the per-element chain needs)
 //   warps 8-15 : the same for query tile 1
-//   warp  16   : TMA loader (Q tiles once, then a 2-stage ring of K and of V tiles)
+//   warp  16   : TMA loader (Q tiles once, then one ring shared by the K and V tiles)
 //   warp  17   : TMEM owner and MMA issuer
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+DH) O1 [384,384+DH).  The bf16 probabilities P
@@ -31,7 +31,7 @@ namespace {
 constexpr int AT_SOFTMAX_WARPS = 16;                 // 2 query tiles x 2 column halves x 4 lane quarters
 constexpr int AT_TMA_WARP = AT_SOFTMAX_WARPS, AT_MMA_WARP = AT_SOFTMAX_WARPS + 1;
 constexpr int AT_THREADS = 32 * (AT_SOFTMAX_WARPS + 2);
-constexpr int BQ = 128, BKV = 128, KV_STAGES = 2;
+constexpr int BQ = 128, BKV = 128;
 constexpr float LOG2E_F = 1.4426950408889634f;
 constexpr float LN2_F = 0.6931471805599453f;
 constexpr float RESCALE_THRESHOLD = 8.0f;      // log2 units
@@ -50,12 +50,15 @@ template <int DH>
 struct AttnSmem {
   static constexpr int TILE_BYTES = 128 * DH * 2;            // one 128-row tile of Q, K or V
   static constexpr int Q_OFF = 0;
-  static constexpr int K_OFF = 2 * TILE_BYTES;
-  static constexpr int V_OFF = K_OFF + KV_STAGES * TILE_BYTES;
-  static constexpr int BAR_OFF = V_OFF + KV_STAGES * TILE_BYTES;
-  // at least 120 KB so that two CTAs (each wanting all 512 TMEM columns) never share an SM
-  static constexpr int XCH_OFF = BAR_OFF + 512;              // float [2 tiles][2 halves][128 rows]: max / sum exchange
-  static constexpr int TOTAL = (XCH_OFF + 2048 + 1024) > 122880 ? (XCH_OFF + 2048 + 1024) : 122880;
+  // K and V tiles share one ring, filled and released in the order K_0 V_0 K_1 V_1 ... (that is also the order
+  // in which the MMAs finish with them): 5 slots at d_h = 128 fill the shared memory, 2.5 tiles of each ahead
+  static constexpr int NSLOT = DH == 128 ? 5 : 8;
+  static constexpr int KV_OFF = 2 * TILE_BYTES;
+  static constexpr int BAR_OFF = KV_OFF + NSLOT * TILE_BYTES;
+  static constexpr int XCH_OFF = BAR_OFF + 256;              // float [2 tiles][2 halves][128 rows]: max / sum exchange
+  // no slack for alignment: the kernel checks that its dynamic shared memory starts on a 1024-byte boundary.
+  // At least 120 KB so that two CTAs (each wanting all 512 TMEM columns) never share an SM.
+  static constexpr int TOTAL = (XCH_OFF + 2048) > 122880 ? (XCH_OFF + 2048) : 122880;
 };
 
 TC_DEVINL void fail(volatile int* abort_flag, int* status, int code) {
@@ -112,18 +115,21 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                    const __grid_constant__ CUtensorMap tmV, AttnParams p) {
   using SM = AttnSmem<DH>;
   constexpr int NBOX = DH / 64;
-  extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  constexpr int NS = SM::NSLOT;
+  extern __shared__ __align__(1024) unsigned char smem_dyn[];
+  unsigned char* smem = smem_dyn;
+  if (smem_u32(smem) & 1023u) {       // the swizzled tiles need it; nothing has been set up yet, so just report
+    if (threadIdx.x == 0) atomicCAS(p.status, 0, ST_BAD_SMEM_ALIGNMENT);
+    return;
+  }
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFF);
   uint64_t* q_full = bars;            // [2]
-  uint64_t* k_full = bars + 2;        // [KV_STAGES]
-  uint64_t* k_empty = bars + 4;
-  uint64_t* v_full = bars + 6;
-  uint64_t* v_empty = bars + 8;
-  uint64_t* s_full = bars + 10;       // [2]  MMA -> softmax: S tile ready
-  uint64_t* p_full = bars + 12;       // [2]  softmax -> MMA: P tile written
-  uint64_t* o_done = bars + 14;       // [2]  MMA -> softmax: last P V finished
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint64_t* kv_full = bars + 2;       // [NS]  slot of the n-th tile of the sequence K_0 V_0 K_1 V_1 ...: n % NS
+  uint64_t* kv_empty = bars + 2 + NS; // [NS]
+  uint64_t* s_full = bars + 2 + 2 * NS;   // [2]  MMA -> softmax: S tile ready
+  uint64_t* p_full = s_full + 2;      // [2]  softmax -> MMA: P tile written
+  uint64_t* o_done = p_full + 2;      // [2]  MMA -> softmax: last P V finished
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_done + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -146,13 +152,13 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(&q_full[i], 1);
-      mbar_init(&k_full[i], 1);
-      mbar_init(&k_empty[i], 1);
-      mbar_init(&v_full[i], 1);
-      mbar_init(&v_empty[i], 1);
       mbar_init(&s_full[i], 1);
       mbar_init(&p_full[i], 256);
       mbar_init(&o_done[i], 1);
+    }
+    for (int i = 0; i < NS; ++i) {
+      mbar_init(&kv_full[i], 1);
+      mbar_init(&kv_empty[i], 1);
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -181,19 +187,15 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           tma_load_3d(smem + SM::Q_OFF + s * SM::TILE_BYTES + c * 16384, &tmQ, hi * DH + c * 64, blk * 256 + s * BQ, b,
                       &q_full[s]);
       }
-      for (int j = 0; j < n_max; ++j) {
-        const int st = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
-        if (!mbar_wait(&k_empty[st], ph ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
-        mbar_expect_tx(&k_full[st], SM::TILE_BYTES);
+      for (int n = 0; n < 2 * n_max; ++n) {        // n-th tile of K_0 V_0 K_1 V_1 ...
+        const int j = n >> 1, sl = n % NS;
+        const uint32_t ph = (n / NS) & 1;
+        if (!mbar_wait(&kv_empty[sl], ph ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
+        mbar_expect_tx(&kv_full[sl], SM::TILE_BYTES);
 #pragma unroll
         for (int c = 0; c < NBOX; ++c)
-          tma_load_3d(smem + SM::K_OFF + st * SM::TILE_BYTES + c * 16384, &tmK, hj * DH + c * 64, j * BKV, b, &k_full[st]);
-        if (!mbar_wait(&v_empty[st], ph ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
-        mbar_expect_tx(&v_full[st], SM::TILE_BYTES);
-#pragma unroll
-        for (int c = 0; c < NBOX; ++c)
-          tma_load_3d(smem + SM::V_OFF + st * SM::TILE_BYTES + c * 16384, &tmV, hj * DH + c * 64, j * BKV, b, &v_full[st]);
+          tma_load_3d(smem + SM::KV_OFF + sl * SM::TILE_BYTES + c * 16384, (n & 1) ? &tmV : &tmK, hj * DH + c * 64, j * BKV, b,
+                      &kv_full[sl]);
       }
     }
   } else if (warp == AT_MMA_WARP) {
@@ -207,14 +209,14 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // descriptor words: low = address >> 4 | leading offset << 16, high = stride offset, version, swizzle
       const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
       const uint32_t q_lo = (smem_u32(smem + SM::Q_OFF) >> 4) | (1u << 16);
-      const uint32_t k_lo = (smem_u32(smem + SM::K_OFF) >> 4) | (1u << 16);
-      const uint32_t v_lo = (smem_u32(smem + SM::V_OFF) >> 4) | ((16384u >> 4) << 16);   // 64-channel chunks 16 KB apart
+      const uint32_t k_lo = (smem_u32(smem + SM::KV_OFF) >> 4) | (1u << 16);
+      const uint32_t v_lo = (smem_u32(smem + SM::KV_OFF) >> 4) | ((16384u >> 4) << 16);   // 64-channel chunks 16 KB apart
       constexpr uint32_t TILE16 = SM::TILE_BYTES >> 4;
       auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
         return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
       };
       auto issue_s = [&](int s, int j) {      // S_s = Q_s K_j^T
-        const uint32_t qa = q_lo + s * TILE16, ka = k_lo + (j & 1) * TILE16;
+        const uint32_t qa = q_lo + s * TILE16, ka = k_lo + ((2 * j) % NS) * TILE16;
         if (leader) {
 #pragma unroll
           for (int kk = 0; kk < DH / 16; ++kk) {
@@ -224,7 +226,7 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
       };
       auto issue_pv = [&](int s, int j) {     // O_s (+)= P_s V_j
-        const uint32_t va = v_lo + (j & 1) * TILE16;
+        const uint32_t va = v_lo + ((2 * j + 1) % NS) * TILE16;
         if (leader) {
 #pragma unroll
           for (int kk = 0; kk < BKV / 16; ++kk)
@@ -237,7 +239,7 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       };
       // prologue: first S tile of each query tile
       if (n_max > 0) {
-        if (!wait_all(&k_full[0], 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+        if (!wait_all(&kv_full[0], 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
         tc_fence_after();
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
@@ -249,21 +251,21 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
       }
       for (int j = 0; j < n_max; ++j) {
-        const int st = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
+        const int vsl = (2 * j + 1) % NS;
+        const uint32_t vph = ((2 * j + 1) / NS) & 1;
         // all S(j) were issued before this point: release K_j when they complete
-        commit(&k_empty[st]);
+        commit(&kv_empty[(2 * j) % NS]);
         bool k_next_ready = false;
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
           if (j >= n_s[s]) continue;
           if (!wait_all(&p_full[s], j & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
-          if (!wait_all(&v_full[st], ph)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+          if (!wait_all(&kv_full[vsl], vph)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
           tc_fence_after();
           issue_pv(s, j);
           if (j + 1 < n_s[s]) {
             if (!k_next_ready) {
-              if (!wait_all(&k_full[(j + 1) & 1], ((j + 1) >> 1) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+              if (!wait_all(&kv_full[(2 * j + 2) % NS], ((2 * j + 2) / NS) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
               tc_fence_after();
               k_next_ready = true;
             }
@@ -273,7 +275,7 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             commit(&o_done[s]);
           }
         }
-        commit(&v_empty[st]);
+        commit(&kv_empty[vsl]);
       }
     }
   } else {

@@ -13,7 +13,7 @@ namespace tc {
 
 // Device status codes written to the handle's status word when a bounded wait gives up.
 enum : int { ST_OK = 0, ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_EPI = 103, ST_TIMEOUT_SOFTMAX = 104,
-             ST_TIMEOUT_CORR = 105 };
+             ST_TIMEOUT_CORR = 105, ST_BAD_SMEM_ALIGNMENT = 110 };
 
 constexpr long long WAIT_CYCLES = 4000000000LL;   // about 2 s at 2 GHz: far beyond any legitimate wait
 
