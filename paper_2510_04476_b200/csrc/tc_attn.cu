@@ -127,8 +127,8 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   uint64_t* kv_full = bars + 2;       // [NS]  slot of the n-th tile of the sequence K_0 V_0 K_1 V_1 ...: n % NS
   uint64_t* kv_empty = bars + 2 + NS; // [NS]
   uint64_t* s_full = bars + 2 + 2 * NS;   // [2]  MMA -> softmax: S tile ready
-  uint64_t* p_full = s_full + 2;      // [2]  softmax -> MMA: P tile written
-  uint64_t* o_done = p_full + 2;      // [2]  MMA -> softmax: last P V finished
+  uint64_t* p_full = s_full + 2;      // [2 tiles][2]  softmax -> MMA: first / second 32 keys of every thread's P written
+  uint64_t* o_done = p_full + 4;      // [2]  MMA -> softmax: last P V finished
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_done + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -153,7 +153,8 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     for (int i = 0; i < 2; ++i) {
       mbar_init(&q_full[i], 1);
       mbar_init(&s_full[i], 1);
-      mbar_init(&p_full[i], 256);
+      mbar_init(&p_full[2 * i], 256);
+      mbar_init(&p_full[2 * i + 1], 256);
       mbar_init(&o_done[i], 1);
     }
     for (int i = 0; i < NS; ++i) {
@@ -225,13 +226,17 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           }
         }
       };
-      auto issue_pv = [&](int s, int j) {     // O_s (+)= P_s V_j
+      // O_s (+)= P_s V_j over the keys whose P is complete after the softmax threads' chunk hf: each thread owns
+      // 64 keys (k-steps 0-3 or 4-7) and finishes them 32 at a time, so chunk hf covers k-steps {2hf, 2hf+1, 4+2hf, 5+2hf}
+      auto issue_pv = [&](int s, int j, int hf) {
         const uint32_t va = v_lo + ((2 * j + 1) % NS) * TILE16;
         if (leader) {
 #pragma unroll
-          for (int kk = 0; kk < BKV / 16; ++kk)
+          for (int i = 0; i < 4; ++i) {
+            const int kk = (i >> 1) * 4 + 2 * hf + (i & 1);
             mma_ts_w(tmem_base + 256 + s * 128, tmem_base + s * 128 + (kk >> 2) * 64 + (kk & 3) * 8, va + kk * (2048 >> 4),
-                     desc_hi, idesc_o, (j | kk) != 0);
+                     desc_hi, idesc_o, (j | hf | i) != 0);
+          }
         }
       };
       auto commit = [&](uint64_t* bar) {
@@ -259,10 +264,13 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
           if (j >= n_s[s]) continue;
-          if (!wait_all(&p_full[s], j & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+          if (!wait_all(&p_full[2 * s], j & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
           if (!wait_all(&kv_full[vsl], vph)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
           tc_fence_after();
-          issue_pv(s, j);
+          issue_pv(s, j, 0);                 // runs while the softmax threads finish their second 32 keys
+          if (!wait_all(&p_full[2 * s + 1], j & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+          tc_fence_after();
+          issue_pv(s, j, 1);
           if (j + 1 < n_s[s]) {
             if (!k_next_ready) {
               if (!wait_all(&kv_full[(2 * j + 2) % NS], ((2 * j + 2) / NS) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
@@ -370,15 +378,15 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           for (int c = 0; c < 4; ++c) exp8<POLY, true>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
         }
         tmem_st16(s_tmem + part * 64 + hf * 16, pk);
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(&p_full[2 * s + hf]);
       }
       {
         uint32_t a, b;
         unpack2u(sum2, a, b);
         l_run += __uint_as_float(a) + __uint_as_float(b);
       }
-      tmem_st_wait();
-      tc_fence_before();
-      mbar_arrive(&p_full[s]);
     }
     if (n_s[s] > 0) {
       // total of the two halves of the row
