@@ -3,15 +3,13 @@
 // 128-row tiles that ping-pong: while the softmax warps of one tile work on S = Q K^T, the tensor core
 // runs the other tile's MMAs.
 //
-//   warps 0-7  : softmax + epilogue of query tile 0: warps 0-3 take score columns 0-63 of a KV tile,
-//                warps 4-7 columns 64-127 (thread = query row = TMEM lane; two threads per row keep four
-//                warps per scheduler busy, which the latency of the per-element chain needs)
-//   warps 8-15 : the same for query tile 1
+//   warps 0-15 : softmax + epilogue; all of them work on one query tile at a time, alternating between the
+//                two tiles (thread = query row = TMEM lane; warps 4p..4p+3 take score columns [32p, 32p+32))
 //   warp  16   : TMA loader (Q tiles once, then one ring shared by the K and V tiles)
 //   warp  17   : TMEM owner and MMA issuer
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+DH) O1 [384,384+DH).  The bf16 probabilities P
-// overwrite columns [0,32) and [64,96) of their S tile and feed the P V MMA directly from TMEM.
+// overwrite the first 16 of every 32 columns of their S tile and feed the P V MMA directly from TMEM.
 // Softmax: with L2-normalised q and k (Eq. 11) every logit is bounded by sqrt(d_h) * beta, so that bound
 // serves as a fixed row maximum: no max pass, no rescale of O (the kernel falls back to the online form,
 // with a lazy rescale when the running maximum grows by more than 2^8, if the latents are not normalised
@@ -153,8 +151,8 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     for (int i = 0; i < 2; ++i) {
       mbar_init(&q_full[i], 1);
       mbar_init(&s_full[i], 1);
-      mbar_init(&p_full[2 * i], 256);
-      mbar_init(&p_full[2 * i + 1], 256);
+      mbar_init(&p_full[2 * i], 512);
+      mbar_init(&p_full[2 * i + 1], 512);
       mbar_init(&o_done[i], 1);
     }
     for (int i = 0; i < NS; ++i) {
@@ -227,14 +225,14 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
       };
       // O_s (+)= P_s V_j over the keys whose P is complete after the softmax threads' chunk hf: each thread owns
-      // 64 keys (k-steps 0-3 or 4-7) and finishes them 32 at a time, so chunk hf covers k-steps {2hf, 2hf+1, 4+2hf, 5+2hf}
+      // 32 keys (k-steps 2 part, 2 part + 1) and finishes them 16 at a time, so chunk hf covers k-steps {hf, 2+hf, 4+hf, 6+hf}
       auto issue_pv = [&](int s, int j, int hf) {
         const uint32_t va = v_lo + ((2 * j + 1) % NS) * TILE16;
         if (leader) {
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const int kk = (i >> 1) * 4 + 2 * hf + (i & 1);
-            mma_ts_w(tmem_base + 256 + s * 128, tmem_base + s * 128 + (kk >> 2) * 64 + (kk & 3) * 8, va + kk * (2048 >> 4),
+            const int kk = 2 * i + hf;
+            mma_ts_w(tmem_base + 256 + s * 128, tmem_base + s * 128 + (kk >> 1) * 32 + (kk & 1) * 8, va + kk * (2048 >> 4),
                      desc_hi, idesc_o, (j | hf | i) != 0);
           }
         }
@@ -288,16 +286,14 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     }
   } else {
     // ---------------------------------------------------------------- softmax + epilogue
-    const int s = warp >> 3;                         // query tile of this warp
-    const int part = (warp >> 2) & 1;                // which 64 score columns of each KV tile
-    const int row = threadIdx.x & 127;
+    // All 16 warps work on one query tile at a time, alternating between the two tiles in the order the MMA
+    // warp produces their S: a tile's softmax then takes half as long as with eight warps per tile, which is
+    // what bounds the loop (the tile waits for its own softmax and then for its own two MMAs).
+    const int part = warp >> 2;                      // which 32 score columns of each KV tile
+    const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t s_tmem = tmem_base + lane_sel + s * 128;          // S tile; P goes to its first 64 columns
-    const uint32_t o_tmem = tmem_base + lane_sel + 256 + s * 128;
-    float* xch = reinterpret_cast<float*>(smem + SM::XCH_OFF) + s * 256;   // [2 halves][128 rows]
-    const int bar_id = 1 + s;                        // named barrier of the 256 threads of this tile
-    const int m0 = blk * 256 + s * BQ;
-    const int tq = m0 + row;
+    float* xch = reinterpret_cast<float*>(smem + SM::XCH_OFF);     // [4 parts][128 rows]
+    auto sync_softmax = [&]() { asm volatile("bar.sync 1, 512;" ::: "memory"); };
     const float c_scale = rsqrtf((float)DH) * LOG2E_F;
     // Fixed maximum: |q| = sqrt(d_h), |k| = sqrt(d_h) beta, so the scaled logit (log2 units) is at most
     // sqrt(d_h) beta log2(e); 1 % covers the bf16 rounding of q and k.  Used while 2^(-2 bound) is a normal
@@ -309,104 +305,116 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       fixed = m_fixed <= 56.f;
     }
     const uint64_t scale2 = pack2f(c_scale, c_scale);
-    float m_run = fixed ? m_fixed : -INFINITY, l_run = 0.f;
-    for (int j = 0; j < n_s[s]; ++j) {
-      if (!mbar_wait(&s_full[s], j & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
-      tc_fence_after();
-      const int k0 = j * BKV + part * 64;            // first key of this thread's columns
-      const bool need_mask = (p.causal && j * BKV + BKV - 1 > m0) || (j * BKV + BKV > p.S);
-      const int lim = p.causal ? min(tq, p.S - 1) : p.S - 1;       // last visible key
-      float m_use = m_run;
-      if (!fixed) {
-        // first pass over this thread's 64 scores for the row maximum (they are read again below)
-        float mx = -INFINITY;
+    float m_run[2] = {fixed ? m_fixed : -INFINITY, fixed ? m_fixed : -INFINITY}, l_run[2] = {0.f, 0.f};
+    for (int j = 0; j < n_max; ++j) {
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          uint32_t v[32];
-          tmem_ld32(s_tmem + part * 64 + hf * 32, v);
-          tmem_ld_wait();
-#pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (!need_mask || k0 + hf * 32 + c <= lim) mx = fmaxf(mx, __uint_as_float(v[c]));
-        }
-        // the other half of the row is another thread's: exchange through shared memory
-        xch[part * 128 + row] = mx;
-        asm volatile("bar.sync %0, 256;" ::"r"(bar_id) : "memory");
-        mx = fmaxf(mx, xch[(part ^ 1) * 128 + row]) * c_scale;
-        asm volatile("bar.sync %0, 256;" ::"r"(bar_id) : "memory");
-        const bool grow = mx > m_run + RESCALE_THRESHOLD;           // also true on the first tile
-        if (grow) m_use = mx;
-        if (m_use == -INFINITY) m_use = 0.f;
-        if (j > 0 && __any_sync(0xffffffffu, grow)) {
-          // rescale this thread's half of the running output (rare)
-          const float alpha = grow ? exp2f(m_run - m_use) : 1.f;
-          l_run *= alpha;
-#pragma unroll 1
-          for (int c = 0; c < DH / 64; ++c) {
-            uint32_t t[32];
-            tmem_ld32(o_tmem + part * (DH / 2) + c * 32, t);
+      for (int s = 0; s < 2; ++s) {
+        if (j >= n_s[s]) continue;
+        const uint32_t s_tmem = tmem_base + lane_sel + s * 128 + part * 32;   // this thread's 32 S columns
+        const uint32_t o_tmem = tmem_base + lane_sel + 256 + s * 128;
+        const int m0 = blk * 256 + s * BQ;
+        const int tq = m0 + row;
+        if (!mbar_wait(&s_full[s], j & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+        tc_fence_after();
+        const int k0 = j * BKV + part * 32;            // first key of this thread's columns
+        const bool need_mask = (p.causal && j * BKV + BKV - 1 > m0) || (j * BKV + BKV > p.S);
+        const int lim = p.causal ? min(tq, p.S - 1) : p.S - 1;       // last visible key
+        float m_use = m_run[s];
+        if (!fixed) {
+          // first pass over this thread's 32 scores for the row maximum (they are read again below)
+          float mx = -INFINITY;
+          {
+            uint32_t v[32];
+            tmem_ld32(s_tmem, v);
             tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) t[i] = __float_as_uint(__uint_as_float(t[i]) * alpha);
-            tmem_st32(o_tmem + part * (DH / 2) + c * 32, t);
+            for (int c = 0; c < 32; ++c)
+              if (!need_mask || k0 + c <= lim) mx = fmaxf(mx, __uint_as_float(v[c]));
           }
+          // the rest of the row belongs to three other threads: exchange through shared memory
+          xch[part * 128 + row] = mx;
+          sync_softmax();
+          mx = fmaxf(fmaxf(xch[row], xch[128 + row]), fmaxf(xch[256 + row], xch[384 + row])) * c_scale;
+          sync_softmax();
+          const bool grow = mx > m_run[s] + RESCALE_THRESHOLD;        // also true on the first tile
+          if (grow) m_use = mx;
+          if (m_use == -INFINITY) m_use = 0.f;
+          if (j > 0 && __any_sync(0xffffffffu, grow)) {
+            // rescale this thread's quarter of the running output (rare)
+            const float alpha = grow ? exp2f(m_run[s] - m_use) : 1.f;
+            l_run[s] *= alpha;
+#pragma unroll 1
+            for (int c = 0; c < DH / 64; ++c) {
+              uint32_t t[16];
+              tmem_ld16(o_tmem + part * (DH / 4) + c * 16, t);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 16; ++i) t[i] = __float_as_uint(__uint_as_float(t[i]) * alpha);
+              tmem_st16(o_tmem + part * (DH / 4) + c * 16, t);
+            }
+            tmem_st_wait();
+          }
+          m_run[s] = m_use;
+        }
+        const uint64_t negm2 = pack2f(-m_use, -m_use);
+        uint64_t sum2 = pack2f(0.f, 0.f);
+        // 16 scores at a time.  The bf16 pairs of P go over the S columns the same thread has already read:
+        // part p reads S columns [32p, 32p+32) and writes P into storage columns [32p, 32p+16); after each
+        // chunk the MMA warp may start on those keys.
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t v[16], pk[8];
+          tmem_ld16(s_tmem + hf * 16, v);
+          tmem_ld_wait();
+          if (need_mask) {
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+              if (k0 + hf * 16 + c > lim) v[c] = 0xff800000u;        // -inf
+#pragma unroll
+            for (int c = 0; c < 2; ++c) exp8<0, false>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
+          } else if (fixed) {
+#pragma unroll
+            for (int c = 0; c < 2; ++c) exp8<POLY, false>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 2; ++c) exp8<POLY, true>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
+          }
+          tmem_st8(s_tmem + hf * 8, pk);
           tmem_st_wait();
+          tc_fence_before();
+          mbar_arrive(&p_full[2 * s + hf]);
         }
-        m_run = m_use;
-      }
-      const uint64_t negm2 = pack2f(-m_use, -m_use);
-      uint64_t sum2 = pack2f(0.f, 0.f);
-      // 32 scores at a time.  The bf16 pairs of P go over the S columns the same thread has already read:
-      // part p reads S columns [64p, 64p+64) and writes P into storage columns [64p, 64p+32), so P of a
-      // KV tile sits in two separate 32-column pieces (the P V MMAs address them piece by piece).
-#pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        uint32_t v[32], pk[16];
-        tmem_ld32(s_tmem + part * 64 + hf * 32, v);
-        tmem_ld_wait();
-        if (need_mask) {
-#pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (k0 + hf * 32 + c > lim) v[c] = 0xff800000u;        // -inf
-#pragma unroll
-          for (int c = 0; c < 4; ++c) exp8<0, false>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
-        } else if (fixed) {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) exp8<POLY, false>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
-        } else {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) exp8<POLY, true>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
+        {
+          uint32_t a, b2;
+          unpack2u(sum2, a, b2);
+          l_run[s] += __uint_as_float(a) + __uint_as_float(b2);
         }
-        tmem_st16(s_tmem + part * 64 + hf * 16, pk);
-        tmem_st_wait();
-        tc_fence_before();
-        mbar_arrive(&p_full[2 * s + hf]);
-      }
-      {
-        uint32_t a, b;
-        unpack2u(sum2, a, b);
-        l_run += __uint_as_float(a) + __uint_as_float(b);
       }
     }
-    if (n_s[s] > 0) {
-      // total of the two halves of the row
-      xch[part * 128 + row] = l_run;
-      asm volatile("bar.sync %0, 256;" ::"r"(bar_id) : "memory");
-      l_run += xch[(part ^ 1) * 128 + row];
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      if (n_s[s] == 0) continue;
+      const uint32_t o_tmem = tmem_base + lane_sel + 256 + s * 128;
+      const int tq = blk * 256 + s * BQ + row;
+      // total of the four parts of the row
+      sync_softmax();
+      xch[part * 128 + row] = l_run[s];
+      sync_softmax();
+      const float l_tot = (xch[row] + xch[128 + row]) + (xch[256 + row] + xch[384 + row]);
       if (!mbar_wait(&o_done[s], 0, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
       tc_fence_after();
-      const float inv_l = 1.f / l_run;
+      const float inv_l = 1.f / l_tot;
       const long long row_g = (long long)b * p.S + tq;
 #pragma unroll 1
       for (int c = 0; c < DH / 64; ++c) {
-        uint32_t t[32];
-        const int col = part * (DH / 2) + c * 32;
-        tmem_ld32(o_tmem + col, t);
+        uint32_t t[16];
+        const int col = part * (DH / 4) + c * 16;
+        tmem_ld16(o_tmem + col, t);
         tmem_ld_wait();
         if (tq < p.S) {
           bf16* dst = p.o + row_g * p.Lq + hi * DH + col;
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
+          for (int i = 0; i < 2; ++i) {
             uint4 w;
             w.x = pack_bf16(__uint_as_float(t[8 * i + 0]) * inv_l, __uint_as_float(t[8 * i + 1]) * inv_l);
             w.y = pack_bf16(__uint_as_float(t[8 * i + 2]) * inv_l, __uint_as_float(t[8 * i + 3]) * inv_l);
@@ -417,14 +425,14 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           if (p.o32) {
             float* d32 = p.o32 + row_g * p.Lq + hi * DH + col;
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
+            for (int i = 0; i < 4; ++i)
               reinterpret_cast<float4*>(d32)[i] =
                   make_float4(__uint_as_float(t[4 * i]) * inv_l, __uint_as_float(t[4 * i + 1]) * inv_l,
                               __uint_as_float(t[4 * i + 2]) * inv_l, __uint_as_float(t[4 * i + 3]) * inv_l);
           }
         }
       }
-      if (part == 0 && tq < p.S) p.lse[((long long)b * p.hq + hi) * p.S + tq] = (m_run + log2f(l_run)) * LN2_F;
+      if (part == 0 && tq < p.S) p.lse[((long long)b * p.hq + hi) * p.S + tq] = (m_run[s] + log2f(l_tot)) * LN2_F;
     }
   }
 done:
