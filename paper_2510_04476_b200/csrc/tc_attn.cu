@@ -488,8 +488,10 @@ int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, cons
   p.status = d_status;
   const long long grid = (long long)p.n_blocks * d.B * d.hq;
   if (grid > 0x7fffffffLL) return 1;
-  p.temp = (s->attn_poly & 8) ? nullptr : temp;
-  const int poly = s->attn_poly & 7;
+  // at d_h = 128 the packed polynomial only moves the bottleneck to the half-rate heavy FMA pipe
+  const int knob = s->attn_poly < 0 ? (d.dh == 128 ? 0 : 1) : s->attn_poly;
+  p.temp = (knob & 8) ? nullptr : temp;
+  const int poly = knob & 7;
   if (d.dh == 128) {
     if (poly == 0) return launch_attn<128, 0>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
     if (poly == 1) return launch_attn<128, 1>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);

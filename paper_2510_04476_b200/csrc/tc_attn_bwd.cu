@@ -133,7 +133,8 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint64_t* dp_full = bars + 13;      // MMA -> compute: dP ready
   uint64_t* ds_full = bars + 14;      // compute -> MMA: dS written, dP consumed (all compute threads)
   uint64_t* dq_done = bars + 15;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint64_t* dp_free = bars + 16;      // compute -> MMA: dP of the tile is in registers (all compute threads)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -159,6 +160,7 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     mbar_init(dp_full, 1);
     mbar_init(ds_full, 32 * BW_COMPUTE_WARPS);
     mbar_init(dq_done, 1);
+    mbar_init(dp_free, 32 * BW_COMPUTE_WARPS);
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmQ);
@@ -227,9 +229,9 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           mma_commit(&s_full[nx]);
         }
       }
-      if (!wait_all(ds_full, j & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
-      tc_fence_after();
       if (j + 1 < n_kv) {
+        // dP(j+1) as soon as the compute warps hold dP(j) in registers: their exponentials then overlap it
+        if (!wait_all(dp_free, j & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
         if (!wait_all(&v_full[nx], nph)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
         tc_fence_after();
         if (leader) {
@@ -238,6 +240,8 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           mma_commit(&v_empty[nx]);
         }
       }
+      if (!wait_all(ds_full, j & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+      tc_fence_after();
       if (leader) {
         mma_tm<DH>(tmem_base + 384, tmem_base + st * 128, k_mn + kst * TILE16, hi_w, j != 0);   // dQ += dS(j) K_j
         mma_commit(&k_empty[kst]);
@@ -264,24 +268,28 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       const int k0 = j * 128 + part * 32;
       const bool need_mask = (p.causal && j * 128 + 127 > m0) || (j * 128 + 128 > p.S);
       const int lim = p.causal ? min(tq, p.S - 1) : p.S - 1;
+      uint32_t sv[32], dv[32];
+      tmem_ld32(s_t, sv);
+      tmem_ld32(dp_t, dv);
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(dp_free);                            // the dP buffer may be overwritten
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
-        uint32_t sv[16], dv[16], pk[8];
-        tmem_ld16(s_t + hf * 16, sv);
-        tmem_ld16(dp_t + hf * 16, dv);
-        tmem_ld_wait();
+        uint32_t pk[8];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-          const uint64_t x = fma2(pack2u(sv[2 * c], sv[2 * c + 1]), scale2, nl2);
-          uint64_t e = (c & 3) < POLY ? exp2_pair<true>(x) : exp2_pair<false>(x);
+          const int e = hf * 16 + 2 * c;
+          const uint64_t x = fma2(pack2u(sv[e], sv[e + 1]), scale2, nl2);
+          uint64_t ex = (c & 3) < POLY ? exp2_pair<true>(x) : exp2_pair<false>(x);
           if (need_mask) {
             uint32_t a, bb;
-            unpack2u(e, a, bb);
-            if (k0 + hf * 16 + 2 * c > lim) a = 0u;
-            if (k0 + hf * 16 + 2 * c + 1 > lim) bb = 0u;
-            e = pack2u(a, bb);
+            unpack2u(ex, a, bb);
+            if (k0 + e > lim) a = 0u;
+            if (k0 + e + 1 > lim) bb = 0u;
+            ex = pack2u(a, bb);
           }
-          pk[c] = cvt_bf16x2(mul2(e, add2(pack2u(dv[2 * c], dv[2 * c + 1]), ndl2)));
+          pk[c] = cvt_bf16x2(mul2(ex, add2(pack2u(dv[e], dv[e + 1]), ndl2)));
         }
         // dS (bf16 pairs) over columns this thread has read: keys 32 part + [0,32) -> columns 32 part + [0,16)
         tmem_st8(s_t + hf * 8, pk);
