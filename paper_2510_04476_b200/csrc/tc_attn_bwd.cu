@@ -647,7 +647,7 @@ int tc_attn_bwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, cons
   p.lse = lse; p.delta = delta; p.dq = dq; p.dk = dk; p.dv = dv;
   p.n_tiles = (d.S + 127) / 128;
   p.status = d_status;
-  const int poly = s->attn_poly_bwd;
+  const int poly = s->attn_poly_bwd < 0 ? (d.dh == 128 ? 0 : 1) : s->attn_poly_bwd;
   if (d.dh == 128) {
     if (poly == 0) return launch_bwd<128, 0>(s, d, tmQ, tmK, tmV, tmDO, tmQh, tmDOh, p, st);
     if (poly == 2) return launch_bwd<128, 2>(s, d, tmQ, tmK, tmV, tmDO, tmQh, tmDOh, p, st);
