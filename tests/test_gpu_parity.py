@@ -85,6 +85,13 @@ SMALL = [
     S_("no_convs", 1, 70, 256, 4, 2, 32, flags=63 & ~3),
     S_("conv1_only_no_rope", 1, 70, 256, 4, 2, 32, flags=1 | 16),
     S_("three_tiles", 1, 300, 512, 8, 2, 64),
+    S_("noncausal_dh64_tiles", 1, 300, 512, 8, 2, 64, causal=0),
+    S_("noncausal_dh128", 1, 260, 1024, 8, 4, 128, causal=0),
+    S_("gqa8_dh64", 1, 200, 512, 8, 1, 64),
+    S_("group_of_one_dh128", 1, 140, 512, 4, 4, 128),
+    S_("fused_projection_ragged_rows", 1, 777, 512, 8, 2, 64),
+    S_("fused_projection_three_sequences", 3, 300, 512, 8, 2, 64),
+    S_("fused_projection_no_v_shift", 2, 300, 512, 8, 2, 64, flags=63 & ~8),
 ]
 
 
@@ -153,7 +160,31 @@ def test_cfg3_prefill16k_sampled_rows(impl):
     cca.close()
 
 
-@pytest.mark.parametrize("S,C", [(1024, 8), (4096, 2)])
+@pytest.mark.parametrize("S,C", [(16384, 4), (65536, 8), (32768, 1)])
+def test_sweep_long_context_forward_sampled_rows(S, C):
+    """Long-context points of the sweep (64k is the longest context of the workloads): one sequence, latents in
+    full, the S^2 stage on sampled query rows."""
+    sh = synth.sweep_shape(S, C).replace(B=1)
+    t = synth.make_inputs(sh, want_dout=False)
+    rows = sample_rows(sh.S, n_random=24)
+    out_ref, o_ref, lse_ref, I = O.forward_rows(oracle_cfg(sh), t, t["x"], rows)
+    dev = to_device(t)
+    cca = _cca(sh)
+    ws = cca.alloc_workspace(sh.B, sh.S, False)
+    out = cca.forward(dev, dev["x"], ws)
+    torch.cuda.synchronize()
+    assert cca.last_status() == 0
+    sv = cca.saved(ws, sh.B, sh.S)
+    for n in ("v", "q", "k"):
+        check_close(n, sv[n], I[n])
+    check_close("o_rows", sv["o"][:, rows], o_ref)
+    check_close("lse_rows", sv["lse"][:, :, rows], lse_ref)
+    check_close("out_rows", out[:, rows], out_ref)
+    assert torch.isfinite(out.float()).all()
+    cca.close()
+
+
+@pytest.mark.parametrize("S,C", [(1024, 8), (4096, 2), (2048, 4)])
 def test_sweep_points_forward_backward(S, C):
     sh = synth.sweep_shape(S, C)
     sh = sh.replace(B=min(sh.B, 2))      # the oracle's share of the batch; sequences are independent
