@@ -23,7 +23,8 @@ Readings taken where the paper is silent (all are runtime parameters):
   * causal = 0 drops only the attention mask; convs and value-shift stay causal.
 
 Pins: see tests/test_oracle_pins.py (brute-force attention, causality and halo,
-MHA reduction, CCGQA -> CCA, closed forms, finite differences, autograd, formulas).
+MHA reduction, CCGQA -> CCA, closed forms, finite differences, autograd, formulas;
+the token-by-token decode against the whole-sequence forward and brute force).
 The RoPE convention, the conv sizes and the RoPE base are "parity unpinned" against
 the authors' kernel (no source or numbers exist); everything else is pinned.
 """
@@ -412,6 +413,119 @@ def backward(cfg: OracleConfig, w: Dict[str, torch.Tensor], I: Dict[str, torch.T
         dx += dxs
     G["d_x"] = dx
     return G
+
+
+# --------------------------------------------------------------------------------------
+# Decode: one new token per sequence against the latent KV cache (comparison table of the
+# paper, KV-cache and decode columns).  The state is what the block's definition needs of
+# the past: the cached latent keys and values (2 L_k numbers per token), the
+# pre-convolution q0|k0 of the last k_seq + k_ch - 2 tokens (the convs' halo) and the
+# previous token's input (the value shift).
+# --------------------------------------------------------------------------------------
+
+def decode_init(cfg: OracleConfig, B: int) -> Dict[str, object]:
+    """Empty state: no cached token, zero history (the convs and the value shift see zeros
+    before the first token)."""
+    pad = cfg.k_seq + cfg.k_ch - 2
+    return {
+        "k": torch.zeros(B, 0, cfg.n_kv_heads, cfg.head_dim, dtype=F64),
+        "v": torch.zeros(B, 0, cfg.n_kv_heads, cfg.head_dim, dtype=F64),
+        "qk0_hist": torch.zeros(B, pad, cfg.L, dtype=F64),      # oldest first
+        "x_prev": torch.zeros(B, cfg.d_model, dtype=F64),
+        "pos": 0,
+    }
+
+
+def decode_step(cfg: OracleConfig, w: Dict[str, torch.Tensor], state: Dict[str, object], x_t):
+    """Eq. 7-11 for the single token x_t [B,E] at position state["pos"], every sequence at the
+    same position.  Returns out [B,E]; the state is advanced in place.  The attention is causal by
+    construction: the new query sees the cached tokens and itself."""
+    x_t = _f64(x_t)
+    B, E = x_t.shape
+    hq, hk, dh, g = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.g
+    Lq, Lk, L = cfg.L_q, cfg.L_k, cfg.L
+    ks = cfg.k_seq if cfg.flags & CONV1 else 1
+    kc = cfg.k_ch if cfg.flags & CONV2 else 1
+    pad = cfg.k_seq + cfg.k_ch - 2
+    pos = int(state["pos"])
+    qk0_t = x_t @ _f64(w["w_qk"]).transpose(0, 1)                                   # Eq. 7
+    win = torch.cat([state["qk0_hist"], qk0_t[:, None, :]], dim=1)                  # tokens pos-pad .. pos
+    # Eq. 8, conv1 at the kc tokens conv2 looks at, then conv2 at the new token
+    y1 = []
+    for r in range(kc):                                   # token pos - (kc-1) + r  = window row pad - (kc-1) + r
+        row = pad - (kc - 1) + r
+        if cfg.flags & CONV1:
+            w0 = _f64(w["conv0_w"])
+            acc = torch.zeros(B, L, dtype=F64)
+            for j in range(ks):
+                acc = acc + win[:, row - (ks - 1) + j, :] * w0[:, j]
+            y1.append(acc)
+        else:
+            y1.append(win[:, row, :])
+    if cfg.flags & CONV2:
+        w1 = _f64(w["conv1_w"]).reshape(hq + hk, dh, dh, kc)
+        y2 = torch.zeros(B, hq + hk, dh, dtype=F64)
+        for r in range(kc):
+            y2 = y2 + torch.einsum("bhi,hoi->bho", y1[r].reshape(B, hq + hk, dh), w1[..., r])
+        y2 = y2.reshape(B, L)
+    else:
+        y2 = y1[-1]
+    q0 = qk0_t[:, :Lq].reshape(B, hq, dh)
+    k0 = qk0_t[:, Lq:].reshape(B, hk, dh)
+    qh = y2[:, :Lq].reshape(B, hq, dh)
+    kh = y2[:, Lq:].reshape(B, hk, dh)
+    if cfg.flags & QK_MEAN:                                                          # Eq. 9
+        mu = 0.5 * (q0 + k0.repeat_interleave(g, dim=1))
+        qh = qh + mu
+        kh = kh + mu.reshape(B, hk, g, dh).mean(dim=2)
+    xs = state["x_prev"] if cfg.flags & V_SHIFT else x_t                             # Eq. 10
+    v_t = torch.cat([x_t @ _f64(w["w_v1"]).transpose(0, 1), xs @ _f64(w["w_v2"]).transpose(0, 1)], dim=-1)
+    v_t = v_t.reshape(B, hk, dh)
+    if cfg.flags & QK_NORM:                                                          # Eq. 11
+        beta = torch.exp(_f64(w["temp"]))
+        qh = qh * math.sqrt(dh) / qh.norm(dim=-1, keepdim=True)
+        kh = kh * (math.sqrt(dh) * beta)[None, :, None] / kh.norm(dim=-1, keepdim=True)
+    if cfg.flags & ROPE:
+        half = dh // 2
+        c = torch.arange(half, dtype=F64)
+        ang = pos * torch.pow(torch.tensor(float(cfg.rope_base), dtype=F64), -2.0 * c / dh)
+        cs, sn = torch.cos(ang), torch.sin(ang)
+
+        def rot(u):
+            a, b = u[..., :half], u[..., half:]
+            return torch.cat([a * cs - b * sn, b * cs + a * sn], dim=-1)
+        qh, kh = rot(qh), rot(kh)
+    state["k"] = torch.cat([state["k"], kh[:, None]], dim=1)
+    state["v"] = torch.cat([state["v"], v_t[:, None]], dim=1)
+    o = torch.zeros(B, hq, dh, dtype=F64)
+    for i in range(hq):
+        j = i // g
+        s = torch.einsum("bd,bsd->bs", qh[:, i], state["k"][:, :, j]) / math.sqrt(dh)
+        p = torch.softmax(s, dim=-1)
+        o[:, i] = torch.einsum("bs,bsd->bd", p, state["v"][:, :, j])
+    out = o.reshape(B, Lq) @ _f64(w["w_o"]).transpose(0, 1)
+    if pad > 0:
+        state["qk0_hist"] = win[:, 1:, :].clone()
+    state["x_prev"] = x_t.clone()
+    state["pos"] = pos + 1
+    state["q_last"], state["o_last"] = qh, o
+    return out
+
+
+def decode_state_after_prefill(cfg: OracleConfig, I: Dict[str, torch.Tensor], S0: int) -> Dict[str, object]:
+    """The decode state after the first S0 tokens of a prefill whose intermediates are I
+    (from pre_attention / forward): cached k, v, the q0|k0 halo and the last input."""
+    pad = cfg.k_seq + cfg.k_ch - 2
+    B = I["x"].shape[0]
+    hist = torch.zeros(B, pad, cfg.L, dtype=F64)
+    n = min(pad, S0)
+    if n > 0:
+        hist[:, pad - n:, :] = I["qk0"][:, S0 - n:S0, :]
+    return {
+        "k": I["k"][:, :S0].clone(), "v": I["v"][:, :S0].clone(), "qk0_hist": hist,
+        "x_prev": I["x"][:, S0 - 1, :].clone() if S0 > 0 else torch.zeros(B, cfg.d_model, dtype=F64),
+        "pos": S0,
+    }
 
 
 # --------------------------------------------------------------------------------------

@@ -479,3 +479,52 @@ def test_forward_rows_equals_forward():
     rows = [0, 3, 15]
     out_r, _, _, _ = O.forward_rows(cfg, t, t["x"], rows)
     assert torch.allclose(out[:, rows], out_r, atol=1e-14)
+
+
+# ------------------------------------------------------------------ decode with the latent KV cache
+
+@pytest.mark.parametrize("k_seq,k_ch", [(2, 2), (1, 1), (3, 2), (2, 4)])
+@pytest.mark.parametrize("flags", [O.ALL_FLAGS, 0, O.ALL_FLAGS & ~O.V_SHIFT, O.ALL_FLAGS & ~O.CONV1,
+                                   O.ALL_FLAGS & ~O.CONV2, O.ALL_FLAGS & ~O.QK_MEAN])
+def test_decode_token_by_token_equals_whole_sequence_forward(k_seq, k_ch, flags):
+    """Feeding the tokens one at a time through the cache must reproduce every row of the causal
+    whole-sequence forward, which is pinned above by other means."""
+    sh = small_shape(S=9, k_seq=k_seq, k_ch=k_ch, flags=flags)
+    cfg, t = cfg_of(sh), inputs64(sh)
+    out, I = O.forward(cfg, t, t["x"])
+    st = O.decode_init(cfg, sh.B)
+    for tok in range(sh.S):
+        o_t = O.decode_step(cfg, t, st, t["x"][:, tok])
+        assert torch.allclose(o_t, out[:, tok], rtol=1e-10, atol=1e-12), tok
+    assert torch.allclose(st["k"], I["k"], rtol=1e-10, atol=1e-12)
+    assert torch.allclose(st["v"], I["v"], rtol=1e-10, atol=1e-12)
+    assert st["k"].numel() + st["v"].numel() == O.describe(cfg, sh.B, sh.S)["kv_cache_elems"]
+
+
+@pytest.mark.parametrize("S0", [0, 1, 2, 5])
+def test_decode_continues_a_prefill(S0):
+    sh = small_shape(S=8, k_seq=3, k_ch=2, n_kv_heads=1)
+    cfg, t = cfg_of(sh), inputs64(sh)
+    out, I = O.forward(cfg, t, t["x"])
+    st = O.decode_state_after_prefill(cfg, I, S0)
+    for tok in range(S0, sh.S):
+        o_t = O.decode_step(cfg, t, st, t["x"][:, tok])
+        assert torch.allclose(o_t, out[:, tok], rtol=1e-10, atol=1e-12), tok
+
+
+def test_decode_first_token_closed_form_and_planted_mistakes():
+    """Position 0: the single key gets probability one, the shifted value half is zero."""
+    sh = small_shape(S=3)
+    cfg, t = cfg_of(sh), inputs64(sh)
+    st = O.decode_init(cfg, sh.B)
+    o0 = O.decode_step(cfg, t, st, t["x"][:, 0])
+    v = torch.cat([t["x"][:, 0] @ t["w_v1"].T, torch.zeros(sh.B, sh.L_k // 2, dtype=F64)], dim=-1)
+    o = v.reshape(sh.B, sh.n_kv_heads, sh.head_dim).repeat_interleave(sh.n_q_heads // sh.n_kv_heads, dim=1)
+    assert torch.allclose(o0, o.reshape(sh.B, sh.L_q) @ t["w_o"].T, rtol=1e-10, atol=1e-12)
+    # a state that forgot the previous input (value shift) or the conv halo must change the next token
+    out, _ = O.forward(cfg, t, t["x"])
+    for key in ("x_prev", "qk0_hist"):
+        st2 = O.decode_init(cfg, sh.B)
+        O.decode_step(cfg, t, st2, t["x"][:, 0])
+        st2[key] = torch.zeros_like(st2[key])
+        assert not torch.allclose(O.decode_step(cfg, t, st2, t["x"][:, 1]), out[:, 1], rtol=1e-6, atol=1e-8), key
