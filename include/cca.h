@@ -176,6 +176,45 @@ int cca_forward_static(cca_handle* h, const cca_weights* w, const void* x, void*
 int cca_attention_forward(cca_handle* h, const void* q, const void* k, const void* v, void* o,
                           float* lse, int64_t B, int64_t S, void* cuda_stream);
 
+/* ---- Decode: one new token per sequence against the latent KV cache ------------------------------
+ * The paper's comparison table gives the cache (2 B S E / C2 numbers: the latent keys and values) and the
+ * decode FLOPs of the block; this is that step.  Besides the cache the block's definition needs, of the
+ * past, the pre-convolution q0|k0 of the last k_seq + k_ch - 2 tokens (Eq. 8: the two causal convs' halo)
+ * and the previous token's input (Eq. 10: half of the value channels come from x_{t-1}).  All of it is
+ * caller-owned device memory described by cca_decode_state; the library keeps nothing between steps. */
+typedef struct {
+  void* k_cache;        /* bf16 [B, S_max, L_k]: keys after norm, temperature and RoPE (Eq. 11), row = position */
+  void* v_cache;        /* bf16 [B, S_max, L_k]: values (Eq. 10)                                                */
+  void* qk0_hist;       /* fp32 [B, k_seq + k_ch - 2, L]: q0|k0 (Eq. 7) of the last tokens, oldest first; all
+                           zeros before a sequence's first token; may be null when k_seq = k_ch = 1           */
+  void* x_prev;         /* bf16 [B, E]: previous token's input; zeros before a sequence's first token          */
+  const int32_t* pos;   /* int32 [B], device: position of each sequence's new token = tokens already cached;
+                           read, never written (the caller advances it after the step)                         */
+  int64_t S_max;        /* capacity of both caches in tokens                                                    */
+} cca_decode_state;
+
+/* Bytes of device workspace one decode step needs for B sequences of at most max_len tokens (the new
+ * token included). */
+int cca_decode_workspace_size(const cca_handle* h, int64_t B, int64_t max_len, size_t* bytes);
+
+/* One decode step, Eq. 7-11 for a single new token per sequence: x device bf16 [B,E] (read), out device
+ * bf16 [B,E] (written).  Sequence b's token sits at position pos[b]; it attends to cached positions
+ * 0..pos[b]-1 and to itself.  On return (stream order) row pos[b] of both caches holds the new key and
+ * value, qk0_hist and x_prev are advanced by one token.  max_len: host-side bound, pos[b] < max_len <=
+ * S_max for every b; it sizes the launch.  A sequence whose pos[b] is outside [0, min(max_len, S_max)) is
+ * skipped (its caches, history and output row are left untouched or undefined, nothing is written out of
+ * bounds) and the device status word becomes 120, which cca_last_status reports.
+ * Needs causal = 1, head_dim in {32,64,128}, L_k and E multiples of 8.  No allocation, no synchronisation.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE_TOO_SMALL, CUDA. */
+int cca_decode_step(cca_handle* h, const cca_weights* w, const void* x, void* out, const cca_decode_state* state,
+                    int64_t max_len, void* workspace, size_t workspace_bytes, int64_t B, void* cuda_stream);
+
+/* Hand-over from a prefill: fills `state` (caches rows 0..S-1, history, previous input) from x [B,S,E] and
+ * the workspace cca_forward left for it, so that the next cca_decode_step continues at pos[b] = S.  Copies
+ * only (stream order); state->pos is not read.  Errors: INVALID_ARG (S > S_max, null), ALIGNMENT, CUDA. */
+int cca_decode_state_from_prefill(cca_handle* h, const void* x, const void* workspace, size_t workspace_bytes,
+                                  int64_t B, int64_t S, const cca_decode_state* state, void* cuda_stream);
+
 /* Select kernel implementations: 0 = plain SIMT kernels, 1 = tcgen05/TMA kernels where they
  * exist (default).  Returns the previous value. */
 int cca_set_impl(cca_handle* h, int impl);
@@ -188,8 +227,8 @@ int cca_set_attention_events(cca_handle* h, void* ev_begin, void* ev_end);
 int64_t cca_launch_count(const cca_handle* h);
 
 /* After the caller has synchronised the stream: copies the device status word.  0 = no error;
- * otherwise the code written by a kernel whose bounded wait expired.  Returns
- * CCA_ERR_DEVICE_TIMEOUT if it is non-zero. */
+ * otherwise the code written by a kernel whose bounded wait expired (or 120: a decode step met a position
+ * outside its cache).  Returns CCA_ERR_DEVICE_TIMEOUT if it is non-zero. */
 int cca_last_status(cca_handle* h, int* device_status);
 
 /* Last CUDA runtime error code seen by this handle, and its string. */

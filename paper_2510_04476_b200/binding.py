@@ -45,6 +45,11 @@ class cca_layout(C.Structure):
                 ("saved_bytes", C.c_int64), ("total_bytes", C.c_int64), ("off_rnorm", C.c_int64)]
 
 
+class cca_decode_state(C.Structure):
+    _fields_ = [("k_cache", C.c_void_p), ("v_cache", C.c_void_p), ("qk0_hist", C.c_void_p), ("x_prev", C.c_void_p),
+                ("pos", C.c_void_p), ("S_max", C.c_int64)]
+
+
 # name -> (restype, argtypes); also the list of symbols the header declares
 SYMBOLS = {
     "cca_init": (C.c_int, [C.POINTER(cca_config), C.c_int, C.POINTER(C.c_void_p)]),
@@ -61,6 +66,11 @@ SYMBOLS = {
                                      C.c_void_p]),
     "cca_attention_forward": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_int64, C.c_int64, C.c_void_p]),
+    "cca_decode_workspace_size": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.POINTER(C.c_size_t)]),
+    "cca_decode_step": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.POINTER(cca_decode_state),
+                                  C.c_int64, C.c_void_p, C.c_size_t, C.c_int64, C.c_void_p]),
+    "cca_decode_state_from_prefill": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_int64, C.c_int64,
+                                                C.POINTER(cca_decode_state), C.c_void_p]),
     "cca_set_impl": (C.c_int, [C.c_void_p, C.c_int]),
     "cca_set_attention_events": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "cca_launch_count": (C.c_int64, [C.c_void_p]),
@@ -224,6 +234,63 @@ class CCA:
         _check(self.lib, self.lib.cca_forward_static(self.handle, C.byref(cw), _ptr(x), _ptr(out), B, S, st),
                self.handle, "cca_forward_static")
         return out
+
+    # ---- decode ---------------------------------------------------------------------------
+    def new_decode_state(self, B: int, S_max: int) -> Dict[str, torch.Tensor]:
+        """Caller-owned tensors of cca_decode_state for B empty sequences (device memory only, no arithmetic)."""
+        c = self.cfg
+        Lk = c.n_kv_heads * c.head_dim
+        L = c.n_q_heads * c.head_dim + Lk
+        pad = c.k_seq + c.k_ch - 2
+        dev = self.device
+        return {"k_cache": torch.zeros(B, S_max, Lk, dtype=torch.bfloat16, device=dev),
+                "v_cache": torch.zeros(B, S_max, Lk, dtype=torch.bfloat16, device=dev),
+                "qk0_hist": torch.zeros(B, max(pad, 1), L, dtype=torch.float32, device=dev)[:, :pad].contiguous(),
+                "x_prev": torch.zeros(B, c.d_model, dtype=torch.bfloat16, device=dev),
+                "pos": torch.zeros(B, dtype=torch.int32, device=dev)}
+
+    @staticmethod
+    def _decode_state(state: Dict[str, torch.Tensor]) -> cca_decode_state:
+        s = cca_decode_state()
+        for n in ("k_cache", "v_cache", "qk0_hist", "x_prev", "pos"):
+            t = state[n]
+            assert t.is_cuda and t.is_contiguous(), n
+            setattr(s, n, t.data_ptr() if t.numel() else None)
+        assert state["pos"].dtype == torch.int32
+        s.S_max = state["k_cache"].shape[1]
+        return s
+
+    def decode_workspace_size(self, B: int, max_len: int) -> int:
+        n = C.c_size_t()
+        _check(self.lib, self.lib.cca_decode_workspace_size(self.handle, B, max_len, C.byref(n)), self.handle,
+               "cca_decode_workspace_size")
+        return int(n.value)
+
+    def alloc_decode_workspace(self, B: int, max_len: int) -> torch.Tensor:
+        return torch.empty(self.decode_workspace_size(B, max_len) + 256, dtype=torch.uint8, device=self.device)
+
+    def decode_step(self, w, x: torch.Tensor, state: Dict[str, torch.Tensor], max_len: int, workspace: torch.Tensor,
+                    out: Optional[torch.Tensor] = None):
+        """cca_decode_step: x [B,E] -> out [B,E]; the state tensors are updated in place except `pos`."""
+        B, E = x.shape
+        assert x.is_cuda and x.is_contiguous() and x.dtype == torch.bfloat16
+        if out is None:
+            out = torch.empty_like(x)
+        cw = self._weights(w)
+        ds = self._decode_state(state)
+        wp, wn = self._ws_ptr(workspace)
+        st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+        _check(self.lib, self.lib.cca_decode_step(self.handle, C.byref(cw), _ptr(x), _ptr(out), C.byref(ds), max_len,
+                                                  wp, wn, B, st), self.handle, "cca_decode_step")
+        return out
+
+    def decode_state_from_prefill(self, x: torch.Tensor, workspace: torch.Tensor, state: Dict[str, torch.Tensor]):
+        B, S, E = x.shape
+        ds = self._decode_state(state)
+        wp, wn = self._ws_ptr(workspace)
+        st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+        _check(self.lib, self.lib.cca_decode_state_from_prefill(self.handle, _ptr(x), wp, wn, B, S, C.byref(ds), st),
+               self.handle, "cca_decode_state_from_prefill")
 
     def backward(self, w, x: torch.Tensor, d_out: torch.Tensor, workspace: torch.Tensor):
         """Returns (d_x bf16, dict of fp32 parameter gradients)."""

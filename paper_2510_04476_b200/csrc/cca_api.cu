@@ -6,6 +6,7 @@
 
 #include "../../include/cca.h"
 #include "common.cuh"
+#include "decode.cuh"
 #include "tc_kernels.cuh"
 
 struct cca_handle {
@@ -276,6 +277,82 @@ int cca_attention_forward(cca_handle* h, const void* q, const void* k, const voi
   // q and k come from the caller: nothing is known about their norms
   return run_attention_fwd(h, d, (const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)o, nullptr, lse, nullptr,
                            (cudaStream_t)cuda_stream);
+}
+
+int cca_decode_workspace_size(const cca_handle* h, int64_t B, int64_t max_len, size_t* bytes) {
+  int r = check_sizes(h, B, max_len);
+  if (r != CCA_OK) return r;
+  if (!bytes) return CCA_ERR_INVALID_ARG;
+  CcaDims d = make_dims(h->cfg, B, 1);
+  *bytes = decode_workspace_bytes(d, (int)max_len, h->sm_count > 0 ? h->sm_count : 148);
+  return CCA_OK;
+}
+
+int cca_decode_step(cca_handle* h, const cca_weights* w, const void* x, void* out, const cca_decode_state* s,
+                    int64_t max_len, void* workspace, size_t workspace_bytes, int64_t B, void* cuda_stream) {
+  int r = check_sizes(h, B, max_len, true);
+  if (r != CCA_OK) return r;
+  if (!w || !x || !out || !s || !workspace) return CCA_ERR_INVALID_ARG;
+  if (!w->w_qk || !w->w_v1 || !w->w_v2 || !w->w_o) return CCA_ERR_INVALID_ARG;
+  const cca_config& c = h->cfg;
+  if ((c.flags & CCA_CONV1) && !w->conv0_w) return CCA_ERR_INVALID_ARG;
+  if ((c.flags & CCA_CONV2) && !w->conv1_w) return CCA_ERR_INVALID_ARG;
+  if ((c.flags & CCA_QK_NORM) && !w->temp) return CCA_ERR_INVALID_ARG;
+  const int pad = c.k_seq + c.k_ch - 2;
+  if (!s->k_cache || !s->v_cache || !s->x_prev || !s->pos || (pad > 0 && !s->qk0_hist)) return CCA_ERR_INVALID_ARG;
+  if (max_len > s->S_max || s->S_max > (int64_t)1 << 24) return CCA_ERR_INVALID_ARG;
+  if (!c.causal) return CCA_ERR_UNSUPPORTED;
+  CcaDims d = make_dims(c, B, 1);
+  if (d.Lk % 8 || d.E % 8 || d.Lq % 8) return CCA_ERR_UNSUPPORTED;
+  if (!aligned16(x) || !aligned16(out) || !aligned16(w->w_qk) || !aligned16(w->w_v1) || !aligned16(w->w_v2) ||
+      !aligned16(w->w_o) || !aligned16(s->k_cache) || !aligned16(s->v_cache) || !aligned16(s->x_prev) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CCA_ERR_ALIGNMENT;
+  if (workspace_bytes < decode_workspace_bytes(d, (int)max_len, h->sm_count)) return CCA_ERR_WORKSPACE_TOO_SMALL;
+  CU(cudaSetDevice(h->device));
+  DecodeWeights dw{(const bf16*)w->w_qk, (const bf16*)w->w_v1, (const bf16*)w->w_v2, (const bf16*)w->w_o,
+                   (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, (const float*)w->temp};
+  DecodeState ds{(bf16*)s->k_cache, (bf16*)s->v_cache, (float*)s->qk0_hist, (bf16*)s->x_prev, s->pos, s->S_max};
+  int rr = launch_decode_step(d, dw, (const bf16*)x, (bf16*)out, ds, (int)max_len, workspace, h->sm_count, h->d_status,
+                              &h->launches, (cudaStream_t)cuda_stream);
+  if (rr < 0) { h->last_cuda = -rr; return CCA_ERR_CUDA; }
+  if (rr > 0) return CCA_ERR_UNSUPPORTED;
+  return CCA_OK;
+}
+
+int cca_decode_state_from_prefill(cca_handle* h, const void* x, const void* workspace, size_t workspace_bytes,
+                                  int64_t B, int64_t S, const cca_decode_state* s, void* cuda_stream) {
+  int r = check_sizes(h, B, S, true);
+  if (r != CCA_OK) return r;
+  if (!x || !workspace || !s) return CCA_ERR_INVALID_ARG;
+  const cca_config& c = h->cfg;
+  const int pad = c.k_seq + c.k_ch - 2;
+  if (!s->k_cache || !s->v_cache || !s->x_prev || (pad > 0 && !s->qk0_hist) || S > s->S_max) return CCA_ERR_INVALID_ARG;
+  Layout l = make_layout(c, B, S);
+  if (workspace_bytes < l.saved_end) return CCA_ERR_WORKSPACE_TOO_SMALL;
+  CU(cudaSetDevice(h->device));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CcaDims d = make_dims(c, B, S);
+  const char* ws = (const char*)workspace;
+  const size_t row_k = (size_t)d.Lk * 2;
+  for (int64_t b = 0; b < B; ++b) {
+    CU(cudaMemcpyAsync((char*)s->k_cache + (size_t)b * s->S_max * row_k, ws + l.k + (size_t)b * S * row_k, (size_t)S * row_k,
+                       cudaMemcpyDeviceToDevice, st));
+    CU(cudaMemcpyAsync((char*)s->v_cache + (size_t)b * s->S_max * row_k, ws + l.v + (size_t)b * S * row_k, (size_t)S * row_k,
+                       cudaMemcpyDeviceToDevice, st));
+  }
+  // previous input: the last token of every sequence (rows S-1 of x, one strided copy)
+  CU(cudaMemcpy2DAsync(s->x_prev, (size_t)d.E * 2, (const char*)x + (size_t)(S - 1) * d.E * 2, (size_t)S * d.E * 2,
+                       (size_t)d.E * 2, (size_t)B, cudaMemcpyDeviceToDevice, st));
+  if (pad > 0) {
+    const size_t row = (size_t)d.L * 4;
+    const int64_t n = S < pad ? S : pad;
+    CU(cudaMemsetAsync(s->qk0_hist, 0, (size_t)B * pad * row, st));
+    CU(cudaMemcpy2DAsync((char*)s->qk0_hist + (size_t)(pad - n) * row, (size_t)pad * row,
+                         ws + l.qk0 + (size_t)(S - n) * row, (size_t)S * row, (size_t)n * row, (size_t)B,
+                         cudaMemcpyDeviceToDevice, st));
+  }
+  return CCA_OK;
 }
 
 int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, void* workspace,

@@ -1,0 +1,604 @@
+// Decode step: one new token per sequence against the latent KV cache (the KV-cache and decode columns of the
+// paper's comparison table).  Everything here is bound by memory traffic -- the weights are read once per step
+// and every cached key and value row once per (sequence, kv head) -- so these are plain CUDA kernels laid out
+// for coalesced 16-byte accesses, not tensor-core tiles:
+//
+//   decode_proj_kernel      out[b, n] = sum_k W[n, k] x[b, k] for a few stacked weight segments (Eq. 7, 10; Eq. 11
+//                           up-projection): one warp per two weight rows, 16 sequences per CTA staged in shared memory
+//   decode_transform_kernel Eq. 8-11 for the new token of one (sequence, head): conv halo from the caller's history,
+//                           q-k-mean, norm, temperature, RoPE at the sequence's own position; appends k, v to the cache
+//   decode_attn_kernel      softmax(q k^T / sqrt(d_h)) v of the new query over a chunk of the cached keys of one
+//                           (sequence, kv head, group of <= 4 query heads); partial results per chunk
+//   decode_combine_kernel   merges the chunks' partial results
+#include <cstring>
+
+#include "common.cuh"
+#include "decode.cuh"
+
+namespace {
+
+constexpr unsigned F_CONV1 = 1, F_CONV2 = 2, F_QK_MEAN = 4, F_V_SHIFT = 8, F_QK_NORM = 16, F_ROPE = 32;
+constexpr int ST_DECODE_BAD_POSITION = 120;
+constexpr float LOG2E = 1.4426950408889634f;
+
+CCA_DEVINL void unpack8(const uint4& u, float* f) {
+  f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
+  f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
+  f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xffff0000u);
+  f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xffff0000u);
+}
+
+// ------------------------------------------------------------------------------------------------ projections
+constexpr int PJ_BT = 16;          // sequences per CTA
+constexpr int PJ_KC = 1024;        // k-chunk staged in shared memory
+constexpr int PJ_WARPS = 4, PJ_RPW = 2, PJ_ROWS = PJ_WARPS * PJ_RPW;
+
+struct ProjSeg {
+  const bf16* W;     // [rows, K] row-major
+  const bf16* X;     // [B, K] row-major
+  int rows;
+  int out_off;       // first output column of this segment
+};
+struct ProjArgs {
+  ProjSeg seg[3];
+  int n_seg, rows_total, K, B;
+  float* out_f32;    // [B, ldo] (one of the two)
+  bf16* out_bf16;
+  int ldo;
+};
+
+__global__ void __launch_bounds__(PJ_WARPS * 32) decode_proj_kernel(ProjArgs a) {
+  __shared__ __align__(16) bf16 xs[PJ_BT][PJ_KC];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b0 = blockIdx.y * PJ_BT;
+  const int row0 = blockIdx.x * PJ_ROWS;          // first row of this CTA in the stacked row space
+  // segments start on multiples of PJ_ROWS in the stacked space (the host pads), so a CTA stays inside one
+  int sidx = 0, base = 0;
+  for (int s = 0; s < a.n_seg; ++s) {
+    const int padded = (a.seg[s].rows + PJ_ROWS - 1) / PJ_ROWS * PJ_ROWS;
+    if (row0 >= base && row0 < base + padded) { sidx = s; break; }
+    base += padded;
+  }
+  const ProjSeg sg = a.seg[sidx];
+  const int r_first = row0 - base + warp * PJ_RPW;
+  float acc[PJ_RPW][PJ_BT];
+#pragma unroll
+  for (int r = 0; r < PJ_RPW; ++r)
+#pragma unroll
+    for (int b = 0; b < PJ_BT; ++b) acc[r][b] = 0.f;
+
+  for (int k0 = 0; k0 < a.K; k0 += PJ_KC) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < PJ_BT * (PJ_KC / 8); i += PJ_WARPS * 32) {
+      const int b = i / (PJ_KC / 8), kv = (i % (PJ_KC / 8)) * 8;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (b0 + b < a.B && k0 + kv < a.K) v = *reinterpret_cast<const uint4*>(sg.X + (size_t)(b0 + b) * a.K + k0 + kv);
+      *reinterpret_cast<uint4*>(&xs[b][kv]) = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < PJ_KC / 256; ++i) {
+      const int kv = i * 256 + lane * 8;
+      float w[PJ_RPW][8];
+#pragma unroll
+      for (int r = 0; r < PJ_RPW; ++r) {
+        uint4 u = make_uint4(0, 0, 0, 0);
+        if (r_first + r < sg.rows && k0 + kv < a.K)
+          u = __ldg(reinterpret_cast<const uint4*>(sg.W + (size_t)(r_first + r) * a.K + k0 + kv));
+        unpack8(u, w[r]);
+      }
+#pragma unroll
+      for (int b = 0; b < PJ_BT; ++b) {
+        float x[8];
+        unpack8(*reinterpret_cast<const uint4*>(&xs[b][kv]), x);
+#pragma unroll
+        for (int r = 0; r < PJ_RPW; ++r)
+#pragma unroll
+          for (int c = 0; c < 8; ++c) acc[r][b] = fmaf(w[r][c], x[c], acc[r][b]);
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < PJ_RPW; ++r)
+#pragma unroll
+    for (int b = 0; b < PJ_BT; ++b) {
+      float v = acc[r][b];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      acc[r][b] = v;
+    }
+  // lane b of the warp stores sequence b
+#pragma unroll
+  for (int r = 0; r < PJ_RPW; ++r) {
+    float mine = 0.f;
+#pragma unroll
+    for (int b = 0; b < PJ_BT; ++b)
+      if (lane == b) mine = acc[r][b];
+    if (lane < PJ_BT && b0 + lane < a.B && r_first + r < sg.rows) {
+      const size_t o = (size_t)(b0 + lane) * a.ldo + sg.out_off + r_first + r;
+      if (a.out_f32) a.out_f32[o] = mine;
+      else a.out_bf16[o] = __float2bfloat16(mine);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ transforms
+struct TrArgs {
+  CcaDims d;
+  const float* lat;      // [B, L + Lk]: q0 | k0 | v1 | v2 of the new token
+  const bf16* x;         // [B, E] new token
+  const bf16* w0;        // [L, k_seq]
+  const bf16* w1;        // [L, d_h, k_ch]
+  const float* temp;
+  float* q;              // [B, Lq] out
+  bf16* k_cache;         // [B, S_max, Lk]
+  bf16* v_cache;
+  float* hist;           // [B, pad, L]
+  bf16* x_prev;          // [B, E]
+  const int* pos;
+  long long S_max;
+  int max_len;
+  int* status;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(128) decode_transform_kernel(TrArgs a) {
+  constexpr int MAXW = 8;                      // window rows: pad + 1 <= 8 (k_seq, k_ch <= 4 each)
+  __shared__ float win[MAXW][DH];
+  __shared__ float y1[4][DH];
+  __shared__ float xh[DH];
+  __shared__ float red[4];
+  const CcaDims& d = a.d;
+  const int b = blockIdx.y, head = blockIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int t = a.pos[b];
+  if (t < 0 || t >= a.S_max || t >= a.max_len) {
+    if (tid == 0) atomicCAS(a.status, 0, ST_DECODE_BAD_POSITION);
+    return;
+  }
+  const int ld_lat = d.L + d.Lk;
+  if (head == d.hq + d.hk) {
+    // value row of the new token (Eq. 10; the projection already took x_{t-1} for the second half) and the
+    // input the next step's value shift needs
+    for (int c = tid; c < d.Lk; c += 128)
+      a.v_cache[((size_t)b * a.S_max + t) * d.Lk + c] = __float2bfloat16(a.lat[(size_t)b * ld_lat + d.L + c]);
+    for (int c = tid; c < d.E / 8; c += 128)
+      reinterpret_cast<uint4*>(a.x_prev + (size_t)b * d.E)[c] = reinterpret_cast<const uint4*>(a.x + (size_t)b * d.E)[c];
+    return;
+  }
+  const bool is_q = head < d.hq;
+  const int ch0 = head * DH;                   // first channel of the head in the q0|k0 latent
+  const int pad = d.k_seq + d.k_ch - 2;
+  const int ks = (d.flags & F_CONV1) ? d.k_seq : 1;
+  const int kc = (d.flags & F_CONV2) ? d.k_ch : 1;
+  const float* lat_b = a.lat + (size_t)b * ld_lat;
+  for (int i = tid; i < (pad + 1) * DH; i += 128) {
+    const int r = i / DH, c = i % DH;
+    win[r][c] = r < pad ? a.hist[((size_t)b * pad + r) * d.L + ch0 + c] : lat_b[ch0 + c];
+  }
+  __syncthreads();
+  // Eq. 8, conv1 at the kc tokens conv2 reads
+  for (int i = tid; i < kc * DH; i += 128) {
+    const int r = i / DH, c = i % DH;
+    const int row = pad - (kc - 1) + r;
+    float acc;
+    if (d.flags & F_CONV1) {
+      acc = 0.f;
+      for (int j = 0; j < ks; ++j)
+        acc = fmaf(__bfloat162float(a.w0[(size_t)(ch0 + c) * d.k_seq + j]), win[row - (ks - 1) + j][c], acc);
+    } else {
+      acc = win[row][c];
+    }
+    y1[r][c] = acc;
+  }
+  __syncthreads();
+  // Eq. 8, conv2 at the new token: one warp per output channel, lanes over (input channel, tap)
+  if (d.flags & F_CONV2) {
+    for (int o = warp; o < DH; o += 4) {
+      const bf16* wr = a.w1 + (size_t)(ch0 + o) * DH * d.k_ch;
+      float acc = 0.f;
+      for (int idx = lane; idx < DH * d.k_ch; idx += 32) {
+        const int i = idx / d.k_ch, r = idx % d.k_ch;
+        acc = fmaf(__bfloat162float(wr[idx]), y1[r][i], acc);
+      }
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+      if (lane == 0) xh[o] = acc;
+    }
+  } else {
+    for (int c = tid; c < DH; c += 128) xh[c] = y1[kc - 1][c];
+  }
+  __syncthreads();
+  // history for the next token: drop the oldest row, append this token's q0|k0 (every read of the old rows is done)
+  for (int i = tid; i < pad * DH; i += 128) {
+    const int r = i / DH, c = i % DH;
+    a.hist[((size_t)b * pad + r) * d.L + ch0 + c] = win[r + 1][c];
+  }
+  // Eq. 9 (q-k-mean), Eq. 11 (norm, temperature, RoPE)
+  float val[DH / 128 > 0 ? DH / 128 : 1];
+  float ssq = 0.f;
+  constexpr int PER = DH >= 128 ? DH / 128 : 1;
+#pragma unroll
+  for (int u = 0; u < PER; ++u) {
+    const int c = tid + u * 128;
+    float v = 0.f;
+    if (c < DH) {
+      v = xh[c];
+      if (d.flags & F_QK_MEAN) {
+        if (is_q) {
+          const int j = head / d.g;
+          v += 0.5f * (lat_b[ch0 + c] + lat_b[d.Lq + j * DH + c]);
+        } else {
+          const int j = head - d.hq;
+          float sq = 0.f;
+          for (int i = 0; i < d.g; ++i) sq += lat_b[(j * d.g + i) * DH + c];
+          v += 0.5f * lat_b[ch0 + c] + 0.5f * sq / (float)d.g;
+        }
+      }
+      ssq = fmaf(v, v, ssq);
+    }
+    val[u] = v;
+  }
+  if (d.flags & F_QK_NORM) {
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, s);
+    if (lane == 0) red[warp] = ssq;
+    __syncthreads();
+    const float tot = red[0] + red[1] + red[2] + red[3];
+    float sc = sqrtf((float)DH) * rsqrtf(tot);
+    if (!is_q) sc *= __expf(a.temp[head - d.hq]);
+#pragma unroll
+    for (int u = 0; u < PER; ++u) val[u] *= sc;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int u = 0; u < PER; ++u)
+    if (tid + u * 128 < DH) xh[tid + u * 128] = val[u];
+  __syncthreads();
+#pragma unroll
+  for (int u = 0; u < PER; ++u) {
+    const int c = tid + u * 128;
+    if (c >= DH) continue;
+    float v = xh[c];
+    if (d.flags & F_ROPE) {
+      const int cc = c % (DH / 2);
+      const double theta = exp2(-2.0 * (double)cc / (double)DH * log2((double)d.rope_base));
+      double sn, cs;
+      sincos((double)t * theta, &sn, &cs);
+      v = c < DH / 2 ? xh[c] * (float)cs - xh[c + DH / 2] * (float)sn : xh[c] * (float)cs + xh[c - DH / 2] * (float)sn;
+    }
+    if (is_q) a.q[(size_t)b * d.Lq + ch0 + c] = v;
+    else a.k_cache[((size_t)b * a.S_max + t) * d.Lk + (ch0 - d.Lq) + c] = __float2bfloat16(v);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ attention
+struct AtArgs {
+  CcaDims d;
+  const float* q;        // [B, Lq]
+  const bf16* k_cache;
+  const bf16* v_cache;
+  const float* temp;     // log key temperature if q, k are normalised, else null
+  const int* pos;
+  long long S_max;
+  int max_len;
+  int chunk, splits;
+  float* part_o;         // [B, hq, splits, DH]
+  float* part_ml;        // [B, hq, splits, 2]
+};
+
+constexpr int DA_WARPS = 4, DA_UNR = 4;
+
+// One CTA: keys [split * chunk, ...) of sequence b, kv head j, query heads [j g + gq0, j g + gq0 + GQ).
+// A key row (d_h bf16) is read by d_h / 8 adjacent lanes, 16 bytes each; a warp reads 256 / d_h keys per load.
+template <int DH, int GQ>
+__global__ void __launch_bounds__(DA_WARPS * 32) decode_attn_kernel(AtArgs a) {
+  constexpr int LPK = DH / 8;                  // lanes per key
+  constexpr int KPW = 32 / LPK;                // keys per warp load
+  const CcaDims& d = a.d;
+  const int split = blockIdx.x, b = blockIdx.z;
+  const int n_grp = (d.g + GQ - 1) / GQ;
+  const int j = blockIdx.y / n_grp, gq0 = (blockIdx.y % n_grp) * GQ;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int sub = lane / LPK, cl = (lane % LPK) * 8;       // key within the load, first channel of this lane
+  const int t = a.pos[b];
+  if (t < 0 || t >= a.S_max || t >= a.max_len) return;     // reported by the transform kernel
+  const int n_keys = t + 1;
+  const int k_begin = split * a.chunk, k_end = min(n_keys, k_begin + a.chunk);
+  const float c_scale = rsqrtf((float)DH) * LOG2E;
+
+  float qf[GQ][8];
+#pragma unroll
+  for (int h = 0; h < GQ; ++h) {
+    const int hi = j * d.g + min(gq0 + h, d.g - 1);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) qf[h][c] = a.q[(size_t)b * d.Lq + hi * DH + cl + c] * c_scale;
+  }
+  float m[GQ], l[GQ], acc[GQ][8];
+  bool fixed = false;
+  float m_fixed = 0.f;
+  if (a.temp != nullptr) {
+    m_fixed = sqrtf((float)DH) * __expf(a.temp[j]) * LOG2E * 1.01f;
+    fixed = m_fixed <= 56.f;
+  }
+#pragma unroll
+  for (int h = 0; h < GQ; ++h) {
+    m[h] = fixed ? m_fixed : -INFINITY;
+    l[h] = 0.f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) acc[h][c] = 0.f;
+  }
+  const bf16* kb = a.k_cache + (size_t)b * a.S_max * d.Lk + j * DH + cl;
+  const bf16* vb = a.v_cache + (size_t)b * a.S_max * d.Lk + j * DH + cl;
+  for (int k0 = k_begin + warp * KPW * DA_UNR; k0 < k_end; k0 += DA_WARPS * KPW * DA_UNR) {
+    uint4 kf[DA_UNR], vf[DA_UNR];
+#pragma unroll
+    for (int u = 0; u < DA_UNR; ++u) {
+      const int key = k0 + u * KPW + sub;
+      kf[u] = vf[u] = make_uint4(0, 0, 0, 0);
+      if (key < k_end) {
+        kf[u] = __ldcs(reinterpret_cast<const uint4*>(kb + (size_t)key * d.Lk));
+        vf[u] = __ldcs(reinterpret_cast<const uint4*>(vb + (size_t)key * d.Lk));
+      }
+    }
+    float s[DA_UNR][GQ];
+#pragma unroll
+    for (int u = 0; u < DA_UNR; ++u) {
+      float kx[8];
+      unpack8(kf[u], kx);
+#pragma unroll
+      for (int h = 0; h < GQ; ++h) {
+        float p = 0.f;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) p = fmaf(qf[h][c], kx[c], p);
+        s[u][h] = p;
+      }
+    }
+#pragma unroll
+    for (int o = LPK / 2; o > 0; o >>= 1)
+#pragma unroll
+      for (int u = 0; u < DA_UNR; ++u)
+#pragma unroll
+        for (int h = 0; h < GQ; ++h) s[u][h] += __shfl_xor_sync(0xffffffffu, s[u][h], o);
+#pragma unroll
+    for (int u = 0; u < DA_UNR; ++u)
+      if (k0 + u * KPW + sub >= k_end)
+#pragma unroll
+        for (int h = 0; h < GQ; ++h) s[u][h] = -INFINITY;
+    if (!fixed) {
+#pragma unroll
+      for (int h = 0; h < GQ; ++h) {
+        float mx = s[0][h];
+#pragma unroll
+        for (int u = 1; u < DA_UNR; ++u) mx = fmaxf(mx, s[u][h]);
+        if (mx > m[h]) {
+          const float alpha = exp2f(m[h] - mx);      // 0 on the first keys (m = -inf)
+          l[h] *= alpha;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) acc[h][c] *= alpha;
+          m[h] = mx;
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < DA_UNR; ++u) {
+      float vx[8];
+      unpack8(vf[u], vx);
+#pragma unroll
+      for (int h = 0; h < GQ; ++h) {
+        const float p = (s[u][h] == -INFINITY) ? 0.f : exp2f(s[u][h] - m[h]);
+        l[h] += p;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[h][c] = fmaf(p, vx[c], acc[h][c]);
+      }
+    }
+  }
+  // merge the key sub-groups of the warp (lanes that hold the same channels of different keys)
+#pragma unroll
+  for (int o = LPK; o < 32; o <<= 1) {
+#pragma unroll
+    for (int h = 0; h < GQ; ++h) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m[h], o);
+      const float l2 = __shfl_xor_sync(0xffffffffu, l[h], o);
+      const float mn = fmaxf(m[h], m2);
+      const float a1 = (m[h] == -INFINITY) ? 0.f : exp2f(m[h] - mn);
+      const float a2 = (m2 == -INFINITY) ? 0.f : exp2f(m2 - mn);
+      l[h] = l[h] * a1 + l2 * a2;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const float o2 = __shfl_xor_sync(0xffffffffu, acc[h][c], o);
+        acc[h][c] = acc[h][c] * a1 + o2 * a2;
+      }
+      m[h] = mn;
+    }
+  }
+  // merge the warps through shared memory
+  __shared__ float sm_o[DA_WARPS][GQ][DH];
+  __shared__ float sm_ml[DA_WARPS][GQ][2];
+  if (sub == 0) {
+#pragma unroll
+    for (int h = 0; h < GQ; ++h) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) sm_o[warp][h][cl + c] = acc[h][c];
+      if (lane == 0) { sm_ml[warp][h][0] = m[h]; sm_ml[warp][h][1] = l[h]; }
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < GQ * DH; i += DA_WARPS * 32) {
+    const int h = i / DH, c = i % DH;
+    if (gq0 + h >= d.g) continue;
+    float mn = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < DA_WARPS; ++w) mn = fmaxf(mn, sm_ml[w][h][0]);
+    float lo = 0.f, oo = 0.f;
+#pragma unroll
+    for (int w = 0; w < DA_WARPS; ++w) {
+      const float al = (sm_ml[w][h][0] == -INFINITY) ? 0.f : exp2f(sm_ml[w][h][0] - mn);
+      lo += sm_ml[w][h][1] * al;
+      oo += sm_o[w][h][c] * al;
+    }
+    const int hi = j * d.g + gq0 + h;
+    const size_t pidx = ((size_t)b * d.hq + hi) * a.splits + split;
+    a.part_o[pidx * DH + c] = oo;
+    if (c == 0) { a.part_ml[pidx * 2] = mn; a.part_ml[pidx * 2 + 1] = lo; }
+  }
+}
+
+struct CbArgs {
+  CcaDims d;
+  const float* part_o;
+  const float* part_ml;
+  const int* pos;
+  long long S_max;
+  int max_len, splits;
+  bf16* o;               // [B, Lq]
+};
+
+template <int DH>
+__global__ void __launch_bounds__(DH < 64 ? 64 : DH) decode_combine_kernel(CbArgs a) {
+  const int hi = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
+  const int t = a.pos[b];
+  if (t < 0 || t >= a.S_max || t >= a.max_len) return;
+  if (c >= DH) return;
+  const size_t p0 = ((size_t)b * a.d.hq + hi) * a.splits;
+  float mn = -INFINITY;
+  for (int s = 0; s < a.splits; ++s) mn = fmaxf(mn, a.part_ml[(p0 + s) * 2]);
+  float lo = 0.f, oo = 0.f;
+  for (int s = 0; s < a.splits; ++s) {
+    const float ms = a.part_ml[(p0 + s) * 2];
+    const float al = (ms == -INFINITY) ? 0.f : exp2f(ms - mn);
+    lo += a.part_ml[(p0 + s) * 2 + 1] * al;
+    oo += a.part_o[(p0 + s) * DH + c] * al;
+  }
+  a.o[(size_t)b * a.d.Lq + hi * DH + c] = __float2bfloat16(oo / lo);
+}
+
+int padded_rows(int rows) { return (rows + PJ_ROWS - 1) / PJ_ROWS * PJ_ROWS; }
+
+cudaError_t launch_proj(ProjArgs& a, cudaStream_t st) {
+  int tot = 0;
+  for (int s = 0; s < a.n_seg; ++s) tot += padded_rows(a.seg[s].rows);
+  a.rows_total = tot;
+  dim3 grid((unsigned)(tot / PJ_ROWS), (unsigned)((a.B + PJ_BT - 1) / PJ_BT));
+  decode_proj_kernel<<<grid, PJ_WARPS * 32, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+template <int DH>
+cudaError_t launch_attn_dh(const AtArgs& a, cudaStream_t st) {
+  const CcaDims& d = a.d;
+  if (d.g >= 4) {
+    dim3 grid((unsigned)a.splits, (unsigned)(d.hk * ((d.g + 3) / 4)), (unsigned)d.B);
+    decode_attn_kernel<DH, 4><<<grid, DA_WARPS * 32, 0, st>>>(a);
+  } else if (d.g >= 2) {
+    dim3 grid((unsigned)a.splits, (unsigned)(d.hk * ((d.g + 1) / 2)), (unsigned)d.B);
+    decode_attn_kernel<DH, 2><<<grid, DA_WARPS * 32, 0, st>>>(a);
+  } else {
+    dim3 grid((unsigned)a.splits, (unsigned)d.hk, (unsigned)d.B);
+    decode_attn_kernel<DH, 1><<<grid, DA_WARPS * 32, 0, st>>>(a);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+void decode_plan(const CcaDims& d, int max_len, int sm_count, int* chunk, int* splits) {
+  const int n_grp = d.g >= 4 ? (d.g + 3) / 4 : (d.g >= 2 ? (d.g + 1) / 2 : 1);
+  const long long base = (long long)d.B * d.hk * n_grp;
+  long long want = (4LL * sm_count + base - 1) / base;         // about four CTAs per SM
+  if (want < 1) want = 1;
+  if (want > 128) want = 128;
+  int ch = (int)((max_len + want - 1) / want);
+  ch = (ch + 127) / 128 * 128;                                 // a warp iteration covers up to 64 keys
+  if (ch < 128) ch = 128;
+  *chunk = ch;
+  *splits = (max_len + ch - 1) / ch;
+}
+
+size_t decode_workspace_bytes(const CcaDims& d, int max_len, int sm_count) {
+  int chunk, splits;
+  decode_plan(d, max_len, sm_count, &chunk, &splits);
+  auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+  size_t n = 0;
+  n += up((size_t)d.B * (d.L + d.Lk) * 4);             // lat
+  n += up((size_t)d.B * d.Lq * 4);                     // q
+  n += up((size_t)d.B * d.hq * splits * d.dh * 4);     // partial o
+  n += up((size_t)d.B * d.hq * splits * 2 * 4);        // partial (m, l)
+  n += up((size_t)d.B * d.Lq * 2);                     // o
+  return n;
+}
+
+int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, bf16* out, const DecodeState& s,
+                       int max_len, void* workspace, int sm_count, int* status, long long* launches, cudaStream_t st) {
+  int chunk, splits;
+  decode_plan(d, max_len, sm_count, &chunk, &splits);
+  auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+  unsigned char* p = static_cast<unsigned char*>(workspace);
+  float* lat = reinterpret_cast<float*>(p); p += up((size_t)d.B * (d.L + d.Lk) * 4);
+  float* q = reinterpret_cast<float*>(p); p += up((size_t)d.B * d.Lq * 4);
+  float* part_o = reinterpret_cast<float*>(p); p += up((size_t)d.B * d.hq * splits * d.dh * 4);
+  float* part_ml = reinterpret_cast<float*>(p); p += up((size_t)d.B * d.hq * splits * 2 * 4);
+  bf16* o = reinterpret_cast<bf16*>(p);
+  cudaError_t e;
+  // Eq. 7 and Eq. 10: q0 | k0 | v1 from x_t, v2 from x_{t-1}
+  ProjArgs pa;
+  memset(&pa, 0, sizeof(pa));
+  pa.n_seg = 3;
+  pa.seg[0] = ProjSeg{w.w_qk, x, d.L, 0};
+  pa.seg[1] = ProjSeg{w.w_v1, x, d.Lk / 2, d.L};
+  pa.seg[2] = ProjSeg{w.w_v2, (d.flags & F_V_SHIFT) ? s.x_prev : x, d.Lk / 2, d.L + d.Lk / 2};
+  pa.K = d.E; pa.B = d.B; pa.out_f32 = lat; pa.ldo = d.L + d.Lk;
+  if ((e = launch_proj(pa, st)) != cudaSuccess) return -(int)e;
+  ++*launches;
+  TrArgs ta;
+  ta.d = d; ta.lat = lat; ta.x = x; ta.w0 = w.conv0_w; ta.w1 = w.conv1_w; ta.temp = w.temp; ta.q = q;
+  ta.k_cache = s.k_cache; ta.v_cache = s.v_cache; ta.hist = s.qk0_hist; ta.x_prev = s.x_prev; ta.pos = s.pos;
+  ta.S_max = s.S_max; ta.max_len = max_len; ta.status = status;
+  {
+    dim3 grid((unsigned)(d.hq + d.hk + 1), (unsigned)d.B);
+    switch (d.dh) {
+      case 32: decode_transform_kernel<32><<<grid, 128, 0, st>>>(ta); break;
+      case 64: decode_transform_kernel<64><<<grid, 128, 0, st>>>(ta); break;
+      case 128: decode_transform_kernel<128><<<grid, 128, 0, st>>>(ta); break;
+      default: return 1;
+    }
+    if ((e = cudaGetLastError()) != cudaSuccess) return -(int)e;
+    ++*launches;
+  }
+  AtArgs aa;
+  aa.d = d; aa.q = q; aa.k_cache = s.k_cache; aa.v_cache = s.v_cache;
+  aa.temp = (d.flags & F_QK_NORM) ? w.temp : nullptr;
+  aa.pos = s.pos; aa.S_max = s.S_max; aa.max_len = max_len; aa.chunk = chunk; aa.splits = splits;
+  aa.part_o = part_o; aa.part_ml = part_ml;
+  switch (d.dh) {
+    case 32: e = launch_attn_dh<32>(aa, st); break;
+    case 64: e = launch_attn_dh<64>(aa, st); break;
+    case 128: e = launch_attn_dh<128>(aa, st); break;
+    default: return 1;
+  }
+  if (e != cudaSuccess) return -(int)e;
+  ++*launches;
+  CbArgs ca;
+  ca.d = d; ca.part_o = part_o; ca.part_ml = part_ml; ca.pos = s.pos; ca.S_max = s.S_max; ca.max_len = max_len;
+  ca.splits = splits; ca.o = o;
+  {
+    dim3 grid((unsigned)d.hq, (unsigned)d.B);
+    switch (d.dh) {
+      case 32: decode_combine_kernel<32><<<grid, 64, 0, st>>>(ca); break;
+      case 64: decode_combine_kernel<64><<<grid, 64, 0, st>>>(ca); break;
+      case 128: decode_combine_kernel<128><<<grid, 128, 0, st>>>(ca); break;
+      default: return 1;
+    }
+    if ((e = cudaGetLastError()) != cudaSuccess) return -(int)e;
+    ++*launches;
+  }
+  // Eq. 11, up-projection
+  ProjArgs pb;
+  memset(&pb, 0, sizeof(pb));
+  pb.n_seg = 1;
+  pb.seg[0] = ProjSeg{w.w_o, o, d.E, 0};
+  pb.K = d.Lq; pb.B = d.B; pb.out_bf16 = out; pb.ldo = d.E;
+  if ((e = launch_proj(pb, st)) != cudaSuccess) return -(int)e;
+  ++*launches;
+  return 0;
+}
