@@ -310,6 +310,178 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+DECODE_WORKLOADS = {
+    # model of the 16k prefill shape; 32 sequences, each with 16384 cached tokens
+    "decode16k": dict(model="cfg3_prefill16k", B=32, context=16384),
+}
+
+
+def decode_bytes(sh, B, context):
+    """Algorithmic HBM bytes of one decode step: every cached key and value row of every sequence once, every
+    weight once, the new token's input and output."""
+    cache = 2 * B * (context + 1) * sh.L_k * 2
+    weights = 2 * (sh.L + sh.L_k) * sh.d_model + 2 * sh.d_model * sh.L_q + 2 * sh.L * (sh.k_seq + sh.head_dim * sh.k_ch)
+    io = 2 * 2 * B * sh.d_model
+    return {"cache": cache, "weights": weights, "io": io, "total": cache + weights + io}
+
+
+def hbm_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (copy)"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def run_decode(args, rank, world, local_rank):
+    """One decode step per timed step: B new tokens against caches of `context` tokens per sequence.  The cache of
+    one really prefilled sequence is replicated over the batch (the step's work does not depend on the values)."""
+    from paper_2510_04476_b200.binding import CCA
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    wl = DECODE_WORKLOADS[args.workload]
+    sh = synth.CONFIGS[wl["model"]]
+    B, ctx = wl["B"], wl["context"]
+    n_steps = max(3, args.warmup) + args.steps + 12
+    S_max = ctx + n_steps + 1
+    t = synth.make_inputs(sh.replace(B=1, S=ctx), want_dout=False)
+    dev = {k: v.cuda(local_rank).contiguous() for k, v in t.items()}
+    cca = CCA.from_shape(sh, device=local_rank)
+    ws = cca.alloc_workspace(1, ctx, False)
+    cca.forward(dev, dev["x"], ws)
+    one = cca.new_decode_state(1, S_max)
+    cca.decode_state_from_prefill(dev["x"], ws, one)
+    st = cca.new_decode_state(B, S_max)
+    for n in ("k_cache", "v_cache", "qk0_hist", "x_prev"):
+        st[n].copy_(one[n].expand_as(st[n]))
+    del ws, one
+    g = torch.Generator().manual_seed(99)
+    xs_host = torch.randn(n_steps, B, sh.d_model, generator=g).to(torch.bfloat16).pin_memory()
+    xs = xs_host.cuda(local_rank)
+    pos_table = (ctx + torch.arange(n_steps, dtype=torch.int32)[:, None].expand(n_steps, B)).contiguous().cuda(local_rank)
+    dws = cca.alloc_decode_workspace(B, S_max)
+    out = torch.empty(B, sh.d_model, dtype=torch.bfloat16, device=dev["x"].device)
+    it = [0]
+
+    def step(x=None):
+        i = it[0]
+        it[0] += 1
+        st["pos"] = pos_table[i]
+        cca.decode_step(dev, xs[i] if x is None else x, st, S_max, dws, out)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in ev:
+        a.record(); b.record()
+    torch.cuda.synchronize()
+    vis = [v for v in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if v]
+    sampler = ClockSampler(vis[local_rank] if local_rank < len(vis) else str(local_rank))
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.15)
+    barrier()
+    l0 = cca.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0 = time.time()
+    e0.record()
+    for i in range(args.steps):
+        cca.set_attention_events(*ev[i])
+        step()
+    e1.record()
+    barrier()
+    w1 = time.time()
+    cca.set_attention_events(None, None)
+    launches = cca.launch_count() - l0
+    clocks = sampler.stop(w0, w1) if rank == 0 else None
+    tm = torch.tensor([e0.elapsed_time(e1)], device="cuda", dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+    ms_step = float(tm.item()) / args.steps
+    attn_ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
+    status = cca.last_status()
+    # end to end: the new tokens come from pinned host memory, the outputs go back to it
+    oh = torch.empty(B, sh.d_model, dtype=torch.bfloat16).pin_memory()
+    xd = torch.empty(B, sh.d_model, dtype=torch.bfloat16, device=out.device)
+    n_e2e = min(args.steps, 10)
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    g0.record()
+    for i in range(n_e2e):
+        xd.copy_(xs_host[it[0]], non_blocking=True)
+        step(xd)
+        oh.copy_(out, non_blocking=True)
+        torch.cuda.synchronize()
+    g1.record()
+    barrier()
+    e2e_ms = torch.tensor([g0.elapsed_time(g1) / n_e2e], device="cuda", dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+    by = decode_bytes(sh, B, ctx)
+    peak, peak_kind = hbm_peak()
+    attn_gbs = by["cache"] / (attn_ms * 1e-3) / 1e9
+    line = {
+        "metric": "CCGQA decode throughput at 16k context (new tokens / device time)", "value": world * B / (ms_step * 1e-3),
+        "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "step": "decode", "B": B, "context": ctx, "d_model": sh.d_model,
+                   "n_q_heads": sh.n_q_heads, "n_kv_heads": sh.n_kv_heads, "head_dim": sh.head_dim, "k_seq": sh.k_seq,
+                   "k_ch": sh.k_ch, "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
+                   "l2": f"no flush: each step streams {by['cache'] / 1e6:.0f} MB of cache, more than the 126 MB L2"},
+        "clocks": clocks,
+        "e2e": {"value": world * B / (float(e2e_ms.item()) * 1e-3), "unit": "tokens/s",
+                "h2d_bytes_per_step": B * sh.d_model * 2, "d2h_bytes_per_step": B * sh.d_model * 2,
+                "ms_per_step": float(e2e_ms.item())},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "decode attention over the latent cache", "achieved": attn_gbs, "peak": peak,
+                     "unit": "GB/s", "frac": attn_gbs / peak, "peak_kind": peak_kind, "ms_per_launch": attn_ms,
+                     "bytes_per_launch": by["cache"], "traffic": None},
+        "step_gbs": by["total"] / (ms_step * 1e-3) / 1e9, "step_bytes": by,
+        "device_status": status,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu:
+        v, dt, sample = oracle_decode_sample(sh, ctx)
+        line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
+                                "sample": sample, "seconds": dt}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    cca.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def oracle_decode_sample(sh, ctx):
+    """The oracle's decode step, as it stands, for one sequence with `ctx` cached tokens (the prefill that fills
+    the cache is not timed)."""
+    from oracle import cca_oracle as O
+    n_new = 2048
+    s1 = sh.replace(B=1, S=ctx + n_new)
+    t = synth.make_inputs(s1, want_dout=False)
+    cfg = O.OracleConfig(sh.d_model, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.k_seq, sh.k_ch, sh.causal, sh.flags,
+                         sh.rope_base)
+    I = O.pre_attention(cfg, t, t["x"][:, :ctx])
+    st = O.decode_state_after_prefill(cfg, I, ctx)
+    t0 = time.perf_counter()
+    n = 0
+    while n < n_new and (n < 4 or time.perf_counter() - t0 < 10.0):
+        O.decode_step(cfg, t, st, t["x"][:, ctx + n])
+        n += 1
+    dt = time.perf_counter() - t0
+    return n / dt, dt, f"{n} consecutive tokens of one sequence with {ctx} cached tokens"
+
+
 def fwd_bwd_same_shape(sh, args, local_rank):
     """The headline shape with the backward as well (the metric asks for forward and forward + backward at
     16k context).  Reported beside the forward-only line; not part of the timed region above."""
@@ -384,7 +556,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg3_prefill16k", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--workload", default="cfg3_prefill16k", choices=sorted(synth.CONFIGS) + sorted(DECODE_WORKLOADS))
     ap.add_argument("--kernels", type=int, default=1, help="0 = SIMT kernels only, 1 = tcgen05 kernels where available")
     ap.add_argument("--backward", action="store_true", help="time forward + backward on a forward-only workload too")
     ap.add_argument("--no-mha", action="store_true")
@@ -393,8 +565,12 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference" and args.workload in DECODE_WORKLOADS:
+        raise SystemExit("the reference arm times the prefill workloads; the decode line carries its own cpu_baseline")
     if args.impl == "reference":
         run_reference(args, rank, world)
+    elif args.workload in DECODE_WORKLOADS:
+        run_decode(args, rank, world, local_rank)
     else:
         run_ours(args, rank, world, local_rank)
 

@@ -314,7 +314,7 @@ int cca_decode_step(cca_handle* h, const cca_weights* w, const void* x, void* ou
                    (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, (const float*)w->temp};
   DecodeState ds{(bf16*)s->k_cache, (bf16*)s->v_cache, (float*)s->qk0_hist, (bf16*)s->x_prev, s->pos, s->S_max};
   int rr = launch_decode_step(d, dw, (const bf16*)x, (bf16*)out, ds, (int)max_len, workspace, h->sm_count, h->d_status,
-                              &h->launches, (cudaStream_t)cuda_stream);
+                              &h->launches, h->ev_attn_begin, h->ev_attn_end, (cudaStream_t)cuda_stream);
   if (rr < 0) { h->last_cuda = -rr; return CCA_ERR_CUDA; }
   if (rr > 0) return CCA_ERR_UNSUPPORTED;
   return CCA_OK;

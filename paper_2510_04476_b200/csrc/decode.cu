@@ -529,7 +529,8 @@ size_t decode_workspace_bytes(const CcaDims& d, int max_len, int sm_count) {
 }
 
 int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, bf16* out, const DecodeState& s,
-                       int max_len, void* workspace, int sm_count, int* status, long long* launches, cudaStream_t st) {
+                       int max_len, void* workspace, int sm_count, int* status, long long* launches, cudaEvent_t ev_attn_begin,
+                       cudaEvent_t ev_attn_end, cudaStream_t st) {
   int chunk, splits;
   decode_plan(d, max_len, sm_count, &chunk, &splits);
   auto up = [](size_t v) { return (v + 255) / 256 * 256; };
@@ -570,6 +571,7 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
   aa.temp = (d.flags & F_QK_NORM) ? w.temp : nullptr;
   aa.pos = s.pos; aa.S_max = s.S_max; aa.max_len = max_len; aa.chunk = chunk; aa.splits = splits;
   aa.part_o = part_o; aa.part_ml = part_ml;
+  if (ev_attn_begin && (e = cudaEventRecord(ev_attn_begin, st)) != cudaSuccess) return -(int)e;
   switch (d.dh) {
     case 32: e = launch_attn_dh<32>(aa, st); break;
     case 64: e = launch_attn_dh<64>(aa, st); break;
@@ -578,6 +580,7 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
   }
   if (e != cudaSuccess) return -(int)e;
   ++*launches;
+  if (ev_attn_end && (e = cudaEventRecord(ev_attn_end, st)) != cudaSuccess) return -(int)e;
   CbArgs ca;
   ca.d = d; ca.part_o = part_o; ca.part_ml = part_ml; ca.pos = s.pos; ca.S_max = s.S_max; ca.max_len = max_len;
   ca.splits = splits; ca.o = o;

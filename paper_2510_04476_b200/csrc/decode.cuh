@@ -20,5 +20,7 @@ struct DecodeState {
 void decode_plan(const CcaDims& d, int max_len, int sm_count, int* chunk, int* splits);
 size_t decode_workspace_bytes(const CcaDims& d, int max_len, int sm_count);
 // 0 = enqueued, 1 = shape not covered, < 0 = minus a cudaError_t.  *launches is advanced by the kernels enqueued.
+// The two events (may be null) are recorded around the attention kernel.
 int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, bf16* out, const DecodeState& s,
-                       int max_len, void* workspace, int sm_count, int* status, long long* launches, cudaStream_t st);
+                       int max_len, void* workspace, int sm_count, int* status, long long* launches, cudaEvent_t ev_attn_begin,
+                       cudaEvent_t ev_attn_end, cudaStream_t st);
