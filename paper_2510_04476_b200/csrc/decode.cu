@@ -1,14 +1,15 @@
 // Decode step: one new token per sequence against the latent KV cache (the KV-cache and decode columns of the
 // paper's comparison table).  Everything here is bound by memory traffic -- the weights are read once per step
 // and every cached key and value row once per (sequence, kv head) -- so these are plain CUDA kernels laid out
-// for coalesced 16-byte accesses, not tensor-core tiles:
+// for coalesced 16-byte accesses, not tcgen05 tiles (the attention uses warp-level tensor-core instructions only to
+// keep its instruction count below what the loads need):
 //
 //   decode_proj_kernel      out[b, n] = sum_k W[n, k] x[b, k] for a few stacked weight segments (Eq. 7, 10; Eq. 11
 //                           up-projection): one warp per two weight rows, 16 sequences per CTA staged in shared memory
 //   decode_transform_kernel Eq. 8-11 for the new token of one (sequence, head): conv halo from the caller's history,
 //                           q-k-mean, norm, temperature, RoPE at the sequence's own position; appends k, v to the cache
 //   decode_attn_kernel      softmax(q k^T / sqrt(d_h)) v of the new query over a chunk of the cached keys of one
-//                           (sequence, kv head, group of <= 4 query heads); partial results per chunk
+//                           (sequence, kv head), all its query heads at once; partial results per chunk
 //   decode_combine_kernel   merges the chunks' partial results
 #include <cstring>
 
@@ -287,146 +288,200 @@ struct AtArgs {
   float* part_ml;        // [B, hq, splits, 2]
 };
 
-constexpr int DA_WARPS = 4, DA_UNR = 4;
+constexpr int DA_WARPS = 4;
 
-// One CTA: keys [split * chunk, ...) of sequence b, kv head j, query heads [j g + gq0, j g + gq0 + GQ).
-// A key row (d_h bf16) is read by d_h / 8 adjacent lanes, 16 bytes each; a warp reads 256 / d_h keys per load.
-template <int DH, int GQ>
+CCA_DEVINL void mma_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+CCA_DEVINL uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Channel of the cached row that output column n (0..7) of PV tile nt holds: thread (g, .) of a warp loads, of
+// every value row, the 16-byte pieces that start at channel 8 g (and 64 + 8 g when d_h = 128), or the 8-byte
+// piece at 4 g when d_h = 32, so that a warp's load covers whole rows; tile nt takes the nt-th of those channels.
+template <int DH>
+CCA_DEVINL int pv_channel(int nt, int n) {
+  if (DH == 32) return n * 4 + nt;
+  return (nt >> 3) * 64 + n * 8 + (nt & 7);
+}
+
+// One CTA: keys [split * chunk, ...) of sequence b, kv head j, up to 16 of its query heads.  The two
+// contractions of a 16-key block run as m16n8k16 tensor-core instructions with the query heads as the 16 rows
+// (most of them padding): one cached row costs a few instructions instead of 4 d_h multiply-adds per head, so the
+// kernel's speed is that of its loads.  Keys and values go from global memory straight into the operand
+// registers: a contraction does not care about the order of its inner index, so each lane takes 16 contiguous
+// bytes per key (QK^T, inner index = channel) and pairs the same channel of two value rows with a byte permute
+// (P V, inner index = key).
+template <int DH>
 __global__ void __launch_bounds__(DA_WARPS * 32) decode_attn_kernel(AtArgs a) {
-  constexpr int LPK = DH / 8;                  // lanes per key
-  constexpr int KPW = 32 / LPK;                // keys per warp load
+  constexpr int NT = DH / 8;                   // output tiles of P V = channels per lane per value row
+  constexpr int CB = DH / 32;                  // 32-channel blocks of Q K^T
+  constexpr int VW = NT / 2;                   // 32-bit words per lane per value row
   const CcaDims& d = a.d;
   const int split = blockIdx.x, b = blockIdx.z;
-  const int n_grp = (d.g + GQ - 1) / GQ;
-  const int j = blockIdx.y / n_grp, gq0 = (blockIdx.y % n_grp) * GQ;
+  const int n_grp = (d.g + 15) / 16;
+  const int j = blockIdx.y / n_grp, h0 = (blockIdx.y % n_grp) * 16;
+  const int nh = min(16, d.g - h0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int sub = lane / LPK, cl = (lane % LPK) * 8;       // key within the load, first channel of this lane
-  const int t = a.pos[b];
-  if (t < 0 || t >= a.S_max || t >= a.max_len) return;     // reported by the transform kernel
-  const int n_keys = t + 1;
+  const int g = lane >> 2, t = lane & 3;
+  const int tpos = a.pos[b];
+  if (tpos < 0 || tpos >= a.S_max || tpos >= a.max_len) return;     // reported by the transform kernel
+  const int n_keys = tpos + 1;
   const int k_begin = split * a.chunk, k_end = min(n_keys, k_begin + a.chunk);
   const float c_scale = rsqrtf((float)DH) * LOG2E;
 
-  float qf[GQ][8];
+  // query fragments: rows g and g + 8 of the 16-row operand are heads h0 + g and h0 + g + 8
+  uint32_t qa[CB][2][4];
 #pragma unroll
-  for (int h = 0; h < GQ; ++h) {
-    const int hi = j * d.g + min(gq0 + h, d.g - 1);
+  for (int cb = 0; cb < CB; ++cb)
 #pragma unroll
-    for (int c = 0; c < 8; ++c) qf[h][c] = a.q[(size_t)b * d.Lq + hi * DH + cl + c] * c_scale;
-  }
-  float m[GQ], l[GQ], acc[GQ][8];
+    for (int mm = 0; mm < 2; ++mm) {
+#pragma unroll
+      for (int hi = 0; hi < 2; ++hi) {
+        float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (g + 8 * hi < nh)
+          qv = *reinterpret_cast<const float4*>(a.q + (size_t)b * d.Lq + (size_t)(j * d.g + h0 + g + 8 * hi) * DH + cb * 32 +
+                                                t * 8 + mm * 4);
+        qa[cb][mm][hi] = pack_bf16x2(qv.x, qv.y);
+        qa[cb][mm][2 + hi] = pack_bf16x2(qv.z, qv.w);
+      }
+    }
   bool fixed = false;
   float m_fixed = 0.f;
   if (a.temp != nullptr) {
     m_fixed = sqrtf((float)DH) * __expf(a.temp[j]) * LOG2E * 1.01f;
     fixed = m_fixed <= 56.f;
   }
+  float m_row[2] = {fixed ? m_fixed : -INFINITY, fixed ? m_fixed : -INFINITY};
+  float l_row[2] = {0.f, 0.f};
+  float o[NT][4];
 #pragma unroll
-  for (int h = 0; h < GQ; ++h) {
-    m[h] = fixed ? m_fixed : -INFINITY;
-    l[h] = 0.f;
+  for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-    for (int c = 0; c < 8; ++c) acc[h][c] = 0.f;
-  }
-  const bf16* kb = a.k_cache + (size_t)b * a.S_max * d.Lk + j * DH + cl;
-  const bf16* vb = a.v_cache + (size_t)b * a.S_max * d.Lk + j * DH + cl;
-  for (int k0 = k_begin + warp * KPW * DA_UNR; k0 < k_end; k0 += DA_WARPS * KPW * DA_UNR) {
-    uint4 kf[DA_UNR], vf[DA_UNR];
+    for (int c = 0; c < 4; ++c) o[nt][c] = 0.f;
+
+  const bf16* kb = a.k_cache + (size_t)b * a.S_max * d.Lk + j * DH;
+  const bf16* vb = a.v_cache + (size_t)b * a.S_max * d.Lk + j * DH;
+  for (int k0 = k_begin + warp * 16; k0 < k_end; k0 += DA_WARPS * 16) {
+    // ---- loads of the 16-key block
+    uint4 kf[2][CB];
 #pragma unroll
-    for (int u = 0; u < DA_UNR; ++u) {
-      const int key = k0 + u * KPW + sub;
-      kf[u] = vf[u] = make_uint4(0, 0, 0, 0);
+    for (int ti = 0; ti < 2; ++ti) {
+      const int key = k0 + ti * 8 + g;
+#pragma unroll
+      for (int cb = 0; cb < CB; ++cb) {
+        kf[ti][cb] = make_uint4(0, 0, 0, 0);
+        if (key < k_end) kf[ti][cb] = __ldcs(reinterpret_cast<const uint4*>(kb + (size_t)key * d.Lk + cb * 32 + t * 8));
+      }
+    }
+    uint32_t vf[4][VW];                        // value rows 2t, 2t+1, 2t+8, 2t+9 of the block
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int key = k0 + 2 * t + (r & 1) + (r >> 1) * 8;
+#pragma unroll
+      for (int w = 0; w < VW; ++w) vf[r][w] = 0u;
       if (key < k_end) {
-        kf[u] = __ldcs(reinterpret_cast<const uint4*>(kb + (size_t)key * d.Lk));
-        vf[u] = __ldcs(reinterpret_cast<const uint4*>(vb + (size_t)key * d.Lk));
-      }
-    }
-    float s[DA_UNR][GQ];
+        const bf16* vr = vb + (size_t)key * d.Lk;
+        if (DH == 32) {
+          const uint2 u = __ldcs(reinterpret_cast<const uint2*>(vr + g * 4));
+          vf[r][0] = u.x; vf[r][1] = u.y;
+        } else {
 #pragma unroll
-    for (int u = 0; u < DA_UNR; ++u) {
-      float kx[8];
-      unpack8(kf[u], kx);
-#pragma unroll
-      for (int h = 0; h < GQ; ++h) {
-        float p = 0.f;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) p = fmaf(qf[h][c], kx[c], p);
-        s[u][h] = p;
-      }
-    }
-#pragma unroll
-    for (int o = LPK / 2; o > 0; o >>= 1)
-#pragma unroll
-      for (int u = 0; u < DA_UNR; ++u)
-#pragma unroll
-        for (int h = 0; h < GQ; ++h) s[u][h] += __shfl_xor_sync(0xffffffffu, s[u][h], o);
-#pragma unroll
-    for (int u = 0; u < DA_UNR; ++u)
-      if (k0 + u * KPW + sub >= k_end)
-#pragma unroll
-        for (int h = 0; h < GQ; ++h) s[u][h] = -INFINITY;
-    if (!fixed) {
-#pragma unroll
-      for (int h = 0; h < GQ; ++h) {
-        float mx = s[0][h];
-#pragma unroll
-        for (int u = 1; u < DA_UNR; ++u) mx = fmaxf(mx, s[u][h]);
-        if (mx > m[h]) {
-          const float alpha = exp2f(m[h] - mx);      // 0 on the first keys (m = -inf)
-          l[h] *= alpha;
-#pragma unroll
-          for (int c = 0; c < 8; ++c) acc[h][c] *= alpha;
-          m[h] = mx;
+          for (int hf = 0; hf < DH / 64; ++hf) {
+            const uint4 u = __ldcs(reinterpret_cast<const uint4*>(vr + hf * 64 + g * 8));
+            vf[r][hf * 4 + 0] = u.x; vf[r][hf * 4 + 1] = u.y; vf[r][hf * 4 + 2] = u.z; vf[r][hf * 4 + 3] = u.w;
+          }
         }
       }
     }
+    // ---- S = Q K^T for the two 8-key tiles
+    float sc[2][4];
 #pragma unroll
-    for (int u = 0; u < DA_UNR; ++u) {
-      float vx[8];
-      unpack8(vf[u], vx);
+    for (int ti = 0; ti < 2; ++ti) {
 #pragma unroll
-      for (int h = 0; h < GQ; ++h) {
-        const float p = (s[u][h] == -INFINITY) ? 0.f : exp2f(s[u][h] - m[h]);
-        l[h] += p;
+      for (int c = 0; c < 4; ++c) sc[ti][c] = 0.f;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) acc[h][c] = fmaf(p, vx[c], acc[h][c]);
+      for (int cb = 0; cb < CB; ++cb) {
+        mma_16816(sc[ti], qa[cb][0], kf[ti][cb].x, kf[ti][cb].y);
+        mma_16816(sc[ti], qa[cb][1], kf[ti][cb].z, kf[ti][cb].w);
       }
+    }
+    // ---- softmax weights of this block; thread (g, t) holds rows g, g + 8 and keys 2t, 2t+1 of each tile
+#pragma unroll
+    for (int ti = 0; ti < 2; ++ti)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int key = k0 + ti * 8 + 2 * t + (c & 1);
+        sc[ti][c] = key < k_end ? sc[ti][c] * c_scale : -INFINITY;
+      }
+    if (!fixed) {
+      float mx[2];
+#pragma unroll
+      for (int hi = 0; hi < 2; ++hi) {
+        mx[hi] = fmaxf(fmaxf(sc[0][2 * hi], sc[0][2 * hi + 1]), fmaxf(sc[1][2 * hi], sc[1][2 * hi + 1]));
+        mx[hi] = fmaxf(mx[hi], __shfl_xor_sync(0xffffffffu, mx[hi], 1));
+        mx[hi] = fmaxf(mx[hi], __shfl_xor_sync(0xffffffffu, mx[hi], 2));
+      }
+      const bool grow = mx[0] > m_row[0] || mx[1] > m_row[1];
+      if (__any_sync(0xffffffffu, grow)) {
+#pragma unroll
+        for (int hi = 0; hi < 2; ++hi) {
+          if (mx[hi] > m_row[hi]) {
+            const float alpha = exp2f(m_row[hi] - mx[hi]);     // 0 while nothing has been seen (m = -inf)
+            l_row[hi] *= alpha;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) { o[nt][2 * hi] *= alpha; o[nt][2 * hi + 1] *= alpha; }
+            m_row[hi] = mx[hi];
+          }
+        }
+      }
+    }
+    uint32_t pa[4];
+#pragma unroll
+    for (int ti = 0; ti < 2; ++ti)
+#pragma unroll
+      for (int hi = 0; hi < 2; ++hi) {
+        const float mu = m_row[hi] == -INFINITY ? 0.f : m_row[hi];
+        const float p0 = exp2f(sc[ti][2 * hi] - mu), p1 = exp2f(sc[ti][2 * hi + 1] - mu);
+        const uint32_t w = pack_bf16x2(p0, p1);
+        pa[2 * ti + hi] = w;
+        // the sum runs over the rounded weights, the ones P V uses
+        l_row[hi] += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
+      }
+    // ---- O += P V
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const int w = nt >> 1;
+      const uint32_t sel = (nt & 1) ? 0x7632u : 0x5410u;
+      const uint32_t b0 = __byte_perm(vf[0][w], vf[1][w], sel);
+      const uint32_t b1 = __byte_perm(vf[2][w], vf[3][w], sel);
+      mma_16816(o[nt], pa, b0, b1);
     }
   }
-  // merge the key sub-groups of the warp (lanes that hold the same channels of different keys)
+  // row sums: the four lanes of a group hold different keys
 #pragma unroll
-  for (int o = LPK; o < 32; o <<= 1) {
-#pragma unroll
-    for (int h = 0; h < GQ; ++h) {
-      const float m2 = __shfl_xor_sync(0xffffffffu, m[h], o);
-      const float l2 = __shfl_xor_sync(0xffffffffu, l[h], o);
-      const float mn = fmaxf(m[h], m2);
-      const float a1 = (m[h] == -INFINITY) ? 0.f : exp2f(m[h] - mn);
-      const float a2 = (m2 == -INFINITY) ? 0.f : exp2f(m2 - mn);
-      l[h] = l[h] * a1 + l2 * a2;
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const float o2 = __shfl_xor_sync(0xffffffffu, acc[h][c], o);
-        acc[h][c] = acc[h][c] * a1 + o2 * a2;
-      }
-      m[h] = mn;
-    }
+  for (int hi = 0; hi < 2; ++hi) {
+    l_row[hi] += __shfl_xor_sync(0xffffffffu, l_row[hi], 1);
+    l_row[hi] += __shfl_xor_sync(0xffffffffu, l_row[hi], 2);
   }
   // merge the warps through shared memory
-  __shared__ float sm_o[DA_WARPS][GQ][DH];
-  __shared__ float sm_ml[DA_WARPS][GQ][2];
-  if (sub == 0) {
+  __shared__ float sm_o[DA_WARPS][16][DH];
+  __shared__ float sm_ml[DA_WARPS][16][2];
 #pragma unroll
-    for (int h = 0; h < GQ; ++h) {
+  for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-      for (int c = 0; c < 8; ++c) sm_o[warp][h][cl + c] = acc[h][c];
-      if (lane == 0) { sm_ml[warp][h][0] = m[h]; sm_ml[warp][h][1] = l[h]; }
-    }
+    for (int c = 0; c < 4; ++c) sm_o[warp][g + 8 * (c >> 1)][pv_channel<DH>(nt, 2 * t + (c & 1))] = o[nt][c];
+  if (t == 0) {
+#pragma unroll
+    for (int hi = 0; hi < 2; ++hi) { sm_ml[warp][g + 8 * hi][0] = m_row[hi]; sm_ml[warp][g + 8 * hi][1] = l_row[hi]; }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < GQ * DH; i += DA_WARPS * 32) {
+  for (int i = threadIdx.x; i < nh * DH; i += DA_WARPS * 32) {
     const int h = i / DH, c = i % DH;
-    if (gq0 + h >= d.g) continue;
     float mn = -INFINITY;
 #pragma unroll
     for (int w = 0; w < DA_WARPS; ++w) mn = fmaxf(mn, sm_ml[w][h][0]);
@@ -437,7 +492,7 @@ __global__ void __launch_bounds__(DA_WARPS * 32) decode_attn_kernel(AtArgs a) {
       lo += sm_ml[w][h][1] * al;
       oo += sm_o[w][h][c] * al;
     }
-    const int hi = j * d.g + gq0 + h;
+    const int hi = j * d.g + h0 + h;
     const size_t pidx = ((size_t)b * d.hq + hi) * a.splits + split;
     a.part_o[pidx * DH + c] = oo;
     if (c == 0) { a.part_ml[pidx * 2] = mn; a.part_ml[pidx * 2 + 1] = lo; }
@@ -487,30 +542,22 @@ cudaError_t launch_proj(ProjArgs& a, cudaStream_t st) {
 template <int DH>
 cudaError_t launch_attn_dh(const AtArgs& a, cudaStream_t st) {
   const CcaDims& d = a.d;
-  if (d.g >= 4) {
-    dim3 grid((unsigned)a.splits, (unsigned)(d.hk * ((d.g + 3) / 4)), (unsigned)d.B);
-    decode_attn_kernel<DH, 4><<<grid, DA_WARPS * 32, 0, st>>>(a);
-  } else if (d.g >= 2) {
-    dim3 grid((unsigned)a.splits, (unsigned)(d.hk * ((d.g + 1) / 2)), (unsigned)d.B);
-    decode_attn_kernel<DH, 2><<<grid, DA_WARPS * 32, 0, st>>>(a);
-  } else {
-    dim3 grid((unsigned)a.splits, (unsigned)d.hk, (unsigned)d.B);
-    decode_attn_kernel<DH, 1><<<grid, DA_WARPS * 32, 0, st>>>(a);
-  }
+  dim3 grid((unsigned)a.splits, (unsigned)(d.hk * ((d.g + 15) / 16)), (unsigned)d.B);
+  decode_attn_kernel<DH><<<grid, DA_WARPS * 32, 0, st>>>(a);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 void decode_plan(const CcaDims& d, int max_len, int sm_count, int* chunk, int* splits) {
-  const int n_grp = d.g >= 4 ? (d.g + 3) / 4 : (d.g >= 2 ? (d.g + 1) / 2 : 1);
+  const int n_grp = (d.g + 15) / 16;
   const long long base = (long long)d.B * d.hk * n_grp;
   long long want = (4LL * sm_count + base - 1) / base;         // about four CTAs per SM
   if (want < 1) want = 1;
   if (want > 128) want = 128;
   int ch = (int)((max_len + want - 1) / want);
-  ch = (ch + 127) / 128 * 128;                                 // a warp iteration covers up to 64 keys
-  if (ch < 128) ch = 128;
+  ch = (ch + 63) / 64 * 64;                                    // the four warps of a CTA take 16 keys each per round
+  if (ch < 64) ch = 64;
   *chunk = ch;
   *splits = (max_len + ch - 1) / ch;
 }
