@@ -300,32 +300,32 @@ CCA_DEVINL uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Channel of the cached row that output column n (0..7) of PV tile nt holds: thread (g, .) of a warp loads, of
-// every value row, the 16-byte pieces that start at channel 8 g (and 64 + 8 g when d_h = 128), or the 8-byte
-// piece at 4 g when d_h = 32, so that a warp's load covers whole rows; tile nt takes the nt-th of those channels.
+// Channel that the ci-th value-row element of lane group g is: a lane loads, of every value row, the 16-byte
+// pieces that start at channel 8 g (and 64 + 8 g when d_h = 128), or the 8-byte piece at 4 g when d_h = 32, so
+// that a warp's load covers whole rows.
 template <int DH>
-CCA_DEVINL int pv_channel(int nt, int n) {
-  if (DH == 32) return n * 4 + nt;
-  return (nt >> 3) * 64 + n * 8 + (nt & 7);
+CCA_DEVINL int pv_channel(int g, int ci) {
+  if (DH == 32) return g * 4 + ci;
+  return (ci >> 3) * 64 + g * 8 + (ci & 7);
 }
 
-// One CTA: keys [split * chunk, ...) of sequence b, kv head j, up to 16 of its query heads.  The two
-// contractions of a 16-key block run as m16n8k16 tensor-core instructions with the query heads as the 16 rows
-// (most of them padding): one cached row costs a few instructions instead of 4 d_h multiply-adds per head, so the
-// kernel's speed is that of its loads.  Keys and values go from global memory straight into the operand
-// registers: a contraction does not care about the order of its inner index, so each lane takes 16 contiguous
-// bytes per key (QK^T, inner index = channel) and pairs the same channel of two value rows with a byte permute
-// (P V, inner index = key).
-template <int DH>
+// One CTA: keys [split * chunk, ...) of sequence b, kv head j, up to 8 NHT of its query heads.  The two
+// contractions of a 16-key block run as m16n8k16 tensor-core instructions -- S = Q K^T with the query heads as
+// rows (padded to 16), O^T = V^T P^T with the heads as the 8 columns -- so one cached row costs a few
+// instructions instead of 4 d_h multiply-adds per head and the kernel's speed is that of its loads.  Keys and
+// values go from global memory straight into the operand registers: a contraction does not care about the order
+// of its inner index nor about how its output rows are numbered, so each lane takes 16 contiguous bytes per key
+// (Q K^T, inner index = channel) and pairs the same channel of two value rows with a byte permute (V^T P^T, inner
+// index = key, output row = whichever channel the lane loaded).
+template <int DH, int NHT>
 __global__ void __launch_bounds__(DA_WARPS * 32) decode_attn_kernel(AtArgs a) {
-  constexpr int NT = DH / 8;                   // output tiles of P V = channels per lane per value row
   constexpr int CB = DH / 32;                  // 32-channel blocks of Q K^T
-  constexpr int VW = NT / 2;                   // 32-bit words per lane per value row
+  constexpr int VW = DH / 16;                  // 32-bit words per lane per value row = 16-channel tiles of O^T
   const CcaDims& d = a.d;
   const int split = blockIdx.x, b = blockIdx.z;
-  const int n_grp = (d.g + 15) / 16;
-  const int j = blockIdx.y / n_grp, h0 = (blockIdx.y % n_grp) * 16;
-  const int nh = min(16, d.g - h0);
+  const int n_grp = (d.g + 8 * NHT - 1) / (8 * NHT);
+  const int j = blockIdx.y / n_grp, h0 = (blockIdx.y % n_grp) * 8 * NHT;
+  const int nh = min(8 * NHT, d.g - h0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
   const int tpos = a.pos[b];
@@ -343,7 +343,7 @@ __global__ void __launch_bounds__(DA_WARPS * 32) decode_attn_kernel(AtArgs a) {
 #pragma unroll
       for (int hi = 0; hi < 2; ++hi) {
         float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (g + 8 * hi < nh)
+        if (hi < NHT && g + 8 * hi < nh)
           qv = *reinterpret_cast<const float4*>(a.q + (size_t)b * d.Lq + (size_t)(j * d.g + h0 + g + 8 * hi) * DH + cb * 32 +
                                                 t * 8 + mm * 4);
         qa[cb][mm][hi] = pack_bf16x2(qv.x, qv.y);
@@ -356,13 +356,18 @@ __global__ void __launch_bounds__(DA_WARPS * 32) decode_attn_kernel(AtArgs a) {
     m_fixed = sqrtf((float)DH) * __expf(a.temp[j]) * LOG2E * 1.01f;
     fixed = m_fixed <= 56.f;
   }
-  float m_row[2] = {fixed ? m_fixed : -INFINITY, fixed ? m_fixed : -INFINITY};
-  float l_row[2] = {0.f, 0.f};
-  float o[NT][4];
+  // softmax state of heads g (and g + 8): every lane of group g carries it; the sums are per-lane partials
+  float m_row[NHT], l_row[NHT];
 #pragma unroll
-  for (int nt = 0; nt < NT; ++nt)
+  for (int hi = 0; hi < NHT; ++hi) { m_row[hi] = fixed ? m_fixed : -INFINITY; l_row[hi] = 0.f; }
+  // O^T tiles: o[hi][mt] = {(channel slot g, head 2t), (g, 2t+1), (g + 8, 2t), (g + 8, 2t+1)} of heads 8 hi + ...
+  float o[NHT][VW][4];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) o[nt][c] = 0.f;
+  for (int hi = 0; hi < NHT; ++hi)
+#pragma unroll
+    for (int mt = 0; mt < VW; ++mt)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) o[hi][mt][c] = 0.f;
 
   const bf16* kb = a.k_cache + (size_t)b * a.S_max * d.Lk + j * DH;
   const bf16* vb = a.v_cache + (size_t)b * a.S_max * d.Lk + j * DH;
@@ -398,7 +403,7 @@ __global__ void __launch_bounds__(DA_WARPS * 32) decode_attn_kernel(AtArgs a) {
         }
       }
     }
-    // ---- S = Q K^T for the two 8-key tiles
+    // ---- S = Q K^T for the two 8-key tiles: thread (g, t) gets heads g, g + 8 x keys 2t, 2t+1 of each tile
     float sc[2][4];
 #pragma unroll
     for (int ti = 0; ti < 2; ++ti) {
@@ -410,74 +415,85 @@ __global__ void __launch_bounds__(DA_WARPS * 32) decode_attn_kernel(AtArgs a) {
         mma_16816(sc[ti], qa[cb][1], kf[ti][cb].z, kf[ti][cb].w);
       }
     }
-    // ---- softmax weights of this block; thread (g, t) holds rows g, g + 8 and keys 2t, 2t+1 of each tile
 #pragma unroll
     for (int ti = 0; ti < 2; ++ti)
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2 * NHT; ++c) {
         const int key = k0 + ti * 8 + 2 * t + (c & 1);
         sc[ti][c] = key < k_end ? sc[ti][c] * c_scale : -INFINITY;
       }
     if (!fixed) {
-      float mx[2];
+      float mx[NHT];
+      bool grow = false;
 #pragma unroll
-      for (int hi = 0; hi < 2; ++hi) {
+      for (int hi = 0; hi < NHT; ++hi) {
         mx[hi] = fmaxf(fmaxf(sc[0][2 * hi], sc[0][2 * hi + 1]), fmaxf(sc[1][2 * hi], sc[1][2 * hi + 1]));
         mx[hi] = fmaxf(mx[hi], __shfl_xor_sync(0xffffffffu, mx[hi], 1));
         mx[hi] = fmaxf(mx[hi], __shfl_xor_sync(0xffffffffu, mx[hi], 2));
+        grow = grow || mx[hi] > m_row[hi];
       }
-      const bool grow = mx[0] > m_row[0] || mx[1] > m_row[1];
       if (__any_sync(0xffffffffu, grow)) {
 #pragma unroll
-        for (int hi = 0; hi < 2; ++hi) {
+        for (int hi = 0; hi < NHT; ++hi) {
+          float alpha = 1.f;
           if (mx[hi] > m_row[hi]) {
-            const float alpha = exp2f(m_row[hi] - mx[hi]);     // 0 while nothing has been seen (m = -inf)
+            alpha = exp2f(m_row[hi] - mx[hi]);                 // 0 while nothing has been seen (m = -inf)
             l_row[hi] *= alpha;
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) { o[nt][2 * hi] *= alpha; o[nt][2 * hi + 1] *= alpha; }
             m_row[hi] = mx[hi];
+          }
+          // the O^T columns of this lane are heads 2t, 2t+1, whose factors live in lane groups 2t, 2t+1
+          const float a0 = __shfl_sync(0xffffffffu, alpha, (2 * t) * 4);
+          const float a1 = __shfl_sync(0xffffffffu, alpha, (2 * t + 1) * 4);
+#pragma unroll
+          for (int mt = 0; mt < VW; ++mt) {
+            o[hi][mt][0] *= a0; o[hi][mt][1] *= a1; o[hi][mt][2] *= a0; o[hi][mt][3] *= a1;
           }
         }
       }
     }
-    uint32_t pa[4];
+    uint32_t pb[NHT][2];                       // P^T operand: keys 2t, 2t+1 (tile 0) and 2t+8, 2t+9 (tile 1) of head g (+ 8)
 #pragma unroll
     for (int ti = 0; ti < 2; ++ti)
 #pragma unroll
-      for (int hi = 0; hi < 2; ++hi) {
+      for (int hi = 0; hi < NHT; ++hi) {
         const float mu = m_row[hi] == -INFINITY ? 0.f : m_row[hi];
         const float p0 = exp2f(sc[ti][2 * hi] - mu), p1 = exp2f(sc[ti][2 * hi + 1] - mu);
         const uint32_t w = pack_bf16x2(p0, p1);
-        pa[2 * ti + hi] = w;
-        // the sum runs over the rounded weights, the ones P V uses
+        pb[hi][ti] = w;
+        // the sum runs over the rounded weights, the ones the second contraction uses
         l_row[hi] += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
       }
-    // ---- O += P V
+    // ---- O^T += V^T P^T
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const int w = nt >> 1;
-      const uint32_t sel = (nt & 1) ? 0x7632u : 0x5410u;
-      const uint32_t b0 = __byte_perm(vf[0][w], vf[1][w], sel);
-      const uint32_t b1 = __byte_perm(vf[2][w], vf[3][w], sel);
-      mma_16816(o[nt], pa, b0, b1);
+    for (int mt = 0; mt < VW; ++mt) {
+      uint32_t va[4];
+      va[0] = __byte_perm(vf[0][mt], vf[1][mt], 0x5410u);
+      va[1] = __byte_perm(vf[0][mt], vf[1][mt], 0x7632u);
+      va[2] = __byte_perm(vf[2][mt], vf[3][mt], 0x5410u);
+      va[3] = __byte_perm(vf[2][mt], vf[3][mt], 0x7632u);
+#pragma unroll
+      for (int hi = 0; hi < NHT; ++hi) mma_16816(o[hi][mt], va, pb[hi][0], pb[hi][1]);
     }
   }
   // row sums: the four lanes of a group hold different keys
 #pragma unroll
-  for (int hi = 0; hi < 2; ++hi) {
+  for (int hi = 0; hi < NHT; ++hi) {
     l_row[hi] += __shfl_xor_sync(0xffffffffu, l_row[hi], 1);
     l_row[hi] += __shfl_xor_sync(0xffffffffu, l_row[hi], 2);
   }
   // merge the warps through shared memory
-  __shared__ float sm_o[DA_WARPS][16][DH];
-  __shared__ float sm_ml[DA_WARPS][16][2];
+  __shared__ float sm_o[DA_WARPS][8 * NHT][DH + 1];
+  __shared__ float sm_ml[DA_WARPS][8 * NHT][2];
 #pragma unroll
-  for (int nt = 0; nt < NT; ++nt)
+  for (int hi = 0; hi < NHT; ++hi)
 #pragma unroll
-    for (int c = 0; c < 4; ++c) sm_o[warp][g + 8 * (c >> 1)][pv_channel<DH>(nt, 2 * t + (c & 1))] = o[nt][c];
+    for (int mt = 0; mt < VW; ++mt)
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        sm_o[warp][8 * hi + 2 * t + (c & 1)][pv_channel<DH>(g, 2 * mt + (c >> 1))] = o[hi][mt][c];
   if (t == 0) {
 #pragma unroll
-    for (int hi = 0; hi < 2; ++hi) { sm_ml[warp][g + 8 * hi][0] = m_row[hi]; sm_ml[warp][g + 8 * hi][1] = l_row[hi]; }
+    for (int hi = 0; hi < NHT; ++hi) { sm_ml[warp][g + 8 * hi][0] = m_row[hi]; sm_ml[warp][g + 8 * hi][1] = l_row[hi]; }
   }
   __syncthreads();
   for (int i = threadIdx.x; i < nh * DH; i += DA_WARPS * 32) {
@@ -542,15 +558,20 @@ cudaError_t launch_proj(ProjArgs& a, cudaStream_t st) {
 template <int DH>
 cudaError_t launch_attn_dh(const AtArgs& a, cudaStream_t st) {
   const CcaDims& d = a.d;
-  dim3 grid((unsigned)a.splits, (unsigned)(d.hk * ((d.g + 15) / 16)), (unsigned)d.B);
-  decode_attn_kernel<DH><<<grid, DA_WARPS * 32, 0, st>>>(a);
+  if (d.g <= 8) {
+    dim3 grid((unsigned)a.splits, (unsigned)d.hk, (unsigned)d.B);
+    decode_attn_kernel<DH, 1><<<grid, DA_WARPS * 32, 0, st>>>(a);
+  } else {
+    dim3 grid((unsigned)a.splits, (unsigned)(d.hk * ((d.g + 15) / 16)), (unsigned)d.B);
+    decode_attn_kernel<DH, 2><<<grid, DA_WARPS * 32, 0, st>>>(a);
+  }
   return cudaGetLastError();
 }
 
 }  // namespace
 
 void decode_plan(const CcaDims& d, int max_len, int sm_count, int* chunk, int* splits) {
-  const int n_grp = (d.g + 15) / 16;
+  const int n_grp = d.g <= 8 ? 1 : (d.g + 15) / 16;
   const long long base = (long long)d.B * d.hk * n_grp;
   long long want = (4LL * sm_count + base - 1) / base;         // about four CTAs per SM
   if (want < 1) want = 1;

@@ -27,6 +27,8 @@ EMPTY_START = [
     S_("dec_mha_g1", 2, 17, 256, 4, 4, 64, flags=0),
     S_("dec_g2", 2, 17, 512, 4, 2, 64),
     S_("dec_g8", 1, 19, 512, 8, 1, 64),
+    S_("dec_g16", 1, 37, 1024, 16, 1, 64),
+    S_("dec_g12_dh128", 2, 21, 1536, 12, 1, 128, flags=63 & ~16),
     S_("dec_k3_k4", 2, 15, 512, 8, 2, 64, k_seq=3, k_ch=4),
     S_("dec_k1_k1", 2, 9, 512, 8, 2, 64, k_seq=1, k_ch=1),
     S_("dec_no_shift", 2, 9, 512, 8, 2, 64, flags=63 & ~8),
