@@ -5,12 +5,15 @@
 // keep its instruction count below what the loads need):
 //
 //   decode_proj_kernel      out[b, n] = sum_k W[n, k] x[b, k] for a few stacked weight segments (Eq. 7, 10; Eq. 11
-//                           up-projection): one warp per two weight rows, 16 sequences per CTA staged in shared memory
-//   decode_transform_kernel Eq. 8-11 for the new token of one (sequence, head): conv halo from the caller's history,
-//                           q-k-mean, norm, temperature, RoPE at the sequence's own position; appends k, v to the cache
+//                           up-projection; also conv2 of Eq. 8, a contraction over (input channel, tap) per head)
+//   decode_conv1_kernel     Eq. 8 conv1 at the tokens conv2 reads, from the caller's history; appends v to the cache,
+//                           advances the history and the previous input
+//   decode_finalize_kernel  Eq. 9, 11 for the new token of one (sequence, head): q-k-mean, norm, temperature, RoPE at
+//                           the sequence's own position; appends k to the cache
 //   decode_attn_kernel      softmax(q k^T / sqrt(d_h)) v of the new query over a chunk of the cached keys of one
 //                           (sequence, kv head), all its query heads at once; partial results per chunk
 //   decode_combine_kernel   merges the chunks' partial results
+#include <cstdlib>
 #include <cstring>
 
 #include "common.cuh"
@@ -22,117 +25,122 @@ constexpr unsigned F_CONV1 = 1, F_CONV2 = 2, F_QK_MEAN = 4, F_V_SHIFT = 8, F_QK_
 constexpr int ST_DECODE_BAD_POSITION = 120;
 constexpr float LOG2E = 1.4426950408889634f;
 
-CCA_DEVINL void unpack8(const uint4& u, float* f) {
-  f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
-  f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
-  f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xffff0000u);
-  f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xffff0000u);
+CCA_DEVINL void mma_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+CCA_DEVINL uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
 }
 
 // ------------------------------------------------------------------------------------------------ projections
-constexpr int PJ_BT = 16;          // sequences per CTA
-constexpr int PJ_KC = 1024;        // k-chunk staged in shared memory
-constexpr int PJ_WARPS = 4, PJ_RPW = 2, PJ_ROWS = PJ_WARPS * PJ_RPW;
+// out[b, n] = sum_k W[n, k] x[b, k]: 16 weight rows per CTA as the rows of m16n8k16 tiles, 32 sequences as four
+// column tiles, the inner dimension split over the 8 warps and summed through shared memory.  A lane loads 16
+// contiguous bytes of a weight row and of an input row and feeds them to two tensor-core instructions (the inner
+// index may be taken in any order as long as both operands agree), so every load is a full 64-byte piece of a row.
+constexpr int PJ_WARPS = 8, PJ_ROWS = 16, PJ_NT = 4, PJ_UNR = 4;
 
 struct ProjSeg {
   const bf16* W;     // [rows, K] row-major
-  const bf16* X;     // [B, K] row-major
+  const bf16* X;     // [B, ldx] row-major
   int rows;
   int out_off;       // first output column of this segment
 };
 struct ProjArgs {
   ProjSeg seg[3];
-  int n_seg, rows_total, K, B;
+  int n_seg, K, B;
+  int ldx;           // row stride of X in elements
+  int x_head_rows;   // > 0: every x_head_rows rows form a head, and head h reads X at column offset h * K
   float* out_f32;    // [B, ldo] (one of the two)
   bf16* out_bf16;
   int ldo;
 };
 
 __global__ void __launch_bounds__(PJ_WARPS * 32) decode_proj_kernel(ProjArgs a) {
-  __shared__ __align__(16) bf16 xs[PJ_BT][PJ_KC];
+  __shared__ float red[PJ_WARPS][PJ_ROWS][PJ_NT * 8 + 1];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b0 = blockIdx.y * PJ_BT;
+  const int g = lane >> 2, t = lane & 3;
+  const int b0 = blockIdx.y * (PJ_NT * 8);
   const int row0 = blockIdx.x * PJ_ROWS;          // first row of this CTA in the stacked row space
   // segments start on multiples of PJ_ROWS in the stacked space (the host pads), so a CTA stays inside one
-  int sidx = 0, base = 0;
-  for (int s = 0; s < a.n_seg; ++s) {
-    const int padded = (a.seg[s].rows + PJ_ROWS - 1) / PJ_ROWS * PJ_ROWS;
-    if (row0 >= base && row0 < base + padded) { sidx = s; break; }
-    base += padded;
+  int base = 0;
+  ProjSeg sg = a.seg[0];
+  if (a.n_seg > 1) {
+    const int p0 = (a.seg[0].rows + PJ_ROWS - 1) / PJ_ROWS * PJ_ROWS;
+    const int p1 = (a.seg[1].rows + PJ_ROWS - 1) / PJ_ROWS * PJ_ROWS;
+    if (row0 >= p0 + p1 && a.n_seg > 2) { sg = a.seg[2]; base = p0 + p1; }
+    else if (row0 >= p0) { sg = a.seg[1]; base = p0; }
   }
-  const ProjSeg sg = a.seg[sidx];
-  const int r_first = row0 - base + warp * PJ_RPW;
-  float acc[PJ_RPW][PJ_BT];
+  const int r_lo = row0 - base + g, r_hi = r_lo + 8;
+  const bool ok_lo = r_lo < sg.rows, ok_hi = r_hi < sg.rows;
+  const bf16* w_lo = sg.W + (size_t)r_lo * a.K + t * 8;
+  const bf16* w_hi = sg.W + (size_t)r_hi * a.K + t * 8;
+  const bf16* xb = sg.X + (a.x_head_rows > 0 ? (size_t)((row0 - base) / a.x_head_rows) * a.K : 0) + t * 8;
+  float acc[PJ_NT][4];
 #pragma unroll
-  for (int r = 0; r < PJ_RPW; ++r)
+  for (int nt = 0; nt < PJ_NT; ++nt)
 #pragma unroll
-    for (int b = 0; b < PJ_BT; ++b) acc[r][b] = 0.f;
-
-  for (int k0 = 0; k0 < a.K; k0 += PJ_KC) {
-    __syncthreads();
-    for (int i = threadIdx.x; i < PJ_BT * (PJ_KC / 8); i += PJ_WARPS * 32) {
-      const int b = i / (PJ_KC / 8), kv = (i % (PJ_KC / 8)) * 8;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (b0 + b < a.B && k0 + kv < a.K) v = *reinterpret_cast<const uint4*>(sg.X + (size_t)(b0 + b) * a.K + k0 + kv);
-      *reinterpret_cast<uint4*>(&xs[b][kv]) = v;
-    }
-    __syncthreads();
+    for (int c = 0; c < 4; ++c) acc[nt][c] = 0.f;
+  const int nkb = a.K / 32;
+  for (int kb0 = warp; kb0 < nkb; kb0 += PJ_WARPS * PJ_UNR) {
+    uint4 wl[PJ_UNR], wh[PJ_UNR], xf[PJ_UNR][PJ_NT];
 #pragma unroll
-    for (int i = 0; i < PJ_KC / 256; ++i) {
-      const int kv = i * 256 + lane * 8;
-      float w[PJ_RPW][8];
-#pragma unroll
-      for (int r = 0; r < PJ_RPW; ++r) {
-        uint4 u = make_uint4(0, 0, 0, 0);
-        if (r_first + r < sg.rows && k0 + kv < a.K)
-          u = __ldg(reinterpret_cast<const uint4*>(sg.W + (size_t)(r_first + r) * a.K + k0 + kv));
-        unpack8(u, w[r]);
+    for (int u = 0; u < PJ_UNR; ++u) {
+      const int kb = kb0 + u * PJ_WARPS;
+      wl[u] = wh[u] = make_uint4(0, 0, 0, 0);
+      if (kb < nkb) {
+        if (ok_lo) wl[u] = __ldcs(reinterpret_cast<const uint4*>(w_lo + kb * 32));
+        if (ok_hi) wh[u] = __ldcs(reinterpret_cast<const uint4*>(w_hi + kb * 32));
       }
 #pragma unroll
-      for (int b = 0; b < PJ_BT; ++b) {
-        float x[8];
-        unpack8(*reinterpret_cast<const uint4*>(&xs[b][kv]), x);
+      for (int nt = 0; nt < PJ_NT; ++nt) {
+        const int seq = b0 + nt * 8 + g;
+        xf[u][nt] = make_uint4(0, 0, 0, 0);
+        if (kb < nkb && seq < a.B) xf[u][nt] = __ldg(reinterpret_cast<const uint4*>(xb + (size_t)seq * a.ldx + kb * 32));
+      }
+    }
 #pragma unroll
-        for (int r = 0; r < PJ_RPW; ++r)
+    for (int u = 0; u < PJ_UNR; ++u) {
+      const uint32_t a1[4] = {wl[u].x, wh[u].x, wl[u].y, wh[u].y};
+      const uint32_t a2[4] = {wl[u].z, wh[u].z, wl[u].w, wh[u].w};
 #pragma unroll
-          for (int c = 0; c < 8; ++c) acc[r][b] = fmaf(w[r][c], x[c], acc[r][b]);
+      for (int nt = 0; nt < PJ_NT; ++nt) {
+        mma_16816(acc[nt], a1, xf[u][nt].x, xf[u][nt].y);
+        mma_16816(acc[nt], a2, xf[u][nt].z, xf[u][nt].w);
       }
     }
   }
 #pragma unroll
-  for (int r = 0; r < PJ_RPW; ++r)
+  for (int nt = 0; nt < PJ_NT; ++nt)
 #pragma unroll
-    for (int b = 0; b < PJ_BT; ++b) {
-      float v = acc[r][b];
+    for (int c = 0; c < 4; ++c) red[warp][g + 8 * (c >> 1)][nt * 8 + 2 * t + (c & 1)] = acc[nt][c];
+  __syncthreads();
+  for (int i = threadIdx.x; i < PJ_ROWS * PJ_NT * 8; i += PJ_WARPS * 32) {
+    const int row = i % PJ_ROWS, seq = i / PJ_ROWS;
+    float v = 0.f;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      acc[r][b] = v;
-    }
-  // lane b of the warp stores sequence b
-#pragma unroll
-  for (int r = 0; r < PJ_RPW; ++r) {
-    float mine = 0.f;
-#pragma unroll
-    for (int b = 0; b < PJ_BT; ++b)
-      if (lane == b) mine = acc[r][b];
-    if (lane < PJ_BT && b0 + lane < a.B && r_first + r < sg.rows) {
-      const size_t o = (size_t)(b0 + lane) * a.ldo + sg.out_off + r_first + r;
-      if (a.out_f32) a.out_f32[o] = mine;
-      else a.out_bf16[o] = __float2bfloat16(mine);
+    for (int w = 0; w < PJ_WARPS; ++w) v += red[w][row][seq];
+    const int r = row0 - base + row;
+    if (r < sg.rows && b0 + seq < a.B) {
+      const size_t o = (size_t)(b0 + seq) * a.ldo + sg.out_off + r;
+      if (a.out_f32) a.out_f32[o] = v;
+      else a.out_bf16[o] = __float2bfloat16(v);
     }
   }
 }
 
 // ------------------------------------------------------------------------------------------------ transforms
-struct TrArgs {
+// Eq. 8, conv1 at the k_ch tokens conv2 reads, for every channel of one sequence; also the value row (Eq. 10),
+// the history for the next token and the input the next step's value shift needs.
+struct C1Args {
   CcaDims d;
   const float* lat;      // [B, L + Lk]: q0 | k0 | v1 | v2 of the new token
   const bf16* x;         // [B, E] new token
   const bf16* w0;        // [L, k_seq]
-  const bf16* w1;        // [L, d_h, k_ch]
-  const float* temp;
-  float* q;              // [B, Lq] out
-  bf16* k_cache;         // [B, S_max, Lk]
+  bf16* y1s;             // [B, L * kc]: conv1 output of channel c at tap r in element c * kc + r (conv2 on)
+  float* y2;             // [B, L]: written here instead when conv2 is off
   bf16* v_cache;
   float* hist;           // [B, pad, L]
   bf16* x_prev;          // [B, E]
@@ -142,103 +150,91 @@ struct TrArgs {
   int* status;
 };
 
+__global__ void __launch_bounds__(256) decode_conv1_kernel(C1Args a) {
+  const CcaDims& d = a.d;
+  const int b = blockIdx.y, tid = threadIdx.x;
+  const int t = a.pos[b];
+  if (t < 0 || t >= a.S_max || t >= a.max_len) {
+    if (tid == 0 && blockIdx.x == 0) atomicCAS(a.status, 0, ST_DECODE_BAD_POSITION);
+    return;
+  }
+  const int ld_lat = d.L + d.Lk;
+  const int pad = d.k_seq + d.k_ch - 2;
+  const int ks = (d.flags & F_CONV1) ? d.k_seq : 1;
+  const int kc = (d.flags & F_CONV2) ? d.k_ch : 1;
+  const float* lat_b = a.lat + (size_t)b * ld_lat;
+  for (int ch = blockIdx.x * 256 + tid; ch < d.L; ch += gridDim.x * 256) {
+    float win[8];                                  // tokens t - pad .. t of this channel (pad + 1 <= 7)
+#pragma unroll
+    for (int r = 0; r < 8; ++r) win[r] = 0.f;
+#pragma unroll
+    for (int r = 0; r < 7; ++r)
+      if (r < pad) win[r] = a.hist[((size_t)b * pad + r) * d.L + ch];
+    win[pad] = lat_b[ch];
+    for (int r = 0; r < kc; ++r) {
+      const int row = pad - (kc - 1) + r;
+      float acc;
+      if (d.flags & F_CONV1) {
+        acc = 0.f;
+        for (int j = 0; j < ks; ++j) acc = fmaf(__bfloat162float(a.w0[(size_t)ch * d.k_seq + j]), win[row - (ks - 1) + j], acc);
+      } else {
+        acc = win[row];
+      }
+      if (d.flags & F_CONV2) a.y1s[((size_t)b * d.L + ch) * kc + r] = __float2bfloat16(acc);
+      else a.y2[(size_t)b * d.L + ch] = acc;
+    }
+#pragma unroll
+    for (int r = 0; r < 7; ++r)
+      if (r < pad) a.hist[((size_t)b * pad + r) * d.L + ch] = win[r + 1];
+  }
+  for (int c = blockIdx.x * 256 + tid; c < d.Lk; c += gridDim.x * 256)
+    a.v_cache[((size_t)b * a.S_max + t) * d.Lk + c] = __float2bfloat16(lat_b[d.L + c]);
+  for (int c = blockIdx.x * 256 + tid; c < d.E / 8; c += gridDim.x * 256)
+    reinterpret_cast<uint4*>(a.x_prev + (size_t)b * d.E)[c] = reinterpret_cast<const uint4*>(a.x + (size_t)b * d.E)[c];
+}
+
+// Eq. 9 (q-k-mean) and Eq. 11 (norm, temperature, RoPE at the sequence's own position) for one (sequence, head);
+// the query goes to the workspace, the key into the cache.
+struct FnArgs {
+  CcaDims d;
+  const float* lat;
+  const float* y2;       // [B, L]: conv output of the new token
+  const float* temp;
+  float* q;              // [B, Lq]
+  bf16* k_cache;
+  const int* pos;
+  long long S_max;
+  int max_len;
+};
+
 template <int DH>
-__global__ void __launch_bounds__(128) decode_transform_kernel(TrArgs a) {
-  constexpr int MAXW = 8;                      // window rows: pad + 1 <= 8 (k_seq, k_ch <= 4 each)
-  __shared__ float win[MAXW][DH];
-  __shared__ float y1[4][DH];
+__global__ void __launch_bounds__(128) decode_finalize_kernel(FnArgs a) {
   __shared__ float xh[DH];
   __shared__ float red[4];
   const CcaDims& d = a.d;
   const int b = blockIdx.y, head = blockIdx.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int t = a.pos[b];
-  if (t < 0 || t >= a.S_max || t >= a.max_len) {
-    if (tid == 0) atomicCAS(a.status, 0, ST_DECODE_BAD_POSITION);
-    return;
-  }
-  const int ld_lat = d.L + d.Lk;
-  if (head == d.hq + d.hk) {
-    // value row of the new token (Eq. 10; the projection already took x_{t-1} for the second half) and the
-    // input the next step's value shift needs
-    for (int c = tid; c < d.Lk; c += 128)
-      a.v_cache[((size_t)b * a.S_max + t) * d.Lk + c] = __float2bfloat16(a.lat[(size_t)b * ld_lat + d.L + c]);
-    for (int c = tid; c < d.E / 8; c += 128)
-      reinterpret_cast<uint4*>(a.x_prev + (size_t)b * d.E)[c] = reinterpret_cast<const uint4*>(a.x + (size_t)b * d.E)[c];
-    return;
-  }
+  if (t < 0 || t >= a.S_max || t >= a.max_len) return;      // reported by the conv1 kernel
   const bool is_q = head < d.hq;
   const int ch0 = head * DH;                   // first channel of the head in the q0|k0 latent
-  const int pad = d.k_seq + d.k_ch - 2;
-  const int ks = (d.flags & F_CONV1) ? d.k_seq : 1;
-  const int kc = (d.flags & F_CONV2) ? d.k_ch : 1;
-  const float* lat_b = a.lat + (size_t)b * ld_lat;
-  for (int i = tid; i < (pad + 1) * DH; i += 128) {
-    const int r = i / DH, c = i % DH;
-    win[r][c] = r < pad ? a.hist[((size_t)b * pad + r) * d.L + ch0 + c] : lat_b[ch0 + c];
-  }
-  __syncthreads();
-  // Eq. 8, conv1 at the kc tokens conv2 reads
-  for (int i = tid; i < kc * DH; i += 128) {
-    const int r = i / DH, c = i % DH;
-    const int row = pad - (kc - 1) + r;
-    float acc;
-    if (d.flags & F_CONV1) {
-      acc = 0.f;
-      for (int j = 0; j < ks; ++j)
-        acc = fmaf(__bfloat162float(a.w0[(size_t)(ch0 + c) * d.k_seq + j]), win[row - (ks - 1) + j][c], acc);
-    } else {
-      acc = win[row][c];
-    }
-    y1[r][c] = acc;
-  }
-  __syncthreads();
-  // Eq. 8, conv2 at the new token: one warp per output channel, lanes over (input channel, tap)
-  if (d.flags & F_CONV2) {
-    for (int o = warp; o < DH; o += 4) {
-      const bf16* wr = a.w1 + (size_t)(ch0 + o) * DH * d.k_ch;
-      float acc = 0.f;
-      for (int idx = lane; idx < DH * d.k_ch; idx += 32) {
-        const int i = idx / d.k_ch, r = idx % d.k_ch;
-        acc = fmaf(__bfloat162float(wr[idx]), y1[r][i], acc);
+  const float* lat_b = a.lat + (size_t)b * (d.L + d.Lk);
+  float v = 0.f, ssq = 0.f;
+  const int c = tid;
+  if (c < DH) {
+    v = a.y2[(size_t)b * d.L + ch0 + c];
+    if (d.flags & F_QK_MEAN) {
+      if (is_q) {
+        const int j = head / d.g;
+        v += 0.5f * (lat_b[ch0 + c] + lat_b[d.Lq + j * DH + c]);
+      } else {
+        const int j = head - d.hq;
+        float sq = 0.f;
+        for (int i = 0; i < d.g; ++i) sq += lat_b[(j * d.g + i) * DH + c];
+        v += 0.5f * lat_b[ch0 + c] + 0.5f * sq / (float)d.g;
       }
-#pragma unroll
-      for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-      if (lane == 0) xh[o] = acc;
     }
-  } else {
-    for (int c = tid; c < DH; c += 128) xh[c] = y1[kc - 1][c];
-  }
-  __syncthreads();
-  // history for the next token: drop the oldest row, append this token's q0|k0 (every read of the old rows is done)
-  for (int i = tid; i < pad * DH; i += 128) {
-    const int r = i / DH, c = i % DH;
-    a.hist[((size_t)b * pad + r) * d.L + ch0 + c] = win[r + 1][c];
-  }
-  // Eq. 9 (q-k-mean), Eq. 11 (norm, temperature, RoPE)
-  float val[DH / 128 > 0 ? DH / 128 : 1];
-  float ssq = 0.f;
-  constexpr int PER = DH >= 128 ? DH / 128 : 1;
-#pragma unroll
-  for (int u = 0; u < PER; ++u) {
-    const int c = tid + u * 128;
-    float v = 0.f;
-    if (c < DH) {
-      v = xh[c];
-      if (d.flags & F_QK_MEAN) {
-        if (is_q) {
-          const int j = head / d.g;
-          v += 0.5f * (lat_b[ch0 + c] + lat_b[d.Lq + j * DH + c]);
-        } else {
-          const int j = head - d.hq;
-          float sq = 0.f;
-          for (int i = 0; i < d.g; ++i) sq += lat_b[(j * d.g + i) * DH + c];
-          v += 0.5f * lat_b[ch0 + c] + 0.5f * sq / (float)d.g;
-        }
-      }
-      ssq = fmaf(v, v, ssq);
-    }
-    val[u] = v;
+    ssq = v * v;
   }
   if (d.flags & F_QK_NORM) {
 #pragma unroll
@@ -248,29 +244,20 @@ __global__ void __launch_bounds__(128) decode_transform_kernel(TrArgs a) {
     const float tot = red[0] + red[1] + red[2] + red[3];
     float sc = sqrtf((float)DH) * rsqrtf(tot);
     if (!is_q) sc *= __expf(a.temp[head - d.hq]);
-#pragma unroll
-    for (int u = 0; u < PER; ++u) val[u] *= sc;
+    v *= sc;
   }
+  if (c < DH) xh[c] = v;
   __syncthreads();
-#pragma unroll
-  for (int u = 0; u < PER; ++u)
-    if (tid + u * 128 < DH) xh[tid + u * 128] = val[u];
-  __syncthreads();
-#pragma unroll
-  for (int u = 0; u < PER; ++u) {
-    const int c = tid + u * 128;
-    if (c >= DH) continue;
-    float v = xh[c];
-    if (d.flags & F_ROPE) {
-      const int cc = c % (DH / 2);
-      const double theta = exp2(-2.0 * (double)cc / (double)DH * log2((double)d.rope_base));
-      double sn, cs;
-      sincos((double)t * theta, &sn, &cs);
-      v = c < DH / 2 ? xh[c] * (float)cs - xh[c + DH / 2] * (float)sn : xh[c] * (float)cs + xh[c - DH / 2] * (float)sn;
-    }
-    if (is_q) a.q[(size_t)b * d.Lq + ch0 + c] = v;
-    else a.k_cache[((size_t)b * a.S_max + t) * d.Lk + (ch0 - d.Lq) + c] = __float2bfloat16(v);
+  if (c >= DH) return;
+  if (d.flags & F_ROPE) {
+    const int cc = c % (DH / 2);
+    const double theta = exp2(-2.0 * (double)cc / (double)DH * log2((double)d.rope_base));
+    double sn, cs;
+    sincos((double)t * theta, &sn, &cs);
+    v = c < DH / 2 ? xh[c] * (float)cs - xh[c + DH / 2] * (float)sn : xh[c] * (float)cs + xh[c - DH / 2] * (float)sn;
   }
+  if (is_q) a.q[(size_t)b * d.Lq + ch0 + c] = v;
+  else a.k_cache[((size_t)b * a.S_max + t) * d.Lk + (ch0 - d.Lq) + c] = __float2bfloat16(v);
 }
 
 // ------------------------------------------------------------------------------------------------ attention
@@ -289,16 +276,6 @@ struct AtArgs {
 };
 
 constexpr int DA_WARPS = 4;
-
-CCA_DEVINL void mma_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-CCA_DEVINL uint32_t pack_bf16x2(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
 
 // Channel that the ci-th value-row element of lane group g is: a lane loads, of every value row, the 16-byte
 // pieces that start at channel 8 g (and 64 + 8 g when d_h = 128), or the 8-byte piece at 4 g when d_h = 32, so
@@ -546,11 +523,10 @@ __global__ void __launch_bounds__(DH < 64 ? 64 : DH) decode_combine_kernel(CbArg
 
 int padded_rows(int rows) { return (rows + PJ_ROWS - 1) / PJ_ROWS * PJ_ROWS; }
 
-cudaError_t launch_proj(ProjArgs& a, cudaStream_t st) {
+cudaError_t launch_proj(const ProjArgs& a, cudaStream_t st) {
   int tot = 0;
   for (int s = 0; s < a.n_seg; ++s) tot += padded_rows(a.seg[s].rows);
-  a.rows_total = tot;
-  dim3 grid((unsigned)(tot / PJ_ROWS), (unsigned)((a.B + PJ_BT - 1) / PJ_BT));
+  dim3 grid((unsigned)(tot / PJ_ROWS), (unsigned)((a.B + PJ_NT * 8 - 1) / (PJ_NT * 8)));
   decode_proj_kernel<<<grid, PJ_WARPS * 32, 0, st>>>(a);
   return cudaGetLastError();
 }
@@ -573,7 +549,13 @@ cudaError_t launch_attn_dh(const AtArgs& a, cudaStream_t st) {
 void decode_plan(const CcaDims& d, int max_len, int sm_count, int* chunk, int* splits) {
   const int n_grp = d.g <= 8 ? 1 : (d.g + 15) / 16;
   const long long base = (long long)d.B * d.hk * n_grp;
-  long long want = (4LL * sm_count + base - 1) / base;         // about four CTAs per SM
+  static int per_sm = 0;                                       // CTAs per SM to aim for (CCA_DECODE_CTAS_PER_SM overrides)
+  if (per_sm == 0) {
+    const char* e = getenv("CCA_DECODE_CTAS_PER_SM");
+    per_sm = e ? atoi(e) : 12;
+    if (per_sm < 1 || per_sm > 64) per_sm = 12;
+  }
+  long long want = ((long long)per_sm * sm_count + base - 1) / base;
   if (want < 1) want = 1;
   if (want > 128) want = 128;
   int ch = (int)((max_len + want - 1) / want);
@@ -593,6 +575,8 @@ size_t decode_workspace_bytes(const CcaDims& d, int max_len, int sm_count) {
   n += up((size_t)d.B * d.hq * splits * d.dh * 4);     // partial o
   n += up((size_t)d.B * d.hq * splits * 2 * 4);        // partial (m, l)
   n += up((size_t)d.B * d.Lq * 2);                     // o
+  n += up((size_t)d.B * d.L * d.k_ch * 2);             // conv1 output at the taps conv2 reads
+  n += up((size_t)d.B * d.L * 4);                      // conv output
   return n;
 }
 
@@ -607,8 +591,12 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
   float* q = reinterpret_cast<float*>(p); p += up((size_t)d.B * d.Lq * 4);
   float* part_o = reinterpret_cast<float*>(p); p += up((size_t)d.B * d.hq * splits * d.dh * 4);
   float* part_ml = reinterpret_cast<float*>(p); p += up((size_t)d.B * d.hq * splits * 2 * 4);
-  bf16* o = reinterpret_cast<bf16*>(p);
+  bf16* o = reinterpret_cast<bf16*>(p); p += up((size_t)d.B * d.Lq * 2);
+  bf16* y1s = reinterpret_cast<bf16*>(p); p += up((size_t)d.B * d.L * d.k_ch * 2);
+  float* y2 = reinterpret_cast<float*>(p);
   cudaError_t e;
+  if (d.dh != 32 && d.dh != 64 && d.dh != 128) return 1;
+  if (d.E % 32 || d.Lq % 32) return 1;
   // Eq. 7 and Eq. 10: q0 | k0 | v1 from x_t, v2 from x_{t-1}
   ProjArgs pa;
   memset(&pa, 0, sizeof(pa));
@@ -616,20 +604,36 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
   pa.seg[0] = ProjSeg{w.w_qk, x, d.L, 0};
   pa.seg[1] = ProjSeg{w.w_v1, x, d.Lk / 2, d.L};
   pa.seg[2] = ProjSeg{w.w_v2, (d.flags & F_V_SHIFT) ? s.x_prev : x, d.Lk / 2, d.L + d.Lk / 2};
-  pa.K = d.E; pa.B = d.B; pa.out_f32 = lat; pa.ldo = d.L + d.Lk;
+  pa.K = d.E; pa.B = d.B; pa.ldx = d.E; pa.out_f32 = lat; pa.ldo = d.L + d.Lk;
   if ((e = launch_proj(pa, st)) != cudaSuccess) return -(int)e;
   ++*launches;
-  TrArgs ta;
-  ta.d = d; ta.lat = lat; ta.x = x; ta.w0 = w.conv0_w; ta.w1 = w.conv1_w; ta.temp = w.temp; ta.q = q;
-  ta.k_cache = s.k_cache; ta.v_cache = s.v_cache; ta.hist = s.qk0_hist; ta.x_prev = s.x_prev; ta.pos = s.pos;
-  ta.S_max = s.S_max; ta.max_len = max_len; ta.status = status;
+  // Eq. 8: conv1 (with the value row, history and previous input), conv2 as a per-head contraction over
+  // (input channel, tap); Eq. 9 and the rest of Eq. 11 per head
+  const int kc = (d.flags & F_CONV2) ? d.k_ch : 1;
+  C1Args c1;
+  c1.d = d; c1.lat = lat; c1.x = x; c1.w0 = w.conv0_w; c1.y1s = y1s; c1.y2 = y2; c1.v_cache = s.v_cache;
+  c1.hist = s.qk0_hist; c1.x_prev = s.x_prev; c1.pos = s.pos; c1.S_max = s.S_max; c1.max_len = max_len; c1.status = status;
+  decode_conv1_kernel<<<dim3((unsigned)((d.L + 255) / 256), (unsigned)d.B), 256, 0, st>>>(c1);
+  if ((e = cudaGetLastError()) != cudaSuccess) return -(int)e;
+  ++*launches;
+  if (d.flags & F_CONV2) {
+    ProjArgs pc;
+    memset(&pc, 0, sizeof(pc));
+    pc.n_seg = 1;
+    pc.seg[0] = ProjSeg{w.conv1_w, y1s, d.L, 0};
+    pc.K = d.dh * kc; pc.B = d.B; pc.ldx = d.L * kc; pc.x_head_rows = d.dh; pc.out_f32 = y2; pc.ldo = d.L;
+    if ((e = launch_proj(pc, st)) != cudaSuccess) return -(int)e;
+    ++*launches;
+  }
+  FnArgs fa;
+  fa.d = d; fa.lat = lat; fa.y2 = y2; fa.temp = w.temp; fa.q = q; fa.k_cache = s.k_cache; fa.pos = s.pos;
+  fa.S_max = s.S_max; fa.max_len = max_len;
   {
-    dim3 grid((unsigned)(d.hq + d.hk + 1), (unsigned)d.B);
+    dim3 grid((unsigned)(d.hq + d.hk), (unsigned)d.B);
     switch (d.dh) {
-      case 32: decode_transform_kernel<32><<<grid, 128, 0, st>>>(ta); break;
-      case 64: decode_transform_kernel<64><<<grid, 128, 0, st>>>(ta); break;
-      case 128: decode_transform_kernel<128><<<grid, 128, 0, st>>>(ta); break;
-      default: return 1;
+      case 32: decode_finalize_kernel<32><<<grid, 128, 0, st>>>(fa); break;
+      case 64: decode_finalize_kernel<64><<<grid, 128, 0, st>>>(fa); break;
+      default: decode_finalize_kernel<128><<<grid, 128, 0, st>>>(fa); break;
     }
     if ((e = cudaGetLastError()) != cudaSuccess) return -(int)e;
     ++*launches;
@@ -668,7 +672,7 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
   memset(&pb, 0, sizeof(pb));
   pb.n_seg = 1;
   pb.seg[0] = ProjSeg{w.w_o, o, d.E, 0};
-  pb.K = d.Lq; pb.B = d.B; pb.out_bf16 = out; pb.ldo = d.E;
+  pb.K = d.Lq; pb.B = d.B; pb.ldx = d.Lq; pb.out_bf16 = out; pb.ldo = d.E;
   if ((e = launch_proj(pb, st)) != cudaSuccess) return -(int)e;
   ++*launches;
   return 0;
