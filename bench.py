@@ -310,6 +310,10 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+# dram bytes (read + write) of one launch of the decode attention kernel as it stands, from the full ncu capture
+# summarised under profiles/ (None when the kernel has changed since)
+DECODE_ATTN_DRAM_BYTES = {"decode16k": 537120512 + 5153792}
+
 DECODE_WORKLOADS = {
     # model of the 16k prefill shape; 32 sequences, each with 16384 cached tokens
     "decode16k": dict(model="cfg3_prefill16k", B=32, context=16384),
@@ -447,7 +451,7 @@ def run_decode(args, rank, world, local_rank):
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "decode attention over the latent cache", "achieved": attn_gbs, "peak": peak,
                      "unit": "GB/s", "frac": attn_gbs / peak, "peak_kind": peak_kind, "ms_per_launch": attn_ms,
-                     "bytes_per_launch": by["cache"], "traffic": None},
+                     "bytes_per_launch": by["cache"], "traffic": DECODE_ATTN_DRAM_BYTES.get(args.workload)},
         "step_gbs": by["total"] / (ms_step * 1e-3) / 1e9, "step_bytes": by,
         "device_status": status,
     }
