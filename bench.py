@@ -25,6 +25,7 @@ if ROOT not in sys.path:
 import torch
 
 from paper_2510_04476_b200 import synth
+from paper_2510_04476_b200.replicas import max_over_ranks
 
 METRIC = "CCGQA block throughput at 16k context (algorithmic causal FLOPs / device time)"
 UNIT = "TFLOP/s"
@@ -228,10 +229,7 @@ def run_ours(args, rank, world, local_rank):
     launches = cca.launch_count() - l0
     clocks = sampler.stop(w0, w1) if rank == 0 else None
     ms_total = e0.elapsed_time(e1)
-    tm = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-    ms_step = float(tm.item()) / args.steps
+    ms_step = max_over_ranks(ms_total, dist, "cuda") / args.steps
     status = cca.last_status()
     fl = flops_of(sh, backward)
     value = world * fl["total"] / (ms_step * 1e-3) / 1e12
@@ -265,10 +263,8 @@ def run_ours(args, rank, world, local_rank):
         e2e_step()
     g1.record()
     barrier()
-    e2e_ms = torch.tensor([g0.elapsed_time(g1) / n_e2e], device="cuda", dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-    e2e_val = world * fl["total"] / (float(e2e_ms.item()) * 1e-3) / 1e12
+    e2e_ms = max_over_ranks(g0.elapsed_time(g1) / n_e2e, dist, "cuda")
+    e2e_val = world * fl["total"] / (e2e_ms * 1e-3) / 1e12
     h2d = act_bytes * (2 if backward else 1)
     d2h = act_bytes
 
@@ -286,7 +282,7 @@ def run_ours(args, rank, world, local_rank):
                    "kernels": "tcgen05+simt" if args.kernels else "simt"},
         "clocks": clocks,
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": float(e2e_ms.item())},
+                "ms_per_step": e2e_ms},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "kernel": "latent attention forward", "achieved": attn_tflops, "peak": peak,
                      "unit": "TFLOP/s", "frac": attn_tflops / peak, "peak_kind": peak_kind,
@@ -410,10 +406,7 @@ def run_decode(args, rank, world, local_rank):
     cca.set_attention_events(None, None)
     launches = cca.launch_count() - l0
     clocks = sampler.stop(w0, w1) if rank == 0 else None
-    tm = torch.tensor([e0.elapsed_time(e1)], device="cuda", dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-    ms_step = float(tm.item()) / args.steps
+    ms_step = max_over_ranks(e0.elapsed_time(e1), dist, "cuda") / args.steps
     attn_ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
     status = cca.last_status()
     # end to end: the new tokens come from pinned host memory, the outputs go back to it
@@ -430,9 +423,7 @@ def run_decode(args, rank, world, local_rank):
         torch.cuda.synchronize()
     g1.record()
     barrier()
-    e2e_ms = torch.tensor([g0.elapsed_time(g1) / n_e2e], device="cuda", dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+    e2e_ms = max_over_ranks(g0.elapsed_time(g1) / n_e2e, dist, "cuda")
     by = decode_bytes(sh, B, ctx)
     peak, peak_kind = hbm_peak()
     attn_gbs = by["cache"] / (attn_ms * 1e-3) / 1e9
@@ -445,9 +436,9 @@ def run_decode(args, rank, world, local_rank):
                    "k_ch": sh.k_ch, "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
                    "l2": f"no flush: each step streams {by['cache'] / 1e6:.0f} MB of cache, more than the 126 MB L2"},
         "clocks": clocks,
-        "e2e": {"value": world * B / (float(e2e_ms.item()) * 1e-3), "unit": "tokens/s",
+        "e2e": {"value": world * B / (e2e_ms * 1e-3), "unit": "tokens/s",
                 "h2d_bytes_per_step": B * sh.d_model * 2, "d2h_bytes_per_step": B * sh.d_model * 2,
-                "ms_per_step": float(e2e_ms.item())},
+                "ms_per_step": e2e_ms},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "decode attention over the latent cache", "achieved": attn_gbs, "peak": peak,
                      "unit": "GB/s", "frac": attn_gbs / peak, "peak_kind": peak_kind, "ms_per_launch": attn_ms,
