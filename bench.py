@@ -172,7 +172,7 @@ def run_reference(args, rank, world):
 
 
 def run_ours(args, rank, world, local_rank):
-    from paper_2510_04476_b200.binding import CCA
+    from paper_2510_04476_b200.binding import CCA, stack_down_projection
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(local_rank)
@@ -184,7 +184,7 @@ def run_ours(args, rank, world, local_rank):
     sh = synth.CONFIGS[args.workload]
     backward = args.workload in TRAIN_WORKLOADS or args.backward
     t = synth.make_inputs(sh, want_dout=backward)
-    dev = {k: v.cuda(local_rank).contiguous() for k, v in t.items()}
+    dev = stack_down_projection({k: v.cuda(local_rank).contiguous() for k, v in t.items()})
     cca = CCA.from_shape(sh, device=local_rank)
     cca.set_impl(args.kernels)
     act_bytes = sh.B * sh.S * sh.d_model * 2
@@ -480,9 +480,9 @@ def oracle_decode_sample(sh, ctx):
 def fwd_bwd_same_shape(sh, args, local_rank):
     """The headline shape with the backward as well (the metric asks for forward and forward + backward at
     16k context).  Reported beside the forward-only line; not part of the timed region above."""
-    from paper_2510_04476_b200.binding import CCA
+    from paper_2510_04476_b200.binding import CCA, stack_down_projection
     t = synth.make_inputs(sh, want_dout=True)
-    dev = {k: v.cuda(local_rank).contiguous() for k, v in t.items()}
+    dev = stack_down_projection({k: v.cuda(local_rank).contiguous() for k, v in t.items()})
     cca = CCA.from_shape(sh, device=local_rank)
     cca.set_impl(args.kernels)
     ws = cca.alloc_workspace(sh.B, sh.S, True)

@@ -62,7 +62,10 @@ typedef struct {
   float rope_base;      /* RoPE base, e.g. 10000                                            */
 } cca_config;
 
-/* Parameters, all device pointers.  q rows of w_qk come first, then k rows (Listing A.1). */
+/* Parameters, all device pointers.  q rows of w_qk come first, then k rows (Listing A.1).
+ * Layout hint: the library contracts x with the stacked matrix [w_qk; w_v1; w_v2].  If the three already lie one
+ * after the other in memory in that order (w_v1 == w_qk + L*E elements, w_v2 == w_v1 + (L_k/2)*E) it reads them in
+ * place; otherwise every forward first copies them into the workspace (12.6 MB at the 16k prefill shape). */
 typedef struct {
   const void* w_qk;     /* bf16 [L_q + L_k, E]   packed q/k down-projection, Eq. 7          */
   const void* w_v1;     /* bf16 [L_k/2, E]       value projection of x_t, Eq. 10            */
@@ -73,7 +76,8 @@ typedef struct {
   const float* temp;    /* fp32 [h_k]            log of the key temperature beta            */
 } cca_weights;
 
-/* Parameter gradients, fp32 device buffers of the parameters' shapes; overwritten. */
+/* Parameter gradients, fp32 device buffers of the parameters' shapes; overwritten.  If d_w_qk, d_w_v1, d_w_v2 lie one
+ * after the other in memory (one [L + L_k, E] block) a single contraction writes all three. */
 typedef struct {
   float* d_w_qk;
   float* d_w_v1;

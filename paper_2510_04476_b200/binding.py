@@ -114,6 +114,16 @@ def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else C.c_void_p(t.data_ptr())
 
 
+def stack_down_projection(w: Dict[str, torch.Tensor]) -> Dict[str, torch.Tensor]:
+    """The same parameters with w_qk, w_v1, w_v2 as views of one [L + L_k, E] device tensor, the layout the library
+    reads in place (see cca_weights in the header).  Memory placement only."""
+    out = dict(w)
+    allw = torch.cat([w["w_qk"], w["w_v1"], w["w_v2"]], dim=0).contiguous()
+    n0, n1 = w["w_qk"].shape[0], w["w_v1"].shape[0]
+    out["w_qk"], out["w_v1"], out["w_v2"] = allw[:n0], allw[n0:n0 + n1], allw[n0 + n1:]
+    return out
+
+
 class CCA:
     """One configured block on one device.  Methods mirror the C entry points."""
 
@@ -292,16 +302,25 @@ class CCA:
         _check(self.lib, self.lib.cca_decode_state_from_prefill(self.handle, _ptr(x), wp, wn, B, S, C.byref(ds), st),
                self.handle, "cca_decode_state_from_prefill")
 
-    def backward(self, w, x: torch.Tensor, d_out: torch.Tensor, workspace: torch.Tensor):
-        """Returns (d_x bf16, dict of fp32 parameter gradients)."""
+    def backward(self, w, x: torch.Tensor, d_out: torch.Tensor, workspace: torch.Tensor, separate_grads: bool = False):
+        """Returns (d_x bf16, dict of fp32 parameter gradients).  separate_grads: give every gradient a buffer of
+        its own instead of one block for the three down-projection gradients."""
         B, S, E = x.shape
         assert d_out.is_cuda and d_out.is_contiguous() and d_out.dtype == torch.bfloat16
         d_x = torch.empty_like(x)
         grads = {}
         cg = cca_weight_grads()
+        # the three down-projection gradients as one block (the library then writes them with one contraction)
+        n0, n1, n2 = w["w_qk"].shape[0], w["w_v1"].shape[0], w["w_v2"].shape[0]
+        if separate_grads:
+            for n in ("w_qk", "w_v1", "w_v2"):
+                grads["d_" + n] = torch.empty((w[n].shape[0] + 3, E), dtype=torch.float32, device=self.device)[:w[n].shape[0]]
+        else:
+            d_all = torch.empty((n0 + n1 + n2, E), dtype=torch.float32, device=self.device)
+            grads["d_w_qk"], grads["d_w_v1"], grads["d_w_v2"] = d_all[:n0], d_all[n0:n0 + n1], d_all[n0 + n1:]
+        for n in ("w_o", "conv0_w", "conv1_w", "temp"):
+            grads["d_" + n] = torch.empty(w[n].shape, dtype=torch.float32, device=self.device)
         for n in ("w_qk", "w_v1", "w_v2", "w_o", "conv0_w", "conv1_w", "temp"):
-            shape = w[n].shape
-            grads["d_" + n] = torch.empty(shape, dtype=torch.float32, device=self.device)
             setattr(cg, "d_" + n, grads["d_" + n].data_ptr())
         cw = self._weights(w)
         wp, wn = self._ws_ptr(workspace)

@@ -69,6 +69,12 @@ CcaDims make_dims(const cca_config& c, int64_t B, int64_t S) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// True if three row blocks of `row_bytes` wide rows already lie one after the other in memory (a then b then c).
+bool adjacent(const void* a, const void* b, const void* c, size_t rows_a, size_t rows_b, size_t row_bytes) {
+  const char* pa = (const char*)a;
+  return pa && (const char*)b == pa + rows_a * row_bytes && (const char*)c == pa + (rows_a + rows_b) * row_bytes;
+}
+
 int check_sizes(const cca_handle* h, int64_t B, int64_t S, bool need_device = false) {
   if (!h || B < 1 || S < 1) return CCA_ERR_INVALID_ARG;
   if (need_device && h->device < 0) return CCA_ERR_INVALID_ARG;
@@ -391,11 +397,16 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
     h->launches++;
   }
   // the three down-projection weights stacked (also the B operand of the input gradient in the backward)
-  bf16* w_all = (bf16*)(ws + l.w_all);
-  CU(cudaMemcpyAsync(w_all, w->w_qk, (size_t)d.L * d.E * 2, cudaMemcpyDeviceToDevice, st));
-  CU(cudaMemcpyAsync(w_all + (size_t)d.L * d.E, w->w_v1, (size_t)(d.Lk / 2) * d.E * 2, cudaMemcpyDeviceToDevice, st));
-  CU(cudaMemcpyAsync(w_all + (size_t)(d.L + d.Lk / 2) * d.E, w->w_v2, (size_t)(d.Lk / 2) * d.E * 2,
-                     cudaMemcpyDeviceToDevice, st));
+  // (no copy if the caller keeps them adjacent in that order already)
+  const bf16* w_all = (const bf16*)w->w_qk;
+  if (!adjacent(w->w_qk, w->w_v1, w->w_v2, d.L, d.Lk / 2, (size_t)d.E * 2)) {
+    bf16* ws_all = (bf16*)(ws + l.w_all);
+    CU(cudaMemcpyAsync(ws_all, w->w_qk, (size_t)d.L * d.E * 2, cudaMemcpyDeviceToDevice, st));
+    CU(cudaMemcpyAsync(ws_all + (size_t)d.L * d.E, w->w_v1, (size_t)(d.Lk / 2) * d.E * 2, cudaMemcpyDeviceToDevice, st));
+    CU(cudaMemcpyAsync(ws_all + (size_t)(d.L + d.Lk / 2) * d.E, w->w_v2, (size_t)(d.Lk / 2) * d.E * 2,
+                       cudaMemcpyDeviceToDevice, st));
+    w_all = ws_all;
+  }
   GemmArgs g{};
   bool fused = false;
   if (h->impl >= 1 && h->tc) {
@@ -502,7 +513,9 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   float* dk = (float*)(ws + l.dk);
   float* dv = (float*)(ws + l.dv);
   bf16* dlat = (bf16*)(ws + l.dlat);
-  bf16* w_all = (bf16*)(ws + l.w_all);
+  // the stacked down-projection weights: the caller's own if they are adjacent, else the forward's copy
+  const bf16* w_all = adjacent(w->w_qk, w->w_v1, w->w_v2, d.L, d.Lk / 2, (size_t)d.E * 2) ? (const bf16*)w->w_qk
+                                                                                         : (const bf16*)(ws + l.w_all);
   const long long ldl = d.L + d.Lk;
 
   CU(cudaMemsetAsync(gr->d_conv0_w, 0, (size_t)d.L * c.k_seq * 4, st));
@@ -556,11 +569,17 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   g = GemmArgs{};
   g.A = mmajor(dlat, ldl); g.B = mmajor(x, d.E);
   g.M = d.L; g.N = d.E; g.K = T; g.seq_len = d.S; g.out_f32 = gr->d_w_qk; g.ldc = d.E;
-  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
-  g.A = mmajor(dlat + d.L, ldl); g.M = d.Lk / 2; g.out_f32 = gr->d_w_v1;
-  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
-  g.A = mmajor(dlat + d.L + d.Lk / 2, ldl); g.out_f32 = gr->d_w_v2;
-  if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  if (adjacent(gr->d_w_qk, gr->d_w_v1, gr->d_w_v2, d.L, d.Lk / 2, (size_t)d.E * 4)) {
+    // the three gradients are one [L + L_k, E] block for the caller: one contraction writes them all
+    g.M = d.L + d.Lk;
+    if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  } else {
+    if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+    g.A = mmajor(dlat + d.L, ldl); g.M = d.Lk / 2; g.out_f32 = gr->d_w_v1;
+    if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+    g.A = mmajor(dlat + d.L + d.Lk / 2, ldl); g.out_f32 = gr->d_w_v2;
+    if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  }
   // input gradient: d_x = [d_qk0, d_v1, d_v2 moved one token earlier] [W_qk; W_v1; W_v2] (stacked by the forward)
   g = GemmArgs{};
   g.A = kmajor(dlat, ldl); g.B = mmajor(w_all, d.E);

@@ -217,3 +217,30 @@ def test_bad_arguments_are_rejected_not_run():
     with pytest.raises(CcaError, match="invalid argument"):
         cca.forward(bad, t["x"], ws)
     cca.close()
+
+
+def test_adjacent_down_projection_weights_are_read_in_place():
+    """w_qk, w_v1, w_v2 laid out as one block (no stacking copy, one weight-gradient contraction) must give the
+    results of the separate-buffer path: same kernels, same operand values."""
+    from paper_2510_04476_b200.binding import stack_down_projection
+    sh = S_("stacked", 2, 600, 512, 8, 2, 64)
+    t = synth.make_inputs(sh)
+    dev = to_device(t)
+    cca = _cca(sh)
+    res = []
+    for i, w in enumerate((dev, stack_down_projection(dev))):
+        ws = cca.alloc_workspace(sh.B, sh.S, True)
+        ws.zero_()
+        out = cca.forward(w, w["x"], ws)
+        d_x, grads = cca.backward(w, w["x"], w["d_out"], ws, separate_grads=(i == 0))
+        torch.cuda.synchronize()
+        assert cca.last_status() == 0
+        res.append((out.clone(), d_x.clone(), {k: v.clone() for k, v in grads.items()}))
+    assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1])
+    cfg = oracle_cfg(sh)
+    _, I = O.forward(cfg, t, t["x"])
+    G = O.backward(cfg, t, I, t["d_out"])
+    for n in ("w_qk", "w_v1", "w_v2"):
+        check_close("d_" + n, res[0][2]["d_" + n], G["d_" + n], scale_abs=True)
+        check_close("d_" + n, res[1][2]["d_" + n], G["d_" + n], scale_abs=True)
+    cca.close()
