@@ -1,5 +1,6 @@
 // Tensor-core kernels, part 6: the large projection GEMMs on CTA pairs.
-//   C[M,N] = sum_k A(m,k) B(n,k), A K-major, B K-major or MN-major, bf16 operands, fp32 accumulate.
+//   C[M,N] = sum_k A(m,k) B(n,k), A and B K-major or MN-major, bf16 operands, fp32 accumulate; optional split of the
+//   k range over several work items whose partial sums are added to a zeroed fp32 output (weight gradients: K = tokens).
 // Two CTAs on neighbouring SMs (a cluster of 2) work on one 256 x 256 tile with tcgen05.mma.cta_group::2:
 // each CTA loads its own 128 rows of A and only HALF of the B tile (128 of the 256 output columns), the
 // tensor cores of both SMs read B from both shared memories.  Per k-block a CTA therefore pulls 32 KB
@@ -29,7 +30,8 @@ struct G2Params {
   float* out_f32;
   long long ldc;
   int tiles_m, tiles_n, num_kb;     // tiles of 256 x 256
-  int b_mn;
+  int a_mn, b_mn;
+  int splits, kb_per_split;   // work item = (tile, split)
   int vec_ok;
   int split_L, split_Lk, split_shift, seq_len;   // fused down-projection output (see GemmArgs)
   int* status;
@@ -107,7 +109,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int num_tiles = p.tiles_m * p.tiles_n;
+  const int num_tiles = p.tiles_m * p.tiles_n * p.splits;       // work items
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < G2_STAGES; ++s) {
@@ -139,15 +141,22 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       int stage = 0;
       uint32_t phase = 0;
       for (int tile = pair; tile < num_tiles; tile += n_pairs) {
-        const int m0 = (tile / p.tiles_n) * (2 * G2_BM) + (int)rank * G2_BM;
-        const int n0 = (tile % p.tiles_n) * G2_BN + (int)rank * (G2_BN / 2);
-        for (int kb = 0; kb < p.num_kb; ++kb) {
+        const int sp = tile % p.splits, mn = tile / p.splits;
+        const int m0 = (mn / p.tiles_n) * (2 * G2_BM) + (int)rank * G2_BM;
+        const int n0 = (mn % p.tiles_n) * G2_BN + (int)rank * (G2_BN / 2);
+        const int kb_end = min(p.num_kb, (sp + 1) * p.kb_per_split);
+        for (int kb = sp * p.kb_per_split; kb < kb_end; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
           unsigned char* sa = smem + stage * SM::STAGE_BYTES;
           unsigned char* sb = sa + SM::A_BYTES;
           if (rank == 0) mbar_expect_tx(&full_bar[stage], 2 * SM::STAGE_BYTES);
           const int k0 = kb * G2_BK;
-          tma_load_2d_pair(sa, &tmA, k0, m0, &full_bar[stage]);
+          if (!p.a_mn) {
+            tma_load_2d_pair(sa, &tmA, k0, m0, &full_bar[stage]);
+          } else {
+            tma_load_2d_pair(sa, &tmA, m0, k0, &full_bar[stage]);
+            tma_load_2d_pair(sa + 8192, &tmA, m0 + 64, k0, &full_bar[stage]);
+          }
           if (!p.b_mn) {
             tma_load_2d_pair(sb, &tmB, k0, n0, &full_bar[stage]);
           } else {
@@ -162,11 +171,11 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (rank == 0) {
       const bool leader = elect_one();
       // M = 256 over the pair, N = 256
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.b_mn << 16) | ((uint32_t)(G2_BN >> 3) << 17) |
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) | ((uint32_t)(G2_BN >> 3) << 17) |
                              ((uint32_t)(256 >> 4) << 24);
       const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
-      const uint32_t a_lbo = 1u << 16, b_lbo = p.b_mn ? ((8192u >> 4) << 16) : (1u << 16);
-      const uint32_t a_step = 32u >> 4, b_step = p.b_mn ? (2048u >> 4) : (32u >> 4);
+      const uint32_t a_lbo = p.a_mn ? ((8192u >> 4) << 16) : (1u << 16), b_lbo = p.b_mn ? ((8192u >> 4) << 16) : (1u << 16);
+      const uint32_t a_step = p.a_mn ? (2048u >> 4) : (32u >> 4), b_step = p.b_mn ? (2048u >> 4) : (32u >> 4);
       const uint32_t smem_lo = smem_u32(smem) >> 4;
       auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
         return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
@@ -180,7 +189,9 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         if (!wait_all(&acc_empty[as], aphase ^ 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + as * G2_BN;
-        for (int kb = 0; kb < p.num_kb; ++kb) {
+        const int sp = tile % p.splits;
+        const int kb_begin = sp * p.kb_per_split, kb_end = min(p.num_kb, kb_begin + p.kb_per_split);
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!wait_all(&full_bar[stage], phase)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
           tc_fence_after();
           const uint32_t sa = (smem_lo + stage * (SM::STAGE_BYTES >> 4)) | a_lbo;
@@ -188,7 +199,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           if (leader) {
 #pragma unroll
             for (int k = 0; k < G2_BK / 16; ++k)
-              mma2_ss_w(d_tmem, sa + k * a_step, desc_hi, sb + k * b_step, desc_hi, idesc, (kb | k) != 0);
+              mma2_ss_w(d_tmem, sa + k * a_step, desc_hi, sb + k * b_step, desc_hi, idesc, (kb != kb_begin) | (k != 0));
             mma2_commit_both(&empty_bar[stage]);
           }
           if (++stage == G2_STAGES) { stage = 0; phase ^= 1; }
@@ -202,7 +213,8 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     for (int tile = pair; tile < num_tiles; tile += n_pairs, ++it) {
       const int as = it & 1;
       const uint32_t aphase = (it >> 1) & 1;
-      const int m0 = (tile / p.tiles_n) * (2 * G2_BM) + (int)rank * G2_BM, n0 = (tile % p.tiles_n) * G2_BN;
+      const int mn = tile / p.splits;
+      const int m0 = (mn / p.tiles_n) * (2 * G2_BM) + (int)rank * G2_BM, n0 = (mn % p.tiles_n) * G2_BN;
       if (!mbar_wait(&acc_full[as], aphase, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
       tc_fence_after();
       const int m = m0 + q * 32 + lane;
@@ -263,7 +275,20 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
           } else {
             float* dst = p.out_f32 + (long long)m * p.ldc + n;
-            if (p.vec_ok && n + 32 <= p.N) {
+            if (p.splits > 1) {
+              if (p.vec_ok && n + 32 <= p.N) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4 * i), "f"(__uint_as_float(r[4 * i])),
+                               "f"(__uint_as_float(r[4 * i + 1])), "f"(__uint_as_float(r[4 * i + 2])),
+                               "f"(__uint_as_float(r[4 * i + 3]))
+                               : "memory");
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (n + i < p.N) atomicAdd(dst + i, __uint_as_float(r[i]));
+              }
+            } else if (p.vec_ok && n + 32 <= p.N) {
 #pragma unroll
               for (int i = 0; i < 8; ++i)
                 reinterpret_cast<uint4*>(dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
@@ -298,7 +323,8 @@ done:
 }
 
 template <int BN>
-int launch_pair(TcState* s, const GemmArgs& g, const G2Params& p0, bool b_mn, long long lda, long long ldb, cudaStream_t st) {
+int launch_pair(TcState* s, const GemmArgs& g, const G2Params& p0, bool a_mn, bool b_mn, long long lda, long long ldb,
+                cudaStream_t st) {
   static bool attr_set = false;
   using SM = G2Smem<BN>;
   if (!attr_set) {
@@ -307,14 +333,33 @@ int launch_pair(TcState* s, const GemmArgs& g, const G2Params& p0, bool b_mn, lo
     attr_set = true;
   }
   CUtensorMap tmA, tmB;
-  if (!tc_make_map_2d(s, &tmA, g.A.p, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)lda, G2_BK, G2_BM)) return 1;
   bool ok;
+  if (!a_mn) ok = tc_make_map_2d(s, &tmA, g.A.p, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)lda, G2_BK, G2_BM);
+  else ok = tc_make_map_2d(s, &tmA, g.A.p, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)lda, 64, G2_BK);
+  if (!ok) return 1;
   if (!b_mn) ok = tc_make_map_2d(s, &tmB, g.B.p, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)ldb, G2_BK, BN / 2);
   else ok = tc_make_map_2d(s, &tmB, g.B.p, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)ldb, 64, G2_BK);
   if (!ok) return 1;
   G2Params p = p0;
   p.tiles_n = (g.N + BN - 1) / BN;
-  const int tiles = p.tiles_m * p.tiles_n;
+  // split the k range when that fills the waves of CTA pairs better (fp32 output that the items can add into)
+  p.splits = 1;
+  if (g.out_f32 && !g.out_bf16 && g.split_L == 0 && g.ldc == g.N && p.num_kb >= 32) {
+    const long long mn = (long long)p.tiles_m * p.tiles_n;
+    double best = 1e30;
+    for (int sp = 1; sp <= 8 && sp * 16 <= p.num_kb; ++sp) {
+      const long long waves = (mn * sp + s->pair_clusters - 1) / s->pair_clusters;
+      const double c = (double)waves / sp * (1.0 + 0.03 * (sp - 1));
+      if (c < best - 1e-9) { best = c; p.splits = sp; }
+    }
+  }
+  p.kb_per_split = (p.num_kb + p.splits - 1) / p.splits;
+  p.splits = (p.num_kb + p.kb_per_split - 1) / p.kb_per_split;     // no empty split
+  if (p.splits > 1) {
+    cudaError_t me = cudaMemsetAsync(g.out_f32, 0, (size_t)g.M * g.N * sizeof(float), st);
+    if (me != cudaSuccess) return -(int)me;
+  }
+  const int tiles = p.tiles_m * p.tiles_n * p.splits;
   const int pairs = tiles < s->pair_clusters ? tiles : s->pair_clusters;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
@@ -334,10 +379,11 @@ int launch_pair(TcState* s, const GemmArgs& g, const G2Params& p0, bool b_mn, lo
 // Returns 0 if enqueued, 1 if the case is outside this kernel's coverage, -cudaError on failure.
 int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) {
   if (!s || !s->encode || !s->use_pairs) return 1;
-  if (g.A.cs != 1 || g.a_row_off != 0) return 1;                  // A K-major, no row shift
-  const int b_mn = g.B.cs != 1;
-  if (b_mn && g.B.rs != 1) return 1;
-  const long long lda = g.A.rs, ldb = b_mn ? g.B.cs : g.B.rs;
+  if (g.a_row_off != 0) return 1;                                 // no row shift
+  const int a_mn = g.A.cs != 1, b_mn = g.B.cs != 1;
+  if ((a_mn && g.A.rs != 1) || (b_mn && g.B.rs != 1)) return 1;
+  if (a_mn && g.split_L > 0) return 1;
+  const long long lda = a_mn ? g.A.cs : g.A.rs, ldb = b_mn ? g.B.cs : g.B.rs;
   if (lda % 8 || ldb % 8) return 1;
   if ((reinterpret_cast<uintptr_t>(g.A.p) & 15) || (reinterpret_cast<uintptr_t>(g.B.p) & 15)) return 1;
   if (g.M < 512 || g.N < 256 || g.K < 64) return 1;
@@ -368,7 +414,8 @@ int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) 
   p.tiles_m = (g.M + 2 * G2_BM - 1) / (2 * G2_BM);
   p.tiles_n = 0;
   p.num_kb = (g.K + G2_BK - 1) / G2_BK;
-  p.b_mn = b_mn;
+  p.a_mn = a_mn; p.b_mn = b_mn;
+  p.splits = 1; p.kb_per_split = p.num_kb;
   const void* outp = g.out_bf16 ? (const void*)g.out_bf16 : (const void*)g.out_f32;
   const int esz = g.out_bf16 ? 2 : 4;
   p.vec_ok = ((reinterpret_cast<uintptr_t>(outp) & 15) == 0) && ((g.ldc * esz) % 16 == 0);
@@ -380,6 +427,6 @@ int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) 
     return ((tiles + s->pair_clusters - 1) / s->pair_clusters) * bn;
   };
   // (an MN-major B half of 96 columns would not be a whole number of 64-column swizzle chunks)
-  if (!b_mn && cost(192) < cost(256)) return launch_pair<192>(s, g, p, b_mn, lda, ldb, st);
-  return launch_pair<256>(s, g, p, b_mn, lda, ldb, st);
+  if (!b_mn && cost(192) < cost(256)) return launch_pair<192>(s, g, p, a_mn, b_mn, lda, ldb, st);
+  return launch_pair<256>(s, g, p, a_mn, b_mn, lda, ldb, st);
 }
