@@ -53,7 +53,7 @@ typedef struct {
   int32_t d_model;      /* E                                                                */
   int32_t n_q_heads;    /* h_q;  L_q = h_q * head_dim = E / C1                              */
   int32_t n_kv_heads;   /* h_k;  L_k = h_k * head_dim = E / C2;  h_q % h_k == 0, L_k even   */
-  int32_t head_dim;     /* d_h, latent per-head size: 32, 64 or 128                         */
+  int32_t head_dim;     /* d_h, latent per-head size: 32, 64, 128; 256 forward only        */
   int32_t compression;  /* C = C1; checked: E == C * h_q * d_h                              */
   int32_t k_seq;        /* taps of conv1_seq (1..4)                                         */
   int32_t k_ch;         /* taps of conv2_seq+ch (1..4)                                      */
@@ -111,7 +111,7 @@ typedef struct cca_handle cca_handle;
 
 /* Validate the configuration for `device`, create a handle.  Paper: Eq. 7-11 parameters.
  * Errors: INVALID_ARG (null, E != C*h_q*d_h, h_q % h_k, odd L_k, bad kernel sizes),
- * UNSUPPORTED (head_dim not in {32,64,128}, h_q > 64, device not compute capability 10.x),
+ * UNSUPPORTED (head_dim not in {32,64,128,256}, h_q > 64, device not compute capability 10.x),
  * CUDA.  device = -1 makes a host-only handle: cca_describe and cca_workspace_size work, every
  * compute entry point returns INVALID_ARG. */
 int cca_init(const cca_config* cfg, int device, cca_handle** out);
@@ -136,7 +136,7 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out,
 /* Backward of the block: given d_out = dLoss/d out (device bf16 [B,S,E]) and the workspace
  * left by cca_forward for the same x and weights, writes d_x (device bf16 [B,S,E]) and every
  * field of `grads` (fp32, overwritten).  The paper prints no backward; this is the exact
- * adjoint of Eq. 7-11.  Errors as cca_forward. */
+ * adjoint of Eq. 7-11.  Errors as cca_forward; UNSUPPORTED for head_dim = 256 (forward only). */
 int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void* d_out,
                  void* workspace, size_t workspace_bytes, void* d_x,
                  const cca_weight_grads* grads, int64_t B, int64_t S, void* cuda_stream);

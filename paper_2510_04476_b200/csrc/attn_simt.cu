@@ -366,6 +366,14 @@ cudaError_t set_smem(K kern, size_t bytes) {
 cudaError_t launch_attn_fwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* o32,
                                  float* lse, cudaStream_t st) {
   dim3 grid((d.S + BT - 1) / BT, d.hq, d.B);
+  if (d.dh == 256) {                       // forward only exists at this head size
+    constexpr int DH = 256;
+    size_t sm = (size_t)(3 * BT * AL<DH>::LD + BT * AL<DH>::PLD) * sizeof(float);
+    cudaError_t e = set_smem(attn_fwd_kernel<DH>, sm);
+    if (e != cudaSuccess) return e;
+    attn_fwd_kernel<DH><<<grid, 256, sm, st>>>(d, q, k, v, o, o32, lse);
+    return cudaGetLastError();
+  }
   DISPATCH_DH(d.dh, {
     size_t sm = (size_t)(3 * BT * AL<DH>::LD + BT * AL<DH>::PLD) * sizeof(float);
     cudaError_t e = set_smem(attn_fwd_kernel<DH>, sm);

@@ -26,7 +26,7 @@ namespace {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
-  size_t qk0, q, k, v, o, lse, rope, rnorm, w_all, saved_end;
+  size_t qk0, q, k, v, o, lse, rope, rnorm, w_all, y1s, y2, saved_end;
   size_t o32, d_o, delta, dq, dk, dv, dlat, dy1, total_end;
 };
 
@@ -45,6 +45,12 @@ Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
   l.rope = take((size_t)S * (c.head_dim / 2) * 8);
   l.rnorm = take(T * (size_t)(c.n_q_heads + c.n_kv_heads) * 4);   // norm scale of every (token, head)
   l.w_all = take((L + Lk) * (size_t)c.d_model * 2);                // [W_qk; W_v1; W_v2] stacked
+  // unfused latent transforms (head sizes the fused kernel does not cover): conv1 taps and conv output
+  l.y1s = l.y2 = off;
+  if (c.head_dim > 128) {
+    l.y1s = take(T * L * (size_t)c.k_ch * 2);
+    l.y2 = take(T * L * 4);
+  }
   l.saved_end = off;
   l.o32 = take(T * Lq * 4);
   l.d_o = take(T * Lq * 2);
@@ -112,7 +118,8 @@ int run_attention_fwd(cca_handle* h, const CcaDims& d, const bf16* q, const bf16
   if (h->ev_attn_begin) CU(cudaEventRecord(h->ev_attn_begin, st));
   bool done = false;
   if (h->impl >= 1 && h->tc) {
-    int r = tc_attn_fwd(h->tc, d, q, k, v, o, o32, lse, temp, h->d_status, st);
+    int r = d.dh == 256 ? tc_attn_fwd256(h->tc, d, q, k, v, o, o32, lse, temp, h->d_status, st)
+                        : tc_attn_fwd(h->tc, d, q, k, v, o, o32, lse, temp, h->d_status, st);
     if (r == 0) done = true;
     if (r < 0) { h->last_cuda = -r; return CCA_ERR_CUDA; }
   }
@@ -151,7 +158,7 @@ static int validate_config(const cca_config* c) {
   if (c->flags & ~(uint32_t)CCA_ALL_STAGES) return CCA_ERR_INVALID_ARG;
   if ((c->flags & CCA_ROPE) && !(c->rope_base > 0.f)) return CCA_ERR_INVALID_ARG;
   if (c->k_seq > 4 || c->k_ch > 4) return CCA_ERR_UNSUPPORTED;
-  if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return CCA_ERR_UNSUPPORTED;
+  if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128 && c->head_dim != 256) return CCA_ERR_UNSUPPORTED;
   if (c->n_q_heads > 64) return CCA_ERR_UNSUPPORTED;
   if (c->d_model % 8 != 0) return CCA_ERR_UNSUPPORTED;
   return CCA_OK;
@@ -434,7 +441,26 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
     if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
   }
   // Eq. 8, 9, 11: convs, q-k-mean, norm, temperature, RoPE
-  {
+  if (d.dh > 128) {
+    // unfused: conv1 at the taps conv2 reads, conv2 as one contraction per head over (input channel, tap), then the
+    // per-(token, head) stages
+    bf16* y1s = (bf16*)(ws + l.y1s);
+    float* y2 = (float*)(ws + l.y2);
+    CU(launch_conv1_taps(d, qk0, (const bf16*)w->conv0_w, y1s, y2, st));
+    h->launches++;
+    if (c.flags & CCA_CONV2) {
+      const int kd = d.dh * c.k_ch;
+      for (int hh = 0; hh < d.hq + d.hk; ++hh) {
+        GemmArgs gc{};
+        gc.A = kmajor(y1s + (size_t)hh * kd, (long long)d.L * c.k_ch);
+        gc.B = kmajor((const bf16*)w->conv1_w + (size_t)hh * d.dh * kd, kd);
+        gc.M = T; gc.N = d.dh; gc.K = kd; gc.seq_len = d.S; gc.out_f32 = y2 + (size_t)hh * d.dh; gc.ldc = d.L;
+        if ((r = run_gemm(h, gc, st)) != CCA_OK) return r;
+      }
+    }
+    CU(launch_finalize(d, qk0, y2, w->temp, rope, q, k, rnorm, st));
+    h->launches++;
+  } else {
     bool done = false;
     if (h->impl >= 1 && h->tc) {
       int tr = tc_transform_fwd(h->tc, d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k,
@@ -489,6 +515,7 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   if (!gr->d_w_qk || !gr->d_w_v1 || !gr->d_w_v2 || !gr->d_w_o || !gr->d_conv0_w || !gr->d_conv1_w || !gr->d_temp)
     return CCA_ERR_INVALID_ARG;
   const cca_config& c = h->cfg;
+  if (c.head_dim > 128) return CCA_ERR_UNSUPPORTED;          // head size 256: forward only
   if (!aligned16(x) || !aligned16(d_out) || !aligned16(d_x) || (reinterpret_cast<uintptr_t>(workspace) & 255))
     return CCA_ERR_ALIGNMENT;
   Layout l = make_layout(c, B, S);

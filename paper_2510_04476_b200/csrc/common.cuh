@@ -70,6 +70,13 @@ cudaError_t launch_transform_bwd_w1(const CcaDims& d, const float* qk0, const bf
 // dlat columns [L, L+Lk) <- dv with the second half moved one token earlier (value-shift adjoint).
 cudaError_t launch_pack_dv(const CcaDims& d, const float* dv, bf16* dlat, long long ld_dlat, cudaStream_t st);
 
+// Same stages without the fused kernels, for head sizes those do not cover: conv1 output at the taps conv2 reads
+// (y1s[t, c * k_ch + r], bf16; y2 [T, L] fp32 directly when conv2 is off), then -- after the caller's per-head
+// contractions have filled y2 -- q-k-mean, norm, temperature and RoPE.
+cudaError_t launch_conv1_taps(const CcaDims& d, const float* qk0, const bf16* w0, bf16* y1s, float* y2, cudaStream_t st);
+cudaError_t launch_finalize(const CcaDims& d, const float* qk0, const float* y2, const float* temp, const float2* rope,
+                            bf16* q, bf16* k, float* rnorm, cudaStream_t st);
+
 // ---- attention (Eq. 11, softmax line), plain SIMT ----
 // o32: optional fp32 copy of o (kept for the backward's delta = rowsum(dO * O)); may be null.
 cudaError_t launch_attn_fwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o,

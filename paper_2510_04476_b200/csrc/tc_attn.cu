@@ -18,6 +18,7 @@
 // fixed share of the exponentials is evaluated on the FMA pipe instead (round to integer + cubic for
 // 2^f, |f| <= 1/2, relative error 7.5e-5, well under the bf16 rounding of P), two at a time with the
 // packed f32x2 instructions.
+#include "tc_attn_common.cuh"
 #include "tc_kernels.cuh"
 #include "tc_ptx.cuh"
 #include "tc_state.cuh"
@@ -30,20 +31,6 @@ constexpr int AT_SOFTMAX_WARPS = 16;                 // 2 query tiles x 2 column
 constexpr int AT_TMA_WARP = AT_SOFTMAX_WARPS, AT_MMA_WARP = AT_SOFTMAX_WARPS + 1;
 constexpr int AT_THREADS = 32 * (AT_SOFTMAX_WARPS + 2);
 constexpr int BQ = 128, BKV = 128;
-constexpr float LOG2E_F = 1.4426950408889634f;
-constexpr float LN2_F = 0.6931471805599453f;
-constexpr float RESCALE_THRESHOLD = 8.0f;      // log2 units
-
-struct AttnParams {
-  int B, S, hq, hk, g, Lq, Lk, causal;
-  bf16* o;
-  float* o32;
-  float* lse;
-  int n_blocks;       // 256-row blocks per sequence
-  int* status;
-  const float* temp;  // log key temperature per kv head if q, k are L2-normalised (Eq. 11), else null
-};
-
 template <int DH>
 struct AttnSmem {
   static constexpr int TILE_BYTES = 128 * DH * 2;            // one 128-row tile of Q, K or V
@@ -59,11 +46,6 @@ struct AttnSmem {
   static constexpr int TOTAL = (XCH_OFF + 2048) > 122880 ? (XCH_OFF + 2048) : 122880;
 };
 
-TC_DEVINL void fail(volatile int* abort_flag, int* status, int code) {
-  *abort_flag = 1;
-  atomicCAS(status, 0, code);
-}
-
 // K-major operand tile [128 rows][DH] stored as DH/64 swizzled boxes of [128][64]: descriptor of the
 // kk-th 16-element slice along the head dimension.
 template <int DH>
@@ -74,38 +56,6 @@ TC_DEVINL uint64_t kmajor_desc(uint32_t tile_addr, int kk) {
 // kk-th 16-key slice; 64-channel chunks are one box (16384 B) apart.
 TC_DEVINL uint64_t v_desc(uint32_t tile_addr, int kk) { return smem_desc_sw128(tile_addr + kk * 2048, 16384, 1024); }
 
-
-// Exponentials of 8 consecutive scores (already in registers) -> 4 packed bf16 pairs; adds the rounded
-// values to the two running partial sums in `sum2`.  POLY of the 4 pairs go through the
-// polynomial.  CLAMP: x may be far below the smallest exponent (online mode); then it is clamped first.
-template <int POLY, bool CLAMP>
-TC_DEVINL void exp8(const uint32_t* v, uint64_t scale2, uint64_t negm2, uint64_t& sum2, uint32_t* out) {
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint64_t x = fma2(pack2u(v[2 * i], v[2 * i + 1]), scale2, negm2);
-    uint64_t e;
-    if (i < POLY) {
-      if (CLAMP) {
-        uint32_t a, b;
-        unpack2u(x, a, b);
-        x = pack2f(fmaxf(__uint_as_float(a), -120.f), fmaxf(__uint_as_float(b), -120.f));
-      }
-      e = exp2_poly2(x);
-    } else {
-      uint32_t a, b;
-      unpack2u(x, a, b);
-      e = pack2f(ex2f(__uint_as_float(a)), ex2f(__uint_as_float(b)));
-    }
-    // The row sum is taken over the bf16-rounded probabilities, the values the P V product really uses, so
-    // that the weights of a row sum to one whatever the rounding did (with a fixed maximum even the
-    // largest probability of a row is rounded).
-    uint32_t a, b;
-    unpack2u(e, a, b);
-    const uint32_t w = pack_bf16(__uint_as_float(a), __uint_as_float(b));
-    out[i] = w;
-    sum2 = add2(sum2, pack2u(w << 16, w & 0xffff0000u));
-  }
-}
 
 template <int DH, int POLY>
 __global__ void __launch_bounds__(AT_THREADS, 1)

@@ -13,6 +13,9 @@ int tc_gemm(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st);
 int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st);
 int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* o32,
                 float* lse, const float* temp, int* d_status, cudaStream_t st);
+// Head size 256 (one query tile per CTA, score buffers alternate over key tiles).
+int tc_attn_fwd256(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* o32, float* lse,
+                   const float* temp, int* d_status, cudaStream_t st);
 // Attention adjoint (dq, dk, dv in fp32) from q, k, v, d_o, the forward's lse and delta = rowsum(dO o O).
 int tc_attn_bwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                 const float* lse, const float* delta, float* dq, float* dk, float* dv, int* d_status, cudaStream_t st);

@@ -244,3 +244,54 @@ def test_adjacent_down_projection_weights_are_read_in_place():
         check_close("d_" + n, res[0][2]["d_" + n], G["d_" + n], scale_abs=True)
         check_close("d_" + n, res[1][2]["d_" + n], G["d_" + n], scale_abs=True)
     cca.close()
+
+
+# ------------------------------------------------------------------ head size 256 (forward only)
+DH256 = [
+    S_("dh256_two_tiles", 2, 300, 1024, 4, 1, 256),
+    S_("dh256_g2_ragged", 1, 777, 2048, 4, 2, 256),
+    S_("dh256_noncausal", 1, 260, 1024, 4, 2, 256, causal=0),
+    S_("dh256_plain_mha", 1, 200, 1024, 4, 4, 256, flags=0),
+    S_("dh256_no_conv2_k3", 2, 140, 1024, 4, 1, 256, flags=63 & ~2, k_seq=3),
+    S_("dh256_k3_k4", 1, 150, 1024, 4, 1, 256, k_seq=3, k_ch=4),
+    S_("dh256_one_token", 2, 1, 1024, 4, 1, 256),
+]
+
+
+@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("sh", DH256, ids=lambda s: s.name)
+def test_head_size_256_forward(sh, impl):
+    run_case(sh, impl, backward=False)
+
+
+def test_head_size_256_backward_is_refused():
+    from paper_2510_04476_b200.binding import CcaError
+    sh = DH256[0]
+    t = synth.make_inputs(sh)
+    dev = to_device(t)
+    cca = _cca(sh)
+    ws = cca.alloc_workspace(sh.B, sh.S, True)
+    cca.forward(dev, dev["x"], ws)
+    with pytest.raises(CcaError):
+        cca.backward(dev, dev["x"], dev["d_out"], ws)
+    cca.close()
+
+
+def test_head_size_256_at_16k_sampled_rows():
+    sh = synth.Shape("dh256_16k", 1, 16384, 2048, 2, 1, 256, seed=77)
+    t = synth.make_inputs(sh, want_dout=False)
+    rows = sample_rows(sh.S, n_random=24)
+    out_ref, o_ref, lse_ref, I = O.forward_rows(oracle_cfg(sh), t, t["x"], rows)
+    dev = to_device(t)
+    cca = _cca(sh)
+    ws = cca.alloc_workspace(sh.B, sh.S, False)
+    out = cca.forward(dev, dev["x"], ws)
+    torch.cuda.synchronize()
+    assert cca.last_status() == 0
+    sv = cca.saved(ws, sh.B, sh.S)
+    for n in ("v", "q", "k"):
+        check_close(n, sv[n], I[n])
+    check_close("o_rows", sv["o"][:, rows], o_ref)
+    check_close("lse_rows", sv["lse"][:, :, rows], lse_ref)
+    check_close("out_rows", out[:, rows], out_ref)
+    cca.close()
