@@ -12,6 +12,11 @@ namespace {
 
 enum : unsigned { F_CONV1 = 1, F_CONV2 = 2, F_QK_MEAN = 4, F_QK_NORM = 16, F_ROPE = 32 };
 
+CCA_DEVINL uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
 // thread = (token, 4 channels)
 __global__ void __launch_bounds__(256) conv1_taps_kernel(CcaDims d, const float* __restrict__ qk0, const bf16* __restrict__ w0,
                                                          bf16* __restrict__ y1s, float* __restrict__ y2) {
@@ -38,12 +43,13 @@ __global__ void __launch_bounds__(256) conv1_taps_kernel(CcaDims d, const float*
 #pragma unroll
     for (int j = 0; j < 4; ++j)
       wt[c][j] = (j < ks) ? ((d.flags & F_CONV1) ? __bfloat162float(w0[(size_t)(ch + c) * d.k_seq + j]) : 1.f) : 0.f;
+  // the thread's 4 channels x kc taps are contiguous in y1s: element (c, r) at (ch + c) * kc + r
+  float yv[4][4];
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
-    if (r >= kc) break;
     // y1 at token t - (kc - 1) + r: taps j = 0..ks-1 read raw tokens t - (kc-1) + r - (ks-1) + j = raw[r + j]
     float y[4] = {0.f, 0.f, 0.f, 0.f};
-    if (t - (kc - 1) + r >= 0) {
+    if (r < kc && t - (kc - 1) + r >= 0) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         if (j < ks) {
@@ -55,12 +61,31 @@ __global__ void __launch_bounds__(256) conv1_taps_kernel(CcaDims d, const float*
         }
       }
     }
-    if (d.flags & F_CONV2) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) y1s[(tok * d.L + ch + c) * kc + r] = __float2bfloat16(y[c]);
-    } else {
-      *reinterpret_cast<float4*>(y2 + tok * d.L + ch) = make_float4(y[0], y[1], y[2], y[3]);
-    }
+    for (int c = 0; c < 4; ++c) yv[c][r] = y[c];
+  }
+  if (!(d.flags & F_CONV2)) {
+    *reinterpret_cast<float4*>(y2 + tok * d.L + ch) = make_float4(yv[0][0], yv[1][0], yv[2][0], yv[3][0]);
+    return;
+  }
+  bf16* dst = y1s + (tok * d.L + ch) * kc;          // 8 kc bytes, 8-byte aligned
+  if (kc == 2) {
+    uint4 w;
+    w.x = pack2(yv[0][0], yv[0][1]); w.y = pack2(yv[1][0], yv[1][1]);
+    w.z = pack2(yv[2][0], yv[2][1]); w.w = pack2(yv[3][0], yv[3][1]);
+    *reinterpret_cast<uint4*>(dst) = w;
+  } else if (kc == 4) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      reinterpret_cast<uint2*>(dst)[c] = make_uint2(pack2(yv[c][0], yv[c][1]), pack2(yv[c][2], yv[c][3]));
+  } else if (kc == 1) {
+    *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(yv[0][0], yv[1][0]), pack2(yv[2][0], yv[3][0]));
+  } else {                                           // kc == 3: 12 elements
+    const float f[12] = {yv[0][0], yv[0][1], yv[0][2], yv[1][0], yv[1][1], yv[1][2],
+                         yv[2][0], yv[2][1], yv[2][2], yv[3][0], yv[3][1], yv[3][2]};
+#pragma unroll
+    for (int i = 0; i < 3; ++i)
+      reinterpret_cast<uint2*>(dst)[i] = make_uint2(pack2(f[4 * i], f[4 * i + 1]), pack2(f[4 * i + 2], f[4 * i + 3]));
   }
 }
 
