@@ -460,6 +460,10 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
     }
     CU(launch_finalize(d, qk0, y2, w->temp, rope, q, k, rnorm, st));
     h->launches++;
+  } else if (h->impl >= 1 && !(c.flags & (CCA_CONV1 | CCA_CONV2)) && (d.dh == 64 || d.dh == 128)) {
+    // no convolution at all (the plain GQA / MHA configurations): the per-(token, head) stages read qk0 directly
+    CU(launch_finalize(d, qk0, qk0, w->temp, rope, q, k, rnorm, st));
+    h->launches++;
   } else {
     bool done = false;
     if (h->impl >= 1 && h->tc) {
