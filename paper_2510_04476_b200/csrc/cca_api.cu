@@ -19,6 +19,8 @@ struct cca_handle {
   long long launches;
   TcState* tc;            // tensor-map cache etc. (may be null if unavailable)
   cudaEvent_t ev_attn_begin, ev_attn_end;   // optional, recorded around the attention kernel
+  cudaStream_t side;                        // the RoPE table is computed here, beside the down-projection
+  cudaEvent_t ev_fork, ev_join;
 };
 
 namespace {
@@ -191,6 +193,7 @@ int cca_init(const cca_config* cfg, int device, cca_handle** out) {
   h->d_status = nullptr;
   h->tc = nullptr;
   h->ev_attn_begin = h->ev_attn_end = nullptr;
+  h->side = nullptr; h->ev_fork = h->ev_join = nullptr;
   if (device >= 0) {
     if (cudaMalloc(&h->d_status, 64) != cudaSuccess || cudaMemset(h->d_status, 0, 64) != cudaSuccess) {
       if (h->d_status) cudaFree(h->d_status);
@@ -198,6 +201,12 @@ int cca_init(const cca_config* cfg, int device, cca_handle** out) {
       return CCA_ERR_CUDA;
     }
     h->tc = tc_create(h->sm_count);
+    if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+      (void)cudaGetLastError();
+      h->side = nullptr;                      // everything then runs on the caller's stream
+    }
   }
   *out = h;
   return CCA_OK;
@@ -206,6 +215,11 @@ int cca_init(const cca_config* cfg, int device, cca_handle** out) {
 int cca_destroy(cca_handle* h) {
   if (!h) return CCA_ERR_INVALID_ARG;
   if (h->tc) tc_destroy(h->tc);
+  if (h->side) {
+    cudaStreamDestroy(h->side);
+    cudaEventDestroy(h->ev_fork);
+    cudaEventDestroy(h->ev_join);
+  }
   if (h->d_status) cudaFree(h->d_status);
   delete h;
   return CCA_OK;
@@ -399,8 +413,18 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   // fp32 copy of o for the backward, kept only if the caller's workspace has the backward region
   float* o32 = workspace_bytes >= l.total_end ? (float*)(ws + l.o32) : nullptr;
 
+  // The RoPE table does not depend on x: it is computed on a side stream while the down-projection runs.
+  bool forked = false;
   if (c.flags & CCA_ROPE) {
-    CU(launch_rope_table(rope, d.S, d.dh, c.rope_base, st));
+    if (h->side) {
+      CU(cudaEventRecord(h->ev_fork, st));
+      CU(cudaStreamWaitEvent(h->side, h->ev_fork, 0));
+      CU(launch_rope_table(rope, d.S, d.dh, c.rope_base, h->side));
+      CU(cudaEventRecord(h->ev_join, h->side));
+      forked = true;
+    } else {
+      CU(launch_rope_table(rope, d.S, d.dh, c.rope_base, st));
+    }
     h->launches++;
   }
   // the three down-projection weights stacked (also the B operand of the input gradient in the backward)
@@ -441,6 +465,7 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
     if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
   }
   // Eq. 8, 9, 11: convs, q-k-mean, norm, temperature, RoPE
+  if (forked) CU(cudaStreamWaitEvent(st, h->ev_join, 0));
   if (d.dh > 128) {
     // unfused: conv1 at the taps conv2 reads, conv2 as one contraction per head over (input channel, tap), then the
     // per-(token, head) stages
