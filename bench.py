@@ -34,7 +34,7 @@ FALLBACK_PEAK_TFLOPS = 1590.0
 TRAIN_WORKLOADS = {"cfg2_small", "cfg4_train"}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the attention-forward kernel as it stands, from
 # the full ncu capture summarised under profiles/ (set to None when the kernel changes until it is re-captured)
-ATTN_FWD_DRAM_BYTES = {"cfg3_prefill16k": 50396672 + 2499840}
+ATTN_FWD_DRAM_BYTES = {"cfg3_prefill16k": 50386432 + 2622464}
 
 
 def flops_of(sh, backward: bool):
