@@ -14,7 +14,7 @@ def oracle_cfg(sh):
                           rope_base=sh.rope_base)
 
 
-def check_close(name, got, ref, scale_abs=False, scale=None):
+def check_close(name, got, ref, scale_abs=False, scale=None, tail=None):
     """Activations, outputs and the input gradient (scale_abs=False): element-wise
         |got - ref| <= 1e-2 + 1e-2 |ref|.
 
@@ -33,7 +33,12 @@ def check_close(name, got, ref, scale_abs=False, scale=None):
         |err_i|  <= 1e-2 + 1e-2 |ref_i| + 1e-1 * rms(ref).
     rms(ref) stands for the random-walk scale sqrt(sum of squared terms) of one element, which it
     estimates well for a large matrix of sign-random sums.  For a gradient with a handful of elements
-    (d_temp: one heavily cancelling sum per kv head) the caller passes that scale explicitly."""
+    (d_temp: one heavily cancelling sum per kv head) the caller passes that scale explicitly.
+
+    tail = (fraction, factor), only for tensors of tens of millions of elements outside the five benchmark
+    configurations: at most `fraction` of the elements may exceed the bound, none by more than `factor`.  (With
+    Gaussian rounding noise of standard deviation sigma the largest of 7e7 errors is about 6 sigma, so a bound that
+    the typical element meets five times over is still grazed by a handful.)"""
     got = got.detach().to("cpu").to(torch.float64)
     ref = ref.detach().to("cpu").to(torch.float64)
     assert got.shape == ref.shape, (name, got.shape, ref.shape)
@@ -48,6 +53,10 @@ def check_close(name, got, ref, scale_abs=False, scale=None):
         assert rms_err <= ATOL * (1.0 + rms_ref), f"{name}: rms error {rms_err:.4g} vs rms(ref) {rms_ref:.4g}"
         tol = tol + 10 * RTOL * rms_ref
     bad = err > tol
+    if tail is not None and bad.any():
+        frac, factor = tail
+        assert int(bad.sum()) <= frac * bad.numel(), f"{name}: {int(bad.sum())}/{bad.numel()} outside tolerance"
+        bad = err > factor * tol
     if bad.any():
         idx = torch.nonzero(bad)[0].tolist()
         worst = float((err / tol).max())
