@@ -141,10 +141,23 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
                  void* workspace, size_t workspace_bytes, void* d_x,
                  const cca_weight_grads* grads, int64_t B, int64_t S, void* cuda_stream);
 
+/* Chunked prefill of one causal sequence: tokens [t_begin, t_end) of a sequence of S_total tokens, given that the
+ * tokens before t_begin have been through this function (or cca_forward) with the same workspace, which holds their
+ * latents.  Eq. 7-11 are causal, so a chunk needs nothing of the tokens after it: out_chunk equals rows
+ * [t_begin, t_end) of cca_forward on the whole sequence.  x_chunk, out_chunk: device bf16 [t_end - t_begin, E].
+ * workspace: as for cca_forward(1, S_total) without the backward part; nothing is kept for a backward (the
+ * log-sum-exp region is scratch here).  Chunks are processed in order of position on one stream.
+ * Limits: t_begin a multiple of 256, at least 512 tokens per chunk, causal = 1, conv2 on, head_dim 64 or 128, the
+ * tensor-core kernels enabled; otherwise UNSUPPORTED (use cca_forward).  Errors: as cca_forward. */
+int cca_forward_chunk(cca_handle* h, const cca_weights* w, const void* x_chunk, void* out_chunk, void* workspace,
+                      size_t workspace_bytes, int64_t S_total, int64_t t_begin, int64_t t_end, void* cuda_stream);
+
 /* Same block, host buffers: copies x (host, ideally pinned) to a staging area inside the
  * workspace, runs cca_forward, copies out back to `out_host`, and synchronises the stream.
  * workspace must be >= cca_workspace_size(h, B, S, 0, ..) + 2 * round_up(B*S*E*2, 256) bytes; nothing is kept
- * for a backward. */
+ * for a backward.  One long causal sequence (B = 1, S a multiple of 2048) goes through as a pipeline of
+ * cca_forward_chunk calls with the copies on two streams of the handle's own (created on the first such call), so
+ * that the transfers in both directions overlap the compute. */
 int cca_forward_host(cca_handle* h, const cca_weights* w, const void* x_host, void* out_host,
                      void* workspace, size_t workspace_bytes, int64_t B, int64_t S,
                      void* cuda_stream);

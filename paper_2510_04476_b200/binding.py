@@ -62,6 +62,8 @@ SYMBOLS = {
                                C.c_void_p, C.POINTER(cca_weight_grads), C.c_int64, C.c_int64, C.c_void_p]),
     "cca_forward_host": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_size_t, C.c_int64, C.c_int64, C.c_void_p]),
+    "cca_forward_chunk": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                    C.c_int64, C.c_int64, C.c_int64, C.c_void_p]),
     "cca_forward_static": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
                                      C.c_void_p]),
     "cca_attention_forward": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -221,6 +223,20 @@ class CCA:
         st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
         _check(self.lib, self.lib.cca_forward(self.handle, C.byref(cw), _ptr(x), _ptr(out), wp, wn, B, S, st),
                self.handle, "cca_forward")
+        return out
+
+    def forward_chunk(self, w, x_chunk: torch.Tensor, workspace: torch.Tensor, S_total: int, t_begin: int,
+                      out: Optional[torch.Tensor] = None):
+        """cca_forward_chunk: tokens [t_begin, t_begin + len(x_chunk)) of one causal sequence of S_total tokens."""
+        n, E = x_chunk.shape
+        assert x_chunk.is_cuda and x_chunk.is_contiguous() and x_chunk.dtype == torch.bfloat16
+        if out is None:
+            out = torch.empty_like(x_chunk)
+        cw = self._weights(w)
+        wp, wn = self._ws_ptr(workspace)
+        st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+        _check(self.lib, self.lib.cca_forward_chunk(self.handle, C.byref(cw), _ptr(x_chunk), _ptr(out), wp, wn, S_total,
+                                                    t_begin, t_begin + n, st), self.handle, "cca_forward_chunk")
         return out
 
     def forward_host(self, w, x_host: torch.Tensor, out_host: torch.Tensor, workspace: torch.Tensor):

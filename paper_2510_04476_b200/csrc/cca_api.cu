@@ -21,6 +21,10 @@ struct cca_handle {
   cudaEvent_t ev_attn_begin, ev_attn_end;   // optional, recorded around the attention kernel
   cudaStream_t side;                        // the RoPE table is computed here, beside the down-projection
   cudaEvent_t ev_fork, ev_join;
+  // cca_forward_host, chunked: copies in and out run on their own streams beside the compute
+  cudaStream_t s_in, s_out;
+  cudaEvent_t ev_chunk[2][64];              // [arrived / computed][chunk]
+  int n_ev;                                 // events created so far
 };
 
 namespace {
@@ -194,6 +198,7 @@ int cca_init(const cca_config* cfg, int device, cca_handle** out) {
   h->tc = nullptr;
   h->ev_attn_begin = h->ev_attn_end = nullptr;
   h->side = nullptr; h->ev_fork = h->ev_join = nullptr;
+  h->s_in = h->s_out = nullptr; h->n_ev = 0;
   if (device >= 0) {
     if (cudaMalloc(&h->d_status, 64) != cudaSuccess || cudaMemset(h->d_status, 0, 64) != cudaSuccess) {
       if (h->d_status) cudaFree(h->d_status);
@@ -215,6 +220,12 @@ int cca_init(const cca_config* cfg, int device, cca_handle** out) {
 int cca_destroy(cca_handle* h) {
   if (!h) return CCA_ERR_INVALID_ARG;
   if (h->tc) tc_destroy(h->tc);
+  if (h->s_in) cudaStreamDestroy(h->s_in);
+  if (h->s_out) cudaStreamDestroy(h->s_out);
+  for (int i = 0; i < h->n_ev; ++i) {
+    cudaEventDestroy(h->ev_chunk[0][i]);
+    cudaEventDestroy(h->ev_chunk[1][i]);
+  }
   if (h->side) {
     cudaStreamDestroy(h->side);
     cudaEventDestroy(h->ev_fork);
@@ -514,6 +525,82 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   return CCA_OK;
 }
 
+// Tokens [t_begin, t_end) of one causal sequence of S_total tokens whose earlier tokens have been through this function
+// (or cca_forward) with the same workspace: see the header.
+int cca_forward_chunk(cca_handle* h, const cca_weights* w, const void* x_chunk, void* out_chunk, void* workspace,
+                      size_t workspace_bytes, int64_t S_total, int64_t t_begin, int64_t t_end, void* cuda_stream) {
+  int r = check_sizes(h, 1, S_total, true);
+  if (r != CCA_OK) return r;
+  if (!w || !x_chunk || !out_chunk || !workspace) return CCA_ERR_INVALID_ARG;
+  if (!w->w_qk || !w->w_v1 || !w->w_v2 || !w->w_o) return CCA_ERR_INVALID_ARG;
+  if (t_begin < 0 || t_begin >= t_end || t_end > S_total || t_begin % 256) return CCA_ERR_INVALID_ARG;
+  const cca_config& c = h->cfg;
+  if ((c.flags & CCA_CONV1) && !w->conv0_w) return CCA_ERR_INVALID_ARG;
+  if (!w->conv1_w || ((c.flags & CCA_QK_NORM) && !w->temp)) return CCA_ERR_INVALID_ARG;
+  // the tensor-core kernels only: causal, fused conv2, head size 64 or 128, at least 512 tokens per chunk
+  if (!c.causal || !(c.flags & CCA_CONV2) || (c.head_dim != 64 && c.head_dim != 128) || h->impl < 1 || !h->tc ||
+      t_end - t_begin < 512)
+    return CCA_ERR_UNSUPPORTED;
+  if (!aligned16(x_chunk) || !aligned16(out_chunk) || !aligned16(w->w_qk) || !aligned16(w->w_v1) || !aligned16(w->w_v2) ||
+      !aligned16(w->w_o) || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CCA_ERR_ALIGNMENT;
+  Layout l = make_layout(c, 1, S_total);
+  if (workspace_bytes < l.saved_end) return CCA_ERR_WORKSPACE_TOO_SMALL;
+  CU(cudaSetDevice(h->device));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CcaDims d = make_dims(c, 1, t_end);            // the sequence as far as it exists now
+  const int M = (int)(t_end - t_begin);
+  char* ws = (char*)workspace;
+  float* qk0 = (float*)(ws + l.qk0);
+  bf16* q = (bf16*)(ws + l.q);
+  bf16* k = (bf16*)(ws + l.k);
+  bf16* v = (bf16*)(ws + l.v);
+  bf16* o = (bf16*)(ws + l.o);
+  float* lse = (float*)(ws + l.lse);
+  float2* rope = (float2*)(ws + l.rope);
+  float* rnorm = (float*)(ws + l.rnorm);
+  if (t_begin == 0 && (c.flags & CCA_ROPE)) {
+    CU(launch_rope_table(rope, (int)S_total, d.dh, c.rope_base, st));
+    h->launches++;
+  }
+  const bf16* w_all = (const bf16*)w->w_qk;
+  if (!adjacent(w->w_qk, w->w_v1, w->w_v2, d.L, d.Lk / 2, (size_t)d.E * 2)) {
+    bf16* ws_all = (bf16*)(ws + l.w_all);
+    CU(cudaMemcpyAsync(ws_all, w->w_qk, (size_t)d.L * d.E * 2, cudaMemcpyDeviceToDevice, st));
+    CU(cudaMemcpyAsync(ws_all + (size_t)d.L * d.E, w->w_v1, (size_t)(d.Lk / 2) * d.E * 2, cudaMemcpyDeviceToDevice, st));
+    CU(cudaMemcpyAsync(ws_all + (size_t)(d.L + d.Lk / 2) * d.E, w->w_v2, (size_t)(d.Lk / 2) * d.E * 2,
+                       cudaMemcpyDeviceToDevice, st));
+    w_all = ws_all;
+  }
+  // Eq. 7 and Eq. 10 for the chunk's rows; the value-shifted half of row t_end goes to the next chunk's first row
+  GemmArgs g{};
+  g.A = kmajor(x_chunk, d.E); g.B = kmajor(w_all, d.E);
+  g.M = M; g.N = d.L + d.Lk; g.K = d.E; g.seq_len = (int)S_total; g.row0 = (int)t_begin;
+  g.out_bf16 = v + (size_t)t_begin * d.Lk; g.out_f32 = qk0 + (size_t)t_begin * d.L; g.ldc = d.L;
+  g.split_L = d.L; g.split_Lk = d.Lk; g.split_shift = (c.flags & CCA_V_SHIFT) ? 1 : 0;
+  int pr = tc_gemm_pair(h->tc, g, h->d_status, st);
+  if (pr < 0) { h->last_cuda = -pr; return CCA_ERR_CUDA; }
+  if (pr != 0) return CCA_ERR_UNSUPPORTED;
+  h->launches++;
+  int tr = tc_transform_fwd(h->tc, d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k, rnorm,
+                            h->d_status, st, (int)t_begin);
+  if (tr < 0) { h->last_cuda = -tr; return CCA_ERR_CUDA; }
+  if (tr != 0) return CCA_ERR_UNSUPPORTED;
+  h->launches++;
+  if (h->ev_attn_begin) CU(cudaEventRecord(h->ev_attn_begin, st));
+  int ar = tc_attn_fwd(h->tc, d, q, k, v, o, nullptr, lse, (c.flags & CCA_QK_NORM) ? w->temp : nullptr, h->d_status, st,
+                       (int)t_begin);
+  if (ar < 0) { h->last_cuda = -ar; return CCA_ERR_CUDA; }
+  if (ar != 0) return CCA_ERR_UNSUPPORTED;
+  h->launches++;
+  if (h->ev_attn_end) CU(cudaEventRecord(h->ev_attn_end, st));
+  g = GemmArgs{};
+  g.A = kmajor(o + (size_t)t_begin * d.Lq, d.Lq); g.B = kmajor(w->w_o, d.Lq);
+  g.M = M; g.N = d.E; g.K = d.Lq; g.seq_len = M;
+  g.out_bf16 = (bf16*)out_chunk; g.ldc = d.E;
+  return run_gemm(h, g, st);
+}
+
 int cca_forward_host(cca_handle* h, const cca_weights* w, const void* x_host, void* out_host, void* workspace,
                      size_t workspace_bytes, int64_t B, int64_t S, void* cuda_stream) {
   int r = check_sizes(h, B, S, true);
@@ -526,6 +613,53 @@ int cca_forward_host(cca_handle* h, const cca_weights* w, const void* x_host, vo
   cudaStream_t st = (cudaStream_t)cuda_stream;
   char* xs = (char*)workspace + l.saved_end;
   char* os = xs + act;
+  // One causal sequence that the tensor-core kernels cover: chunks of the sequence go through the copy engines and
+  // the kernels as a pipeline (tokens in on one stream, compute on the caller's, results out on a third), since a
+  // chunk needs nothing of the tokens after it.
+  const cca_config& c = h->cfg;
+  const int64_t CH = 2048;
+  if (B == 1 && S >= 2 * CH && S % CH == 0 && S / CH <= 64 && c.causal && (c.flags & CCA_CONV2) &&
+      (c.head_dim == 64 || c.head_dim == 128) && h->impl >= 1 && h->tc) {
+    if (!h->s_in) {
+      if (cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking) != cudaSuccess ||
+          cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking) != cudaSuccess) {
+        (void)cudaGetLastError();
+        if (h->s_in) cudaStreamDestroy(h->s_in);
+        h->s_in = h->s_out = nullptr;
+      }
+    }
+    const int n_ch = (int)(S / CH);
+    while (h->s_in && h->n_ev < n_ch) {
+      if (cudaEventCreateWithFlags(&h->ev_chunk[0][h->n_ev], cudaEventDisableTiming) != cudaSuccess) break;
+      if (cudaEventCreateWithFlags(&h->ev_chunk[1][h->n_ev], cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventDestroy(h->ev_chunk[0][h->n_ev]);
+        break;
+      }
+      h->n_ev++;
+    }
+    if (h->s_in && h->n_ev >= n_ch) {
+      const size_t row = (size_t)c.d_model * 2;
+      // the copy streams start after whatever the caller's stream has queued so far
+      CU(cudaEventRecord(h->ev_chunk[1][0], st));
+      CU(cudaStreamWaitEvent(h->s_in, h->ev_chunk[1][0], 0));
+      CU(cudaStreamWaitEvent(h->s_out, h->ev_chunk[1][0], 0));
+      for (int i = 0; i < n_ch; ++i) {
+        const size_t off = (size_t)i * CH * row;
+        CU(cudaMemcpyAsync(xs + off, (const char*)x_host + off, (size_t)CH * row, cudaMemcpyHostToDevice, h->s_in));
+        CU(cudaEventRecord(h->ev_chunk[0][i], h->s_in));
+        CU(cudaStreamWaitEvent(st, h->ev_chunk[0][i], 0));
+        r = cca_forward_chunk(h, w, xs + off, os + off, workspace, l.saved_end, S, (int64_t)i * CH, (int64_t)(i + 1) * CH,
+                              cuda_stream);
+        if (r != CCA_OK) return r;
+        CU(cudaEventRecord(h->ev_chunk[1][i], st));
+        CU(cudaStreamWaitEvent(h->s_out, h->ev_chunk[1][i], 0));
+        CU(cudaMemcpyAsync((char*)out_host + off, os + off, (size_t)CH * row, cudaMemcpyDeviceToHost, h->s_out));
+      }
+      CU(cudaStreamSynchronize(h->s_out));
+      CU(cudaStreamSynchronize(st));
+      return CCA_OK;
+    }
+  }
   CU(cudaMemcpyAsync(xs, x_host, (size_t)B * S * h->cfg.d_model * 2, cudaMemcpyHostToDevice, st));
   r = cca_forward(h, w, xs, os, workspace, l.saved_end, B, S, cuda_stream);
   if (r != CCA_OK) return r;

@@ -42,6 +42,7 @@ struct GemmArgs {
   float* out_f32;
   long long ldc;
   int split_L, split_Lk, split_shift;
+  int row0;          // fused output only: position inside its sequence of row 0 of A (a chunk of a longer sequence)
 };
 
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);

@@ -84,7 +84,7 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
   // work item: heavy (late) query blocks first
   const int per_blk = p.B * p.hq;
-  const int blk = p.n_blocks - 1 - (int)(blockIdx.x / per_blk);
+  const int blk = p.blk0 + p.n_blocks - 1 - (int)(blockIdx.x / per_blk);
   const int rem = blockIdx.x % per_blk;
   const int b = rem / p.hq, hi = rem % p.hq, hj = hi / p.g;
   const int n_kv_total = (p.S + BKV - 1) / BKV;
@@ -420,7 +420,8 @@ int launch_attn(TcState* s, const CUtensorMap& tmQ, const CUtensorMap& tmK, cons
 }  // namespace
 
 int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* o32,
-                float* lse, const float* temp, int* d_status, cudaStream_t st) {
+                float* lse, const float* temp, int* d_status, cudaStream_t st, int t_first) {
+  if (t_first % 256 || t_first < 0 || t_first >= d.S) return 1;
   if (!s || !s->encode) return 1;
   if (d.dh != 64 && d.dh != 128) return 1;
   if (d.Lq % 8 || d.Lk % 8) return 1;
@@ -434,7 +435,8 @@ int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, cons
   AttnParams p;
   p.B = d.B; p.S = d.S; p.hq = d.hq; p.hk = d.hk; p.g = d.g; p.Lq = d.Lq; p.Lk = d.Lk; p.causal = d.causal;
   p.o = o; p.o32 = o32; p.lse = lse;
-  p.n_blocks = (d.S + 255) / 256;
+  p.blk0 = t_first / 256;
+  p.n_blocks = (d.S - t_first + 255) / 256;
   p.status = d_status;
   const long long grid = (long long)p.n_blocks * d.B * d.hq;
   if (grid > 0x7fffffffLL) return 1;

@@ -360,6 +360,7 @@ int tc_attn_fwd256(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, c
   AttnParams p;
   p.B = d.B; p.S = d.S; p.hq = d.hq; p.hk = d.hk; p.g = d.g; p.Lq = d.Lq; p.Lk = d.Lk; p.causal = d.causal;
   p.o = o; p.o32 = o32; p.lse = lse;
+  p.blk0 = 0;
   p.n_blocks = (d.S + BQ6 - 1) / BQ6;
   p.status = d_status;
   p.temp = temp;

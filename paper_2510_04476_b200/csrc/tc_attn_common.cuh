@@ -15,7 +15,8 @@ struct AttnParams {
   bf16* o;
   float* o32;
   float* lse;
-  int n_blocks;       // 256-row blocks per sequence
+  int n_blocks;       // query blocks per sequence that this launch covers
+  int blk0;           // first of them (0: whole sequences)
   int* status;
   const float* temp;  // log key temperature per kv head if q, k are L2-normalised (Eq. 11), else null
 };

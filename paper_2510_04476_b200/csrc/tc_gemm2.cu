@@ -33,7 +33,7 @@ struct G2Params {
   int a_mn, b_mn;
   int splits, kb_per_split;   // work item = (tile, split)
   int vec_ok;
-  int split_L, split_Lk, split_shift, seq_len;   // fused down-projection output (see GemmArgs)
+  int split_L, split_Lk, split_shift, seq_len, row0;   // fused down-projection output (see GemmArgs)
   int* status;
 };
 
@@ -235,7 +235,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             } else {
               const int vc = n - p.split_L;
               const bool late = p.split_shift && vc >= p.split_Lk / 2;
-              const int t = m % p.seq_len;
+              const int t = (m + p.row0) % p.seq_len;
               bf16* dst = p.out_bf16 + (long long)(m + (late ? 1 : 0)) * p.split_Lk + vc;
               if (!late || t + 1 < p.seq_len) {
 #pragma unroll
@@ -420,6 +420,7 @@ int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) 
   const int esz = g.out_bf16 ? 2 : 4;
   p.vec_ok = ((reinterpret_cast<uintptr_t>(outp) & 15) == 0) && ((g.ldc * esz) % 16 == 0);
   p.split_L = g.split_L; p.split_Lk = g.split_Lk; p.split_shift = g.split_shift; p.seq_len = g.seq_len > 0 ? g.seq_len : 1;
+  p.row0 = g.row0;
   p.status = d_status;
   // tile width: fewer, fuller waves of CTA pairs win (time of a wave is proportional to the tile width)
   auto cost = [&](int bn) {

@@ -11,8 +11,9 @@ void tc_destroy(TcState* s);
 int tc_gemm(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st);
 // Same contraction on CTA pairs (256 x 256 tiles); covers large K-major-A cases only.
 int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st);
+// t_first > 0 (a multiple of 256): only the query rows [t_first, d.S) of every sequence; keys and values [0, d.S).
 int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* o32,
-                float* lse, const float* temp, int* d_status, cudaStream_t st);
+                float* lse, const float* temp, int* d_status, cudaStream_t st, int t_first = 0);
 // Head size 256 (one query tile per CTA, score buffers alternate over key tiles).
 int tc_attn_fwd256(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o, float* o32, float* lse,
                    const float* temp, int* d_status, cudaStream_t st);
@@ -24,4 +25,4 @@ int tc_transform_bwd(TcState* s, const CcaDims& d, const float* qk0, const bf16*
                      const float* dkh, float* dy1, float* d_w1, int* d_status, cudaStream_t st);
 int tc_transform_fwd(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
                      const float* temp, const float2* rope, bf16* q, bf16* k, float* rnorm, int* d_status,
-                     cudaStream_t st);
+                     cudaStream_t st, int t_first = 0);   // t_first > 0 (multiple of 128): only tokens [t_first, d.S)

@@ -64,7 +64,8 @@ struct TrParams {
   bf16* k;
   float* rnorm;         // [B*S, hq+hk] norm scale kept for the backward
   int* status;
-  int n_tiles;          // 128-token tiles per sequence
+  int n_tiles;          // 128-token tiles per sequence (of the token range that is processed)
+  int t_first;          // first token of that range (0: whole sequences)
   int units_per_head;   // B * n_tiles
   int total_units;
   int cost_q, cost_k;   // relative cost of a unit of a q head / of a kv head (kv units read g more rows)
@@ -141,7 +142,7 @@ __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const T
     int it = 0;
     for (int u = u_begin; u < u_end; ++u, ++it) {
       const int h = u / p.units_per_head, rem = u % p.units_per_head;
-      const int b = rem / p.n_tiles, t0 = (rem % p.n_tiles) * 128;
+      const int b = rem / p.n_tiles, t0 = p.t_first + (rem % p.n_tiles) * 128;
       const bool is_q = h < d.hq;
       const int hj = is_q ? h / d.g : h - d.hq;
       const int ch = h * DH + cq;
@@ -343,7 +344,7 @@ __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const T
     int it = 0;
     for (int u = u_begin; u < u_end; ++u, ++it) {
       const int h = u / p.units_per_head, rem = u % p.units_per_head;
-      const int b = rem / p.n_tiles, t0 = (rem % p.n_tiles) * 128;
+      const int b = rem / p.n_tiles, t0 = p.t_first + (rem % p.n_tiles) * 128;
       const bool is_q = h < d.hq;
       const int hj = is_q ? h / d.g : h - d.hq;
       const int buf = it & 1;
@@ -461,7 +462,7 @@ done:
 
 template <int DH, int KC>
 int launch_tr(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1, const float* temp,
-              const float2* rope, bf16* q, bf16* k, float* rnorm, int* status, cudaStream_t st) {
+              const float2* rope, bf16* q, bf16* k, float* rnorm, int t_first, int* status, cudaStream_t st) {
   static bool attr_done = false;
   using SM = TrSmem<DH, KC>;
   if (!attr_done) {
@@ -471,7 +472,8 @@ int launch_tr(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, co
   }
   TrParams p;
   p.d = d; p.qk0 = qk0; p.w0 = w0; p.w1 = w1; p.temp = temp; p.rope = rope; p.q = q; p.k = k; p.rnorm = rnorm; p.status = status;
-  p.n_tiles = (d.S + 127) / 128;
+  p.t_first = t_first;
+  p.n_tiles = (d.S - t_first + 127) / 128;
   const long long uph = (long long)d.B * p.n_tiles, total = uph * (d.hq + d.hk);
   if (total > 0x7fffffffLL) return 1;
   p.units_per_head = (int)uph;
@@ -488,21 +490,22 @@ int launch_tr(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, co
 
 int tc_transform_fwd(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
                      const float* temp, const float2* rope, bf16* q, bf16* k, float* rnorm, int* d_status,
-                     cudaStream_t st) {
+                     cudaStream_t st, int t_first) {
+  if (t_first % 128 || t_first < 0 || t_first >= d.S) return 1;
   if (!s || s->sm_count < 1) return 1;
   if (!(d.flags & F_CONV2)) return 1;                 // no contraction to run: the SIMT kernel is the right tool
   if (d.L % 4 || d.Lq % 8 || d.Lk % 8) return 1;
   if ((reinterpret_cast<uintptr_t>(w1) & 15) || (reinterpret_cast<uintptr_t>(qk0) & 15)) return 1;
   if (d.dh == 128) {
-    if (d.k_ch == 1) return launch_tr<128, 1>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
-    if (d.k_ch == 2) return launch_tr<128, 2>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
+    if (d.k_ch == 1) return launch_tr<128, 1>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, t_first, d_status, st);
+    if (d.k_ch == 2) return launch_tr<128, 2>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, t_first, d_status, st);
     return 1;
   }
   if (d.dh == 64) {
-    if (d.k_ch == 1) return launch_tr<64, 1>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
-    if (d.k_ch == 2) return launch_tr<64, 2>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
-    if (d.k_ch == 3) return launch_tr<64, 3>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
-    if (d.k_ch == 4) return launch_tr<64, 4>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, d_status, st);
+    if (d.k_ch == 1) return launch_tr<64, 1>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, t_first, d_status, st);
+    if (d.k_ch == 2) return launch_tr<64, 2>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, t_first, d_status, st);
+    if (d.k_ch == 3) return launch_tr<64, 3>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, t_first, d_status, st);
+    if (d.k_ch == 4) return launch_tr<64, 4>(s, d, qk0, w0, w1, temp, rope, q, k, rnorm, t_first, d_status, st);
   }
   return 1;
 }

@@ -305,3 +305,71 @@ def test_head_size_256_at_16k_sampled_rows():
     check_close("lse_rows", sv["lse"][:, :, rows], lse_ref)
     check_close("out_rows", out[:, rows], out_ref)
     cca.close()
+
+
+# ------------------------------------------------------------------ chunked prefill
+@pytest.mark.parametrize("sh,cuts", [(S_("chunk_dh64", 1, 2304, 512, 8, 2, 64), [0, 1024, 1792, 2304]),
+                                     (S_("chunk_dh128_ragged_end", 1, 1900, 1024, 8, 2, 128), [0, 768, 1900]),
+                                     (S_("chunk_no_shift_k3", 1, 1536, 512, 8, 2, 64, flags=63 & ~8, k_seq=3), [0, 512, 1536])],
+                         ids=lambda v: v.name if hasattr(v, "name") else "cuts")
+def test_chunked_prefill_equals_whole_sequence(sh, cuts):
+    """Chunks of one causal sequence fed in order reproduce the whole-sequence forward (oracle and library)."""
+    t = synth.make_inputs(sh, want_dout=False)
+    out_ref, I = O.forward(oracle_cfg(sh), t, t["x"])
+    dev = to_device(t)
+    cca = _cca(sh)
+    ws = cca.alloc_workspace(1, sh.S, False)
+    whole = cca.forward(dev, dev["x"], ws).clone()
+    ws2 = cca.alloc_workspace(1, sh.S, False)
+    ws2.zero_()
+    parts = []
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        parts.append(cca.forward_chunk(dev, dev["x"][0, a:b].contiguous(), ws2, sh.S, a))
+    torch.cuda.synchronize()
+    assert cca.last_status() == 0
+    out = torch.cat(parts, dim=0)[None]
+    check_close("out", out, out_ref)
+    sv = cca.saved(ws2, 1, sh.S)
+    for n in ("q", "k", "v", "o"):
+        check_close(n, sv[n].reshape(I[n].shape), I[n])
+    assert torch.equal(out, whole)                      # same kernels, same operands, row by row
+    cca.close()
+
+
+def test_chunked_prefill_argument_checks():
+    from paper_2510_04476_b200.binding import CcaError
+    sh = S_("chunk_args", 1, 2048, 512, 8, 2, 64)
+    t = synth.make_inputs(sh, want_dout=False)
+    dev = to_device(t)
+    cca = _cca(sh)
+    ws = cca.alloc_workspace(1, sh.S, False)
+    x = dev["x"][0]
+    with pytest.raises(CcaError):
+        cca.forward_chunk(dev, x[100:1000].contiguous(), ws, sh.S, 100)        # start not on a 256-token boundary
+    with pytest.raises(CcaError):
+        cca.forward_chunk(dev, x[0:256].contiguous(), ws, sh.S, 0)             # fewer than 512 tokens
+    with pytest.raises(CcaError):
+        cca.forward_chunk(dev, x[1024:2048].contiguous(), ws, 1536, 1024)      # runs past the sequence
+    nc = _cca(sh.replace(causal=0))
+    with pytest.raises(CcaError):
+        nc.forward_chunk(dev, x[0:1024].contiguous(), ws, sh.S, 0)             # needs the keys after the chunk
+    nc.close()
+    cca.close()
+
+
+def test_forward_host_pipeline_equals_device_forward():
+    """One long causal sequence from host memory goes through as a pipeline of chunks; same result as cca_forward."""
+    sh = S_("host_pipeline", 1, 6144, 512, 8, 2, 64)
+    t = synth.make_inputs(sh, want_dout=False)
+    dev = to_device(t)
+    cca = _cca(sh)
+    ws = cca.alloc_workspace(1, sh.S, False, extra=2 * sh.S * sh.d_model * 2 + 1024)
+    ref = cca.forward(dev, dev["x"], ws).cpu()
+    xh = t["x"].pin_memory()
+    oh = torch.empty_like(t["x"]).pin_memory()
+    for _ in range(2):                                   # the second call reuses the handle's streams and events
+        oh.zero_()
+        cca.forward_host(dev, xh, oh, ws)
+        assert torch.equal(oh, ref)
+    assert cca.last_status() == 0
+    cca.close()
