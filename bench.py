@@ -34,6 +34,7 @@ FALLBACK_PEAK_TFLOPS = 1590.0
 TRAIN_WORKLOADS = {"cfg2_small", "cfg4_train"}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the attention-forward kernel as it stands, from
 # the full ncu capture summarised under profiles/ (set to None when the kernel changes until it is re-captured)
+ATTN_BWD_DRAM_BYTES = {"cfg4_train": 109093632 + 11924736 + 87101184 + 29619456}     # dK/dV kernel + dQ kernel
 ATTN_FWD_DRAM_BYTES = {"cfg3_prefill16k": 50386432 + 2622464}
 
 
@@ -44,7 +45,7 @@ def flops_of(sh, backward: bool):
     attn = (2 if sh.causal else 4) * sh.B * sh.S * sh.S * sh.L_q
     fwd = proj + conv + attn
     total = fwd + (2 * (proj + conv) + 2.5 * attn if backward else 0)
-    return {"total": total, "fwd": fwd, "attn_fwd": attn, "proj": proj, "conv": conv}
+    return {"total": total, "fwd": fwd, "attn_fwd": attn, "attn_bwd": 2.5 * attn, "proj": proj, "conv": conv}
 
 
 def measured_peak():
@@ -269,7 +270,10 @@ def run_ours(args, rank, world, local_rank):
     d2h = act_bytes
 
     peak, peak_kind, _ = measured_peak()
-    attn_tflops = fl["attn_fwd"] / (attn_ms * 1e-3) / 1e12
+    # the events bracket the last attention stage of a step: the forward kernel, or the two adjoint kernels of a
+    # training step (2.5 x the forward's FLOPs: five contractions against two)
+    attn_key = "attn_bwd" if backward else "attn_fwd"
+    attn_tflops = fl[attn_key] / (attn_ms * 1e-3) / 1e12
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -284,11 +288,14 @@ def run_ours(args, rank, world, local_rank):
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "tensor", "kernel": "latent attention forward", "achieved": attn_tflops, "peak": peak,
+        "roofline": {"bound": "tensor",
+                     "kernel": "latent attention backward (dQ and dK/dV kernels)" if backward else "latent attention forward",
+                     "achieved": attn_tflops, "peak": peak,
                      "unit": "TFLOP/s", "frac": attn_tflops / peak, "peak_kind": peak_kind,
                      "frac_of_nominal_2250": attn_tflops / NOMINAL_BF16_TFLOPS, "ms_per_launch": attn_ms,
-                     "flops_per_launch": fl["attn_fwd"],
-                     "traffic": ATTN_FWD_DRAM_BYTES.get(sh.name) if args.kernels else None},
+                     "flops_per_launch": fl[attn_key],
+                     "traffic": ATTN_FWD_DRAM_BYTES.get(sh.name) if args.kernels and not backward else
+                                (ATTN_BWD_DRAM_BYTES.get(sh.name) if args.kernels else None)},
         "pct_of_nominal_bf16_peak": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
         "device_status": status,
     }

@@ -237,7 +237,9 @@ int cca_decode_state_from_prefill(cca_handle* h, const void* x, const void* work
 int cca_set_impl(cca_handle* h, int impl);
 
 /* Profiling hook: two cudaEvent_t (or null to clear) that every later attention stage records on the
- * caller's stream immediately before and after its kernel. */
+ * caller's stream immediately before and after its kernel: the forward attention kernel in cca_forward, the decode
+ * attention kernel in cca_decode_step, the two attention-adjoint kernels (dQ, dK/dV) together in cca_backward,
+ * which therefore overwrites what the forward of the same step recorded. */
 int cca_set_attention_events(cca_handle* h, void* ev_begin, void* ev_end);
 
 /* Number of kernel launches the library has enqueued through this handle so far. */

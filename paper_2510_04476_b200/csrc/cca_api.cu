@@ -724,6 +724,7 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   CU(launch_attn_delta(d, o32, d_o, delta, st));
   h->launches++;
   {
+    if (h->ev_attn_begin) CU(cudaEventRecord(h->ev_attn_begin, st));
     bool done = false;
     if (h->impl >= 1 && h->tc) {
       int tr = tc_attn_bwd(h->tc, d, q, k, v, d_o, lse, delta, dq, dk, dv, h->d_status, st);
@@ -732,6 +733,7 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
     }
     if (!done) CU(launch_attn_bwd_simt(d, q, k, v, o32, d_o, lse, delta, dq, dk, dv, st));
     h->launches += 2;
+    if (h->ev_attn_end) CU(cudaEventRecord(h->ev_attn_end, st));
   }
   // latent-transform adjoints
   CU(launch_transform_bwd_norm(d, q, k, rnorm, w->temp, rope, dq, dk, gr->d_temp, st));
