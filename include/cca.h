@@ -221,7 +221,7 @@ int cca_decode_workspace_size(const cca_handle* h, int64_t B, int64_t max_len, s
  * S_max for every b; it sizes the launch.  A sequence whose pos[b] is outside [0, min(max_len, S_max)) is
  * skipped (its caches, history and output row are left untouched or undefined, nothing is written out of
  * bounds) and the device status word becomes 120, which cca_last_status reports.
- * Needs causal = 1, head_dim in {32,64,128}, L_k and E multiples of 8.  No allocation, no synchronisation.
+ * Needs causal = 1, L_k and E multiples of 8 (at head_dim = 256 at most 8 query heads per kv head).  No allocation, no synchronisation.
  * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE_TOO_SMALL, CUDA. */
 int cca_decode_step(cca_handle* h, const cca_weights* w, const void* x, void* out, const cca_decode_state* state,
                     int64_t max_len, void* workspace, size_t workspace_bytes, int64_t B, void* cuda_stream);

@@ -208,9 +208,10 @@ struct FnArgs {
 };
 
 template <int DH>
-__global__ void __launch_bounds__(128) decode_finalize_kernel(FnArgs a) {
+__global__ void __launch_bounds__(DH < 128 ? 128 : DH) decode_finalize_kernel(FnArgs a) {
+  constexpr int NW = (DH < 128 ? 128 : DH) / 32;      // warps per block
   __shared__ float xh[DH];
-  __shared__ float red[4];
+  __shared__ float red[NW];
   const CcaDims& d = a.d;
   const int b = blockIdx.y, head = blockIdx.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -241,7 +242,9 @@ __global__ void __launch_bounds__(128) decode_finalize_kernel(FnArgs a) {
     for (int s = 16; s > 0; s >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, s);
     if (lane == 0) red[warp] = ssq;
     __syncthreads();
-    const float tot = red[0] + red[1] + red[2] + red[3];
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < NW; ++i) tot += red[i];
     float sc = sqrtf((float)DH) * rsqrtf(tot);
     if (!is_q) sc *= __expf(a.temp[head - d.hq]);
     v *= sc;
@@ -537,9 +540,11 @@ cudaError_t launch_attn_dh(const AtArgs& a, cudaStream_t st) {
   if (d.g <= 8) {
     dim3 grid((unsigned)a.splits, (unsigned)d.hk, (unsigned)d.B);
     decode_attn_kernel<DH, 1><<<grid, DA_WARPS * 32, 0, st>>>(a);
-  } else {
+  } else if constexpr (DH <= 128) {
     dim3 grid((unsigned)a.splits, (unsigned)(d.hk * ((d.g + 15) / 16)), (unsigned)d.B);
     decode_attn_kernel<DH, 2><<<grid, DA_WARPS * 32, 0, st>>>(a);
+  } else {
+    return cudaErrorInvalidValue;          // head size 256: up to 8 query heads per kv head
   }
   return cudaGetLastError();
 }
@@ -595,8 +600,9 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
   bf16* y1s = reinterpret_cast<bf16*>(p); p += up((size_t)d.B * d.L * d.k_ch * 2);
   float* y2 = reinterpret_cast<float*>(p);
   cudaError_t e;
-  if (d.dh != 32 && d.dh != 64 && d.dh != 128) return 1;
+  if (d.dh != 32 && d.dh != 64 && d.dh != 128 && d.dh != 256) return 1;
   if (d.E % 32 || d.Lq % 32) return 1;
+  if (d.dh == 256 && d.g > 8) return 1;
   // Eq. 7 and Eq. 10: q0 | k0 | v1 from x_t, v2 from x_{t-1}
   ProjArgs pa;
   memset(&pa, 0, sizeof(pa));
@@ -633,7 +639,8 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
     switch (d.dh) {
       case 32: decode_finalize_kernel<32><<<grid, 128, 0, st>>>(fa); break;
       case 64: decode_finalize_kernel<64><<<grid, 128, 0, st>>>(fa); break;
-      default: decode_finalize_kernel<128><<<grid, 128, 0, st>>>(fa); break;
+      case 128: decode_finalize_kernel<128><<<grid, 128, 0, st>>>(fa); break;
+      default: decode_finalize_kernel<256><<<grid, 256, 0, st>>>(fa); break;
     }
     if ((e = cudaGetLastError()) != cudaSuccess) return -(int)e;
     ++*launches;
@@ -648,6 +655,7 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
     case 32: e = launch_attn_dh<32>(aa, st); break;
     case 64: e = launch_attn_dh<64>(aa, st); break;
     case 128: e = launch_attn_dh<128>(aa, st); break;
+    case 256: e = launch_attn_dh<256>(aa, st); break;
     default: return 1;
   }
   if (e != cudaSuccess) return -(int)e;
@@ -662,6 +670,7 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
       case 32: decode_combine_kernel<32><<<grid, 64, 0, st>>>(ca); break;
       case 64: decode_combine_kernel<64><<<grid, 64, 0, st>>>(ca); break;
       case 128: decode_combine_kernel<128><<<grid, 128, 0, st>>>(ca); break;
+      case 256: decode_combine_kernel<256><<<grid, 256, 0, st>>>(ca); break;
       default: return 1;
     }
     if ((e = cudaGetLastError()) != cudaSuccess) return -(int)e;

@@ -36,6 +36,8 @@ EMPTY_START = [
     S_("dec_no_norm", 2, 9, 512, 8, 2, 64, flags=63 & ~16),
     S_("dec_no_mean_no_rope", 2, 9, 512, 8, 2, 64, flags=63 & ~4 & ~32),
     S_("dec_batch_over_16", 19, 6, 256, 4, 2, 64),
+    S_("dec_dh256_g2", 2, 25, 1024, 4, 2, 256),
+    S_("dec_dh256_g4_no_norm", 1, 37, 1024, 4, 1, 256, flags=63 & ~16),
 ]
 
 
@@ -67,7 +69,8 @@ def test_decode_from_empty_state_matches_oracle(sh):
 
 @pytest.mark.parametrize("sh,S0", [(S_("dec_prefill_dh64", 2, 712, 512, 8, 2, 64), 700),
                                    (S_("dec_prefill_dh128", 1, 1300, 1024, 8, 2, 128), 1290),
-                                   (S_("dec_prefill_one", 2, 6, 512, 8, 2, 64, k_seq=3, k_ch=3), 1)],
+                                   (S_("dec_prefill_one", 2, 6, 512, 8, 2, 64, k_seq=3, k_ch=3), 1),
+                                   (S_("dec_prefill_dh256", 1, 1034, 1024, 4, 1, 256), 1024)],
                          ids=lambda v: v.name if hasattr(v, "name") else str(v))
 def test_decode_continues_a_gpu_prefill(sh, S0):
     """Prefill S0 tokens with cca_forward, hand the workspace over, decode the rest: every decoded row must
