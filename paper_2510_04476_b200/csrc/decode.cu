@@ -21,6 +21,29 @@
 
 namespace {
 
+// Programmatic dependent launch: every kernel of the step lets the next one be scheduled as soon as all of its own
+// CTAs have started, and waits for the kernel before it (completion and visibility of its writes) before it touches
+// global memory.  The wait comes first in every CTA, also in those that return early, so that "kernel N complete"
+// always implies "kernel N - 1 complete".
+CCA_DEVINL void pdl_enter() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute at;
+  at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 constexpr unsigned F_CONV1 = 1, F_CONV2 = 2, F_QK_MEAN = 4, F_V_SHIFT = 8, F_QK_NORM = 16, F_ROPE = 32;
 constexpr int ST_DECODE_BAD_POSITION = 120;
 constexpr float LOG2E = 1.4426950408889634f;
@@ -59,6 +82,7 @@ struct ProjArgs {
 };
 
 __global__ void __launch_bounds__(PJ_WARPS * 32) decode_proj_kernel(ProjArgs a) {
+  pdl_enter();
   __shared__ float red[PJ_WARPS][PJ_ROWS][PJ_NT * 8 + 1];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -151,6 +175,7 @@ struct C1Args {
 };
 
 __global__ void __launch_bounds__(256) decode_conv1_kernel(C1Args a) {
+  pdl_enter();
   const CcaDims& d = a.d;
   const int b = blockIdx.y, tid = threadIdx.x;
   const int t = a.pos[b];
@@ -209,6 +234,7 @@ struct FnArgs {
 
 template <int DH>
 __global__ void __launch_bounds__(DH < 128 ? 128 : DH) decode_finalize_kernel(FnArgs a) {
+  pdl_enter();
   constexpr int NW = (DH < 128 ? 128 : DH) / 32;      // warps per block
   __shared__ float xh[DH];
   __shared__ float red[NW];
@@ -299,6 +325,7 @@ CCA_DEVINL int pv_channel(int g, int ci) {
 // index = key, output row = whichever channel the lane loaded).
 template <int DH, int NHT>
 __global__ void __launch_bounds__(DA_WARPS * 32) decode_attn_kernel(AtArgs a) {
+  pdl_enter();
   constexpr int CB = DH / 32;                  // 32-channel blocks of Q K^T
   constexpr int VW = DH / 16;                  // 32-bit words per lane per value row = 16-channel tiles of O^T
   const CcaDims& d = a.d;
@@ -507,6 +534,7 @@ struct CbArgs {
 
 template <int DH>
 __global__ void __launch_bounds__(DH < 64 ? 64 : DH) decode_combine_kernel(CbArgs a) {
+  pdl_enter();
   const int hi = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
   const int t = a.pos[b];
   if (t < 0 || t >= a.S_max || t >= a.max_len) return;
@@ -530,8 +558,7 @@ cudaError_t launch_proj(const ProjArgs& a, cudaStream_t st) {
   int tot = 0;
   for (int s = 0; s < a.n_seg; ++s) tot += padded_rows(a.seg[s].rows);
   dim3 grid((unsigned)(tot / PJ_ROWS), (unsigned)((a.B + PJ_NT * 8 - 1) / (PJ_NT * 8)));
-  decode_proj_kernel<<<grid, PJ_WARPS * 32, 0, st>>>(a);
-  return cudaGetLastError();
+  return launch_pdl(decode_proj_kernel, grid, dim3(PJ_WARPS * 32), st, a);
 }
 
 template <int DH>
@@ -539,10 +566,10 @@ cudaError_t launch_attn_dh(const AtArgs& a, cudaStream_t st) {
   const CcaDims& d = a.d;
   if (d.g <= 8) {
     dim3 grid((unsigned)a.splits, (unsigned)d.hk, (unsigned)d.B);
-    decode_attn_kernel<DH, 1><<<grid, DA_WARPS * 32, 0, st>>>(a);
+    return launch_pdl(decode_attn_kernel<DH, 1>, grid, dim3(DA_WARPS * 32), st, a);
   } else if constexpr (DH <= 128) {
     dim3 grid((unsigned)a.splits, (unsigned)(d.hk * ((d.g + 15) / 16)), (unsigned)d.B);
-    decode_attn_kernel<DH, 2><<<grid, DA_WARPS * 32, 0, st>>>(a);
+    return launch_pdl(decode_attn_kernel<DH, 2>, grid, dim3(DA_WARPS * 32), st, a);
   } else {
     return cudaErrorInvalidValue;          // head size 256: up to 8 query heads per kv head
   }
@@ -619,8 +646,8 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
   C1Args c1;
   c1.d = d; c1.lat = lat; c1.x = x; c1.w0 = w.conv0_w; c1.y1s = y1s; c1.y2 = y2; c1.v_cache = s.v_cache;
   c1.hist = s.qk0_hist; c1.x_prev = s.x_prev; c1.pos = s.pos; c1.S_max = s.S_max; c1.max_len = max_len; c1.status = status;
-  decode_conv1_kernel<<<dim3((unsigned)((d.L + 255) / 256), (unsigned)d.B), 256, 0, st>>>(c1);
-  if ((e = cudaGetLastError()) != cudaSuccess) return -(int)e;
+  if ((e = launch_pdl(decode_conv1_kernel, dim3((unsigned)((d.L + 255) / 256), (unsigned)d.B), dim3(256), st, c1)) != cudaSuccess)
+    return -(int)e;
   ++*launches;
   if (d.flags & F_CONV2) {
     ProjArgs pc;
@@ -637,12 +664,12 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
   {
     dim3 grid((unsigned)(d.hq + d.hk), (unsigned)d.B);
     switch (d.dh) {
-      case 32: decode_finalize_kernel<32><<<grid, 128, 0, st>>>(fa); break;
-      case 64: decode_finalize_kernel<64><<<grid, 128, 0, st>>>(fa); break;
-      case 128: decode_finalize_kernel<128><<<grid, 128, 0, st>>>(fa); break;
-      default: decode_finalize_kernel<256><<<grid, 256, 0, st>>>(fa); break;
+      case 32: e = launch_pdl(decode_finalize_kernel<32>, grid, dim3(128), st, fa); break;
+      case 64: e = launch_pdl(decode_finalize_kernel<64>, grid, dim3(128), st, fa); break;
+      case 128: e = launch_pdl(decode_finalize_kernel<128>, grid, dim3(128), st, fa); break;
+      default: e = launch_pdl(decode_finalize_kernel<256>, grid, dim3(256), st, fa); break;
     }
-    if ((e = cudaGetLastError()) != cudaSuccess) return -(int)e;
+    if (e != cudaSuccess) return -(int)e;
     ++*launches;
   }
   AtArgs aa;
@@ -667,13 +694,13 @@ int launch_decode_step(const CcaDims& d, const DecodeWeights& w, const bf16* x, 
   {
     dim3 grid((unsigned)d.hq, (unsigned)d.B);
     switch (d.dh) {
-      case 32: decode_combine_kernel<32><<<grid, 64, 0, st>>>(ca); break;
-      case 64: decode_combine_kernel<64><<<grid, 64, 0, st>>>(ca); break;
-      case 128: decode_combine_kernel<128><<<grid, 128, 0, st>>>(ca); break;
-      case 256: decode_combine_kernel<256><<<grid, 256, 0, st>>>(ca); break;
+      case 32: e = launch_pdl(decode_combine_kernel<32>, grid, dim3(64), st, ca); break;
+      case 64: e = launch_pdl(decode_combine_kernel<64>, grid, dim3(64), st, ca); break;
+      case 128: e = launch_pdl(decode_combine_kernel<128>, grid, dim3(128), st, ca); break;
+      case 256: e = launch_pdl(decode_combine_kernel<256>, grid, dim3(256), st, ca); break;
       default: return 1;
     }
-    if ((e = cudaGetLastError()) != cudaSuccess) return -(int)e;
+    if (e != cudaSuccess) return -(int)e;
     ++*launches;
   }
   // Eq. 11, up-projection
