@@ -4,6 +4,7 @@ non-causal, for CCGQA (C = 4, four query heads per kv head) and for the same ker
 (no compression, four query heads per kv head, latent transforms off) and as MHA.
 
     python -m paper_2510_04476_b200.kernel_grid [--tokens 32768] [--steps 5] [--head-dims 64,128]
+    python -m paper_2510_04476_b200.kernel_grid --sweep          # context x compression sweep, forward and backward
 
 Prints one JSON line per (method, head size, sequence length) and a markdown table at the end.  Every number
 is a CUDA-event time on the launching stream after three warm-up steps; the batch is tokens / S sequences.
@@ -17,7 +18,7 @@ import sys
 import torch
 
 from . import synth
-from .binding import CCA
+from .binding import CCA, stack_down_projection
 
 
 def shapes_for(dh: int, S: int, tokens: int):
@@ -79,6 +80,56 @@ def time_shape(sh: synth.Shape, steps: int, device: int):
     return res
 
 
+def sweep(steps: int, device: int):
+    """Context x compression sweep of the benchmark (d_model 2048, latent head size 64, 32 / C query heads, a quarter as
+    many kv heads, 65536 tokens per point): forward and forward + backward, causal, ms and algorithmic TFLOP/s."""
+    rows = []
+    for C in (1, 2, 4, 8):
+        for S in (1024, 4096, 16384, 32768, 65536):
+            sh = synth.sweep_shape(S, C)
+            t = synth.make_inputs(sh, want_dout=True)
+            dev = stack_down_projection({k: v.cuda(device).contiguous() for k, v in t.items()})
+            out = torch.empty_like(dev["x"])
+            cca = CCA.from_shape(sh, device=device)
+            ws = cca.alloc_workspace(sh.B, sh.S, True)
+            for _ in range(2):
+                cca.forward(dev, dev["x"], ws, out)
+                cca.backward(dev, dev["x"], dev["d_out"], ws)
+            torch.cuda.synchronize()
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            fwd = bwd = 0.0
+            for _ in range(steps):
+                e0.record()
+                cca.forward(dev, dev["x"], ws, out)
+                e1.record()
+                cca.backward(dev, dev["x"], dev["d_out"], ws)
+                e2.record()
+                torch.cuda.synchronize()
+                fwd += e0.elapsed_time(e1) / steps
+                bwd += e1.elapsed_time(e2) / steps
+            st = cca.last_status()
+            cca.close()
+            if st != 0:
+                raise RuntimeError(f"device status {st} at {sh.name}")
+            T = sh.B * sh.S
+            proj = 2 * T * sh.d_model * (sh.L_q + 2 * sh.L_k) + 2 * T * sh.L_q * sh.d_model
+            conv = 2 * T * (sh.L * sh.k_seq + sh.L * sh.head_dim * sh.k_ch)
+            attn = 2 * sh.B * sh.S * sh.S * sh.L_q
+            f_fwd, f_all = proj + conv + attn, 3 * (proj + conv) + 3.5 * attn
+            rec = {"C": C, "S": S, "B": sh.B, "heads": [sh.n_q_heads, sh.n_kv_heads], "fwd_ms": round(fwd, 4),
+                   "fwd_bwd_ms": round(fwd + bwd, 4), "fwd_tflops": round(f_fwd / fwd / 1e9, 1),
+                   "fwd_bwd_tflops": round(f_all / (fwd + bwd) / 1e9, 1)}
+            print(json.dumps(rec), flush=True)
+            rows.append(rec)
+            del ws, dev, out
+            torch.cuda.empty_cache()
+    print("\n| C | S | B | forward ms (TFLOP/s) | forward + backward ms (TFLOP/s) |")
+    print("|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['C']} | {r['S']} | {r['B']} | {r['fwd_ms']:.3f} ({r['fwd_tflops']:.0f}) | {r['fwd_bwd_ms']:.3f} ({r['fwd_bwd_tflops']:.0f}) |")
+    return 0
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--tokens", type=int, default=32768)
@@ -86,10 +137,13 @@ def main(argv=None):
     ap.add_argument("--head-dims", default="64,128")
     ap.add_argument("--seq-lens", default="512,1024,2048,4096,8192,16384")
     ap.add_argument("--device", type=int, default=0)
+    ap.add_argument("--sweep", action="store_true", help="the context x compression sweep instead of the head-size grid")
     a = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("kernel_grid needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(a.device)
+    if a.sweep:
+        return sweep(a.steps, a.device)
     rows = []
     for dh in [int(v) for v in a.head_dims.split(",")]:
         for S in [int(v) for v in a.seq_lens.split(",")]:
