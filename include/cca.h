@@ -3,14 +3,16 @@
  *
  * One block = down-projection of x to latent q/k/v, the latent transforms on q and k
  * (two causal convolutions, q-k-mean, L2 norm with key temperature, RoPE), value-shift,
- * causal softmax attention with grouped kv heads inside the latent, up-projection; and the
- * matching backward.  The method is the paper's Section 2.2 (Eq. 7-11) and Listing A.1.
+ * causal softmax attention with grouped kv heads inside the latent, up-projection; the
+ * matching backward; chunked prefill and the decode step against the latent KV cache.  The
+ * method is the paper's Section 2.2 (Eq. 7-11) and Listing A.1.
  *
  * Conventions
  *   - Every pointer named "device" is CUDA device memory on the handle's device, owned by the
  *     caller.  The library allocates nothing on the device except a 64-byte status word per
- *     handle; cca_forward / cca_backward never allocate, never synchronise, never fall back to
- *     the CPU.  All work is enqueued on the caller's stream.
+ *     handle; cca_forward / cca_backward / cca_decode_step never allocate, never synchronise,
+ *     never fall back to the CPU.  All work is enqueued on the caller's stream (the forward
+ *     computes its RoPE table on a stream of the handle's own, joined back before it is used).
  *   - Activations are row-major [B, S, width] (the paper's listing is [S, B, width]; sequences
  *     are independent so the result is the same).  bf16 = 16-bit brain float, raw bits.
  *   - Linear weights are [out, in] row-major, like torch.nn.Linear.
