@@ -220,6 +220,7 @@ __global__ void __launch_bounds__(256) transform_fwd_kernel(CcaDims d, const flo
 // y is taken from the stored bf16 q / k (rotated back), r in fp32: the 1/|x| amplification is exact,
 // the projection direction carries the bf16 rounding of q.
 // ------------------------------------------------------------------------------------------
+constexpr int BWD_NORM_TOK = 16;
 template <int DH>
 __global__ void __launch_bounds__(256) transform_bwd_norm_kernel(CcaDims d, const bf16* __restrict__ q,
                                                                  const bf16* __restrict__ k,
@@ -229,15 +230,25 @@ __global__ void __launch_bounds__(256) transform_bwd_norm_kernel(CcaDims d, cons
                                                                  float* dk, float* d_temp) {
   constexpr int HALF = DH / 2, TPR = HALF / 4;     // lanes per row
   const int H = d.hq + d.hk;
-  const long long gt = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long long w = gt / TPR;
-  const int sub = (int)(gt % TPR);
-  const long long total = (long long)d.B * d.S * H;
-  const bool act = w < total;
-  const long long wc = act ? w : 0;
-  const int h = (int)(wc % H);
-  const long long row = wc / H;
-  const int t = (int)(row % d.S);
+  // a block walks BWD_NORM_TOK consecutive tokens; work item = (token, head, lane of the row), 32-bit arithmetic
+  __shared__ float temp_acc[64];
+  for (int i = threadIdx.x; i < d.hk && i < 64; i += blockDim.x) temp_acc[i] = 0.f;
+  __syncthreads();
+  const long long row0 = (long long)blockIdx.x * BWD_NORM_TOK;
+  const long long n_rows = (long long)d.B * d.S;
+  const int rows_here = (int)min((long long)BWD_NORM_TOK, n_rows - row0);
+  const unsigned per_row = (unsigned)H * TPR, items = (unsigned)rows_here * per_row;
+  const int t_first = (int)(row0 % d.S);
+  for (unsigned it0 = 0; it0 < items; it0 += blockDim.x) {
+  const unsigned item = it0 + threadIdx.x;
+  const bool act = item < items;
+  const unsigned ic = act ? item : 0u;
+  const unsigned rl = ic / per_row, rem_i = ic - rl * per_row;
+  const int h = (int)(rem_i / TPR);
+  const int sub = (int)(rem_i % TPR);
+  const long long row = row0 + rl;
+  int t = t_first + (int)rl;
+  if (t >= d.S) t -= d.S * (t / d.S);
   const bool is_q = h < d.hq;
   const int hj = is_q ? h : h - d.hq;
   float* g = (is_q ? dq + row * d.Lq : dk + row * d.Lk) + hj * DH + sub * 4;
@@ -277,7 +288,7 @@ __global__ void __launch_bounds__(256) transform_bwd_norm_kernel(CcaDims d, cons
     const float beta = is_q ? 1.f : __expf(temp[hj]);
     const float r = rnorm[row * H + h];
     const float proj = dot / ((float)DH * beta * beta);
-    if (act && !is_q && sub == 0) atomicAdd(d_temp + hj, dot);
+    if (act && !is_q && sub == 0) atomicAdd(&temp_acc[hj & 63], dot);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       ga[i] = r * (ga[i] - ya[i] * proj);
@@ -287,6 +298,11 @@ __global__ void __launch_bounds__(256) transform_bwd_norm_kernel(CcaDims d, cons
   if (act) {
     *reinterpret_cast<float4*>(g) = make_float4(ga[0], ga[1], ga[2], ga[3]);
     *reinterpret_cast<float4*>(g + HALF) = make_float4(gb[0], gb[1], gb[2], gb[3]);
+  }
+  }
+  if (d.flags & F_QK_NORM) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < d.hk && i < 64; i += blockDim.x) atomicAdd(d_temp + i, temp_acc[i]);
   }
 }
 
@@ -523,17 +539,28 @@ __global__ void rope_table_kernel(float2* tab, int S, int half, double log2_base
   tab[idx] = make_float2((float)co, (float)s);
 }
 
-__global__ void pack_dv_kernel(CcaDims d, const float* __restrict__ dv, bf16* __restrict__ dlat, long long ld) {
-  long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  long long total = (long long)d.B * d.S * d.Lk;
-  if (idx >= total) return;
-  int c = (int)(idx % d.Lk);
-  long long row = idx / d.Lk;
-  int t = (int)(row % d.S);
-  float val;
-  if (c < d.Lk / 2 || !(d.flags & F_V_SHIFT)) val = dv[idx];
-  else val = (t + 1 < d.S) ? dv[(row + 1) * d.Lk + c] : 0.f;
-  dlat[row * ld + d.L + c] = __float2bfloat16(val);
+// One thread per 4 consecutive value channels; a block covers PACK_ROWS tokens.
+constexpr int PACK_ROWS = 8;
+__global__ void __launch_bounds__(256) pack_dv_kernel(CcaDims d, const float* __restrict__ dv, bf16* __restrict__ dlat,
+                                                      long long ld) {
+  const int quads = d.Lk / 4;
+  const long long row0 = (long long)blockIdx.x * PACK_ROWS, n_rows = (long long)d.B * d.S;
+  const int rows_here = (int)min((long long)PACK_ROWS, n_rows - row0);
+  const int t_first = (int)(row0 % d.S);
+  for (int i = threadIdx.x; i < rows_here * quads; i += 256) {
+    const int rl = i / quads, c = (i - rl * quads) * 4;
+    const long long row = row0 + rl;
+    int t = t_first + rl;
+    if (t >= d.S) t -= d.S * (t / d.S);
+    float4 v;
+    if (c < d.Lk / 2 || !(d.flags & F_V_SHIFT)) v = *reinterpret_cast<const float4*>(dv + row * d.Lk + c);
+    else v = (t + 1 < d.S) ? *reinterpret_cast<const float4*>(dv + (row + 1) * d.Lk + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(dlat + row * ld + d.L + c) = pk;
+  }
 }
 
 template <typename K>
@@ -575,11 +602,9 @@ cudaError_t launch_transform_bwd_norm(const CcaDims& d, const bf16* q, const bf1
                                       const float* temp, const float2* rope_tab, float* dq, float* dk, float* d_temp,
                                       cudaStream_t st) {
   if (!(d.flags & (F_QK_NORM | F_ROPE))) return cudaSuccess;
-  const long long rows = (long long)d.B * d.S * (d.hq + d.hk);
+  const long long blocks = ((long long)d.B * d.S + BWD_NORM_TOK - 1) / BWD_NORM_TOK;
   DISPATCH_DH(d.dh, {
-    const long long threads = rows * (DH / 8);
-    transform_bwd_norm_kernel<DH><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(d, q, k, rnorm, temp, rope_tab, dq,
-                                                                                     dk, d_temp);
+    transform_bwd_norm_kernel<DH><<<(unsigned)blocks, 256, 0, st>>>(d, q, k, rnorm, temp, rope_tab, dq, dk, d_temp);
   });
   return cudaGetLastError();
 }
@@ -610,8 +635,8 @@ cudaError_t launch_transform_bwd_w1(const CcaDims& d, const float* qk0, const bf
 }
 
 cudaError_t launch_pack_dv(const CcaDims& d, const float* dv, bf16* dlat, long long ld_dlat, cudaStream_t st) {
-  long long total = (long long)d.B * d.S * d.Lk;
-  pack_dv_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(d, dv, dlat, ld_dlat);
+  const long long blocks = ((long long)d.B * d.S + PACK_ROWS - 1) / PACK_ROWS;
+  pack_dv_kernel<<<(unsigned)blocks, 256, 0, st>>>(d, dv, dlat, ld_dlat);
   return cudaGetLastError();
 }
 
