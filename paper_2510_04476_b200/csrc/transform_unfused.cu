@@ -20,13 +20,12 @@ CCA_DEVINL uint32_t pack2(float lo, float hi) {
 // thread = (token, 4 channels)
 __global__ void __launch_bounds__(256) conv1_taps_kernel(CcaDims d, const float* __restrict__ qk0, const bf16* __restrict__ w0,
                                                          bf16* __restrict__ y1s, float* __restrict__ y2) {
-  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
-  const int quads = d.L / 4;
-  const long long T = (long long)d.B * d.S;
-  if (idx >= T * quads) return;
-  const long long tok = idx / quads;
-  const int ch = (int)(idx % quads) * 4;
-  const int t = (int)(tok % d.S);
+  // blockIdx.x = token (of all sequences), blockIdx.y * 256 + thread = channel quad: no per-thread division
+  const int quad = blockIdx.y * 256 + threadIdx.x;
+  if (quad >= d.L / 4) return;
+  const long long tok = blockIdx.x;
+  const int ch = quad * 4;
+  const int t = (int)(blockIdx.x % (unsigned)d.S);
   const int ks = (d.flags & F_CONV1) ? d.k_seq : 1;
   const int kc = (d.flags & F_CONV2) ? d.k_ch : 1;
   const int span = ks + kc - 1;                      // raw tokens t - span + 1 .. t
@@ -96,13 +95,10 @@ __global__ void __launch_bounds__(256) finalize_kernel(CcaDims d, const float* _
                                                        bf16* __restrict__ q, bf16* __restrict__ k, float* __restrict__ rnorm) {
   constexpr int U = DH / 32;
   const int lane = threadIdx.x & 31;
-  const long long w = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int heads = d.hq + d.hk;
-  const long long T = (long long)d.B * d.S;
-  if (w >= T * heads) return;
-  const long long tok = w / heads;
-  const int h = (int)(w % heads);
-  const int t = (int)(tok % d.S);
+  const long long tok = blockIdx.x;                  // token of all sequences; the block's 8 warps walk its heads
+  const int t = (int)(blockIdx.x % (unsigned)d.S);
+  for (int h = threadIdx.x >> 5; h < heads; h += 8) {
   const bool is_q = h < d.hq;
   const int hj = is_q ? h / d.g : h - d.hq;
   const float* lat = qk0 + tok * d.L;
@@ -146,20 +142,20 @@ __global__ void __launch_bounds__(256) finalize_kernel(CcaDims d, const float* _
     dst[c] = __float2bfloat16(a);
     dst[c + DH / 2] = __float2bfloat16(b);
   }
+  }
 }
 
 }  // namespace
 
 cudaError_t launch_conv1_taps(const CcaDims& d, const float* qk0, const bf16* w0, bf16* y1s, float* y2, cudaStream_t st) {
-  const long long n = (long long)d.B * d.S * (d.L / 4);
-  conv1_taps_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(d, qk0, w0, y1s, y2);
+  dim3 grid((unsigned)((long long)d.B * d.S), (unsigned)((d.L / 4 + 255) / 256));
+  conv1_taps_kernel<<<grid, 256, 0, st>>>(d, qk0, w0, y1s, y2);
   return cudaGetLastError();
 }
 
 cudaError_t launch_finalize(const CcaDims& d, const float* qk0, const float* y2, const float* temp, const float2* rope,
                             bf16* q, bf16* k, float* rnorm, cudaStream_t st) {
-  const long long warps = (long long)d.B * d.S * (d.hq + d.hk);
-  const unsigned grid = (unsigned)((warps + 7) / 8);
+  const unsigned grid = (unsigned)((long long)d.B * d.S);
   switch (d.dh) {
     case 64: finalize_kernel<64><<<grid, 256, 0, st>>>(d, qk0, y2, temp, rope, q, k, rnorm); break;
     case 128: finalize_kernel<128><<<grid, 256, 0, st>>>(d, qk0, y2, temp, rope, q, k, rnorm); break;
