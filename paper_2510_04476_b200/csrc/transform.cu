@@ -472,36 +472,41 @@ __global__ void __launch_bounds__(128) conv1_adjoint_kernel(CcaDims d, const flo
     w[j] = conv1 ? ldbf(w0 + c * KS + j) : 1.f;
     dw[j] = 0.f;
   }
-  const long long seq = (long long)b * d.S;
-  auto dy_at = [&](int t) { return t < d.S ? dy1[(seq + t) * d.L + c] : 0.f; };
-  auto q_at = [&](int t) { return t >= 0 ? qk0[(seq + t) * d.L + c] : 0.f; };
+  // every address is a pointer that advances by a row per token: no multiplications or divisions in the loop
+  const long long row0 = (long long)b * d.S + t_begin;
+  const float* pdy = dy1 + row0 * d.L + c;              // dy1 of token t_begin
+  const float* pq0 = qk0 + row0 * d.L + c;              // qk0 of token t_begin
+  bf16* pout = dlat + row0 * ld + c;
   // win[m] = dy1[t + m], qwin[m] = qk0[t - (KS-1) + m]
 #pragma unroll
   for (int m = 0; m < KS; ++m) {
-    win[m] = dy_at(t_begin + m);
-    qwin[m] = q_at(t_begin - (KS - 1) + m);
+    win[m] = t_begin + m < d.S ? pdy[(long long)m * d.L] : 0.f;
+    qwin[m] = t_begin - (KS - 1) + m >= 0 ? pq0[(long long)(m - (KS - 1)) * d.L] : 0.f;
   }
+  // q-k-mean adjoint: a q channel takes half of its own d_hat and 1/(2g) of its kv head's; a k channel half of its
+  // own and half of the sum over its g query heads
   const bool is_q = c < d.Lq;
-  const int cj = is_q ? c : c - d.Lq, hh = cj / d.dh, o = cj % d.dh;
+  const int cj = is_q ? c : c - d.Lq, hh = cj / d.dh, o = cj - hh * d.dh;
   const bool mean = (d.flags & F_QK_MEAN) != 0;
+  const float* pa = is_q ? dqh + row0 * d.Lq + c : dkh + row0 * d.Lk + cj;                       // own d_hat
+  const float* pb = is_q ? dkh + row0 * d.Lk + (hh / d.g) * d.dh + o : dqh + row0 * d.Lq + (hh * d.g) * d.dh + o;
+  const int sa = is_q ? d.Lq : d.Lk, sb = is_q ? d.Lk : d.Lq;                                   // row strides
+  const int n_b = is_q ? 1 : d.g;
+  const float scale_b = is_q ? 0.5f / (float)d.g : 0.5f;
+  const int sL = d.L;
   constexpr int U = 4;                               // tokens per batch: all loads of a batch are issued together
   for (int tb = t_begin; tb < t_end; tb += U) {
     float ndy[U], nq[U], dir[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int t = tb + u;
-      ndy[u] = dy_at(t + KS);
-      nq[u] = (t + 1 < d.S) ? q_at(t + 1) : 0.f;
+      ndy[u] = t + KS < d.S ? pdy[(u + KS) * sL] : 0.f;
+      nq[u] = t + 1 < d.S ? pq0[(u + 1) * sL] : 0.f;
       dir[u] = 0.f;
       if (mean && t < t_end) {
-        const long long row = seq + t;
-        if (is_q) {
-          dir[u] = 0.5f * (dqh[row * d.Lq + c] + dkh[row * d.Lk + (hh / d.g) * d.dh + o] / d.g);
-        } else {
-          float sg = dkh[row * d.Lk + cj];
-          for (int m = 0; m < d.g; ++m) sg += dqh[row * d.Lq + (hh * d.g + m) * d.dh + o];
-          dir[u] = 0.5f * sg;
-        }
+        float sbv = pb[u * sb];
+        for (int m = 1; m < n_b; ++m) sbv += pb[u * sb + m * d.dh];
+        dir[u] = 0.5f * pa[u * sa] + scale_b * sbv;
       }
     }
 #pragma unroll
@@ -513,7 +518,7 @@ __global__ void __launch_bounds__(128) conv1_adjoint_kernel(CcaDims d, const flo
         for (int j = 0; j < KS; ++j) gq = fmaf(w[j], win[KS - 1 - j], gq);
 #pragma unroll
         for (int j = 0; j < KS; ++j) dw[j] = fmaf(win[0], qwin[j], dw[j]);
-        dlat[(seq + t) * ld + c] = __float2bfloat16(gq);
+        pout[(long long)u * ld] = __float2bfloat16(gq);
 #pragma unroll
         for (int m = 0; m < KS - 1; ++m) {
           win[m] = win[m + 1];
@@ -523,6 +528,11 @@ __global__ void __launch_bounds__(128) conv1_adjoint_kernel(CcaDims d, const flo
         qwin[KS - 1] = nq[u];
       }
     }
+    pdy += U * sL;
+    pq0 += U * sL;
+    pout += (long long)U * ld;
+    pa += U * sa;
+    pb += U * sb;
   }
   if (conv1)
 #pragma unroll
