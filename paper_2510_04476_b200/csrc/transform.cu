@@ -455,7 +455,7 @@ __global__ void __launch_bounds__(256) transform_bwd_w1_kernel(CcaDims d, const 
 //   d_qk0[t][c]  = sum_j w0[c][j] dy1[t + (ks-1) - j][c]  +  (direct q-k-mean terms of d_hat)
 //   d_w0[c][j]  += sum_t dy1[t][c] qk0[t - (ks-1) + j][c]
 // One thread per channel (coalesced over channels), walking CONV1_TOK consecutive tokens with sliding windows.
-constexpr int CONV1_TOK = 32;
+constexpr int CONV1_TOK = 16;
 template <int KS>
 __global__ void __launch_bounds__(128) conv1_adjoint_kernel(CcaDims d, const float* __restrict__ dy1,
                                                             const float* __restrict__ dqh, const float* __restrict__ dkh,
