@@ -128,17 +128,22 @@ int cca_workspace_size(const cca_handle* h, int64_t B, int64_t S, int need_backw
 
 /* Forward of the whole block, Eq. 7-11: out = W_o [ softmax(q k^T / sqrt(d_h)) v ]_heads.
  *   x   device bf16 [B,S,E] (read), out device bf16 [B,S,E] (written).
- *   workspace: device, 256-byte aligned, >= cca_workspace_size(..., need_backward).  On return
- *   (stream order) it holds qk0 (fp32), q, k, v, o (bf16), lse and the norm scales (fp32) at the cca_layout offsets; keep it untouched
- *   until cca_backward if gradients are wanted.
+ *   workspace: device, 256-byte aligned, >= cca_workspace_size(h, B, S, save_for_backward, ..).  On return
+ *   (stream order) it holds qk0 (fp32), q, k, v, o (bf16), lse and the norm scales (fp32) at the cca_layout offsets.
+ *   save_for_backward != 0: an fp32 copy of o is kept as well (the backward's delta = rowsum(dO * O) needs it) and
+ *   the handle remembers (workspace, B, S); keep the workspace untouched until cca_backward.  With 0 nothing beyond
+ *   saved_bytes is touched and a later cca_backward on this workspace is refused.
  * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE_TOO_SMALL, CUDA. */
 int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out,
-                void* workspace, size_t workspace_bytes, int64_t B, int64_t S, void* cuda_stream);
+                void* workspace, size_t workspace_bytes, int64_t B, int64_t S, int save_for_backward,
+                void* cuda_stream);
 
 /* Backward of the block: given d_out = dLoss/d out (device bf16 [B,S,E]) and the workspace
- * left by cca_forward for the same x and weights, writes d_x (device bf16 [B,S,E]) and every
- * field of `grads` (fp32, overwritten).  The paper prints no backward; this is the exact
- * adjoint of Eq. 7-11.  Errors as cca_forward; UNSUPPORTED for head_dim = 256 (forward only). */
+ * left by cca_forward(..., save_for_backward = 1, ..) for the same x, weights, B and S, writes d_x (device bf16
+ * [B,S,E]) and every field of `grads` (fp32, overwritten).  The paper prints no backward; this is the exact
+ * adjoint of Eq. 7-11.  Errors as cca_forward (weights and gradient buffers 16-byte aligned; the conv weights and
+ * temp non-null when their stage is on); INVALID_ARG also when `workspace`, B, S are not those of this handle's
+ * last forward with save_for_backward set (nothing is launched). */
 int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void* d_out,
                  void* workspace, size_t workspace_bytes, void* d_x,
                  const cca_weight_grads* grads, int64_t B, int64_t S, void* cuda_stream);
@@ -213,7 +218,8 @@ typedef struct {
 } cca_decode_state;
 
 /* Bytes of device workspace one decode step needs for B sequences of at most max_len tokens (the new
- * token included). */
+ * token included).  The size depends on the device's SM count (the key range is split over the SMs); a
+ * host-only handle assumes 148. */
 int cca_decode_workspace_size(const cca_handle* h, int64_t B, int64_t max_len, size_t* bytes);
 
 /* One decode step, Eq. 7-11 for a single new token per sequence: x device bf16 [B,E] (read), out device
@@ -223,14 +229,16 @@ int cca_decode_workspace_size(const cca_handle* h, int64_t B, int64_t max_len, s
  * S_max for every b; it sizes the launch.  A sequence whose pos[b] is outside [0, min(max_len, S_max)) is
  * skipped (its caches, history and output row are left untouched or undefined, nothing is written out of
  * bounds) and the device status word becomes 120, which cca_last_status reports.
- * Needs causal = 1, L_k and E multiples of 8 (at head_dim = 256 at most 8 query heads per kv head).  No allocation, no synchronisation.
+ * Needs causal = 1, L_k a multiple of 8, E and L_q multiples of 32 (at head_dim = 256 at most 8 query heads per
+ * kv head); otherwise UNSUPPORTED.  No allocation, no synchronisation.
  * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE_TOO_SMALL, CUDA. */
 int cca_decode_step(cca_handle* h, const cca_weights* w, const void* x, void* out, const cca_decode_state* state,
                     int64_t max_len, void* workspace, size_t workspace_bytes, int64_t B, void* cuda_stream);
 
 /* Hand-over from a prefill: fills `state` (caches rows 0..S-1, history, previous input) from x [B,S,E] and
  * the workspace cca_forward left for it, so that the next cca_decode_step continues at pos[b] = S.  Copies
- * only (stream order); state->pos is not read.  Errors: INVALID_ARG (S > S_max, null), ALIGNMENT, CUDA. */
+ * only (stream order); state->pos is not read.  Errors: INVALID_ARG (S > S_max, null), ALIGNMENT (x, the caches,
+ * x_prev, qk0_hist 16-byte, workspace 256-byte), WORKSPACE_TOO_SMALL, CUDA. */
 int cca_decode_state_from_prefill(cca_handle* h, const void* x, const void* workspace, size_t workspace_bytes,
                                   int64_t B, int64_t S, const cca_decode_state* state, void* cuda_stream);
 
@@ -248,9 +256,22 @@ int cca_set_attention_events(cca_handle* h, void* ev_begin, void* ev_end);
 int64_t cca_launch_count(const cca_handle* h);
 
 /* After the caller has synchronised the stream: copies the device status word.  0 = no error;
- * otherwise the code written by a kernel whose bounded wait expired (or 120: a decode step met a position
- * outside its cache).  Returns CCA_ERR_DEVICE_TIMEOUT if it is non-zero. */
+ * otherwise the code written by a kernel whose bounded wait expired (101..105 by role, 109 from
+ * cca_wait_selftest; or 120: a decode step met a position outside its cache).  Returns
+ * CCA_ERR_DEVICE_TIMEOUT if it is non-zero, and clears the word. */
 int cca_last_status(cca_handle* h, int* device_status);
+
+/* Limit of every bounded device-side wait of this handle's kernels, in SM clock cycles (about 0.5 ns each).
+ * 0 restores the default (4e9, about 2 s).  Values below 2^21 cycles (about 1 ms) are raised to that: the waits
+ * of a healthy kernel last microseconds, and a limit they could reach would turn a slow tile into an error.
+ * A kernel whose wait runs out records a status code, lets its copies in flight land, frees its tensor memory
+ * and returns; nothing traps.  Synchronous (one small copy to the device).  Errors: INVALID_ARG, CUDA. */
+int cca_set_wait_limit(cca_handle* h, int64_t sm_cycles);
+
+/* Enqueues one 64-thread kernel whose only wait is on a barrier that nothing ever arrives at, so that the wait
+ * runs into the handle's limit: after the caller synchronises, cca_last_status returns CCA_ERR_DEVICE_TIMEOUT
+ * with status 109, and the handle stays usable.  A check of the error path, not part of the method. */
+int cca_wait_selftest(cca_handle* h, void* cuda_stream);
 
 /* Last CUDA runtime error code seen by this handle, and its string. */
 int cca_last_cuda_error(const cca_handle* h);

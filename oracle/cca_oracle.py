@@ -393,6 +393,7 @@ def backward(cfg: OracleConfig, w: Dict[str, torch.Tensor], I: Dict[str, torch.T
         dy1, G["d_conv1_w"] = conv2_seq_ch_adjoint(dy2, I["y1"], _f64(w["conv1_w"]), hq + hk, dh)
     else:
         dy1, G["d_conv1_w"] = dy2, torch.zeros(L, dh, cfg.k_ch, dtype=F64)
+    G["d_y2"], G["d_y1"] = dy2, dy1
     if cfg.flags & CONV1:
         dqk0, G["d_conv0_w"] = conv1_seq_adjoint(dy1, I["qk0"], _f64(w["conv0_w"]))
     else:

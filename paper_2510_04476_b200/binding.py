@@ -57,7 +57,7 @@ SYMBOLS = {
     "cca_describe": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.POINTER(cca_layout)]),
     "cca_workspace_size": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int, C.POINTER(C.c_size_t)]),
     "cca_forward": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
-                              C.c_int64, C.c_int64, C.c_void_p]),
+                              C.c_int64, C.c_int64, C.c_int, C.c_void_p]),
     "cca_backward": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                C.c_void_p, C.POINTER(cca_weight_grads), C.c_int64, C.c_int64, C.c_void_p]),
     "cca_forward_host": (C.c_int, [C.c_void_p, C.POINTER(cca_weights), C.c_void_p, C.c_void_p, C.c_void_p,
@@ -77,6 +77,8 @@ SYMBOLS = {
     "cca_set_attention_events": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "cca_launch_count": (C.c_int64, [C.c_void_p]),
     "cca_last_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int)]),
+    "cca_set_wait_limit": (C.c_int, [C.c_void_p, C.c_int64]),
+    "cca_wait_selftest": (C.c_int, [C.c_void_p, C.c_void_p]),
     "cca_last_cuda_error": (C.c_int, [C.c_void_p]),
     "cca_status_string": (C.c_char_p, [C.c_int]),
 }
@@ -213,17 +215,35 @@ class CCA:
             setattr(cw, n, t.data_ptr() if t is not None else None)
         return cw
 
-    def forward(self, w, x: torch.Tensor, workspace: torch.Tensor, out: Optional[torch.Tensor] = None):
+    def forward(self, w, x: torch.Tensor, workspace: torch.Tensor, out: Optional[torch.Tensor] = None,
+                save_for_backward: Optional[bool] = None):
+        """cca_forward.  save_for_backward=None: keep the activations for a backward exactly when the workspace was
+        sized for one (alloc_workspace(..., need_backward=True))."""
         B, S, E = x.shape
         assert x.is_cuda and x.is_contiguous() and x.dtype == torch.bfloat16
         if out is None:
             out = torch.empty_like(x)
         cw = self._weights(w)
         wp, wn = self._ws_ptr(workspace)
+        if save_for_backward is None:
+            save_for_backward = wn >= self.workspace_size(B, S, True)
         st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
-        _check(self.lib, self.lib.cca_forward(self.handle, C.byref(cw), _ptr(x), _ptr(out), wp, wn, B, S, st),
-               self.handle, "cca_forward")
+        _check(self.lib, self.lib.cca_forward(self.handle, C.byref(cw), _ptr(x), _ptr(out), wp, wn, B, S,
+                                              int(bool(save_for_backward)), st), self.handle, "cca_forward")
         return out
+
+    def set_wait_limit(self, sm_cycles: int):
+        _check(self.lib, self.lib.cca_set_wait_limit(self.handle, int(sm_cycles)), self.handle, "cca_set_wait_limit")
+
+    def wait_selftest(self):
+        st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+        _check(self.lib, self.lib.cca_wait_selftest(self.handle, st), self.handle, "cca_wait_selftest")
+
+    def last_status_code(self):
+        """(return code of cca_last_status, device status word)."""
+        s = C.c_int()
+        rc = self.lib.cca_last_status(self.handle, C.byref(s))
+        return int(rc), int(s.value)
 
     def forward_chunk(self, w, x_chunk: torch.Tensor, workspace: torch.Tensor, S_total: int, t_begin: int,
                       out: Optional[torch.Tensor] = None):
@@ -334,8 +354,12 @@ class CCA:
         else:
             d_all = torch.empty((n0 + n1 + n2, E), dtype=torch.float32, device=self.device)
             grads["d_w_qk"], grads["d_w_v1"], grads["d_w_v2"] = d_all[:n0], d_all[n0:n0 + n1], d_all[n0 + n1:]
-        for n in ("w_o", "conv0_w", "conv1_w", "temp"):
-            grads["d_" + n] = torch.empty(w[n].shape, dtype=torch.float32, device=self.device)
+        c = self.cfg
+        L = (c.n_q_heads + c.n_kv_heads) * c.head_dim
+        shapes = {"w_o": (E, c.n_q_heads * c.head_dim), "conv0_w": (L, c.k_seq), "conv1_w": (L, c.head_dim, c.k_ch),
+                  "temp": (c.n_kv_heads,)}
+        for n, shp in shapes.items():
+            grads["d_" + n] = torch.empty(shp, dtype=torch.float32, device=self.device)
         for n in ("w_qk", "w_v1", "w_v2", "w_o", "conv0_w", "conv1_w", "temp"):
             setattr(cg, "d_" + n, grads["d_" + n].data_ptr())
         cw = self._weights(w)

@@ -8,6 +8,7 @@
 #include "common.cuh"
 #include "decode.cuh"
 #include "tc_kernels.cuh"
+#include "tc_ptx.cuh"
 
 struct cca_handle {
   cca_config cfg;
@@ -25,6 +26,9 @@ struct cca_handle {
   cudaStream_t s_in, s_out;
   cudaEvent_t ev_chunk[2][64];              // [arrived / computed][chunk]
   int n_ev;                                 // events created so far
+  // what the last cca_forward kept for a backward: cca_backward refuses anything else
+  const void* saved_ws;
+  int64_t saved_B, saved_S;
 };
 
 namespace {
@@ -199,6 +203,7 @@ int cca_init(const cca_config* cfg, int device, cca_handle** out) {
   h->ev_attn_begin = h->ev_attn_end = nullptr;
   h->side = nullptr; h->ev_fork = h->ev_join = nullptr;
   h->s_in = h->s_out = nullptr; h->n_ev = 0;
+  h->saved_ws = nullptr; h->saved_B = h->saved_S = 0;
   if (device >= 0) {
     if (cudaMalloc(&h->d_status, 64) != cudaSuccess || cudaMemset(h->d_status, 0, 64) != cudaSuccess) {
       if (h->d_status) cudaFree(h->d_status);
@@ -259,9 +264,48 @@ int cca_last_status(cca_handle* h, int* device_status) {
   CU(cudaMemcpy(host, h->d_status, 64, cudaMemcpyDeviceToHost));
   *device_status = host[0];
   if (host[0] != 0) {
-    cudaMemset(h->d_status, 0, 64);
+    cudaMemset(h->d_status, 0, 4);           // word 0 only: word 1 is the wait limit
     return CCA_ERR_DEVICE_TIMEOUT;
   }
+  return CCA_OK;
+}
+
+int cca_set_wait_limit(cca_handle* h, int64_t sm_cycles) {
+  if (!h || h->device < 0 || sm_cycles < 0) return CCA_ERR_INVALID_ARG;
+  long long k = sm_cycles == 0 ? 0 : (sm_cycles + 1023) / 1024;      // 0 = default
+  if (k != 0 && k < tc::WAIT_KCYCLES_MIN) k = tc::WAIT_KCYCLES_MIN;
+  if (k > 0x7fffffffLL) k = 0x7fffffffLL;
+  const int word = (int)k;
+  CU(cudaSetDevice(h->device));
+  CU(cudaMemcpy(h->d_status + 1, &word, 4, cudaMemcpyHostToDevice));
+  return CCA_OK;
+}
+
+namespace {
+// One CTA whose only wait is on a barrier that nothing arrives at: the wait runs into the handle's limit, the
+// kernel records ST_TIMEOUT_PROBE and returns.  Nothing traps, nothing spins without a bound.
+__global__ void wait_probe_kernel(int* status) {
+  __shared__ uint64_t bar;
+  __shared__ int ctl[2];
+  if (threadIdx.x == 0) {
+    tc::mbar_init(&bar, 1);
+    tc::wait_ctl_init(ctl, status);
+    tc::fence_barrier_init();
+  }
+  __syncthreads();
+  if (!tc::mbar_wait(&bar, 0, ctl)) {
+    ctl[0] = 1;
+    atomicCAS(status, 0, (int)tc::ST_TIMEOUT_PROBE);
+  }
+}
+}  // namespace
+
+int cca_wait_selftest(cca_handle* h, void* cuda_stream) {
+  if (!h || h->device < 0) return CCA_ERR_INVALID_ARG;
+  CU(cudaSetDevice(h->device));
+  wait_probe_kernel<<<1, 64, 0, (cudaStream_t)cuda_stream>>>(h->d_status);
+  CU(cudaGetLastError());
+  h->launches++;
   return CCA_OK;
 }
 
@@ -341,7 +385,7 @@ int cca_decode_step(cca_handle* h, const cca_weights* w, const void* x, void* ou
   if (max_len > s->S_max || s->S_max > (int64_t)1 << 24) return CCA_ERR_INVALID_ARG;
   if (!c.causal) return CCA_ERR_UNSUPPORTED;
   CcaDims d = make_dims(c, B, 1);
-  if (d.Lk % 8 || d.E % 8 || d.Lq % 8) return CCA_ERR_UNSUPPORTED;
+  if (d.Lk % 8 || d.E % 32 || d.Lq % 32) return CCA_ERR_UNSUPPORTED;
   if (!aligned16(x) || !aligned16(out) || !aligned16(w->w_qk) || !aligned16(w->w_v1) || !aligned16(w->w_v2) ||
       !aligned16(w->w_o) || !aligned16(s->k_cache) || !aligned16(s->v_cache) || !aligned16(s->x_prev) ||
       (reinterpret_cast<uintptr_t>(workspace) & 255))
@@ -366,6 +410,9 @@ int cca_decode_state_from_prefill(cca_handle* h, const void* x, const void* work
   const cca_config& c = h->cfg;
   const int pad = c.k_seq + c.k_ch - 2;
   if (!s->k_cache || !s->v_cache || !s->x_prev || (pad > 0 && !s->qk0_hist) || S > s->S_max) return CCA_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(s->k_cache) || !aligned16(s->v_cache) || !aligned16(s->x_prev) ||
+      (pad > 0 && !aligned16(s->qk0_hist)) || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CCA_ERR_ALIGNMENT;
   Layout l = make_layout(c, B, S);
   if (workspace_bytes < l.saved_end) return CCA_ERR_WORKSPACE_TOO_SMALL;
   CU(cudaSetDevice(h->device));
@@ -394,7 +441,7 @@ int cca_decode_state_from_prefill(cca_handle* h, const void* x, const void* work
 }
 
 int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, void* workspace,
-                size_t workspace_bytes, int64_t B, int64_t S, void* cuda_stream) {
+                size_t workspace_bytes, int64_t B, int64_t S, int save_for_backward, void* cuda_stream) {
   int r = check_sizes(h, B, S, true);
   if (r != CCA_OK) return r;
   if (!w || !x || !out || !workspace) return CCA_ERR_INVALID_ARG;
@@ -407,7 +454,8 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
       !aligned16(w->w_o) || (reinterpret_cast<uintptr_t>(workspace) & 255))
     return CCA_ERR_ALIGNMENT;
   Layout l = make_layout(c, B, S);
-  if (workspace_bytes < l.saved_end) return CCA_ERR_WORKSPACE_TOO_SMALL;
+  if (workspace_bytes < (save_for_backward ? l.total_end : l.saved_end)) return CCA_ERR_WORKSPACE_TOO_SMALL;
+  h->saved_ws = nullptr;                       // set again below once everything is enqueued
   CU(cudaSetDevice(h->device));
   cudaStream_t st = (cudaStream_t)cuda_stream;
   CcaDims d = make_dims(c, B, S);
@@ -421,8 +469,8 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   float* lse = (float*)(ws + l.lse);
   float2* rope = (float2*)(ws + l.rope);
   float* rnorm = (float*)(ws + l.rnorm);
-  // fp32 copy of o for the backward, kept only if the caller's workspace has the backward region
-  float* o32 = workspace_bytes >= l.total_end ? (float*)(ws + l.o32) : nullptr;
+  // fp32 copy of o for the backward's delta = rowsum(dO * O)
+  float* o32 = save_for_backward ? (float*)(ws + l.o32) : nullptr;
 
   // The RoPE table does not depend on x: it is computed on a side stream while the down-projection runs.
   bool forked = false;
@@ -522,6 +570,7 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   g.M = T; g.N = d.E; g.K = d.Lq; g.a_row_off = 0; g.seq_len = d.S;
   g.out_bf16 = (bf16*)out; g.ldc = d.E;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  if (save_for_backward) { h->saved_ws = workspace; h->saved_B = B; h->saved_S = S; }
   return CCA_OK;
 }
 
@@ -661,7 +710,7 @@ int cca_forward_host(cca_handle* h, const cca_weights* w, const void* x_host, vo
     }
   }
   CU(cudaMemcpyAsync(xs, x_host, (size_t)B * S * h->cfg.d_model * 2, cudaMemcpyHostToDevice, st));
-  r = cca_forward(h, w, xs, os, workspace, l.saved_end, B, S, cuda_stream);
+  r = cca_forward(h, w, xs, os, workspace, l.saved_end, B, S, 0, cuda_stream);
   if (r != CCA_OK) return r;
   CU(cudaMemcpyAsync(out_host, os, (size_t)B * S * h->cfg.d_model * 2, cudaMemcpyDeviceToHost, st));
   CU(cudaStreamSynchronize(st));
@@ -678,11 +727,19 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   if (!gr->d_w_qk || !gr->d_w_v1 || !gr->d_w_v2 || !gr->d_w_o || !gr->d_conv0_w || !gr->d_conv1_w || !gr->d_temp)
     return CCA_ERR_INVALID_ARG;
   const cca_config& c = h->cfg;
+  if ((c.flags & CCA_CONV1) && !w->conv0_w) return CCA_ERR_INVALID_ARG;
+  if ((c.flags & CCA_CONV2) && !w->conv1_w) return CCA_ERR_INVALID_ARG;
+  if ((c.flags & CCA_QK_NORM) && !w->temp) return CCA_ERR_INVALID_ARG;
   if (c.head_dim > 128) return CCA_ERR_UNSUPPORTED;          // head size 256: forward only
-  if (!aligned16(x) || !aligned16(d_out) || !aligned16(d_x) || (reinterpret_cast<uintptr_t>(workspace) & 255))
+  if (!aligned16(x) || !aligned16(d_out) || !aligned16(d_x) || !aligned16(w->w_qk) || !aligned16(w->w_v1) ||
+      !aligned16(w->w_v2) || !aligned16(w->w_o) || !aligned16(gr->d_w_qk) || !aligned16(gr->d_w_v1) ||
+      !aligned16(gr->d_w_v2) || !aligned16(gr->d_w_o) || (reinterpret_cast<uintptr_t>(workspace) & 255))
     return CCA_ERR_ALIGNMENT;
   Layout l = make_layout(c, B, S);
   if (workspace_bytes < l.total_end) return CCA_ERR_WORKSPACE_TOO_SMALL;
+  // the workspace must be the one the last cca_forward(..., save_for_backward = 1) filled for this B and S:
+  // without it the fp32 copy of o (and hence delta and every gradient) would be read from unwritten memory
+  if (h->saved_ws != workspace || h->saved_B != B || h->saved_S != S) return CCA_ERR_INVALID_ARG;
   CU(cudaSetDevice(h->device));
   cudaStream_t st = (cudaStream_t)cuda_stream;
   CcaDims d = make_dims(c, B, S);
@@ -814,7 +871,7 @@ int cca_forward_static(cca_handle* h, const cca_weights* w, const void* x, void*
   }
   // Every region of the forward workspace is written in full before it is read, so the previous call's
   // contents need no clearing.  Passing exactly the forward-only size keeps the fp32 copy of o off.
-  return cca_forward(h, w, x, out, ws, l.saved_end, B, S, cuda_stream);
+  return cca_forward(h, w, x, out, ws, l.saved_end, B, S, 0, cuda_stream);
 }
 
 }  // extern "C"

@@ -109,7 +109,7 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       mbar_init(&kv_full[i], 1);
       mbar_init(&kv_empty[i], 1);
     }
-    *abort_flag = 0;
+    wait_ctl_init(abort_flag, p.status);
     fence_barrier_init();
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmK);
@@ -406,12 +406,12 @@ namespace {
 template <int DH, int POLY>
 int launch_attn(TcState* s, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnParams& p,
                 unsigned grid, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[TC_MAX_DEVICES] = {};
+  if (!attr_set[s->device]) {
     cudaError_t e = cudaFuncSetAttribute(tc_attn_fwd_kernel<DH, POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          AttnSmem<DH>::TOTAL);
     if (e != cudaSuccess) return -(int)e;
-    attr_set = true;
+    attr_set[s->device] = true;
   }
   tc_attn_fwd_kernel<DH, POLY><<<grid, AT_THREADS, AttnSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, p);
   cudaError_t e = cudaGetLastError();

@@ -74,7 +74,7 @@ tc_attn_fwd256_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mbar_init(&p_full[2 * i + 1], 512);
     }
     mbar_init(pv_done, 1);
-    *abort_flag = 0;
+    wait_ctl_init(abort_flag, p.status);
     fence_barrier_init();
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmK);
@@ -331,13 +331,13 @@ done:
 }
 
 template <int POLY>
-int launch_attn256(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnParams& p, unsigned grid,
-                   cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
+int launch_attn256(TcState* s, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnParams& p,
+                   unsigned grid, cudaStream_t st) {
+  static bool attr_set[TC_MAX_DEVICES] = {};
+  if (!attr_set[s->device]) {
     cudaError_t e = cudaFuncSetAttribute(tc_attn_fwd256_kernel<POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, A6_TOTAL);
     if (e != cudaSuccess) return -(int)e;
-    attr_set = true;
+    attr_set[s->device] = true;
   }
   tc_attn_fwd256_kernel<POLY><<<grid, A6_THREADS, A6_TOTAL, st>>>(tmQ, tmK, tmV, p);
   cudaError_t e = cudaGetLastError();
@@ -367,5 +367,5 @@ int tc_attn_fwd256(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, c
   const long long grid = (long long)p.n_blocks * d.B * d.hq;
   if (grid > 0x7fffffffLL) return 1;
   // one exponential per 4 * 256 tensor FLOPs: the transcendental unit has time to spare, no polynomial share
-  return launch_attn256<0>(tmQ, tmK, tmV, p, (unsigned)grid, st);
+  return launch_attn256<0>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
 }

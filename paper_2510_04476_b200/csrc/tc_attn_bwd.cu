@@ -161,7 +161,7 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     mbar_init(ds_full, 32 * BW_COMPUTE_WARPS);
     mbar_init(dq_done, 1);
     mbar_init(dp_free, 32 * BW_COMPUTE_WARPS);
-    *abort_flag = 0;
+    wait_ctl_init(abort_flag, p.status);
     fence_barrier_init();
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmK);
@@ -382,7 +382,7 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     mbar_init(acc_done, 1);
     mbar_init(&stat_ready[0], 256);
     mbar_init(&stat_ready[1], 256);
-    *abort_flag = 0;
+    wait_ctl_init(abort_flag, p.status);
     fence_barrier_init();
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmK);
@@ -607,13 +607,13 @@ template <int DH, int POLY>
 int launch_bwd(TcState* s, const CcaDims& d, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                const CUtensorMap& tmDO, const CUtensorMap& tmQh, const CUtensorMap& tmDOh, const BwdParams& p,
                cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[TC_MAX_DEVICES] = {};
+  if (!attr_set[s->device]) {
     cudaError_t e = cudaFuncSetAttribute(tc_attn_bwd_dq_kernel<DH, POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<DH>::TOTAL);
     if (e != cudaSuccess) return -(int)e;
     e = cudaFuncSetAttribute(tc_attn_bwd_dkv_kernel<DH, POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<DH>::TOTAL);
     if (e != cudaSuccess) return -(int)e;
-    attr_set = true;
+    attr_set[s->device] = true;
   }
   const long long g_kv = (long long)p.n_tiles * d.B * d.hk, g_q = (long long)p.n_tiles * d.B * d.hq;
   if (g_q > 0x7fffffffLL) return 1;

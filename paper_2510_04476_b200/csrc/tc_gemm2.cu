@@ -120,7 +120,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       mbar_init(&acc_full[s], 1);
       mbar_init(&acc_empty[s], 8);          // four epilogue warps of each CTA
     }
-    *abort_flag = 0;
+    wait_ctl_init(abort_flag, p.status);
     fence_barrier_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
@@ -325,12 +325,12 @@ done:
 template <int BN>
 int launch_pair(TcState* s, const GemmArgs& g, const G2Params& p0, bool a_mn, bool b_mn, long long lda, long long ldb,
                 cudaStream_t st) {
-  static bool attr_set = false;
+  static bool attr_set[TC_MAX_DEVICES] = {};
   using SM = G2Smem<BN>;
-  if (!attr_set) {
+  if (!attr_set[s->device]) {
     cudaError_t e = cudaFuncSetAttribute(tc_gemm2_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL);
     if (e != cudaSuccess) return -(int)e;
-    attr_set = true;
+    attr_set[s->device] = true;
   }
   CUtensorMap tmA, tmB;
   bool ok;

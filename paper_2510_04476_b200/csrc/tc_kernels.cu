@@ -76,7 +76,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(&acc_full[s], 1);
       mbar_init(&acc_empty[s], 4);
     }
-    *abort_flag = 0;
+    wait_ctl_init(abort_flag, p.status);
     fence_barrier_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
@@ -272,6 +272,12 @@ TcState* tc_create(int sm_count) {
   TcState* s = new (std::nothrow) TcState();
   if (!s) return nullptr;
   s->sm_count = sm_count;
+  s->device = 0;
+  if (cudaGetDevice(&s->device) != cudaSuccess || s->device < 0 || s->device >= TC_MAX_DEVICES) {
+    (void)cudaGetLastError();
+    delete s;
+    return nullptr;
+  }
   s->encode = nullptr;
   s->attr_set_128 = s->attr_set_256 = false;
   s->pair_clusters = -1;

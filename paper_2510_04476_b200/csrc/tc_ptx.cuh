@@ -13,9 +13,20 @@ namespace tc {
 
 // Device status codes written to the handle's status word when a bounded wait gives up.
 enum : int { ST_OK = 0, ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_EPI = 103, ST_TIMEOUT_SOFTMAX = 104,
-             ST_TIMEOUT_CORR = 105, ST_BAD_SMEM_ALIGNMENT = 110 };
+             ST_TIMEOUT_CORR = 105, ST_TIMEOUT_PROBE = 109, ST_BAD_SMEM_ALIGNMENT = 110 };
 
-constexpr long long WAIT_CYCLES = 4000000000LL;   // about 2 s at 2 GHz: far beyond any legitimate wait
+// Wait limit.  The handle's 64-byte device status block holds, in word 1, the limit of every bounded wait in
+// units of 1024 SM clock cycles (0 = default).  Each kernel copies it next to its abort flag in shared memory
+// (wait_ctl_init), where mbar_wait reads it on its slow path only.
+constexpr int WAIT_KCYCLES_DEFAULT = 3906250;     // * 1024 = 4e9 cycles, about 2 s: far beyond any legitimate wait
+constexpr int WAIT_KCYCLES_MIN = 2048;            // about 1 ms: still far beyond any legitimate wait (microseconds)
+
+// abort_flag[0] = 0 (no role has given up), abort_flag[1] = the wait limit.  One thread, before the CTA's first barrier.
+TC_DEVINL void wait_ctl_init(volatile int* abort_flag, const int* status) {
+  const int k = status ? status[1] : 0;
+  abort_flag[0] = 0;
+  abort_flag[1] = k >= WAIT_KCYCLES_MIN ? k : WAIT_KCYCLES_DEFAULT;
+}
 
 TC_DEVINL uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -42,16 +53,17 @@ TC_DEVINL bool mbar_try(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false if the barrier did not flip within WAIT_CYCLES or another role already
-// gave up (*abort != 0); the caller then records a status code and leaves its loop.
+// Bounded wait.  Returns false if the barrier did not flip within the wait limit (abort_flag[1], see
+// wait_ctl_init) or another role already gave up (abort_flag[0] != 0); the caller then records a status code
+// and leaves its loop.
 TC_DEVINL bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   int spins = 0;
   while (!mbar_try(bar, parity)) {
     if ((++spins & 1023) == 0) {
-      if (*abort_flag != 0) return false;
-      if (clock64() - t0 > WAIT_CYCLES) return false;
+      if (abort_flag[0] != 0) return false;
+      if (clock64() - t0 > ((long long)abort_flag[1] << 10)) return false;
     }
   }
   return true;

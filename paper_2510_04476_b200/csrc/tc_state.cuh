@@ -8,8 +8,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// cudaFuncSetAttribute is per device; each launcher remembers per device (index = TcState::device) whether its
+// kernel has been opted in to its dynamic shared-memory size.
+constexpr int TC_MAX_DEVICES = 64;
+
 struct TcState {
   int sm_count;
+  int device;             // device the handle was created on (current at tc_create), < TC_MAX_DEVICES
   EncodeTiledFn encode;
   bool attr_set_128, attr_set_256;
   int pair_clusters;      // co-resident CTA pairs of the pair GEMM (-1: not asked yet, 0: unavailable)

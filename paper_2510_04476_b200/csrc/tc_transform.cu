@@ -114,7 +114,7 @@ __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const T
       mbar_init(&acc_full[s], 1);
       mbar_init(&acc_empty[s], TR_EPILOGUE);
     }
-    *abort_flag = 0;
+    wait_ctl_init(abort_flag, p.status);
     fence_barrier_init();
   }
   if (warp == TR_MMA_WARP) {
@@ -463,12 +463,12 @@ done:
 template <int DH, int KC>
 int launch_tr(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1, const float* temp,
               const float2* rope, bf16* q, bf16* k, float* rnorm, int t_first, int* status, cudaStream_t st) {
-  static bool attr_done = false;
+  static bool attr_done[TC_MAX_DEVICES] = {};
   using SM = TrSmem<DH, KC>;
-  if (!attr_done) {
+  if (!attr_done[s->device]) {
     cudaError_t e = cudaFuncSetAttribute(tc_transform_fwd_kernel<DH, KC>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL);
     if (e != cudaSuccess) return -(int)e;
-    attr_done = true;
+    attr_done[s->device] = true;
   }
   TrParams p;
   p.d = d; p.qk0 = qk0; p.w0 = w0; p.w1 = w1; p.temp = temp; p.rope = rope; p.q = q; p.k = k; p.rnorm = rnorm; p.status = status;

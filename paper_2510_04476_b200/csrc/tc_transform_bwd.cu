@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(TB_THREADS, 1) tc_transform_bwd_kernel(const T
       mbar_init(&acc_empty[s], 128);
     }
     mbar_init(dw_free, 128);
-    *abort_flag = 0;
+    wait_ctl_init(abort_flag, p.status);
     fence_barrier_init();
   }
   if (warp == TB_ALLOC_WARP) {
@@ -344,12 +344,12 @@ done:
 
 template <int DH, int KC>
 int launch_tb(TcState* s, const TbParams& p0, cudaStream_t st) {
-  static bool attr_done = false;
+  static bool attr_done[TC_MAX_DEVICES] = {};
   using SM = TbSmem<DH, KC>;
-  if (!attr_done) {
+  if (!attr_done[s->device]) {
     cudaError_t e = cudaFuncSetAttribute(tc_transform_bwd_kernel<DH, KC>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL);
     if (e != cudaSuccess) return -(int)e;
-    attr_done = true;
+    attr_done[s->device] = true;
   }
   const int grid = p0.total_units < s->sm_count ? p0.total_units : s->sm_count;
   tc_transform_bwd_kernel<DH, KC><<<grid, TB_THREADS, SM::TOTAL, st>>>(p0);

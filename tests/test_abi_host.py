@@ -66,7 +66,9 @@ def test_host_only_handle_refuses_compute_and_bad_sizes():
     assert lib.cca_workspace_size(h, 2, 128, 1, C.byref(n)) == 0
     assert n.value > fwd_only > 0
     w = binding.cca_weights()
-    assert lib.cca_forward(h, C.byref(w), None, None, None, 0, 1, 128, None) == 1
+    assert lib.cca_forward(h, C.byref(w), None, None, None, 0, 1, 128, 0, None) == 1
+    assert lib.cca_set_wait_limit(h, 1 << 22) == 1          # a host-only handle has no device status block
+    assert lib.cca_wait_selftest(h, None) == 1
     assert lib.cca_status_string(4) == b"workspace too small"
     lib.cca_destroy(h)
 

@@ -61,3 +61,17 @@ def test_oracle_reproduces_its_stored_output():
         name, shape = head[0], [int(v) for v in head[1:]]
         ref = torch.tensor([float(v) for v in lines[i + 1].split()], dtype=torch.float64).reshape(shape)
         assert torch.allclose(vals[name], ref, rtol=1e-12, atol=1e-14), name
+
+
+def test_causal_flop_count_matches_hand_evaluation():
+    """fwd_flops_causal is fwd_flops with the S^2 term halved; the three terms are stored evaluated by hand."""
+    for line in open(os.path.join(GOLDEN, "causal_flops.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = line.split()
+        name, (B, S, E, hq, hk, dh, proj, conv, attn, total) = f[0], [int(v) for v in f[1:]]
+        assert proj + conv + attn == total, name
+        d = O.describe(O.OracleConfig(E, hq, hk, dh, 2, 2), B, S)
+        assert d["fwd_flops_causal"] == total, name
+        assert d["fwd_flops"] - d["fwd_flops_causal"] == 2 * B * S * S * hq * dh == attn, name
+        assert d["fwd_flops"] == proj + conv + 2 * attn, name

@@ -1,8 +1,12 @@
 """Random shapes outside the benchmark configurations: forward, backward, decode continuation and chunked prefill
-against the oracle.  A guard against logic errors (indexing, tails, flag combinations), so the element-wise bound
-1e-2 + 1e-2 |ref| is applied with a tail allowance: at the widest shapes drawn here (E = 4096, 16 query heads) the
-bf16-operand pipeline leaves up to 0.03 % of the input-gradient elements above it, by a factor of at most 2.2 (rms
-error 0.3-0.6 % of the rms value); a wrong index or a dropped term is off by orders of magnitude more."""
+against the oracle.  A guard against logic errors (indexing, tails, flag combinations).  Outputs (prefill and
+decode) get no tail allowance: every element is within 1e-2 + 1e-2 |ref| plus six standard deviations of the
+rounding noise of its own sum (tests/util.py::check_out_wide; the widest shapes drawn here, d_model 4096 against
+65 keys, have outputs of rms 1.1, where the bf16 rounding of o alone is a third of the absolute 1e-2).  The input
+gradient gets a tail allowance:
+at the widest shapes drawn here (E = 4096, 16 query heads) the bf16-operand pipeline leaves up to 0.03 % of its
+elements above the bound, by a factor of at most 2.2 (rms error 0.3-0.6 % of the rms value); a wrong index or a
+dropped term is off by orders of magnitude more.  Parameter gradients: tests/util.py::check_param_grads."""
 import random
 
 import pytest
@@ -10,11 +14,10 @@ import torch
 
 from oracle import cca_oracle as O
 from paper_2510_04476_b200 import synth
-from tests.test_gpu_parity import temp_scale
-from tests.util import PARAM_NAMES, check_close, oracle_cfg, to_device
+from tests.util import check_close, check_out_wide, check_param_grads, oracle_cfg, to_device
 
 pytestmark = pytest.mark.gpu
-TAIL = (1e-3, 3.0)
+DX_TAIL = (1e-3, 3.0)       # input gradient only
 
 
 def draw(seed):
@@ -55,11 +58,9 @@ def test_random_shape(seed):
     d_x, grads = cca.backward(dev, dev["x"], dev["d_out"], ws)
     torch.cuda.synchronize()
     assert cca.last_status() == 0
-    check_close("out", out, out_ref, tail=TAIL)
-    check_close("d_x", d_x, G["d_x"], tail=TAIL)
-    rss = temp_scale(sh, t, I, G)
-    for n in PARAM_NAMES:
-        check_close("d_" + n, grads["d_" + n], G["d_" + n], scale_abs=True, scale=rss if n == "temp" else None, tail=TAIL)
+    model = check_out_wide(cfg, t, I, "out", out, out_ref)
+    check_close("d_x", d_x, G["d_x"], tail=DX_TAIL)
+    check_param_grads(cfg, t, I, G, grads, model=model)
     if sh.causal and sh.S >= 2:
         # the last three tokens again, one at a time against the cache of a shorter prefill
         S0 = max(1, sh.S - 3)
@@ -73,7 +74,7 @@ def test_random_shape(seed):
         for tok in range(S0, sh.S):
             o = cca.decode_step(dev, dev["x"][:, tok].contiguous(), st, sh.S, dws)
             st["pos"] += 1
-            check_close(f"decode[{tok}]", o, out_ref[:, tok], tail=TAIL)
+            check_out_wide(cfg, t, I, f"decode[{tok}]", o, out_ref[:, tok], rows=tok, model=model)
     if sh.causal and sh.B == 1 and (sh.flags & 2) and (sh.head_dim == 64 or (sh.head_dim == 128 and sh.k_ch <= 2)):
         cut = (sh.S // 2) // 256 * 256
         if cut >= 512 and sh.S - cut >= 512:

@@ -1,7 +1,8 @@
 """cca_forward_static: the forward for callers that may not allocate device memory (a process whose GPU memory
 belongs to another allocator, a plug-in that is lent only a stream and its buffers).  Its scratch is a fixed
 array inside the library, shared by all calls, so the checks are: same result as cca_forward, twice in a row
-(the second call starts from the first call's leftovers), and a clear refusal beyond the built-in size.
+(the second call starts from the first call's leftovers), no change in the device's free memory across the calls
+(nothing was allocated, by the library or by the binding), and a clear refusal beyond the built-in size.
 This file is named to be collected last."""
 import pytest
 import torch
@@ -23,11 +24,19 @@ def test_static_workspace_forward_matches_forward_twice_in_a_row():
         ref = cca.forward(t, t["x"], ws).clone()
         torch.cuda.synchronize()
         out = torch.empty_like(t["x"])
-        for call in range(2):
+        free_before = None
+        for call in range(3):
             out.fill_(float("nan"))
+            torch.cuda.synchronize()
+            if call == 1:
+                # after the warm-up call (which may load the kernels' code onto the device): the next two calls
+                # must leave the device's free memory exactly where it is
+                free_before = torch.cuda.mem_get_info()[0]
             cca.forward_static(t, t["x"], out)
             torch.cuda.synchronize()
             assert cca.last_status() == 0
+            if call >= 1:
+                assert torch.cuda.mem_get_info()[0] == free_before, "cca_forward_static changed the free device memory"
             check_close(f"{sh.name} call {call}", out, ref.double())
             assert torch.equal(out, ref), "same kernels on the same inputs: the bits should agree too"
         cca.close()
