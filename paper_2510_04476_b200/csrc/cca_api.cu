@@ -36,9 +36,11 @@ namespace {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
-  size_t qk0, q, k, v, o, lse, rope, rnorm, w_all, y1s, y2, saved_end;
+  size_t qk0, q, k, v, o, lse, rope, rnorm, w_all, y1s, y2, qk0b, wc, saved_end;
   size_t o32, d_o, delta, dq, dk, dv, dlat, dy1, total_end;
 };
+
+CcaDims make_dims(const cca_config& c, int64_t B, int64_t S);
 
 Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
   Layout l;
@@ -60,6 +62,15 @@ Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
   if (c.head_dim > 128) {
     l.y1s = take(T * L * (size_t)c.k_ch * 2);
     l.y2 = take(T * L * 4);
+  }
+  // operands of the TMA-fed latent-transform kernel: a bf16 copy of qk0 and the composed conv weights
+  l.qk0b = l.wc = off;
+  {
+    CcaDims dd = make_dims(c, B, S);
+    if (tc_transform2_covers(dd)) {
+      l.qk0b = take(T * L * 2);
+      l.wc = take(tc_transform2_weight_bytes(dd));
+    }
   }
   l.saved_end = off;
   l.o32 = take(T * Lq * 4);
@@ -472,19 +483,31 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   // fp32 copy of o for the backward's delta = rowsum(dO * O)
   float* o32 = save_for_backward ? (float*)(ws + l.o32) : nullptr;
 
-  // The RoPE table does not depend on x: it is computed on a side stream while the down-projection runs.
+  // The RoPE table and the composed conv weights do not depend on x: they are computed on a side stream while the
+  // down-projection runs.
+  const bool use_t2 = h->impl >= 1 && h->tc && tc_transform2_covers(d) && w->conv1_w;
+  bf16* qk0b = use_t2 ? (bf16*)(ws + l.qk0b) : nullptr;
+  bf16* wc = use_t2 ? (bf16*)(ws + l.wc) : nullptr;
   bool forked = false;
-  if (c.flags & CCA_ROPE) {
+  if ((c.flags & CCA_ROPE) || use_t2) {
+    cudaStream_t ss = st;
     if (h->side) {
       CU(cudaEventRecord(h->ev_fork, st));
       CU(cudaStreamWaitEvent(h->side, h->ev_fork, 0));
-      CU(launch_rope_table(rope, d.S, d.dh, c.rope_base, h->side));
-      CU(cudaEventRecord(h->ev_join, h->side));
+      ss = h->side;
       forked = true;
-    } else {
-      CU(launch_rope_table(rope, d.S, d.dh, c.rope_base, st));
     }
-    h->launches++;
+    if (c.flags & CCA_ROPE) {
+      CU(launch_rope_table(rope, d.S, d.dh, c.rope_base, ss));
+      h->launches++;
+    }
+    if (use_t2) {
+      int cr = tc_transform2_compose(d, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, wc, ss);
+      if (cr < 0) { h->last_cuda = -cr; return CCA_ERR_CUDA; }
+      if (cr != 0) return CCA_ERR_INVALID_ARG;
+      h->launches++;
+    }
+    if (forked) CU(cudaEventRecord(h->ev_join, h->side));
   }
   // the three down-projection weights stacked (also the B operand of the input gradient in the backward)
   // (no copy if the caller keeps them adjacent in that order already)
@@ -505,10 +528,12 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
     g.M = T; g.N = d.L + d.Lk; g.K = d.E; g.a_row_off = 0; g.seq_len = d.S;
     g.out_bf16 = v; g.out_f32 = qk0; g.ldc = d.L;
     g.split_L = d.L; g.split_Lk = d.Lk; g.split_shift = (c.flags & CCA_V_SHIFT) ? 1 : 0;
+    g.out_lat_bf16 = (use_t2 && d.L % 32 == 0) ? qk0b : nullptr;
     int pr = tc_gemm_pair(h->tc, g, h->d_status, st);
     if (pr < 0) { h->last_cuda = -pr; return CCA_ERR_CUDA; }
     if (pr == 0) { fused = true; h->launches++; }
   }
+  const bool have_qk0b = fused && g.out_lat_bf16 != nullptr;
   if (!fused) {
     // Eq. 7: packed q/k down-projection
     g = GemmArgs{};
@@ -550,7 +575,12 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
     h->launches++;
   } else {
     bool done = false;
-    if (h->impl >= 1 && h->tc) {
+    if (have_qk0b) {
+      int tr = tc_transform2_fwd(h->tc, d, qk0, qk0b, wc, w->temp, rope, q, k, rnorm, h->d_status, st);
+      if (tr == 0) done = true;
+      if (tr < 0) { h->last_cuda = -tr; return CCA_ERR_CUDA; }
+    }
+    if (!done && h->impl >= 1 && h->tc) {
       int tr = tc_transform_fwd(h->tc, d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k,
                                 rnorm, h->d_status, st);
       if (tr == 0) done = true;
@@ -627,12 +657,24 @@ int cca_forward_chunk(cca_handle* h, const cca_weights* w, const void* x_chunk, 
   g.M = M; g.N = d.L + d.Lk; g.K = d.E; g.seq_len = (int)S_total; g.row0 = (int)t_begin;
   g.out_bf16 = v + (size_t)t_begin * d.Lk; g.out_f32 = qk0 + (size_t)t_begin * d.L; g.ldc = d.L;
   g.split_L = d.L; g.split_Lk = d.Lk; g.split_shift = (c.flags & CCA_V_SHIFT) ? 1 : 0;
+  // the TMA-fed transform kernel where it covers the configuration: bf16 copy of the chunk's qk0 rows, composed weights
+  const bool use_t2 = tc_transform2_covers(d) && d.L % 32 == 0;
+  bf16* qk0b = (bf16*)(ws + l.qk0b);
+  bf16* wc = (bf16*)(ws + l.wc);
+  if (use_t2) {
+    g.out_lat_bf16 = qk0b + (size_t)t_begin * d.L;
+    int cr = tc_transform2_compose(d, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, wc, st);
+    if (cr < 0) { h->last_cuda = -cr; return CCA_ERR_CUDA; }
+    if (cr != 0) return CCA_ERR_INVALID_ARG;
+    h->launches++;
+  }
   int pr = tc_gemm_pair(h->tc, g, h->d_status, st);
   if (pr < 0) { h->last_cuda = -pr; return CCA_ERR_CUDA; }
   if (pr != 0) return CCA_ERR_UNSUPPORTED;
   h->launches++;
-  int tr = tc_transform_fwd(h->tc, d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k, rnorm,
-                            h->d_status, st, (int)t_begin);
+  int tr = use_t2 ? tc_transform2_fwd(h->tc, d, qk0, qk0b, wc, w->temp, rope, q, k, rnorm, h->d_status, st, (int)t_begin)
+                  : tc_transform_fwd(h->tc, d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k,
+                                     rnorm, h->d_status, st, (int)t_begin);
   if (tr < 0) { h->last_cuda = -tr; return CCA_ERR_CUDA; }
   if (tr != 0) return CCA_ERR_UNSUPPORTED;
   h->launches++;

@@ -43,6 +43,7 @@ struct GemmArgs {
   long long ldc;
   int split_L, split_Lk, split_shift;
   int row0;          // fused output only: position inside its sequence of row 0 of A (a chunk of a longer sequence)
+  bf16* out_lat_bf16;   // fused output only, optional: a bf16 copy of columns [0, split_L) (row stride split_L)
 };
 
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);

@@ -34,6 +34,7 @@ struct G2Params {
   int splits, kb_per_split;   // work item = (tile, split)
   int vec_ok;
   int split_L, split_Lk, split_shift, seq_len, row0;   // fused down-projection output (see GemmArgs)
+  bf16* out_lat_bf16;
   int* status;
 };
 
@@ -232,6 +233,18 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
               for (int i = 0; i < 8; ++i)
                 reinterpret_cast<uint4*>(dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+              if (p.out_lat_bf16) {            // the operand copy the latent-transform kernel loads by TMA
+                bf16* dlb = p.out_lat_bf16 + (long long)m * p.split_L + n;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  uint4 v;
+                  v.x = pack_bf16(__uint_as_float(r[8 * i + 0]), __uint_as_float(r[8 * i + 1]));
+                  v.y = pack_bf16(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]));
+                  v.z = pack_bf16(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]));
+                  v.w = pack_bf16(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7]));
+                  reinterpret_cast<uint4*>(dlb)[i] = v;
+                }
+              }
             } else {
               const int vc = n - p.split_L;
               const bool late = p.split_shift && vc >= p.split_Lk / 2;
@@ -421,6 +434,8 @@ int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) 
   p.vec_ok = ((reinterpret_cast<uintptr_t>(outp) & 15) == 0) && ((g.ldc * esz) % 16 == 0);
   p.split_L = g.split_L; p.split_Lk = g.split_Lk; p.split_shift = g.split_shift; p.seq_len = g.seq_len > 0 ? g.seq_len : 1;
   p.row0 = g.row0;
+  p.out_lat_bf16 = (g.split_L > 0 && g.split_L % 32 == 0 && !(reinterpret_cast<uintptr_t>(g.out_lat_bf16) & 15)) ? g.out_lat_bf16 : nullptr;
+  if (g.out_lat_bf16 && !p.out_lat_bf16) return 1;
   p.status = d_status;
   // tile width: fewer, fuller waves of CTA pairs win (time of a wave is proportional to the tile width)
   auto cost = [&](int bn) {

@@ -23,6 +23,13 @@ int tc_attn_bwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, cons
 // Adjoint of conv2: dy1 [T, L] fp32 <- d_hat (dqh, dkh); d_w1 accumulates the conv2 weight gradient.
 int tc_transform_bwd(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1, const float* dqh,
                      const float* dkh, float* dy1, float* d_w1, int* d_status, cudaStream_t st);
+// The same stage with TMA-fed operands (tc_transform2.cu): needs a bf16 copy of qk0 (the fused down-projection writes
+// it) and the composed conv1 * conv2 weights wc that tc_transform2_compose forms from w0, w1 (tc_transform2_weight_bytes).
+size_t tc_transform2_weight_bytes(const CcaDims& d);
+bool tc_transform2_covers(const CcaDims& d);
+int tc_transform2_compose(const CcaDims& d, const bf16* w0, const bf16* w1, bf16* wc, cudaStream_t st);
+int tc_transform2_fwd(TcState* s, const CcaDims& d, const float* qk0, const bf16* qk0b, const bf16* wc, const float* temp,
+                      const float2* rope, bf16* q, bf16* k, float* rnorm, int* d_status, cudaStream_t st, int t_first = 0);
 int tc_transform_fwd(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1,
                      const float* temp, const float2* rope, bf16* q, bf16* k, float* rnorm, int* d_status,
                      cudaStream_t st, int t_first = 0);   // t_first > 0 (multiple of 128): only tokens [t_first, d.S)

@@ -30,37 +30,55 @@ def _r(x):
     return x.to(torch.bfloat16).to(F64)
 
 
-def term_rss(cfg, t, I, G):
-    """sqrt(sum over tokens of term^2) for every element of every matrix-shaped parameter gradient."""
+def term_rss(cfg, t, I, G, power=2):
+    """power = 2: sqrt(sum over tokens of term^2) for every element of every matrix-shaped parameter gradient (the
+    scale of a random walk over the terms).  power = 1: sum of |term| (the scale of the worst case, every rounding
+    in the same direction; used where a sum has too few terms for a random walk)."""
     B, S, E = I["x"].shape
     T = B * S
     L, Lk, dh = cfg.L, cfg.L_k, cfg.head_dim
     H = cfg.n_q_heads + cfg.n_kv_heads
-    x2 = I["x"].reshape(T, E) ** 2
+
+    def pw(v):
+        return v ** 2 if power == 2 else v.abs()
+
+    def root(v):
+        return v.sqrt() if power == 2 else v
+
+    def noisy_factor(v):
+        """|v| of the computed (hence noisy) factor of a term, floored per token by the rms over its head's channels:
+        the rounding noise of a latent-gradient element is at the scale of its head's typical element, not of its
+        own value, which may be a cancelling sum (over the query heads of a group, over the queries of a key)."""
+        vh = v.reshape(*v.shape[:-1], -1, dh)
+        floor = vh.pow(2).mean(dim=-1, keepdim=True).sqrt()
+        return torch.maximum(vh.abs(), floor).reshape(v.shape)
+
+    x2 = pw(I["x"].reshape(T, E))
     r = {}
-    r["w_qk"] = ((G["d_qk0"].reshape(T, L) ** 2).T @ x2).sqrt()
-    dv = G["d_v"].reshape(T, Lk)
-    r["w_v1"] = ((dv[:, :Lk // 2] ** 2).T @ x2).sqrt()
-    r["w_v2"] = ((dv[:, Lk // 2:] ** 2).T @ (I["xs"].reshape(T, E) ** 2)).sqrt()
-    r["w_o"] = ((O._f64(t["d_out"]).reshape(T, E) ** 2).T @ (I["o"].reshape(T, -1) ** 2)).sqrt()
+    r["w_qk"] = root(pw(noisy_factor(G["d_qk0"].reshape(T, L))).T @ x2)
+    dv = noisy_factor(G["d_v"].reshape(T, Lk))
+    r["w_v1"] = root(pw(dv[:, :Lk // 2]).T @ x2)
+    r["w_v2"] = root(pw(dv[:, Lk // 2:]).T @ pw(I["xs"].reshape(T, E)))
+    r["w_o"] = root(pw(O._f64(t["d_out"]).reshape(T, E)).T @ pw(noisy_factor(I["o"].reshape(T, -1))))
     k = cfg.k_seq
     c0 = torch.zeros(L, k, dtype=F64)
     if cfg.flags & O.CONV1:
+        dy1 = noisy_factor(G["d_y1"])
         for j in range(k):
             lag = k - 1 - j
             if lag < S:
-                c0[:, j] = (G["d_y1"][:, lag:] ** 2 * I["qk0"][:, :S - lag] ** 2).sum(dim=(0, 1))
-    r["conv0_w"] = c0.sqrt()
+                c0[:, j] = (pw(dy1[:, lag:]) * pw(I["qk0"][:, :S - lag])).sum(dim=(0, 1))
+    r["conv0_w"] = root(c0)
     k = cfg.k_ch
     c1 = torch.zeros(H, dh, dh, k, dtype=F64)
     if cfg.flags & O.CONV2:
-        dy2 = G["d_y2"].reshape(B, S, H, dh) ** 2
-        y1 = I["y1"].reshape(B, S, H, dh) ** 2
+        dy2 = pw(noisy_factor(G["d_y2"]).reshape(B, S, H, dh))
+        y1 = pw(I["y1"].reshape(B, S, H, dh))
         for j in range(k):
             lag = k - 1 - j
             if lag < S:
                 c1[..., j] = torch.einsum("bsho,bshi->hoi", dy2[:, lag:], y1[:, :S - lag])
-    r["conv1_w"] = c1.reshape(L, dh, k).sqrt()
+    r["conv1_w"] = root(c1.reshape(L, dh, k))
     return r
 
 
@@ -71,10 +89,15 @@ def out_term_rss(t, I):
     return (o2 @ (O._f64(t["w_o"]) ** 2).transpose(0, 1)).sqrt()
 
 
-def temp_term_rss(cfg, I, G):
-    """sqrt(sum of term^2) of d_temp, one number per kv head.  d_temp[j] = sum over the (query, key) pairs of the
-    group's heads of dS * logit (Eq. 11: the temperature scales every logit of its kv head), so the terms are
-    those products; they come from the oracle's q, k, v, o and d_o exactly as its attention adjoint forms them."""
+def temp_term_rss(cfg, I, G, power=2):
+    """Noise scale of d_temp, one number per kv head.  d_temp[j] = sum over the (query, key) pairs of the group's
+    heads of dS * logit (Eq. 11: the temperature scales every logit of its kv head), so the terms are those
+    products, formed from the oracle's q, k, v, o and d_o exactly as its attention adjoint forms them: sqrt(sum of
+    term^2) (power = 2) or sum of |term| (power = 1).  One more contribution enters in quadrature (power = 2) or
+    is added (power = 1): a row of dS sums to zero only as far as delta = rowsum(dO * O) agrees with the
+    probabilities the backward recomputes, and O was accumulated from bf16-rounded probabilities; the residual of row
+    t, of scale sqrt(sum_s (P_s (dP_s - delta_t))^2) roundings, multiplies the row's mean logit sum_s P_s s_s, which
+    is not small when the keys a row attends to are aligned with its query."""
     q, k, v, o, do = I["q"], I["k"], I["v"], I["o"], G["d_o"]
     B, S, hq, dh = q.shape
     g = cfg.g
@@ -96,8 +119,13 @@ def temp_term_rss(cfg, I, G):
                 doi = do[b, r0:r1, i, :]
                 D = (doi * o[b, r0:r1, i, :]).sum(dim=-1, keepdim=True)
                 ds = p * (doi @ vj.transpose(0, 1) - D)
-                acc[j] += (ds * s).pow(2).sum()
-    return acc.sqrt()
+                s0 = torch.where(torch.isfinite(sm), s, torch.zeros_like(s))
+                sbar = (p * s0).sum(dim=-1)
+                if power == 2:
+                    acc[j] += (ds * s0).pow(2).sum() + (sbar.pow(2) * ds.pow(2).sum(dim=-1)).sum()
+                else:
+                    acc[j] += (ds * s0).abs().sum() + (sbar.abs() * ds.abs().sum(dim=-1)).sum()
+    return acc.sqrt() if power == 2 else acc
 
 
 def _attention_bf16_storage(q, k, v, do, g, causal):
@@ -215,10 +243,17 @@ def noisy(rss):
     return U * rss > NOISE_FLOOR
 
 
+MIN_NOISY = 64            # fewer noisy elements than this measure nothing
+
+
 def kappa(model, exact, rss):
     """Effective number of bf16 roundings per term: rms of the model's error in units of 2^-9 * rss, over the
-    `noisy` elements.  Never below 1 (one rounding is the least such a path can have)."""
+    `noisy` elements (over every element with terms at all if fewer than MIN_NOISY are noisy: the gradient is then
+    tiny against the absolute 1e-2 and the figure hardly matters).  Never below 1 (one rounding is the least such a
+    path can have)."""
     m = noisy(rss)
+    if int(m.sum()) < MIN_NOISY:
+        m = rss > 0
     if not bool(m.any()):
         return 1.0
     z = (model - exact)[m] / (U * rss[m])
