@@ -32,10 +32,25 @@ UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAK_TFLOPS = 1590.0
 TRAIN_WORKLOADS = {"cfg2_small", "cfg4_train"}
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the attention-forward kernel as it stands, from
-# the full ncu capture summarised under profiles/ (set to None when the kernel changes until it is re-captured)
-ATTN_BWD_DRAM_BYTES = {"cfg4_train": 109093632 + 11924736 + 87101184 + 29619456}     # dK/dV kernel + dQ kernel
-ATTN_FWD_DRAM_BYTES = {"cfg3_prefill16k": 50386432 + 2622464}
+
+
+def dram_traffic(kernel: str, workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of `kernel` at `workload`, from the ncu captures
+    recorded in profiles/dram_traffic.json.  An entry names the source file of its kernel and that file's sha256 at
+    capture time: once the file has changed the figure is stale and None is returned."""
+    import hashlib
+    try:
+        entries = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic.json")))["entries"]
+    except Exception:
+        return None
+    for e in entries:
+        if e.get("kernel") == kernel and e.get("workload") == workload:
+            try:
+                cur = hashlib.sha256(open(os.path.join(ROOT, e["source"]), "rb").read()).hexdigest()
+            except Exception:
+                return None
+            return int(e["bytes"]) if cur == e.get("source_sha256") else None
+    return None
 
 
 def flops_of(sh, backward: bool):
@@ -57,6 +72,103 @@ def measured_peak():
         except Exception:
             pass
     return FALLBACK_PEAK_TFLOPS, "fallback", {}
+
+
+def stage_table(sh, backward):
+    """(name, first event, last event, bound, algorithmic work per launch) of every stage between two stage events.
+    Tensor stages: FLOPs of the contraction.  HBM stages: the bytes the stage must move if nothing is re-read
+    (latents in the precision they are kept in)."""
+    T, E, L, Lq, Lk, dh = sh.B * sh.S, sh.d_model, sh.L, sh.L_q, sh.L_k, sh.head_dim
+    attn = (2 if sh.causal else 4) * sh.B * sh.S * sh.S * Lq
+    H = sh.n_q_heads + sh.n_kv_heads
+    rows = [
+        ("down-projection (q|k|v in one contraction)", "fwd_begin", "fwd_proj", "tensor", 2 * T * E * (L + Lk)),
+        ("latent transforms (convs, q-k-mean, norm, RoPE)", "fwd_proj", "fwd_transform", "hbm", 2 * T * L + 2 * T * L),
+        ("latent attention forward", "fwd_transform", "fwd_attn", "tensor", attn),
+        ("up-projection", "fwd_attn", "fwd_end", "tensor", 2 * T * Lq * E),
+    ]
+    if backward:
+        rows += [
+            ("d_o = d_out W_o", "bwd_begin", "bwd_do", "tensor", 2 * T * E * Lq),
+            ("d_W_o = d_out^T o", "bwd_do", "bwd_dwo", "tensor", 2 * T * E * Lq),
+            ("delta = rowsum(dO o O)", "bwd_dwo", "bwd_delta", "hbm", 4 * T * Lq + 2 * T * Lq + 4 * T * sh.n_q_heads),
+            ("latent attention backward (dK/dV and dQ kernels)", "bwd_delta", "bwd_attn", "tensor", 2.5 * attn),
+            ("norm / RoPE adjoint, d_temp", "bwd_attn", "bwd_norm", "hbm", 2 * (4 * T * L) + 2 * T * L + 4 * T * H),
+            ("conv2 adjoint, d_conv1_w", "bwd_norm", "bwd_conv2", "hbm", 4 * T * L + 4 * T * L + 4 * T * L),
+            ("conv1 and q-k-mean adjoint, d_conv0_w", "bwd_conv2", "bwd_conv1", "hbm", 3 * (4 * T * L) + 2 * T * L),
+            ("value-unshift", "bwd_conv1", "bwd_pack", "hbm", 4 * T * Lk + 2 * T * Lk),
+            ("down-projection weight gradients", "bwd_pack", "bwd_dw", "tensor", 2 * T * (L + Lk) * E),
+            ("d_x", "bwd_dw", "bwd_end", "tensor", 2 * T * (L + Lk) * E),
+        ]
+    return rows
+
+
+def per_kernel_roofline(cca, step, sh, backward, n=5):
+    """Every stage of the step bracketed by CUDA events the library records on the launching stream
+    (cca_set_stage_events); a few extra steps outside the timed region.  Fractions are of the measured peaks."""
+    from paper_2510_04476_b200.binding import CCA
+    names = CCA.STAGE_EVENTS
+    sets = [[torch.cuda.Event(enable_timing=True) for _ in names] for _ in range(n)]
+    torch.cuda.synchronize()
+    for evs in sets:
+        for e in evs:
+            e.record()
+    torch.cuda.synchronize()
+    for evs in sets:
+        cca.set_stage_events(evs)
+        step()
+    torch.cuda.synchronize()
+    cca.set_stage_events(None)
+    tf_peak, tf_kind, _ = measured_peak()
+    hbm, hbm_kind = hbm_peak()
+    idx = {nm: i for i, nm in enumerate(names)}
+    out = []
+    for name, a, b, bound, work in stage_table(sh, backward):
+        try:
+            ms = sum(evs[idx[a]].elapsed_time(evs[idx[b]]) for evs in sets) / n
+        except Exception:
+            continue
+        if ms <= 0:
+            continue
+        if bound == "tensor":
+            ach, peak, unit, kind = work / (ms * 1e-3) / 1e12, tf_peak, "TFLOP/s", tf_kind
+        else:
+            ach, peak, unit, kind = work / (ms * 1e-3) / 1e9, hbm, "GB/s", hbm_kind
+        out.append({"kernel": name, "bound": bound, "ms": ms, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                    "peak_kind": kind, "work_per_launch": work})
+    return out
+
+
+def sustained(step, barrier, fl_total, seconds, index):
+    """The step back to back for `seconds`: throughput under the power cap, with the SM clock sampled meanwhile,
+    against the measured sustained GEMM rate."""
+    sampler = ClockSampler(index)
+    sampler.start()
+    time.sleep(0.15)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0 = time.time()
+    e0.record()
+    n = 0
+    while time.time() - w0 < seconds:
+        for _ in range(50):
+            step()
+        n += 50
+        if n % 500 == 0:
+            torch.cuda.synchronize()             # keep the launch queue bounded
+    e1.record()
+    barrier()
+    w1 = time.time()
+    clocks = sampler.stop(w0, w1)
+    ms = e0.elapsed_time(e1) / n
+    tf = fl_total / (ms * 1e-3) / 1e12
+    try:
+        peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops_sustained"])
+        kind = "measured (cuBLAS bf16, seconds-long loop)"
+    except Exception:
+        peak, kind = 1400.0, "fallback"
+    return {"seconds": w1 - w0, "steps": n, "ms_per_step": ms, "tflops": tf, "peak": peak, "peak_kind": kind,
+            "frac": tf / peak, "clocks": clocks}
 
 
 class ClockSampler:
@@ -294,11 +406,16 @@ def run_ours(args, rank, world, local_rank):
                      "unit": "TFLOP/s", "frac": attn_tflops / peak, "peak_kind": peak_kind,
                      "frac_of_nominal_2250": attn_tflops / NOMINAL_BF16_TFLOPS, "ms_per_launch": attn_ms,
                      "flops_per_launch": fl[attn_key],
-                     "traffic": ATTN_FWD_DRAM_BYTES.get(sh.name) if args.kernels and not backward else
-                                (ATTN_BWD_DRAM_BYTES.get(sh.name) if args.kernels else None)},
+                     "traffic": (dram_traffic("attention_backward" if backward else "attention_forward", sh.name)
+                                 if args.kernels else None)},
         "pct_of_nominal_bf16_peak": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
         "device_status": status,
     }
+    if rank == 0 and args.kernels:
+        line["roofline_per_kernel"] = per_kernel_roofline(cca, step, sh, backward)
+    if rank == 0 and world == 1 and args.sustain > 0:
+        line["sustained"] = sustained(step, barrier, fl["total"], args.sustain,
+                                      vis[local_rank] if local_rank < len(vis) else str(local_rank))
     if rank == 0 and world == 1 and not args.no_mha and not backward:
         line["mha_same_shape"] = mha_compare(sh, args, ms_step, attn_ms, local_rank)
         line["forward_backward_same_shape"] = fwd_bwd_same_shape(sh, args, local_rank)
@@ -312,10 +429,6 @@ def run_ours(args, rank, world, local_rank):
     if dist is not None:
         dist.destroy_process_group()
 
-
-# dram bytes (read + write) of one launch of the decode attention kernel as it stands, from the full ncu capture
-# summarised under profiles/ (None when the kernel has changed since)
-DECODE_ATTN_DRAM_BYTES = {"decode16k": 537121536 + 5351936}
 
 DECODE_WORKLOADS = {
     # model of the 16k prefill shape; 32 sequences, each with 16384 cached tokens
@@ -449,7 +562,7 @@ def run_decode(args, rank, world, local_rank):
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "decode attention over the latent cache", "achieved": attn_gbs, "peak": peak,
                      "unit": "GB/s", "frac": attn_gbs / peak, "peak_kind": peak_kind, "ms_per_launch": attn_ms,
-                     "bytes_per_launch": by["cache"], "traffic": DECODE_ATTN_DRAM_BYTES.get(args.workload)},
+                     "bytes_per_launch": by["cache"], "traffic": dram_traffic("decode_attention", args.workload)},
         "step_gbs": by["total"] / (ms_step * 1e-3) / 1e9, "step_bytes": by,
         "device_status": status,
     }
@@ -562,6 +675,8 @@ def main():
     ap.add_argument("--kernels", type=int, default=1, help="0 = SIMT kernels only, 1 = tcgen05 kernels where available")
     ap.add_argument("--backward", action="store_true", help="time forward + backward on a forward-only workload too")
     ap.add_argument("--no-mha", action="store_true")
+    ap.add_argument("--sustain", type=float, default=3.0,
+                    help="seconds of back-to-back steps for the sustained (power-capped) figure; 0 = skip")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

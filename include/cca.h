@@ -252,6 +252,22 @@ int cca_set_impl(cca_handle* h, int impl);
  * which therefore overwrites what the forward of the same step recorded. */
 int cca_set_attention_events(cca_handle* h, void* ev_begin, void* ev_end);
 
+/* Profiling hook, finer: CCA_N_STAGE_EVENTS cudaEvent_t (or null to clear) that cca_forward and cca_backward record on
+ * the caller's stream at their stage boundaries, so that the time between two consecutive events is one stage:
+ * forward   BEGIN | down-projection (Eq. 7, 10) | PROJ | latent transforms (Eq. 8, 9, 11) | TRANSFORM | attention
+ *           (Eq. 11) | ATTN | up-projection | END;
+ * backward  BEGIN | d_o = d_out W_o | DO | d_W_o | DWO | delta | DELTA | attention adjoint | ATTN | norm / RoPE
+ *           adjoint | NORM | conv2 adjoint | CONV2 | conv1 and q-k-mean adjoint | CONV1 | value-unshift | PACK |
+ *           down-projection weight gradients | DW | d_x | END.
+ * Events the configuration's path does not reach (CONV2 without the tensor-core conv2 adjoint) are not recorded.
+ * Recording costs a little stream time: time whole steps without it. */
+enum {
+  CCA_EV_FWD_BEGIN = 0, CCA_EV_FWD_PROJ, CCA_EV_FWD_TRANSFORM, CCA_EV_FWD_ATTN, CCA_EV_FWD_END,
+  CCA_EV_BWD_BEGIN, CCA_EV_BWD_DO, CCA_EV_BWD_DWO, CCA_EV_BWD_DELTA, CCA_EV_BWD_ATTN, CCA_EV_BWD_NORM, CCA_EV_BWD_CONV2,
+  CCA_EV_BWD_CONV1, CCA_EV_BWD_PACK, CCA_EV_BWD_DW, CCA_EV_BWD_END, CCA_N_STAGE_EVENTS
+};
+int cca_set_stage_events(cca_handle* h, void* const* events, int n);
+
 /* Number of kernel launches the library has enqueued through this handle so far. */
 int64_t cca_launch_count(const cca_handle* h);
 

@@ -75,6 +75,7 @@ SYMBOLS = {
                                                 C.POINTER(cca_decode_state), C.c_void_p]),
     "cca_set_impl": (C.c_int, [C.c_void_p, C.c_int]),
     "cca_set_attention_events": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cca_set_stage_events": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
     "cca_launch_count": (C.c_int64, [C.c_void_p]),
     "cca_last_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int)]),
     "cca_set_wait_limit": (C.c_int, [C.c_void_p, C.c_int64]),
@@ -195,6 +196,21 @@ class CCA:
         b = C.c_void_p(begin.cuda_event) if begin is not None else None
         e = C.c_void_p(end.cuda_event) if end is not None else None
         _check(self.lib, self.lib.cca_set_attention_events(self.handle, b, e), self.handle, "set_attention_events")
+
+    STAGE_EVENTS = ["fwd_begin", "fwd_proj", "fwd_transform", "fwd_attn", "fwd_end", "bwd_begin", "bwd_do", "bwd_dwo",
+                    "bwd_delta", "bwd_attn", "bwd_norm", "bwd_conv2", "bwd_conv1", "bwd_pack", "bwd_dw", "bwd_end"]
+
+    def set_stage_events(self, events):
+        """cca_set_stage_events: a list of len(STAGE_EVENTS) torch.cuda.Event(enable_timing=True), or None to clear."""
+        if events is None:
+            _check(self.lib, self.lib.cca_set_stage_events(self.handle, None, 0), self.handle, "cca_set_stage_events")
+            return
+        assert len(events) == len(self.STAGE_EVENTS)
+        for e in events:
+            if e.cuda_event == 0:
+                e.record(torch.cuda.current_stream(self.device))      # forces creation of the handle
+        arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+        _check(self.lib, self.lib.cca_set_stage_events(self.handle, arr, len(events)), self.handle, "cca_set_stage_events")
 
     def launch_count(self) -> int:
         return int(self.lib.cca_launch_count(self.handle))

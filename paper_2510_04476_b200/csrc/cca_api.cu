@@ -26,6 +26,7 @@ struct cca_handle {
   cudaStream_t s_in, s_out;
   cudaEvent_t ev_chunk[2][64];              // [arrived / computed][chunk]
   int n_ev;                                 // events created so far
+  cudaEvent_t stage_ev[CCA_N_STAGE_EVENTS]; // optional, recorded at the stage boundaries of forward and backward
   // what the last cca_forward kept for a backward: cca_backward refuses anything else
   const void* saved_ws;
   int64_t saved_B, saved_S;
@@ -116,6 +117,11 @@ int check_sizes(const cca_handle* h, int64_t B, int64_t S, bool need_device = fa
       h->last_cuda = (int)e_;                      \
       return CCA_ERR_CUDA;                         \
     }                                              \
+  } while (0)
+
+#define STAGE(idx)                                                         \
+  do {                                                                     \
+    if (h->stage_ev[idx]) CU(cudaEventRecord(h->stage_ev[idx], st));       \
   } while (0)
 
 GemmOperand kmajor(const void* p, long long ld) { return GemmOperand{(const bf16*)p, ld, 1}; }
@@ -215,6 +221,7 @@ int cca_init(const cca_config* cfg, int device, cca_handle** out) {
   h->side = nullptr; h->ev_fork = h->ev_join = nullptr;
   h->s_in = h->s_out = nullptr; h->n_ev = 0;
   h->saved_ws = nullptr; h->saved_B = h->saved_S = 0;
+  for (int i = 0; i < CCA_N_STAGE_EVENTS; ++i) h->stage_ev[i] = nullptr;
   if (device >= 0) {
     if (cudaMalloc(&h->d_status, 64) != cudaSuccess || cudaMemset(h->d_status, 0, 64) != cudaSuccess) {
       if (h->d_status) cudaFree(h->d_status);
@@ -263,6 +270,12 @@ int cca_set_attention_events(cca_handle* h, void* ev_begin, void* ev_end) {
   if (!h) return CCA_ERR_INVALID_ARG;
   h->ev_attn_begin = (cudaEvent_t)ev_begin;
   h->ev_attn_end = (cudaEvent_t)ev_end;
+  return CCA_OK;
+}
+
+int cca_set_stage_events(cca_handle* h, void* const* events, int n) {
+  if (!h || (events && n != CCA_N_STAGE_EVENTS)) return CCA_ERR_INVALID_ARG;
+  for (int i = 0; i < CCA_N_STAGE_EVENTS; ++i) h->stage_ev[i] = events ? (cudaEvent_t)events[i] : nullptr;
   return CCA_OK;
 }
 
@@ -483,6 +496,7 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   // fp32 copy of o for the backward's delta = rowsum(dO * O)
   float* o32 = save_for_backward ? (float*)(ws + l.o32) : nullptr;
 
+  STAGE(CCA_EV_FWD_BEGIN);
   // The RoPE table and the composed conv weights do not depend on x: they are computed on a side stream while the
   // down-projection runs.
   const bool use_t2 = h->impl >= 1 && h->tc && tc_transform2_covers(d) && w->conv1_w;
@@ -550,6 +564,7 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
   }
   // Eq. 8, 9, 11: convs, q-k-mean, norm, temperature, RoPE
   if (forked) CU(cudaStreamWaitEvent(st, h->ev_join, 0));
+  STAGE(CCA_EV_FWD_PROJ);
   if (d.dh > 128) {
     // unfused: conv1 at the taps conv2 reads, conv2 as one contraction per head over (input channel, tap), then the
     // per-(token, head) stages
@@ -590,16 +605,19 @@ int cca_forward(cca_handle* h, const cca_weights* w, const void* x, void* out, v
       CU(launch_transform_fwd(d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, w->temp, rope, q, k, rnorm, st));
     h->launches++;
   }
+  STAGE(CCA_EV_FWD_TRANSFORM);
   // Eq. 11: attention in the latent
   // with the norm stage on, the logits are bounded by sqrt(d_h) exp(temp): the kernel may use that as the row maximum
   if ((r = run_attention_fwd(h, d, q, k, v, o, o32, lse, (c.flags & CCA_QK_NORM) ? w->temp : nullptr, st)) != CCA_OK)
     return r;
+  STAGE(CCA_EV_FWD_ATTN);
   // Eq. 11: up-projection
   g = GemmArgs{};
   g.A = kmajor(o, d.Lq); g.B = kmajor(w->w_o, d.Lq);
   g.M = T; g.N = d.E; g.K = d.Lq; g.a_row_off = 0; g.seq_len = d.S;
   g.out_bf16 = (bf16*)out; g.ldc = d.E;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  STAGE(CCA_EV_FWD_END);
   if (save_for_backward) { h->saved_ws = workspace; h->saved_B = B; h->saved_S = S; }
   return CCA_OK;
 }
@@ -807,6 +825,7 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
                                                                                          : (const bf16*)(ws + l.w_all);
   const long long ldl = d.L + d.Lk;
 
+  STAGE(CCA_EV_BWD_BEGIN);
   CU(cudaMemsetAsync(gr->d_conv0_w, 0, (size_t)d.L * c.k_seq * 4, st));
   CU(cudaMemsetAsync(gr->d_conv1_w, 0, (size_t)d.L * d.dh * c.k_ch * 4, st));
   CU(cudaMemsetAsync(gr->d_temp, 0, (size_t)d.hk * 4, st));
@@ -815,13 +834,16 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   g.A = kmajor(d_out, d.E); g.B = mmajor(w->w_o, d.Lq);
   g.M = T; g.N = d.Lq; g.K = d.E; g.seq_len = d.S; g.out_bf16 = d_o; g.ldc = d.Lq;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  STAGE(CCA_EV_BWD_DO);
   g = GemmArgs{};
   g.A = mmajor(d_out, d.E); g.B = mmajor(o, d.Lq);
   g.M = d.E; g.N = d.Lq; g.K = T; g.seq_len = d.S; g.out_f32 = gr->d_w_o; g.ldc = d.Lq;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  STAGE(CCA_EV_BWD_DWO);
   // attention adjoint
   CU(launch_attn_delta(d, o32, d_o, delta, st));
   h->launches++;
+  STAGE(CCA_EV_BWD_DELTA);
   {
     if (h->ev_attn_begin) CU(cudaEventRecord(h->ev_attn_begin, st));
     bool done = false;
@@ -834,8 +856,10 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
     h->launches += 2;
     if (h->ev_attn_end) CU(cudaEventRecord(h->ev_attn_end, st));
   }
+  STAGE(CCA_EV_BWD_ATTN);
   // latent-transform adjoints
   CU(launch_transform_bwd_norm(d, q, k, rnorm, w->temp, rope, dq, dk, gr->d_temp, st));
+  STAGE(CCA_EV_BWD_NORM);
   {
     bool done = false;
     if (h->impl >= 1 && h->tc) {
@@ -844,6 +868,7 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
                                 gr->d_conv1_w, h->d_status, st);
       if (tr < 0) { h->last_cuda = -tr; return CCA_ERR_CUDA; }
       if (tr == 0) {
+        STAGE(CCA_EV_BWD_CONV2);
         CU(launch_conv1_adjoint(d, dy1, dq, dk, qk0, (const bf16*)w->conv0_w, dlat, ldl, gr->d_conv0_w, st));
         done = true;
       }
@@ -854,8 +879,10 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
       CU(launch_transform_bwd_w1(d, qk0, (const bf16*)w->conv0_w, dq, dk, gr->d_conv1_w, st));
     }
   }
+  STAGE(CCA_EV_BWD_CONV1);
   CU(launch_pack_dv(d, dv, dlat, ldl, st));
   h->launches += 4;
+  STAGE(CCA_EV_BWD_PACK);
   // down-projection adjoints: parameter gradients
   g = GemmArgs{};
   g.A = mmajor(dlat, ldl); g.B = mmajor(x, d.E);
@@ -871,11 +898,13 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
     g.A = mmajor(dlat + d.L + d.Lk / 2, ldl); g.out_f32 = gr->d_w_v2;
     if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
   }
+  STAGE(CCA_EV_BWD_DW);
   // input gradient: d_x = [d_qk0, d_v1, d_v2 moved one token earlier] [W_qk; W_v1; W_v2] (stacked by the forward)
   g = GemmArgs{};
   g.A = kmajor(dlat, ldl); g.B = mmajor(w_all, d.E);
   g.M = T; g.N = d.E; g.K = (int)ldl; g.seq_len = d.S; g.out_bf16 = (bf16*)d_x; g.ldc = d.E;
   if ((r = run_gemm(h, g, st)) != CCA_OK) return r;
+  STAGE(CCA_EV_BWD_END);
   return CCA_OK;
 }
 

@@ -633,6 +633,11 @@ int tc_attn_bwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, cons
   if (!s || !s->encode) return 1;
   if (d.dh != 64 && d.dh != 128) return 1;
   if (d.Lq % 8 || d.Lk % 8) return 1;
+  if (d.dh == 64 && s->attn_bwd_fused) {
+    // one kernel that visits every (query, key) pair once; dQ by vector reductions into memory
+    const int r = tc_attn_bwd_fused(s, d, q, k, v, d_o, lse, delta, dq, dk, dv, d_status, st);
+    if (r != 1) return r;
+  }
   CUtensorMap tmQ, tmK, tmV, tmDO;
   const uint64_t S = (uint64_t)d.S, B = (uint64_t)d.B, Lq = (uint64_t)d.Lq, Lk = (uint64_t)d.Lk;
   if (!tc_make_map_3d(s, &tmQ, q, Lq, S, B, Lq, S * Lq, 64, 128)) return 1;

@@ -1,0 +1,427 @@
+// Tensor-core kernels, part 4b: adjoint of the softmax attention of Eq. 11 in ONE kernel (head size 64).
+//
+// The two-kernel adjoint (tc_attn_bwd.cu) recomputes S and dP in each kernel: seven contractions and two
+// exponentials per (query, key) pair where the adjoint itself has five and one.  At head size 64 a score costs only
+// 256 tensor FLOPs per contraction, so the exponentials and the element-wise chain bound both kernels; here every
+// pair is visited once.
+//
+// One CTA = 128 keys of one (sequence, kv head); it walks the g query heads of the group and, for each, the query
+// tiles that see these keys (thread = key, transposed tiles S^T = K Q^T, dP^T = V dO^T as in the dK/dV kernel), so
+// that dV += P^T dO and dK += dS^T Q accumulate in TMEM over the whole walk with P^T and dS^T as TMEM operands.
+// The compute warps also leave dS^T as bf16 in shared memory ([key][query], 128-byte swizzle): read with the queries
+// as the M dimension it is the A operand of   dQ_tile = dS K   (M = 128 queries, N = d_h, K = 128 keys; the resident
+// K tile read along its rows is the B operand).  A query tile's dQ gets such a contribution from every key tile it
+// sees, i.e. from different CTAs: they are added into the zeroed fp32 dq with vector reductions (red.global.add.v4),
+// 16 values per thread and tile.  The sum order of dq therefore varies from run to run (fp32 rounding only).
+//
+// TMEM columns: S^T two 64-query buffers [0,128), dP^T likewise [128,256), dV [256,320), dK [320,384),
+// dQ two buffers [384,448) [448,512).
+#include "tc_kernels.cuh"
+#include "tc_ptx.cuh"
+#include "tc_state.cuh"
+
+using namespace tc;
+
+namespace {
+
+constexpr int FB_COMPUTE_WARPS = 16;
+constexpr int FB_TMA_WARP = FB_COMPUTE_WARPS, FB_MMA_WARP = FB_COMPUTE_WARPS + 1;
+constexpr int FB_THREADS = 32 * (FB_COMPUTE_WARPS + 2);
+constexpr float FB_LOG2E = 1.4426950408889634f;
+constexpr int DH = 64;
+
+struct FbParams {
+  int B, S, hq, hk, g, Lq, Lk, causal;
+  const float* lse;     // [B, hq, S] natural-log sum of exponentials from the forward
+  const float* delta;   // [B, hq, S]
+  float* dq;            // [B*S, Lq], zeroed before the launch
+  float* dk;            // [B*S, Lk]
+  float* dv;            // [B*S, Lk]
+  int n_tiles;          // 128-row tiles per sequence
+  int* status;
+};
+
+struct FbSmem {
+  static constexpr int TILE = 128 * DH * 2;            // 16 KB: K, V
+  static constexpr int HALF_TILE = 64 * DH * 2;        // 64 queries of Q or dO
+  static constexpr int STAGES = 6;                     // ring of (Q, dO) half-tile pairs
+  static constexpr int DS_TILE = 128 * 128 * 2;        // dS^T [128 keys][128 queries] bf16: two 64-query boxes
+  static constexpr int FIX_OFF = 0;
+  static constexpr int RING_OFF = 2 * TILE;
+  static constexpr int DS_OFF = RING_OFF + STAGES * 2 * HALF_TILE;
+  static constexpr int BAR_OFF = DS_OFF + 2 * DS_TILE;
+  static constexpr int STAT_OFF = BAR_OFF + 256;       // float [2 groups][2 buffers][2][128]
+  static constexpr int TOTAL = STAT_OFF + 4096 + 1024;
+};
+
+TC_DEVINL void fail(volatile int* abort_flag, int* status, int code) {
+  *abort_flag = 1;
+  atomicCAS(status, 0, code);
+}
+template <bool POLY>
+TC_DEVINL uint64_t exp2_pair(uint64_t x) {
+  uint32_t a, b;
+  unpack2u(x, a, b);
+  if (POLY) return exp2_poly2(pack2f(fmaxf(__uint_as_float(a), -120.f), fmaxf(__uint_as_float(b), -120.f)));
+  return pack2f(ex2f(__uint_as_float(a)), ex2f(__uint_as_float(b)));
+}
+TC_DEVINL uint32_t cvt_bf16x2(uint64_t v) {
+  uint32_t a, b;
+  unpack2u(v, a, b);
+  return pack_bf16(__uint_as_float(a), __uint_as_float(b));
+}
+TC_DEVINL uint32_t lo_kmajor(uint32_t addr) { return (addr >> 4) | (1u << 16); }
+TC_DEVINL uint32_t lo_mnmajor(uint32_t addr) { return (addr >> 4) | ((16384u >> 4) << 16); }
+
+template <int POLY>
+__global__ void __launch_bounds__(FB_THREADS, 1)
+tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO, FbParams p) {
+  using SM = FbSmem;
+  constexpr int NST = SM::STAGES;
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  unsigned char* sK = smem + SM::FIX_OFF;
+  unsigned char* sV = sK + SM::TILE;
+  unsigned char* sRing = smem + SM::RING_OFF;         // [NST] stages of (Q half-tile, dO half-tile): 64 queries each
+  unsigned char* sDS = smem + SM::DS_OFF;             // [2] dS^T of a query tile
+  float* stat = reinterpret_cast<float*>(smem + SM::STAT_OFF);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFF);
+  uint64_t* kv_full = bars;
+  uint64_t* qdo_full = bars + 1;              // [NST]
+  uint64_t* qdo_empty = bars + 1 + NST;       // [NST]
+  uint64_t* sdp_full = bars + 1 + 2 * NST;    // [2] MMA -> compute: S^T and dP^T of a 64-query sub-tile ready
+  uint64_t* pds_full = sdp_full + 2;          // [2] compute group -> MMA: P^T, dS^T written (TMEM and shared memory)
+  uint64_t* acc_done = pds_full + 2;
+  uint64_t* stat_ready = acc_done + 1;        // [2] per compute group
+  uint64_t* dq_full = stat_ready + 2;         // [2] MMA -> compute: dQ of a query tile ready in its TMEM buffer
+  uint64_t* dq_empty = dq_full + 2;           // [2] compute -> MMA: that buffer has been added to memory (512 arrivals)
+  uint64_t* ds_free = dq_empty + 2;           // [2] MMA -> compute: the dQ contraction has read the dS^T tile
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ds_free + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // heavy (early) key tiles first
+  const int per_tile = p.B * p.hk;
+  const int tile = (int)(blockIdx.x / per_tile);
+  const int rem = blockIdx.x % per_tile;
+  const int b = rem / p.hk, hj = rem % p.hk;
+  const int n0 = tile * 128;
+  const int i0 = p.causal ? tile : 0;                  // first query tile that sees these keys
+  const int n_q = p.n_tiles - i0;
+  const int n_it = n_q * p.g;                          // iteration it = (gi, i): gi = it / n_q, i = i0 + it % n_q
+
+  if (threadIdx.x == 0) {
+    mbar_init(kv_full, 1);
+    for (int i = 0; i < NST; ++i) {
+      mbar_init(&qdo_full[i], 1);
+      mbar_init(&qdo_empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sdp_full[i], 1);
+      mbar_init(&pds_full[i], 256);
+      mbar_init(&stat_ready[i], 256);
+      mbar_init(&dq_full[i], 1);
+      mbar_init(&dq_empty[i], 32 * FB_COMPUTE_WARPS);
+      mbar_init(&ds_free[i], 1);
+    }
+    mbar_init(acc_done, 1);
+    wait_ctl_init(abort_flag, p.status);
+    fence_barrier_init();
+    prefetch_tmap(&tmQ);
+    prefetch_tmap(&tmK);
+    prefetch_tmap(&tmV);
+    prefetch_tmap(&tmDO);
+  }
+  if (warp == FB_MMA_WARP) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == FB_TMA_WARP) {
+    if (lane == 0) {
+      mbar_expect_tx(kv_full, 2 * SM::TILE);
+      tma_load_3d(sK, &tmK, hj * DH, n0, b, kv_full);
+      tma_load_3d(sV, &tmV, hj * DH, n0, b, kv_full);
+      for (int sub = 0; sub < 2 * n_it; ++sub) {
+        const int it = sub >> 1, st = sub % NST;
+        const uint32_t ph = (sub / NST) & 1;
+        const int hi = hj * p.g + it / n_q, m0 = (i0 + it % n_q) * 128 + (sub & 1) * 64;
+        if (!mbar_wait(&qdo_empty[st], ph ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_TMA); goto done; }
+        mbar_expect_tx(&qdo_full[st], 2 * SM::HALF_TILE);
+        unsigned char* dst = sRing + st * 2 * SM::HALF_TILE;
+        tma_load_3d(dst, &tmQ, hi * DH, m0, b, &qdo_full[st]);
+        tma_load_3d(dst + SM::HALF_TILE, &tmDO, hi * DH, m0, b, &qdo_full[st]);
+      }
+    }
+  } else if (warp == FB_MMA_WARP) {
+    const bool leader = elect_one();
+    const uint32_t hi_w = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
+    const uint32_t k_lo = lo_kmajor(smem_u32(sK)), v_lo = lo_kmajor(smem_u32(sV)), k_mn = lo_mnmajor(smem_u32(sK));
+    const uint32_t ds_mn = lo_mnmajor(smem_u32(sDS));
+    const uint32_t ring16 = smem_u32(sRing) >> 4;
+    constexpr uint32_t STAGE16 = (2 * SM::HALF_TILE) >> 4, HALF16 = SM::HALF_TILE >> 4, DS16 = SM::DS_TILE >> 4;
+    const int n_sub = 2 * n_it;
+    auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+    };
+    auto issue_sdp = [&](int sub) {     // S^T = K Q^T and dP^T = V dO^T for 64 queries
+      const int sb = sub & 1;
+      const uint32_t idesc = idesc_bf16(64, 0, 0);
+      const uint32_t qb = (ring16 + (sub % NST) * STAGE16) | (1u << 16), ob = qb + HALF16;
+      if (leader) {
+#pragma unroll
+        for (int kk = 0; kk < DH / 16; ++kk)
+          mma_ss_w(tmem_base + sb * 64, k_lo + kk * 2, hi_w, qb + kk * 2, hi_w, idesc, kk != 0);
+#pragma unroll
+        for (int kk = 0; kk < DH / 16; ++kk)
+          mma_ss_w(tmem_base + 128 + sb * 64, v_lo + kk * 2, hi_w, ob + kk * 2, hi_w, idesc, kk != 0);
+        mma_commit(&sdp_full[sb]);
+      }
+    };
+    auto issue_dvdk = [&](int sub) {    // dV += P^T dO, dK += dS^T Q over the sub-tile's 64 queries
+      const int sb = sub & 1, st = sub % NST;
+      const uint32_t idesc = idesc_bf16(DH, 0, 1);
+      const uint32_t qb = (ring16 + st * STAGE16) | ((8192u >> 4) << 16), ob = qb + HALF16;
+      if (leader) {
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          mma_ts_w(tmem_base + 256, tmem_base + sb * 64 + (kk >> 1) * 32 + (kk & 1) * 8, ob + kk * (2048 >> 4), hi_w, idesc,
+                   (sub | kk) != 0);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          mma_ts_w(tmem_base + 320, tmem_base + 128 + sb * 64 + (kk >> 1) * 32 + (kk & 1) * 8, qb + kk * (2048 >> 4), hi_w,
+                   idesc, (sub | kk) != 0);
+        mma_commit(&qdo_empty[st]);
+      }
+    };
+    auto issue_dq = [&](int it) {       // dQ_tile = dS K: A = dS^T tile read with the queries as M, B = K tile rows
+      const int buf = it & 1;
+      const uint32_t idesc = idesc_bf16(DH, 1, 1);
+      if (leader) {
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ss_w(tmem_base + 384 + buf * 64, ds_mn + buf * DS16 + kk * (2048 >> 4), hi_w, k_mn + kk * (2048 >> 4), hi_w, idesc,
+                   kk != 0);
+        mma_commit(&dq_full[buf]);
+        mma_commit(&ds_free[buf]);
+      }
+    };
+    if (!wait_all(kv_full, 0)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+    for (int s0 = 0; s0 < 2 && s0 < n_sub; ++s0) {
+      if (!wait_all(&qdo_full[s0 % NST], (s0 / NST) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+      tc_fence_after();
+      issue_sdp(s0);
+    }
+    for (int sub = 0; sub < n_sub; ++sub) {
+      if (!wait_all(&pds_full[sub & 1], (sub >> 1) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+      tc_fence_after();
+      issue_dvdk(sub);
+      if (sub + 2 < n_sub) {
+        const int nx = sub + 2;
+        if (!wait_all(&qdo_full[nx % NST], (nx / NST) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+        tc_fence_after();
+        issue_sdp(nx);
+      }
+      if (sub & 1) {
+        const int it = sub >> 1;
+        if (!wait_all(&dq_empty[it & 1], ((it >> 1) & 1) ^ 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+        tc_fence_after();
+        issue_dq(it);
+      }
+    }
+    if (leader) mma_commit(acc_done);
+  } else {
+    // ------------------------------------------------------------------ compute, thread = key
+    const int gsel = warp >> 3;                        // sub-tile (queries [64 gsel, 64 gsel + 64) of every query tile)
+    const int part = (warp >> 2) & 1;                  // which 32 of the sub-tile's 64 queries
+    const int row = (warp & 3) * 32 + lane;
+    const int ct = threadIdx.x & 255;
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+    const int tk = n0 + row;
+    const float c_scale = rsqrtf((float)DH) * FB_LOG2E;
+    const float q_scale = rsqrtf((float)DH);
+    float* gstat = stat + gsel * 512;
+    auto fetch_stat = [&](int it) -> float {
+      const int hi = hj * p.g + it / n_q, m0 = (i0 + it % n_q) * 128;
+      const int tq = m0 + (ct & 127);
+      const long long idx = ((long long)b * p.hq + hi) * p.S + tq;
+      if (ct < 128) return tq < p.S ? -p.lse[idx] * FB_LOG2E : -INFINITY;
+      return tq < p.S ? -p.delta[idx] : 0.f;
+    };
+    // adds the finished dQ of iteration `it` (its TMEM buffer) into memory: thread = query row, 16 channels
+    auto flush_dq = [&](int it) -> bool {
+      const int buf = it & 1;
+      if (!mbar_wait(&dq_full[buf], (it >> 1) & 1, abort_flag)) return false;
+      tc_fence_after();
+      uint32_t t[16];
+      const int col = (warp >> 2) * 16;
+      tmem_ld16(tmem_base + lane_sel + 384 + buf * 64 + col, t);
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(&dq_empty[buf]);
+      const int hi = hj * p.g + it / n_q, tq = (i0 + it % n_q) * 128 + row;
+      if (tq < p.S) {
+        float* dst = p.dq + ((long long)b * p.S + tq) * p.Lq + hi * DH + col;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4 * i), "f"(__uint_as_float(t[4 * i]) * q_scale),
+                       "f"(__uint_as_float(t[4 * i + 1]) * q_scale), "f"(__uint_as_float(t[4 * i + 2]) * q_scale),
+                       "f"(__uint_as_float(t[4 * i + 3]) * q_scale)
+                       : "memory");
+      }
+      return true;
+    };
+    float next_stat = n_it > 0 ? fetch_stat(0) : 0.f;
+    const uint64_t scale2 = pack2f(c_scale, c_scale);
+    const uint32_t s_t = tmem_base + lane_sel + gsel * 64 + part * 32;
+    const uint32_t dp_t = tmem_base + lane_sel + 128 + gsel * 64 + part * 32;
+    const int qoff = gsel * 64 + part * 32;            // first query (within the tile) of this thread's columns
+    // this thread's 64 bytes of a dS^T row: box gsel, row `row`, 16-byte chunks 4 part + [0,4) (swizzled)
+    unsigned char* ds_row = sDS + gsel * 16384 + row * 128;
+    for (int it = 0; it < n_it; ++it) {
+      const int stb = it & 1;
+      gstat[stb * 256 + ct] = next_stat;
+      if (it + 1 < n_it) next_stat = fetch_stat(it + 1);
+      mbar_arrive(&stat_ready[gsel]);
+      if (!mbar_wait(&stat_ready[gsel], it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+      const int m0 = (i0 + it % n_q) * 128;
+      const bool diag = p.causal && m0 == n0;
+      // the dS^T tile of two iterations ago must have been read by its dQ contraction
+      if (!mbar_wait(&ds_free[stb], ((it >> 1) & 1) ^ 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+      if (!mbar_wait(&sdp_full[gsel], it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+      tc_fence_after();
+      const ulonglong2* nlv = reinterpret_cast<const ulonglong2*>(gstat + stb * 256 + qoff);
+      const ulonglong2* ndv = reinterpret_cast<const ulonglong2*>(gstat + stb * 256 + 128 + qoff);
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t sv[16], dv[16], pk[8], dk_[8];
+        tmem_ld16(s_t + hf * 16, sv);
+        tmem_ld16(dp_t + hf * 16, dv);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const ulonglong2 nl = nlv[hf * 4 + c], nd = ndv[hf * 4 + c];
+          uint64_t e0 = fma2(pack2u(sv[4 * c + 0], sv[4 * c + 1]), scale2, nl.x);
+          uint64_t e1 = fma2(pack2u(sv[4 * c + 2], sv[4 * c + 3]), scale2, nl.y);
+          e0 = (2 * c & 3) < POLY ? exp2_pair<true>(e0) : exp2_pair<false>(e0);
+          e1 = ((2 * c + 1) & 3) < POLY ? exp2_pair<true>(e1) : exp2_pair<false>(e1);
+          if (diag) {
+            const int q0 = m0 + qoff + hf * 16 + 4 * c;
+            uint32_t a0, a1, a2, a3;
+            unpack2u(e0, a0, a1);
+            unpack2u(e1, a2, a3);
+            if (tk > q0) a0 = 0u;
+            if (tk > q0 + 1) a1 = 0u;
+            if (tk > q0 + 2) a2 = 0u;
+            if (tk > q0 + 3) a3 = 0u;
+            e0 = pack2u(a0, a1);
+            e1 = pack2u(a2, a3);
+          }
+          pk[2 * c] = cvt_bf16x2(e0);
+          pk[2 * c + 1] = cvt_bf16x2(e1);
+          dk_[2 * c] = cvt_bf16x2(mul2(e0, add2(pack2u(dv[4 * c + 0], dv[4 * c + 1]), nd.x)));
+          dk_[2 * c + 1] = cvt_bf16x2(mul2(e1, add2(pack2u(dv[4 * c + 2], dv[4 * c + 3]), nd.y)));
+        }
+        tmem_st8(s_t + hf * 8, pk);                    // P^T over S^T columns this thread has read
+        tmem_st8(dp_t + hf * 8, dk_);                  // dS^T over dP^T columns this thread has read
+        // the same dS^T values for the dQ contraction: queries qoff + 16 hf + [0,16) of row `row`
+        unsigned char* dsb = ds_row + stb * SM::DS_TILE;
+        const int ch = part * 4 + hf * 2;
+        *reinterpret_cast<uint4*>(dsb + (((ch) ^ (row & 7)) << 4)) = make_uint4(dk_[0], dk_[1], dk_[2], dk_[3]);
+        *reinterpret_cast<uint4*>(dsb + (((ch + 1) ^ (row & 7)) << 4)) = make_uint4(dk_[4], dk_[5], dk_[6], dk_[7]);
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      fence_proxy_async();                             // shared-memory writes -> visible to the tensor core
+      mbar_arrive(&pds_full[gsel]);
+      if (it >= 1 && !flush_dq(it - 1)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+    }
+    if (n_it > 0 && !flush_dq(n_it - 1)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
+    if (!mbar_wait(acc_done, 0, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
+    tc_fence_after();
+    {
+#pragma unroll 1
+      for (int c = 0; c < 1; ++c) {
+        uint32_t t[16], u[16];
+        const int col = (gsel * 2 + part) * (DH / 4);
+        tmem_ld16(tmem_base + lane_sel + 256 + col, t);
+        tmem_ld16(tmem_base + lane_sel + 320 + col, u);
+        tmem_ld_wait();
+        if (tk < p.S) {
+          const long long off = ((long long)b * p.S + tk) * p.Lk + hj * DH + col;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            reinterpret_cast<float4*>(p.dv + off)[i] = make_float4(__uint_as_float(t[4 * i]), __uint_as_float(t[4 * i + 1]),
+                                                                    __uint_as_float(t[4 * i + 2]), __uint_as_float(t[4 * i + 3]));
+            reinterpret_cast<float4*>(p.dk + off)[i] =
+                make_float4(__uint_as_float(u[4 * i]) * q_scale, __uint_as_float(u[4 * i + 1]) * q_scale,
+                            __uint_as_float(u[4 * i + 2]) * q_scale, __uint_as_float(u[4 * i + 3]) * q_scale);
+          }
+        }
+      }
+    }
+  }
+done:
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000) {}
+    __syncthreads();
+  }
+  if (warp == FB_MMA_WARP) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+template <int POLY>
+int launch_fused(TcState* s, const CcaDims& d, const CUtensorMap& tmQh, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                 const CUtensorMap& tmDOh, const FbParams& p, cudaStream_t st) {
+  static bool attr_set[TC_MAX_DEVICES] = {};
+  if (!attr_set[s->device]) {
+    cudaError_t e = cudaFuncSetAttribute(tc_attn_bwd_fused_kernel<POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, FbSmem::TOTAL);
+    if (e != cudaSuccess) return -(int)e;
+    attr_set[s->device] = true;
+  }
+  const long long g_kv = (long long)p.n_tiles * d.B * d.hk;
+  if (g_kv > 0x7fffffffLL) return 1;
+  cudaError_t e = cudaMemsetAsync(p.dq, 0, (size_t)d.B * d.S * d.Lq * sizeof(float), st);
+  if (e != cudaSuccess) return -(int)e;
+  tc_attn_bwd_fused_kernel<POLY><<<(unsigned)g_kv, FB_THREADS, FbSmem::TOTAL, st>>>(tmQh, tmK, tmV, tmDOh, p);
+  e = cudaGetLastError();
+  return e == cudaSuccess ? 0 : -(int)e;
+}
+
+}  // namespace
+
+// Head size 64 only.  delta must already hold rowsum(dO o O).  Returns 0 if the work was enqueued (a memset of dq and one
+// kernel), 1 if the case is not covered.
+int tc_attn_bwd_fused(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                      const float* lse, const float* delta, float* dq, float* dk, float* dv, int* d_status, cudaStream_t st) {
+  if (!s || !s->encode) return 1;
+  if (d.dh != 64) return 1;
+  if (d.Lq % 8 || d.Lk % 8) return 1;
+  if (reinterpret_cast<uintptr_t>(dq) & 15) return 1;
+  CUtensorMap tmK, tmV, tmQh, tmDOh;
+  const uint64_t S = (uint64_t)d.S, B = (uint64_t)d.B, Lq = (uint64_t)d.Lq, Lk = (uint64_t)d.Lk;
+  if (!tc_make_map_3d(s, &tmQh, q, Lq, S, B, Lq, S * Lq, 64, 64)) return 1;
+  if (!tc_make_map_3d(s, &tmDOh, d_o, Lq, S, B, Lq, S * Lq, 64, 64)) return 1;
+  if (!tc_make_map_3d(s, &tmK, k, Lk, S, B, Lk, S * Lk, 64, 128)) return 1;
+  if (!tc_make_map_3d(s, &tmV, v, Lk, S, B, Lk, S * Lk, 64, 128)) return 1;
+  FbParams p;
+  p.B = d.B; p.S = d.S; p.hq = d.hq; p.hk = d.hk; p.g = d.g; p.Lq = d.Lq; p.Lk = d.Lk; p.causal = d.causal;
+  p.lse = lse; p.delta = delta; p.dq = dq; p.dk = dk; p.dv = dv;
+  p.n_tiles = (d.S + 127) / 128;
+  p.status = d_status;
+  const int poly = s->attn_poly_bwd < 0 ? 1 : s->attn_poly_bwd;
+  if (poly == 0) return launch_fused<0>(s, d, tmQh, tmK, tmV, tmDOh, p, st);
+  if (poly == 2) return launch_fused<2>(s, d, tmQh, tmK, tmV, tmDOh, p, st);
+  return launch_fused<1>(s, d, tmQh, tmK, tmV, tmDOh, p, st);
+}

@@ -286,6 +286,8 @@ TcState* tc_create(int sm_count) {
   s->attn_attr_set[0] = s->attn_attr_set[1] = false;
   s->attn_poly = -1;      // -1: per head size (0 at d_h = 128, 1 at d_h = 64)
   if (const char* e = getenv("CCA_ATTN_POLY")) s->attn_poly = atoi(e);
+  s->attn_bwd_fused = 1;
+  if (const char* e = getenv("CCA_ATTN_BWD_FUSED")) s->attn_bwd_fused = atoi(e);
   s->attn_poly_bwd = -1;
   if (const char* e = getenv("CCA_ATTN_POLY_BWD")) s->attn_poly_bwd = atoi(e);
   void* fn = nullptr;

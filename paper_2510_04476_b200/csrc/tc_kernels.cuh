@@ -20,6 +20,9 @@ int tc_attn_fwd256(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, c
 // Attention adjoint (dq, dk, dv in fp32) from q, k, v, d_o, the forward's lse and delta = rowsum(dO o O).
 int tc_attn_bwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                 const float* lse, const float* delta, float* dq, float* dk, float* dv, int* d_status, cudaStream_t st);
+// The same adjoint as one kernel (head size 64): every (query, key) pair once; dq is zeroed, then summed by reductions.
+int tc_attn_bwd_fused(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                      const float* lse, const float* delta, float* dq, float* dk, float* dv, int* d_status, cudaStream_t st);
 // Adjoint of conv2: dy1 [T, L] fp32 <- d_hat (dqh, dkh); d_w1 accumulates the conv2 weight gradient.
 int tc_transform_bwd(TcState* s, const CcaDims& d, const float* qk0, const bf16* w0, const bf16* w1, const float* dqh,
                      const float* dkh, float* dy1, float* d_w1, int* d_status, cudaStream_t st);

@@ -21,6 +21,7 @@ struct TcState {
   int use_pairs;          // 0 disables the pair GEMM
   bool attn_attr_set[2];
   int attn_poly_bwd;      // the same share in the backward kernels
+  int attn_bwd_fused;     // head size 64: the one-kernel attention adjoint (0: the dQ and dK/dV kernels)
   int attn_poly;          // of every 4 score pairs, how many take the polynomial exp2 (0..3)
 };
 

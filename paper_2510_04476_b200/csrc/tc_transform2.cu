@@ -15,8 +15,12 @@
 //   warp 8   TMA: the head's NT weight tiles when the head changes, one operand tile per unit (ring of stages)
 //   warp 9   MMA issue: acc = sum_m A_m W_m^T into one of two TMEM accumulators (128 tokens x d_h, fp32)
 //   warps 0-7  epilogue, thread = token, two groups of four warps that take every other unit: adds the q-k-mean term
-//            of Eq. 9 in fp32 from the fp32 latent (coalescing is per thread: 16 bytes at a time along its own row),
-//            L2 norm * sqrt(d_h) (* exp(temp)), RoPE from the table, bf16 store; the norm scale is kept for the backward.
+//            of Eq. 9 in fp32 from the fp32 latent, L2 norm * sqrt(d_h) (* exp(temp)), RoPE from the table, bf16
+//            store; the norm scale is kept for the backward.  A thread needs 128 bytes of its own token's row at a
+//            time (32 fp32 channels, or 16 (cos, sin) pairs); fetched by the thread itself that would be one memory
+//            transaction per thread and 16 bytes.  Instead lane 0 of each warp has TMA bring the warp's 32 rows x 128
+//            bytes into a private shared-memory slot (two slots per warp, the next box in flight while one is read),
+//            and the threads read their rows from there, swizzled, without bank conflicts.
 #include "tc_kernels.cuh"
 #include "tc_ptx.cuh"
 #include "tc_state.cuh"
@@ -38,13 +42,19 @@ struct T2Smem {
   static constexpr int WT = DH * DH * 2;                 // one tap's weight tile
   static constexpr int W_BYTES = NT * WT;
   static constexpr int BUDGET = 232448 - 512;            // 227 KB minus barriers
-  static constexpr int STAGES_FIT = (BUDGET - W_BYTES) / A_BYTES;
-  static constexpr int STAGES = STAGES_FIT > 4 ? 4 : STAGES_FIT;
+  // per epilogue warp: slots for boxes of 32 rows x 128 bytes, as many as fit beside one operand tile (2..4)
+  static constexpr int NSLOT_FIT = (BUDGET - W_BYTES - A_BYTES) / (8 * 4096);
+  static constexpr int NSLOT = NSLOT_FIT > 4 ? 4 : NSLOT_FIT;
+  static constexpr int SLOT_BYTES = 8 * NSLOT * 4096;
+  static constexpr int STAGES_FIT = (BUDGET - W_BYTES - SLOT_BYTES) / A_BYTES;
+  static constexpr int STAGES = STAGES_FIT > 2 ? 2 : STAGES_FIT;   // one is enough: the contraction of a unit is short
+  static_assert(NSLOT >= 2, "box slots do not fit");
   static constexpr int W_OFF = 0;
   static constexpr int A_OFF = W_BYTES;
-  static constexpr int BAR_OFF = A_OFF + STAGES * A_BYTES;
-  static constexpr int TOTAL = BAR_OFF + 256;
-  static_assert(STAGES >= 2, "operand ring needs two stages");
+  static constexpr int SLOT_OFF = A_OFF + STAGES * A_BYTES;
+  static constexpr int BAR_OFF = SLOT_OFF + SLOT_BYTES;
+  static constexpr int TOTAL = BAR_OFF + 512;
+  static_assert(STAGES >= 1, "operand tile does not fit");
   static_assert(NT - 1 <= ROWS - 128, "halo rows");
 };
 
@@ -79,7 +89,8 @@ TC_DEVINL Unit unit_of(const T2Params& p, int u) {
 
 template <int DH, int NT>
 __global__ void __launch_bounds__(T2_THREADS, 1)
-tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const T2Params p) {
+tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                     const __grid_constant__ CUtensorMap tmF, const __grid_constant__ CUtensorMap tmR, const T2Params p) {
   using SM = T2Smem<DH, NT>;
   constexpr int ST = SM::STAGES;
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -94,7 +105,8 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   uint64_t* w_empty = w_full + 1;          // MMA -> TMA: every contraction with the previous head's weights is done
   uint64_t* acc_full = w_empty + 1;        // [2] MMA -> epilogue group (commit)
   uint64_t* acc_empty = acc_full + 2;      // [2] epilogue group -> MMA (128 arrivals)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* slot_full = acc_empty + 2;     // [8 warps][NSLOT] TMA -> the warp's threads
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(slot_full + 8 * SM::NSLOT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const CcaDims& d = p.d;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -120,10 +132,13 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       mbar_init(&acc_full[s], 1);
       mbar_init(&acc_empty[s], 128);
     }
+    for (int s = 0; s < 8 * SM::NSLOT; ++s) mbar_init(&slot_full[s], 1);
     wait_ctl_init(abort_flag, p.status);
     fence_barrier_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmW);
+    prefetch_tmap(&tmF);
+    prefetch_tmap(&tmR);
   }
   if (warp == T2_MMA_WARP) {
     tmem_alloc(tmem_slot, 2 * DH);
@@ -200,10 +215,63 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   } else {
     // ------------------------------------------------------------------ epilogue, thread = token
     constexpr int HALF = DH / 2;
+    constexpr int NS = SM::NSLOT;
     const int grp = warp >> 2;                              // units with (it & 1) == grp, accumulator grp
     const int rho = (warp & 3) * 32 + lane;
     const uint32_t acc = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + grp * DH;
-    const bool use_mean = (d.flags & F_QK_MEAN) != 0;
+    const bool use_mean = (d.flags & F_QK_MEAN) != 0, use_rope = (d.flags & F_ROPE) != 0;
+    unsigned char* my_slots = smem + SM::SLOT_OFF + warp * NS * 4096;
+    uint64_t* my_full = slot_full + warp * NS;
+    // this thread's 16-byte chunk i of its row in a slot (rows of 128 bytes, 128-byte swizzle)
+    uint32_t ch_off[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) ch_off[i] = (uint32_t)lane * 128u + (((uint32_t)i ^ (uint32_t)(lane & 7)) << 4);
+    uint32_t nb = 0;                                        // boxes this warp has consumed so far (all units)
+    // The boxes of a unit, in the order they are read: for every 32-channel chunk the own rows then the other heads'
+    // rows (fp32 latent), then the RoPE table rows, 16 (cos, sin) pairs at a time; rows past the end come as zeros.
+    // Box layout of unit u (warp-uniform):
+    struct Boxes {
+      int h, b, row0, oth_col, per_chunk, n_mean, n_box;
+    };
+    auto boxes_of = [&](int u) -> Boxes {
+      const Unit un = unit_of(p, u);
+      const bool is_q = un.h < d.hq;
+      const int hj = is_q ? un.h / d.g : un.h - d.hq;
+      Boxes x;
+      x.h = un.h; x.b = un.b; x.row0 = un.t0 + (warp & 3) * 32;
+      x.oth_col = is_q ? d.Lq + hj * DH : hj * d.g * DH;
+      x.per_chunk = use_mean ? 1 + (is_q ? 1 : d.g) : 0;
+      x.n_mean = (DH / 32) * x.per_chunk;
+      x.n_box = x.n_mean + (use_rope ? HALF / 16 : 0);
+      return x;
+    };
+    // Issue cursor (lane 0 acts, every lane tracks): the next box to ask for is box pn of unit pu; it runs NS boxes
+    // ahead of the reads, across unit boundaries, so that the slots never sit empty between two units.
+    int pu = u_begin + grp, pn = 0;
+    uint32_t issued = 0;
+    Boxes pbx = pu < u_end ? boxes_of(pu) : Boxes{0, 0, 0, 0, 0, 0, 0};
+    auto issue_next = [&]() {
+      while (pu < u_end && pn >= pbx.n_box) {               // next unit of this group (units without boxes are skipped)
+        pu += 2;
+        pn = 0;
+        if (pu < u_end) pbx = boxes_of(pu);
+      }
+      if (pu >= u_end) return;
+      if (lane == 0) {
+        unsigned char* dst = my_slots + (issued % NS) * 4096;
+        uint64_t* bar = &my_full[issued % NS];
+        mbar_expect_tx(bar, 4096);
+        if (pn < pbx.n_mean) {
+          const int c = pn / pbx.per_chunk, j = pn % pbx.per_chunk;
+          tma_load_3d(dst, &tmF, (j == 0 ? pbx.h * DH : pbx.oth_col + (j - 1) * DH) + c * 32, pbx.row0, pbx.b, bar);
+        } else {
+          tma_load_2d(dst, &tmR, (pn - pbx.n_mean) * 32, pbx.row0, bar);
+        }
+      }
+      ++issued;
+      ++pn;
+    };
+    for (int i = 0; i < NS; ++i) issue_next();
     int it = grp;
     for (int u = u_begin + grp; u < u_end; u += 2, it += 2) {
       const Unit un = unit_of(p, u);
@@ -212,11 +280,24 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       const int t = un.t0 + rho;
       const bool valid = t < d.S;
       const long long tok = (long long)un.b * d.S + (valid ? t : 0);
-      const float* own = p.qk0 + tok * d.L + un.h * DH;
-      // the other operand of the q-k-mean: the kv head's k0 for a q head, the group's q0 heads for a kv head
-      const float* oth = p.qk0 + tok * d.L + (is_q ? d.Lq + hj * DH : hj * d.g * DH);
       const int n_oth = is_q ? 1 : d.g;
       const float oth_scale = is_q ? 0.5f : 0.5f / (float)d.g;
+      const int per_chunk = use_mean ? 1 + n_oth : 0;
+      const int n_mean = (DH / 32) * per_chunk;
+      const int n_box = n_mean + (use_rope ? HALF / 16 : 0);
+      auto wait_box = [&](int n) -> bool {
+        const uint32_t g = nb + (uint32_t)n;
+        return mbar_wait(&my_full[g % NS], (g / NS) & 1, abort_flag);
+      };
+      // Every lane has used a box: its slot takes the next box of the stream.  The TMA write goes through the
+      // asynchronous proxy and is not ordered behind shared-memory loads that are still in flight; release_box is
+      // therefore called only after the arithmetic that consumes the loaded values has been issued (instructions
+      // issue in order, so the values have arrived), and every lane has got there (__syncwarp).
+      auto release_box = [&]() {
+        __syncwarp();
+        if (lane == 0) fence_proxy_async();
+        issue_next();
+      };
       if (!mbar_wait(&acc_full[grp], (it >> 1) & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
       tc_fence_after();
       // pass 1: pre-norm latent = conv output + mean term (Eq. 9), its squared norm; kept in the accumulator
@@ -226,30 +307,25 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         uint32_t r[32];
         tmem_ld32(acc + c * 32, r);
         if (use_mean) {
-          float4 a[8], o[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            a[i] = valid ? __ldg(reinterpret_cast<const float4*>(own + c * 32) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-            o[i] = valid ? __ldg(reinterpret_cast<const float4*>(oth + c * 32) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-          }
-          for (int m = 1; m < n_oth; ++m) {
+          for (int j = 0; j < per_chunk; ++j) {            // j = 0: own rows (weight 1/2), then the other heads' rows
+            const int n = c * per_chunk + j;
+            if (!wait_box(n)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
+            const unsigned char* src = my_slots + ((nb + n) % NS) * 4096;
+            const float wgt = j == 0 ? 0.5f : oth_scale;
+            if (j == 0) tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-              const float4 e = valid ? __ldg(reinterpret_cast<const float4*>(oth + m * DH + c * 32) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-              o[i].x += e.x; o[i].y += e.y; o[i].z += e.z; o[i].w += e.w;
+              const float4 e = *reinterpret_cast<const float4*>(src + ch_off[i]);
+              r[4 * i + 0] = __float_as_uint(fmaf(wgt, e.x, __uint_as_float(r[4 * i + 0])));
+              r[4 * i + 1] = __float_as_uint(fmaf(wgt, e.y, __uint_as_float(r[4 * i + 1])));
+              r[4 * i + 2] = __float_as_uint(fmaf(wgt, e.z, __uint_as_float(r[4 * i + 2])));
+              r[4 * i + 3] = __float_as_uint(fmaf(wgt, e.w, __uint_as_float(r[4 * i + 3])));
             }
+            asm volatile("" ::"r"(r[0]), "r"(r[31]) : "memory");      // the sums exist before the slot is handed over
+            release_box();
           }
-          tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const float v0 = __uint_as_float(r[4 * i + 0]) + fmaf(oth_scale, o[i].x, 0.5f * a[i].x);
-            const float v1 = __uint_as_float(r[4 * i + 1]) + fmaf(oth_scale, o[i].y, 0.5f * a[i].y);
-            const float v2 = __uint_as_float(r[4 * i + 2]) + fmaf(oth_scale, o[i].z, 0.5f * a[i].z);
-            const float v3 = __uint_as_float(r[4 * i + 3]) + fmaf(oth_scale, o[i].w, 0.5f * a[i].w);
-            ss = fmaf(v0, v0, ss); ss = fmaf(v1, v1, ss); ss = fmaf(v2, v2, ss); ss = fmaf(v3, v3, ss);
-            r[4 * i + 0] = __float_as_uint(v0); r[4 * i + 1] = __float_as_uint(v1);
-            r[4 * i + 2] = __float_as_uint(v2); r[4 * i + 3] = __float_as_uint(v3);
-          }
+          for (int i = 0; i < 32; ++i) ss = fmaf(__uint_as_float(r[i]), __uint_as_float(r[i]), ss);
           tmem_st32(acc + c * 32, r);
         } else {
           tmem_ld_wait();
@@ -265,20 +341,22 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       }
       // pass 2: scale, rotate the pairs (c, c + d_h/2), store
       bf16* dst = is_q ? p.q + tok * d.Lq + un.h * DH : p.k + tok * d.Lk + hj * DH;
-      const float4* tab = reinterpret_cast<const float4*>(p.rope + (long long)(valid ? t : 0) * HALF);
 #pragma unroll 1
       for (int c = 0; c < HALF / 16; ++c) {
         uint32_t ra[16], rb[16];
         tmem_ld16(acc + c * 16, ra);
         tmem_ld16(acc + HALF + c * 16, rb);
         float4 cs[8];
-        if (d.flags & F_ROPE) {
+        if (use_rope) {
+          const int n = n_mean + c;
+          if (!wait_box(n)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
+          const unsigned char* src = my_slots + ((nb + n) % NS) * 4096;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) cs[i] = __ldg(tab + c * 8 + i);        // (cos, sin) of two pairs
+          for (int i = 0; i < 8; ++i) cs[i] = *reinterpret_cast<const float4*>(src + ch_off[i]);   // (cos, sin) x 2
         }
         tmem_ld_wait();
         float lo[16], hi[16];
-        if (d.flags & F_ROPE) {
+        if (use_rope) {
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const float a0 = __uint_as_float(ra[2 * i]) * sc, b0 = __uint_as_float(rb[2 * i]) * sc;
@@ -288,6 +366,8 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             lo[2 * i + 1] = a1 * cs[i].z - b1 * cs[i].w;
             hi[2 * i + 1] = b1 * cs[i].z + a1 * cs[i].w;
           }
+          asm volatile("" ::"f"(lo[0]), "f"(hi[15]) : "memory");
+          release_box();
         } else {
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
@@ -312,6 +392,7 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           }
         }
       }
+      nb += (uint32_t)n_box;
       tc_fence_before();
       mbar_arrive(&acc_empty[grp]);
     }
@@ -365,12 +446,30 @@ int launch_t2(TcState* s, const CcaDims& d, const bf16* qk0b, const bf16* wc, co
     if (e != cudaSuccess) return -(int)e;
     attr_done[s->device] = true;
   }
-  CUtensorMap tmA, tmW;
+  CUtensorMap tmA, tmW, tmF, tmR;
   if (!tc_make_map_3d(s, &tmA, qk0b, (uint64_t)d.L, (uint64_t)d.S, (uint64_t)d.B, (uint64_t)d.L, (uint64_t)d.S * d.L, 64, SM::ROWS))
     return 1;
   if (!tc_make_map_2d(s, &tmW, wc, (uint64_t)DH, (uint64_t)(d.hq + d.hk) * NT * DH, (uint64_t)DH, 64, DH)) return 1;
+  // fp32 boxes of 32 rows x 32 values (128 bytes): the latent [B][S][L] and the RoPE table [S][d_h/2 pairs = d_h floats]
+  {
+    cuuint64_t dims[3] = {(cuuint64_t)d.L, (cuuint64_t)d.S, (cuuint64_t)d.B};
+    cuuint64_t strides[2] = {(cuuint64_t)d.L * 4, (cuuint64_t)d.S * d.L * 4};
+    cuuint32_t box[3] = {32, 32, 1}, estr[3] = {1, 1, 1};
+    if (s->encode(&tmF, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(p0.qk0), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return 1;
+    cuuint64_t rdims[2] = {(cuuint64_t)DH, (cuuint64_t)d.S};
+    cuuint64_t rstrides[1] = {(cuuint64_t)DH * 4};
+    cuuint32_t rbox[2] = {32, 32}, restr[2] = {1, 1};
+    const void* rp = (d.flags & F_ROPE) ? (const void*)p0.rope : (const void*)p0.qk0;      // unused without RoPE
+    if (s->encode(&tmR, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(rp), rdims, rstrides, rbox, restr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return 1;
+  }
   const int grid = p0.total_units < s->sm_count ? p0.total_units : s->sm_count;
-  tc_transform2_kernel<DH, NT><<<grid, T2_THREADS, SM::TOTAL, st>>>(tmA, tmW, p0);
+  tc_transform2_kernel<DH, NT><<<grid, T2_THREADS, SM::TOTAL, st>>>(tmA, tmW, tmF, tmR, p0);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 0 : -(int)e;
 }
