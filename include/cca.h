@@ -55,7 +55,7 @@ typedef struct {
   int32_t d_model;      /* E                                                                */
   int32_t n_q_heads;    /* h_q;  L_q = h_q * head_dim = E / C1                              */
   int32_t n_kv_heads;   /* h_k;  L_k = h_k * head_dim = E / C2;  h_q % h_k == 0, L_k even   */
-  int32_t head_dim;     /* d_h, latent per-head size: 32, 64, 128; 256 forward only        */
+  int32_t head_dim;     /* d_h, latent per-head size: 32, 64, 128, 256                      */
   int32_t compression;  /* C = C1; checked: E == C * h_q * d_h                              */
   int32_t k_seq;        /* taps of conv1_seq (1..4)                                         */
   int32_t k_ch;         /* taps of conv2_seq+ch (1..4)                                      */

@@ -385,6 +385,11 @@ cudaError_t launch_attn_fwd_simt(const CcaDims& d, const bf16* q, const bf16* k,
 
 cudaError_t launch_attn_delta(const CcaDims& d, const float* o32, const bf16* d_o, float* delta, cudaStream_t st) {
   const long long rows = (long long)d.B * d.S * d.hq;
+  if (d.dh == 256) {
+    const long long threads = rows * (256 / 8);
+    attn_delta_kernel<256><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(d, o32, d_o, delta);
+    return cudaGetLastError();
+  }
   DISPATCH_DH(d.dh, {
     const long long threads = rows * (DH / 8);
     attn_delta_kernel<DH><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(d, o32, d_o, delta);

@@ -39,6 +39,9 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 struct Layout {
   size_t qk0, q, k, v, o, lse, rope, rnorm, w_all, y1s, y2, qk0b, wc, saved_end;
   size_t o32, d_o, delta, dq, dk, dv, dlat, dy1, total_end;
+  size_t u_s, u_dp, u_p, u_ds, u_dy1s;   // head size 256: scratch of the unfused adjoints
+  int u_rows;                            // query rows per chunk of the unfused attention adjoint
+  size_t u_ld;                           // row stride (keys) of its score chunks
 };
 
 CcaDims make_dims(const cca_config& c, int64_t B, int64_t S);
@@ -82,6 +85,16 @@ Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
   l.dv = take(T * Lk * 4);
   l.dlat = take(T * (L + Lk) * 2);
   l.dy1 = take(T * L * 4);
+  l.u_s = l.u_dp = l.u_p = l.u_ds = l.u_dy1s = off;
+  l.u_rows = 1024;
+  l.u_ld = align_up((size_t)S, 128);
+  if (c.head_dim > 128) {
+    l.u_s = take((size_t)l.u_rows * l.u_ld * 4);
+    l.u_dp = take((size_t)l.u_rows * l.u_ld * 4);
+    l.u_p = take((size_t)l.u_rows * l.u_ld * 2);
+    l.u_ds = take((size_t)l.u_rows * l.u_ld * 2);
+    l.u_dy1s = take(T * L * (size_t)c.k_ch * 4);
+  }
   l.total_end = off;
   return l;
 }
@@ -790,7 +803,6 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   if ((c.flags & CCA_CONV1) && !w->conv0_w) return CCA_ERR_INVALID_ARG;
   if ((c.flags & CCA_CONV2) && !w->conv1_w) return CCA_ERR_INVALID_ARG;
   if ((c.flags & CCA_QK_NORM) && !w->temp) return CCA_ERR_INVALID_ARG;
-  if (c.head_dim > 128) return CCA_ERR_UNSUPPORTED;          // head size 256: forward only
   if (!aligned16(x) || !aligned16(d_out) || !aligned16(d_x) || !aligned16(w->w_qk) || !aligned16(w->w_v1) ||
       !aligned16(w->w_v2) || !aligned16(w->w_o) || !aligned16(gr->d_w_qk) || !aligned16(gr->d_w_v1) ||
       !aligned16(gr->d_w_v2) || !aligned16(gr->d_w_o) || (reinterpret_cast<uintptr_t>(workspace) & 255))
@@ -847,7 +859,53 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   {
     if (h->ev_attn_begin) CU(cudaEventRecord(h->ev_attn_begin, st));
     bool done = false;
-    if (h->impl >= 1 && h->tc) {
+    if (d.dh > 128) {
+      // Head size 256: the adjoint as plain contractions over chunks of query rows of one (sequence, query head) at a
+      // time.  S = Q K^T and dP = dO V^T (fp32), P and dS / sqrt(d_h) (bf16, element-wise), then dQ = dS K,
+      // dV += P^T dO, dK += dS^T Q, the latter two accumulated over chunks and over the g heads of a group.
+      float* s32 = (float*)(ws + l.u_s);
+      float* dp32 = (float*)(ws + l.u_dp);
+      bf16* pb = (bf16*)(ws + l.u_p);
+      bf16* dsb = (bf16*)(ws + l.u_ds);
+      const long long ld = (long long)l.u_ld;
+      CU(cudaMemsetAsync(dk, 0, (size_t)T * d.Lk * 4, st));
+      CU(cudaMemsetAsync(dv, 0, (size_t)T * d.Lk * 4, st));
+      for (int b = 0; b < d.B; ++b)
+        for (int i = 0; i < d.hq; ++i) {
+          const int j = i / d.g;
+          const bf16* kj = k + (size_t)b * d.S * d.Lk + (size_t)j * d.dh;
+          const bf16* vj = v + (size_t)b * d.S * d.Lk + (size_t)j * d.dh;
+          const float* lse_i = lse + ((size_t)b * d.hq + i) * d.S;
+          const float* delta_i = delta + ((size_t)b * d.hq + i) * d.S;
+          for (int m0 = 0; m0 < d.S; m0 += l.u_rows) {
+            const int rows = d.S - m0 < l.u_rows ? d.S - m0 : l.u_rows;
+            const int n_keys = d.causal ? m0 + rows : d.S;
+            const size_t qoff = ((size_t)b * d.S + m0) * d.Lq + (size_t)i * d.dh;
+            GemmArgs ga{};
+            ga.A = kmajor(q + qoff, d.Lq); ga.B = kmajor(kj, d.Lk);
+            ga.M = rows; ga.N = n_keys; ga.K = d.dh; ga.seq_len = rows; ga.out_f32 = s32; ga.ldc = ld;
+            if ((r = run_gemm(h, ga, st)) != CCA_OK) return r;
+            ga.A = kmajor(d_o + qoff, d.Lq); ga.B = kmajor(vj, d.Lk); ga.out_f32 = dp32;
+            if ((r = run_gemm(h, ga, st)) != CCA_OK) return r;
+            CU(launch_pds(s32, dp32, ld, lse_i, delta_i, m0, rows, n_keys, d.S, d.causal, d.dh, pb, dsb, st));
+            h->launches++;
+            ga = GemmArgs{};
+            ga.A = kmajor(dsb, ld); ga.B = mmajor(kj, d.Lk);
+            ga.M = rows; ga.N = d.dh; ga.K = n_keys; ga.seq_len = rows; ga.out_f32 = dq + qoff; ga.ldc = d.Lq;
+            if ((r = run_gemm(h, ga, st)) != CCA_OK) return r;
+            ga = GemmArgs{};
+            ga.A = mmajor(pb, ld); ga.B = mmajor(d_o + qoff, d.Lq);
+            ga.M = n_keys; ga.N = d.dh; ga.K = rows; ga.seq_len = n_keys; ga.ldc = d.Lk; ga.accumulate = 1;
+            ga.out_f32 = dv + (size_t)b * d.S * d.Lk + (size_t)j * d.dh;
+            if ((r = run_gemm(h, ga, st)) != CCA_OK) return r;
+            ga.A = mmajor(dsb, ld); ga.B = mmajor(q + qoff, d.Lq);
+            ga.out_f32 = dk + (size_t)b * d.S * d.Lk + (size_t)j * d.dh;
+            if ((r = run_gemm(h, ga, st)) != CCA_OK) return r;
+          }
+        }
+      done = true;
+    }
+    if (!done && h->impl >= 1 && h->tc) {
       int tr = tc_attn_bwd(h->tc, d, q, k, v, d_o, lse, delta, dq, dk, dv, h->d_status, st);
       if (tr == 0) done = true;
       if (tr < 0) { h->last_cuda = -tr; return CCA_ERR_CUDA; }
@@ -862,7 +920,37 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   STAGE(CCA_EV_BWD_NORM);
   {
     bool done = false;
-    if (h->impl >= 1 && h->tc) {
+    if (d.dh > 128) {
+      // Head size 256: conv2's adjoint as one contraction per head on the stored conv1 taps (the forward's y1s),
+      // dy1s = d_hat W_head and d_conv1_w[head] = d_hat^T y1s, then the taps folded back onto their tokens.
+      float* dy1 = (float*)(ws + l.dy1);
+      if (c.flags & CCA_CONV2) {
+        bf16* dhat = dlat;                      // the latent-gradient buffer is free until conv1's adjoint writes it
+        const bf16* y1s = (const bf16*)(ws + l.y1s);
+        float* dy1s = (float*)(ws + l.u_dy1s);
+        const int kd = d.dh * c.k_ch;
+        CU(launch_cast_dhat(d, dq, dk, dhat, nullptr, st));
+        for (int hh = 0; hh < d.hq + d.hk; ++hh) {
+          GemmArgs gc{};
+          gc.A = kmajor(dhat + (size_t)hh * d.dh, d.L);
+          gc.B = mmajor((const bf16*)w->conv1_w + (size_t)hh * d.dh * kd, kd);
+          gc.M = T; gc.N = kd; gc.K = d.dh; gc.seq_len = d.S; gc.out_f32 = dy1s + (size_t)hh * kd; gc.ldc = (long long)d.L * c.k_ch;
+          if ((r = run_gemm(h, gc, st)) != CCA_OK) return r;
+          gc = GemmArgs{};
+          gc.A = mmajor(dhat + (size_t)hh * d.dh, d.L);
+          gc.B = mmajor(y1s + (size_t)hh * kd, (long long)d.L * c.k_ch);
+          gc.M = d.dh; gc.N = kd; gc.K = T; gc.seq_len = d.S; gc.out_f32 = gr->d_conv1_w + (size_t)hh * d.dh * kd; gc.ldc = kd;
+          if ((r = run_gemm(h, gc, st)) != CCA_OK) return r;
+        }
+        CU(launch_taps_adjoint(d, dy1s, dy1, st));
+      } else {
+        CU(launch_cast_dhat(d, dq, dk, nullptr, dy1, st));
+      }
+      STAGE(CCA_EV_BWD_CONV2);
+      CU(launch_conv1_adjoint(d, dy1, dq, dk, qk0, (const bf16*)w->conv0_w, dlat, ldl, gr->d_conv0_w, st));
+      done = true;
+    }
+    if (!done && h->impl >= 1 && h->tc) {
       float* dy1 = (float*)(ws + l.dy1);
       int tr = tc_transform_bwd(h->tc, d, qk0, (const bf16*)w->conv0_w, (const bf16*)w->conv1_w, dq, dk, dy1,
                                 gr->d_conv1_w, h->d_status, st);

@@ -44,6 +44,7 @@ struct GemmArgs {
   int split_L, split_Lk, split_shift;
   int row0;          // fused output only: position inside its sequence of row 0 of A (a chunk of a longer sequence)
   bf16* out_lat_bf16;   // fused output only, optional: a bf16 copy of columns [0, split_L) (row stride split_L)
+  int accumulate;       // out_f32 only: add the product to what the output holds (atomic adds) instead of overwriting
 };
 
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
@@ -78,6 +79,15 @@ cudaError_t launch_pack_dv(const CcaDims& d, const float* dv, bf16* dlat, long l
 cudaError_t launch_conv1_taps(const CcaDims& d, const float* qk0, const bf16* w0, bf16* y1s, float* y2, cudaStream_t st);
 cudaError_t launch_finalize(const CcaDims& d, const float* qk0, const float* y2, const float* temp, const float2* rope,
                             bf16* q, bf16* k, float* rnorm, cudaStream_t st);
+
+// ---- element-wise pieces of the backward at head sizes without fused adjoint kernels (bwd_unfused.cu) ----
+// P (bf16) and dS / sqrt(d_h) (bf16) of one chunk of `rows` query rows starting at m0 of one (sequence, query head) from
+// its scores s and dP (fp32, row stride ld, keys [0, n_keys)); lse, delta: that head's rows.  Columns >= n_keys get 0.
+cudaError_t launch_pds(const float* s, const float* dp, long long ld, const float* lse, const float* delta, int m0, int rows,
+                       int n_keys, int S, int causal, int dh, bf16* p_out, bf16* ds_out, cudaStream_t st);
+cudaError_t launch_cast_dhat(const CcaDims& d, const float* dqh, const float* dkh, bf16* out_bf16, float* out_f32, cudaStream_t st);
+// dy1 [T, L] from dy1s [T, L * k_ch] (gradient of the conv1 output stored at the k_ch positions conv2 reads).
+cudaError_t launch_taps_adjoint(const CcaDims& d, const float* dy1s, float* dy1, cudaStream_t st);
 
 // ---- attention (Eq. 11, softmax line), plain SIMT ----
 // o32: optional fp32 copy of o (kept for the backward's delta = rowsum(dO * O)); may be null.

@@ -103,6 +103,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
       if (n >= g.N) continue;
       long long idx = (long long)m * g.ldc + n;
       if (g.out_bf16) g.out_bf16[idx] = __float2bfloat16(acc[i][j]);
+      else if (g.accumulate) atomicAdd(g.out_f32 + idx, acc[i][j]);
       else g.out_f32[idx] = acc[i][j];
     }
   }

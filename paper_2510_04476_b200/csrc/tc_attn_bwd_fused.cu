@@ -11,8 +11,10 @@
 // The compute warps also leave dS^T as bf16 in shared memory ([key][query], 128-byte swizzle): read with the queries
 // as the M dimension it is the A operand of   dQ_tile = dS K   (M = 128 queries, N = d_h, K = 128 keys; the resident
 // K tile read along its rows is the B operand).  A query tile's dQ gets such a contribution from every key tile it
-// sees, i.e. from different CTAs: they are added into the zeroed fp32 dq with vector reductions (red.global.add.v4),
-// 16 values per thread and tile.  The sum order of dq therefore varies from run to run (fp32 rounding only).
+// sees, i.e. from different CTAs: the compute warps copy the finished tile from TMEM to a shared-memory stage and a
+// reduce warp adds it into the zeroed fp32 dq with TMA reductions (cp.reduce.async.bulk.tensor, whole 128-byte lines;
+// rows past the end of the sequence are clipped by the tensor map).  The sum order of dq therefore varies from run to
+// run (fp32 rounding only).
 //
 // TMEM columns: S^T two 64-query buffers [0,128), dP^T likewise [128,256), dV [256,320), dK [320,384),
 // dQ two buffers [384,448) [448,512).
@@ -25,8 +27,8 @@ using namespace tc;
 namespace {
 
 constexpr int FB_COMPUTE_WARPS = 16;
-constexpr int FB_TMA_WARP = FB_COMPUTE_WARPS, FB_MMA_WARP = FB_COMPUTE_WARPS + 1;
-constexpr int FB_THREADS = 32 * (FB_COMPUTE_WARPS + 2);
+constexpr int FB_TMA_WARP = FB_COMPUTE_WARPS, FB_MMA_WARP = FB_COMPUTE_WARPS + 1, FB_RED_WARP = FB_COMPUTE_WARPS + 2;
+constexpr int FB_THREADS = 32 * (FB_COMPUTE_WARPS + 3);
 constexpr float FB_LOG2E = 1.4426950408889634f;
 constexpr int DH = 64;
 
@@ -44,12 +46,14 @@ struct FbParams {
 struct FbSmem {
   static constexpr int TILE = 128 * DH * 2;            // 16 KB: K, V
   static constexpr int HALF_TILE = 64 * DH * 2;        // 64 queries of Q or dO
-  static constexpr int STAGES = 6;                     // ring of (Q, dO) half-tile pairs
+  static constexpr int STAGES = 4;                     // ring of (Q, dO) half-tile pairs
   static constexpr int DS_TILE = 128 * 128 * 2;        // dS^T [128 keys][128 queries] bf16: two 64-query boxes
+  static constexpr int DQ_STAGE = 128 * DH * 4;        // one dQ tile in fp32: two boxes of [128 queries][32 channels]
   static constexpr int FIX_OFF = 0;
   static constexpr int RING_OFF = 2 * TILE;
   static constexpr int DS_OFF = RING_OFF + STAGES * 2 * HALF_TILE;
-  static constexpr int BAR_OFF = DS_OFF + 2 * DS_TILE;
+  static constexpr int DQ_OFF = DS_OFF + 2 * DS_TILE;
+  static constexpr int BAR_OFF = DQ_OFF + DQ_STAGE;
   static constexpr int STAT_OFF = BAR_OFF + 256;       // float [2 groups][2 buffers][2][128]
   static constexpr int TOTAL = STAT_OFF + 4096 + 1024;
 };
@@ -76,7 +80,8 @@ TC_DEVINL uint32_t lo_mnmajor(uint32_t addr) { return (addr >> 4) | ((16384u >> 
 template <int POLY>
 __global__ void __launch_bounds__(FB_THREADS, 1)
 tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO, FbParams p) {
+                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO,
+                         const __grid_constant__ CUtensorMap tmDQ, FbParams p) {
   using SM = FbSmem;
   constexpr int NST = SM::STAGES;
   extern __shared__ unsigned char smem_dyn[];
@@ -97,7 +102,9 @@ tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   uint64_t* dq_full = stat_ready + 2;         // [2] MMA -> compute: dQ of a query tile ready in its TMEM buffer
   uint64_t* dq_empty = dq_full + 2;           // [2] compute -> MMA: that buffer has been added to memory (512 arrivals)
   uint64_t* ds_free = dq_empty + 2;           // [2] MMA -> compute: the dQ contraction has read the dS^T tile
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ds_free + 2);
+  uint64_t* stg_full = ds_free + 2;           // compute -> reduce warp: a dQ tile is in the stage (512 arrivals)
+  uint64_t* stg_free = stg_full + 1;          // reduce warp -> compute: the TMA reduction has read the stage
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(stg_free + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -126,12 +133,15 @@ tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       mbar_init(&ds_free[i], 1);
     }
     mbar_init(acc_done, 1);
+    mbar_init(stg_full, 32 * FB_COMPUTE_WARPS);
+    mbar_init(stg_free, 1);
     wait_ctl_init(abort_flag, p.status);
     fence_barrier_init();
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmV);
     prefetch_tmap(&tmDO);
+    prefetch_tmap(&tmDQ);
   }
   if (warp == FB_MMA_WARP) {
     tmem_alloc(tmem_slot, 512);
@@ -235,6 +245,24 @@ tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       }
     }
     if (leader) mma_commit(acc_done);
+  } else if (warp == FB_RED_WARP) {
+    // ------------------------------------------------------------------ dQ reductions into memory
+    if (lane == 0) {
+      unsigned char* stg = smem + SM::DQ_OFF;
+      for (int it = 0; it < n_it; ++it) {
+        if (!mbar_wait(stg_full, it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_CORR); goto done; }
+        const int hi = hj * p.g + it / n_q, m0 = (i0 + it % n_q) * 128;
+#pragma unroll
+        for (int c = 0; c < DH / 32; ++c)
+          asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+                       ::"l"(&tmDQ), "r"(hi * DH + c * 32), "r"(m0), "r"(b), "r"(smem_u32(stg + c * 16384))
+                       : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        mbar_arrive(stg_free);
+      }
+      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    }
   } else {
     // ------------------------------------------------------------------ compute, thread = key
     const int gsel = warp >> 3;                        // sub-tile (queries [64 gsel, 64 gsel + 64) of every query tile)
@@ -253,27 +281,27 @@ tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       if (ct < 128) return tq < p.S ? -p.lse[idx] * FB_LOG2E : -INFINITY;
       return tq < p.S ? -p.delta[idx] : 0.f;
     };
-    // adds the finished dQ of iteration `it` (its TMEM buffer) into memory: thread = query row, 16 channels
+    // hands the finished dQ of iteration `it` (its TMEM buffer) to the reduce warp: thread = query row, 16 channels,
+    // written into the fp32 stage (rows of 128 bytes, 128-byte swizzle, two 32-channel boxes)
+    unsigned char* stg_row = smem + SM::DQ_OFF + ((warp >> 2) >> 1) * 16384 + row * 128;
+    const int stg_ch = ((warp >> 2) & 1) * 4;
     auto flush_dq = [&](int it) -> bool {
       const int buf = it & 1;
       if (!mbar_wait(&dq_full[buf], (it >> 1) & 1, abort_flag)) return false;
       tc_fence_after();
       uint32_t t[16];
-      const int col = (warp >> 2) * 16;
-      tmem_ld16(tmem_base + lane_sel + 384 + buf * 64 + col, t);
+      tmem_ld16(tmem_base + lane_sel + 384 + buf * 64 + (warp >> 2) * 16, t);
       tmem_ld_wait();
       tc_fence_before();
       mbar_arrive(&dq_empty[buf]);
-      const int hi = hj * p.g + it / n_q, tq = (i0 + it % n_q) * 128 + row;
-      if (tq < p.S) {
-        float* dst = p.dq + ((long long)b * p.S + tq) * p.Lq + hi * DH + col;
+      if (!mbar_wait(stg_free, (it & 1) ^ 1, abort_flag)) return false;     // the previous tile has left the stage
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-          asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4 * i), "f"(__uint_as_float(t[4 * i]) * q_scale),
-                       "f"(__uint_as_float(t[4 * i + 1]) * q_scale), "f"(__uint_as_float(t[4 * i + 2]) * q_scale),
-                       "f"(__uint_as_float(t[4 * i + 3]) * q_scale)
-                       : "memory");
-      }
+      for (int i = 0; i < 4; ++i)
+        *reinterpret_cast<float4*>(stg_row + (((stg_ch + i) ^ (row & 7)) << 4)) =
+            make_float4(__uint_as_float(t[4 * i]) * q_scale, __uint_as_float(t[4 * i + 1]) * q_scale,
+                        __uint_as_float(t[4 * i + 2]) * q_scale, __uint_as_float(t[4 * i + 3]) * q_scale);
+      fence_proxy_async();
+      mbar_arrive(stg_full);
       return true;
     };
     float next_stat = n_it > 0 ? fetch_stat(0) : 0.f;
@@ -383,7 +411,7 @@ done:
 
 template <int POLY>
 int launch_fused(TcState* s, const CcaDims& d, const CUtensorMap& tmQh, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                 const CUtensorMap& tmDOh, const FbParams& p, cudaStream_t st) {
+                 const CUtensorMap& tmDOh, const CUtensorMap& tmDQ, const FbParams& p, cudaStream_t st) {
   static bool attr_set[TC_MAX_DEVICES] = {};
   if (!attr_set[s->device]) {
     cudaError_t e = cudaFuncSetAttribute(tc_attn_bwd_fused_kernel<POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, FbSmem::TOTAL);
@@ -394,7 +422,7 @@ int launch_fused(TcState* s, const CcaDims& d, const CUtensorMap& tmQh, const CU
   if (g_kv > 0x7fffffffLL) return 1;
   cudaError_t e = cudaMemsetAsync(p.dq, 0, (size_t)d.B * d.S * d.Lq * sizeof(float), st);
   if (e != cudaSuccess) return -(int)e;
-  tc_attn_bwd_fused_kernel<POLY><<<(unsigned)g_kv, FB_THREADS, FbSmem::TOTAL, st>>>(tmQh, tmK, tmV, tmDOh, p);
+  tc_attn_bwd_fused_kernel<POLY><<<(unsigned)g_kv, FB_THREADS, FbSmem::TOTAL, st>>>(tmQh, tmK, tmV, tmDOh, tmDQ, p);
   e = cudaGetLastError();
   return e == cudaSuccess ? 0 : -(int)e;
 }
@@ -415,13 +443,22 @@ int tc_attn_bwd_fused(TcState* s, const CcaDims& d, const bf16* q, const bf16* k
   if (!tc_make_map_3d(s, &tmDOh, d_o, Lq, S, B, Lq, S * Lq, 64, 64)) return 1;
   if (!tc_make_map_3d(s, &tmK, k, Lk, S, B, Lk, S * Lk, 64, 128)) return 1;
   if (!tc_make_map_3d(s, &tmV, v, Lk, S, B, Lk, S * Lk, 64, 128)) return 1;
+  CUtensorMap tmDQ;       // fp32 dq [B][S][Lq]: boxes of 128 rows x 32 channels for the reductions
+  {
+    cuuint64_t dims[3] = {(cuuint64_t)Lq, (cuuint64_t)S, (cuuint64_t)B};
+    cuuint64_t strides[2] = {(cuuint64_t)Lq * 4, (cuuint64_t)S * Lq * 4};
+    cuuint32_t box[3] = {32, 128, 1}, estr[3] = {1, 1, 1};
+    if (s->encode(&tmDQ, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dq, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return 1;
+  }
   FbParams p;
   p.B = d.B; p.S = d.S; p.hq = d.hq; p.hk = d.hk; p.g = d.g; p.Lq = d.Lq; p.Lk = d.Lk; p.causal = d.causal;
   p.lse = lse; p.delta = delta; p.dq = dq; p.dk = dk; p.dv = dv;
   p.n_tiles = (d.S + 127) / 128;
   p.status = d_status;
   const int poly = s->attn_poly_bwd < 0 ? 1 : s->attn_poly_bwd;
-  if (poly == 0) return launch_fused<0>(s, d, tmQh, tmK, tmV, tmDOh, p, st);
-  if (poly == 2) return launch_fused<2>(s, d, tmQh, tmK, tmV, tmDOh, p, st);
-  return launch_fused<1>(s, d, tmQh, tmK, tmV, tmDOh, p, st);
+  if (poly == 0) return launch_fused<0>(s, d, tmQh, tmK, tmV, tmDOh, tmDQ, p, st);
+  if (poly == 2) return launch_fused<2>(s, d, tmQh, tmK, tmV, tmDOh, tmDQ, p, st);
+  return launch_fused<1>(s, d, tmQh, tmK, tmV, tmDOh, tmDQ, p, st);
 }

@@ -391,6 +391,7 @@ int launch_pair(TcState* s, const GemmArgs& g, const G2Params& p0, bool a_mn, bo
 
 // Returns 0 if enqueued, 1 if the case is outside this kernel's coverage, -cudaError on failure.
 int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) {
+  if (g.accumulate) return 1;                       // the one-CTA kernel handles accumulation into the output
   if (!s || !s->encode || !s->use_pairs) return 1;
   if (g.a_row_off != 0) return 1;                                 // no row shift
   const int a_mn = g.A.cs != 1, b_mn = g.B.cs != 1;

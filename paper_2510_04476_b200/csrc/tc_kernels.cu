@@ -34,6 +34,7 @@ struct TcGemmParams {
   int splits, kb_per_split;   // split-K: work item = (tile, split); partial sums are added atomically (fp32 output)
   int a_mn, b_mn;
   int vec_ok;            // rows of C are 16-byte aligned: vector stores allowed
+  int atomic_out;        // add into the fp32 output (split-K partial sums, or the caller's accumulate)
   int* status;
 };
 
@@ -204,7 +205,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           } else {
             float* dst = p.out_f32 + (long long)m * p.ldc + n;
-            if (p.splits > 1) {
+            if (p.atomic_out) {
 #pragma unroll
               for (int i = 0; i < 32; ++i)
                 if (n + i < p.N) atomicAdd(dst + i, __uint_as_float(r[i]));
@@ -341,10 +342,12 @@ int tc_gemm(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) {
   }
   p.kb_per_split = (p.num_kb + p.splits - 1) / p.splits;
   p.splits = (p.num_kb + p.kb_per_split - 1) / p.kb_per_split;     // no empty split
-  if (p.splits > 1) {
+  if (g.accumulate && !g.out_f32) return 1;
+  if (p.splits > 1 && !g.accumulate) {
     cudaError_t me = cudaMemsetAsync(g.out_f32, 0, (size_t)g.M * g.N * sizeof(float), st);
     if (me != cudaSuccess) return -(int)me;
   }
+  p.atomic_out = (p.splits > 1 || g.accumulate) ? 1 : 0;
   p.a_mn = a_mn; p.b_mn = b_mn;
   const void* outp = g.out_bf16 ? (const void*)g.out_bf16 : (const void*)g.out_f32;
   const int esz = g.out_bf16 ? 2 : 4;

@@ -613,6 +613,10 @@ cudaError_t launch_transform_bwd_norm(const CcaDims& d, const bf16* q, const bf1
                                       cudaStream_t st) {
   if (!(d.flags & (F_QK_NORM | F_ROPE))) return cudaSuccess;
   const long long blocks = ((long long)d.B * d.S + BWD_NORM_TOK - 1) / BWD_NORM_TOK;
+  if (d.dh == 256) {
+    transform_bwd_norm_kernel<256><<<(unsigned)blocks, 256, 0, st>>>(d, q, k, rnorm, temp, rope_tab, dq, dk, d_temp);
+    return cudaGetLastError();
+  }
   DISPATCH_DH(d.dh, {
     transform_bwd_norm_kernel<DH><<<(unsigned)blocks, 256, 0, st>>>(d, q, k, rnorm, temp, rope_tab, dq, dk, d_temp);
   });

@@ -315,7 +315,7 @@ def test_adjacent_down_projection_weights_are_read_in_place():
     cca.close()
 
 
-# ------------------------------------------------------------------ head size 256 (forward only)
+# ------------------------------------------------------------------ head size 256
 DH256 = [
     S_("dh256_two_tiles", 2, 300, 1024, 4, 1, 256),
     S_("dh256_g2_ragged", 1, 777, 2048, 4, 2, 256),
@@ -329,21 +329,14 @@ DH256 = [
 
 @pytest.mark.parametrize("impl", [1, 0])
 @pytest.mark.parametrize("sh", DH256, ids=lambda s: s.name)
-def test_head_size_256_forward(sh, impl):
-    run_case(sh, impl, backward=False)
+def test_head_size_256_forward_backward(sh, impl):
+    run_case(sh, impl)
 
 
-def test_head_size_256_backward_is_refused():
-    from paper_2510_04476_b200.binding import CcaError
-    sh = DH256[0]
-    t = synth.make_inputs(sh)
-    dev = to_device(t)
-    cca = _cca(sh)
-    ws = cca.alloc_workspace(sh.B, sh.S, True)
-    cca.forward(dev, dev["x"], ws)
-    with pytest.raises(CcaError):
-        cca.backward(dev, dev["x"], dev["d_out"], ws)
-    cca.close()
+def test_head_size_256_backward_over_several_query_chunks():
+    """The adjoint at head size 256 walks the queries in chunks of 1024 rows and accumulates dK, dV over the chunks and
+    over the query heads of a group: two sequences of 2500 tokens, 4 query heads on 2 kv heads."""
+    run_case(S_("dh256_chunks", 2, 2500, 2048, 4, 2, 256), 1)
 
 
 def test_head_size_256_at_16k_sampled_rows():
