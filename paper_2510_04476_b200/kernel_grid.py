@@ -60,7 +60,7 @@ def time_shape(sh: synth.Shape, steps: int, device: int):
         key = "causal" if causal else "noncausal"
         res[f"fwd_{key}_ms"] = e0.elapsed_time(e1) / steps
         res[f"attn_fwd_{key}_ms"] = sum(a.elapsed_time(b) for a, b in ev) / steps
-        if not causal and sh.head_dim <= 128:          # head size 256 has no backward
+        if not causal:
             for _ in range(2):
                 cca.forward(dev, dev["x"], ws, out)
                 cca.backward(dev, dev["x"], dev["d_out"], ws)
