@@ -242,6 +242,35 @@ int cca_decode_step(cca_handle* h, const cca_weights* w, const void* x, void* ou
 int cca_decode_state_from_prefill(cca_handle* h, const void* x, const void* workspace, size_t workspace_bytes,
                                   int64_t B, int64_t S, const cca_decode_state* state, void* cuda_stream);
 
+/* ---- MLA baseline --------------------------------------------------------------------------------
+ * Multi-Latent Attention as the paper's Section 2.1 defines it (Eq. 3-6), one of the methods its kernel study compares
+ * CCA with, run on this library's GEMM and attention kernels: forward only.  C_KV = x W_DKV, C_Q = x W_DQ (Eq. 3);
+ * per-head q, k, v up-projected from the latents (Eq. 4); a RoPE part per query head from C_Q and ONE RoPE key part from
+ * x shared by every head, concatenated behind the position-free parts (Eq. 6); causal softmax attention per head with
+ * scale 1 / sqrt(d_nope + d_rope); output projection.
+ * The handle describes the attention: n_q_heads = n_kv_heads = n_h, head_dim = d_nope + d_rope (also the value head
+ * size), d_model = E, causal; its stage flags are not used.  All weights bf16 device, [out, in] row-major. */
+typedef struct {
+  int32_t d_nope, d_rope;   /* per-head sizes of the position-free and the RoPE part (multiples of 8 / 16)        */
+  int32_t d_ckv, d_cq;      /* widths of the shared KV latent (E / c_kv) and of the query latent (E / c_q)        */
+} cca_mla_dims;
+typedef struct {
+  const void* w_dq;     /* [d_cq, E]               Eq. 3 */
+  const void* w_dkv;    /* [d_ckv, E]              Eq. 3 */
+  const void* w_uq;     /* [n_h * d_nope, d_cq]    Eq. 4 */
+  const void* w_uqr;    /* [n_h * d_rope, d_cq]    Eq. 6 */
+  const void* w_uk;     /* [n_h * d_nope, d_ckv]   Eq. 4 */
+  const void* w_uv;     /* [n_h * head_dim, d_ckv] Eq. 4 */
+  const void* w_kr;     /* [d_rope, E]             Eq. 6 */
+  const void* w_o;      /* [E, n_h * head_dim]           */
+} cca_mla_weights;
+int cca_mla_workspace_size(const cca_handle* h, const cca_mla_dims* m, int64_t B, int64_t S, size_t* bytes);
+/* x, out: device bf16 [B,S,E].  workspace: device, 256-byte aligned, >= cca_mla_workspace_size; on return it holds the
+ * latents and q, k, v, o ([B,S,n_h,head_dim] bf16) and lse.  Errors: INVALID_ARG (null, sizes that do not add up to
+ * the handle's head_dim, n_q_heads != n_kv_heads), UNSUPPORTED, ALIGNMENT, WORKSPACE_TOO_SMALL, CUDA. */
+int cca_mla_forward(cca_handle* h, const cca_mla_dims* m, const cca_mla_weights* w, const void* x, void* out, void* workspace,
+                    size_t workspace_bytes, int64_t B, int64_t S, void* cuda_stream);
+
 /* Select kernel implementations: 0 = plain SIMT kernels, 1 = tcgen05/TMA kernels where they
  * exist (default).  Returns the previous value. */
 int cca_set_impl(cca_handle* h, int impl);

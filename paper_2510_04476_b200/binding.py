@@ -45,6 +45,17 @@ class cca_layout(C.Structure):
                 ("saved_bytes", C.c_int64), ("total_bytes", C.c_int64), ("off_rnorm", C.c_int64)]
 
 
+class cca_mla_dims(C.Structure):
+    _fields_ = [("d_nope", C.c_int32), ("d_rope", C.c_int32), ("d_ckv", C.c_int32), ("d_cq", C.c_int32)]
+
+
+MLA_WEIGHTS = ("w_dq", "w_dkv", "w_uq", "w_uqr", "w_uk", "w_uv", "w_kr", "w_o")
+
+
+class cca_mla_weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in MLA_WEIGHTS]
+
+
 class cca_decode_state(C.Structure):
     _fields_ = [("k_cache", C.c_void_p), ("v_cache", C.c_void_p), ("qk0_hist", C.c_void_p), ("x_prev", C.c_void_p),
                 ("pos", C.c_void_p), ("S_max", C.c_int64)]
@@ -73,6 +84,9 @@ SYMBOLS = {
                                   C.c_int64, C.c_void_p, C.c_size_t, C.c_int64, C.c_void_p]),
     "cca_decode_state_from_prefill": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_int64, C.c_int64,
                                                 C.POINTER(cca_decode_state), C.c_void_p]),
+    "cca_mla_workspace_size": (C.c_int, [C.c_void_p, C.POINTER(cca_mla_dims), C.c_int64, C.c_int64, C.POINTER(C.c_size_t)]),
+    "cca_mla_forward": (C.c_int, [C.c_void_p, C.POINTER(cca_mla_dims), C.POINTER(cca_mla_weights), C.c_void_p, C.c_void_p,
+                                  C.c_void_p, C.c_size_t, C.c_int64, C.c_int64, C.c_void_p]),
     "cca_set_impl": (C.c_int, [C.c_void_p, C.c_int]),
     "cca_set_attention_events": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "cca_set_stage_events": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
@@ -384,6 +398,31 @@ class CCA:
         _check(self.lib, self.lib.cca_backward(self.handle, C.byref(cw), _ptr(x), _ptr(d_out), wp, wn, _ptr(d_x),
                                                C.byref(cg), B, S, st), self.handle, "cca_backward")
         return d_x, grads
+
+    def mla_forward(self, dims, w, x: torch.Tensor, out: Optional[torch.Tensor] = None):
+        """cca_mla_forward.  dims = (d_nope, d_rope, d_ckv, d_cq); w: dict of the eight bf16 weights.  Returns (out, workspace)."""
+        B, S, E = x.shape
+        md = cca_mla_dims(*dims)
+        n = C.c_size_t()
+        _check(self.lib, self.lib.cca_mla_workspace_size(self.handle, C.byref(md), B, S, C.byref(n)), self.handle,
+               "cca_mla_workspace_size")
+        key = (B, S, tuple(dims))
+        if getattr(self, "_mla_ws_key", None) != key:              # the workspace is kept between calls of one shape
+            self._mla_ws = torch.empty(int(n.value) + 256, dtype=torch.uint8, device=self.device)
+            self._mla_ws_key = key
+        ws = self._mla_ws
+        if out is None:
+            out = torch.empty_like(x)
+        mw = cca_mla_weights()
+        for name in MLA_WEIGHTS:
+            t = w[name]
+            assert t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16, name
+            setattr(mw, name, t.data_ptr())
+        wp, wn = self._ws_ptr(ws)
+        st = C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+        _check(self.lib, self.lib.cca_mla_forward(self.handle, C.byref(md), C.byref(mw), _ptr(x), _ptr(out), wp, wn, B, S, st),
+               self.handle, "cca_mla_forward")
+        return out, ws
 
     def attention_forward(self, q, k, v, o=None, lse=None):
         B, S, hq, dh = q.shape

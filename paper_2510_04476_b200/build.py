@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcca.so")
-SOURCES = ["cca_api.cu", "gemm_simt.cu", "transform.cu", "attn_simt.cu", "tc_kernels.cu", "tc_gemm2.cu", "tc_attn.cu", "tc_attn_bwd.cu", "tc_attn_bwd_fused.cu", "tc_transform.cu", "tc_transform2.cu", "tc_transform_bwd.cu", "decode.cu", "tc_attn256.cu", "transform_unfused.cu", "bwd_unfused.cu"]
+SOURCES = ["cca_api.cu", "gemm_simt.cu", "transform.cu", "attn_simt.cu", "tc_kernels.cu", "tc_gemm2.cu", "tc_attn.cu", "tc_attn_bwd.cu", "tc_attn_bwd_fused.cu", "tc_transform.cu", "tc_transform2.cu", "tc_transform_bwd.cu", "decode.cu", "tc_attn256.cu", "transform_unfused.cu", "bwd_unfused.cu", "mla.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "--use_fast_math", "-Xptxas", "-v",

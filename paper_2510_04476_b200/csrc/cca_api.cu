@@ -996,6 +996,103 @@ int cca_backward(cca_handle* h, const cca_weights* w, const void* x, const void*
   return CCA_OK;
 }
 
+// ---- MLA baseline ---------------------------------------------------------------------------------
+namespace {
+struct MlaLayout {
+  size_t cq, ckv, kr, qn, qr, kn, q, k, v, o, lse, rope, end;
+};
+MlaLayout make_mla_layout(const cca_config& c, const cca_mla_dims& m, int64_t B, int64_t S) {
+  MlaLayout l;
+  const size_t T = (size_t)B * S, nh = c.n_q_heads, dh = c.head_dim;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  l.cq = take(T * m.d_cq * 2);
+  l.ckv = take(T * m.d_ckv * 2);
+  l.kr = take(T * m.d_rope * 2);
+  l.qn = take(T * nh * m.d_nope * 2);
+  l.qr = take(T * nh * m.d_rope * 2);
+  l.kn = take(T * nh * m.d_nope * 2);
+  l.q = take(T * nh * dh * 2);
+  l.k = take(T * nh * dh * 2);
+  l.v = take(T * nh * dh * 2);
+  l.o = take(T * nh * dh * 2);
+  l.lse = take((size_t)B * nh * S * 4);
+  l.rope = take((size_t)S * (m.d_rope / 2) * 8);
+  l.end = off;
+  return l;
+}
+int check_mla(const cca_handle* h, const cca_mla_dims* m) {
+  if (!h || !m) return CCA_ERR_INVALID_ARG;
+  const cca_config& c = h->cfg;
+  if (m->d_nope < 8 || m->d_rope < 8 || m->d_ckv < 8 || m->d_cq < 8) return CCA_ERR_INVALID_ARG;
+  if (m->d_nope + m->d_rope != c.head_dim || c.n_q_heads != c.n_kv_heads) return CCA_ERR_INVALID_ARG;
+  if (m->d_nope % 8 || m->d_rope % 16 || m->d_ckv % 8 || m->d_cq % 8) return CCA_ERR_UNSUPPORTED;
+  return CCA_OK;
+}
+}  // namespace
+
+int cca_mla_workspace_size(const cca_handle* h, const cca_mla_dims* m, int64_t B, int64_t S, size_t* bytes) {
+  int r = check_sizes(h, B, S);
+  if (r != CCA_OK) return r;
+  if ((r = check_mla(h, m)) != CCA_OK) return r;
+  if (!bytes) return CCA_ERR_INVALID_ARG;
+  *bytes = make_mla_layout(h->cfg, *m, B, S).end;
+  return CCA_OK;
+}
+
+int cca_mla_forward(cca_handle* h, const cca_mla_dims* m, const cca_mla_weights* w, const void* x, void* out, void* workspace,
+                    size_t workspace_bytes, int64_t B, int64_t S, void* cuda_stream) {
+  int r = check_sizes(h, B, S, true);
+  if (r != CCA_OK) return r;
+  if ((r = check_mla(h, m)) != CCA_OK) return r;
+  if (!w || !x || !out || !workspace) return CCA_ERR_INVALID_ARG;
+  if (!w->w_dq || !w->w_dkv || !w->w_uq || !w->w_uqr || !w->w_uk || !w->w_uv || !w->w_kr || !w->w_o) return CCA_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(out) || !aligned16(w->w_dq) || !aligned16(w->w_dkv) || !aligned16(w->w_uq) ||
+      !aligned16(w->w_uqr) || !aligned16(w->w_uk) || !aligned16(w->w_uv) || !aligned16(w->w_kr) || !aligned16(w->w_o) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CCA_ERR_ALIGNMENT;
+  const cca_config& c = h->cfg;
+  MlaLayout l = make_mla_layout(c, *m, B, S);
+  if (workspace_bytes < l.end) return CCA_ERR_WORKSPACE_TOO_SMALL;
+  CU(cudaSetDevice(h->device));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CcaDims d = make_dims(c, B, S);
+  const int T = d.B * d.S, nh = d.hq, dn = m->d_nope, dr = m->d_rope, E = d.E;
+  char* ws = (char*)workspace;
+  bf16 *cq = (bf16*)(ws + l.cq), *ckv = (bf16*)(ws + l.ckv), *kr = (bf16*)(ws + l.kr), *qn = (bf16*)(ws + l.qn);
+  bf16 *qr = (bf16*)(ws + l.qr), *kn = (bf16*)(ws + l.kn), *q = (bf16*)(ws + l.q), *k = (bf16*)(ws + l.k);
+  bf16 *v = (bf16*)(ws + l.v), *o = (bf16*)(ws + l.o);
+  float* lse = (float*)(ws + l.lse);
+  float2* rope = (float2*)(ws + l.rope);
+  STAGE(CCA_EV_FWD_BEGIN);
+  CU(launch_rope_table(rope, d.S, dr, c.rope_base > 0.f ? c.rope_base : 10000.f, st));
+  h->launches++;
+  auto gemm = [&](const void* a, long long lda, const void* bw, int N, int K, bf16* dst) -> int {
+    GemmArgs g{};
+    g.A = kmajor(a, lda); g.B = kmajor(bw, K);
+    g.M = T; g.N = N; g.K = K; g.seq_len = d.S; g.out_bf16 = dst; g.ldc = N;
+    return run_gemm(h, g, st);
+  };
+  // Eq. 3: the two latents (and the shared key's RoPE part straight from x, Eq. 6)
+  if ((r = gemm(x, E, w->w_dq, m->d_cq, E, cq)) != CCA_OK) return r;
+  if ((r = gemm(x, E, w->w_dkv, m->d_ckv, E, ckv)) != CCA_OK) return r;
+  if ((r = gemm(x, E, w->w_kr, dr, E, kr)) != CCA_OK) return r;
+  // Eq. 4 and Eq. 6: per-head up-projections
+  if ((r = gemm(cq, m->d_cq, w->w_uq, nh * dn, m->d_cq, qn)) != CCA_OK) return r;
+  if ((r = gemm(cq, m->d_cq, w->w_uqr, nh * dr, m->d_cq, qr)) != CCA_OK) return r;
+  if ((r = gemm(ckv, m->d_ckv, w->w_uk, nh * dn, m->d_ckv, kn)) != CCA_OK) return r;
+  if ((r = gemm(ckv, m->d_ckv, w->w_uv, nh * d.dh, m->d_ckv, v)) != CCA_OK) return r;
+  STAGE(CCA_EV_FWD_PROJ);
+  CU(launch_mla_assemble(T, d.S, nh, dn, dr, qn, qr, kn, kr, rope, q, k, st));
+  h->launches++;
+  STAGE(CCA_EV_FWD_TRANSFORM);
+  if ((r = run_attention_fwd(h, d, q, k, v, o, nullptr, lse, nullptr, st)) != CCA_OK) return r;
+  STAGE(CCA_EV_FWD_ATTN);
+  if ((r = gemm(o, d.Lq, w->w_o, E, d.Lq, (bf16*)out)) != CCA_OK) return r;
+  STAGE(CCA_EV_FWD_END);
+  return CCA_OK;
+}
+
 // ---- forward without any caller-provided or allocated workspace ---------------------------------
 // The scratch of cca_forward_static: one array in the library's device image.  Every GPU that loads the
 // library reserves these bytes until the process exits.  In host code `g_static_ws` is only a handle for

@@ -89,6 +89,10 @@ cudaError_t launch_cast_dhat(const CcaDims& d, const float* dqh, const float* dk
 // dy1 [T, L] from dy1s [T, L * k_ch] (gradient of the conv1 output stored at the k_ch positions conv2 reads).
 cudaError_t launch_taps_adjoint(const CcaDims& d, const float* dy1s, float* dy1, cudaStream_t st);
 
+// ---- MLA baseline (Eq. 6): attention operands from the up-projected parts (mla.cu) ----
+cudaError_t launch_mla_assemble(long long tokens, int S, int nh, int dn, int dr, const bf16* qn, const bf16* qr, const bf16* kn,
+                                const bf16* kr, const float2* rope, bf16* q, bf16* k, cudaStream_t st);
+
 // ---- attention (Eq. 11, softmax line), plain SIMT ----
 // o32: optional fp32 copy of o (kept for the backward's delta = rowsum(dO * O)); may be null.
 cudaError_t launch_attn_fwd_simt(const CcaDims& d, const bf16* q, const bf16* k, const bf16* v, bf16* o,

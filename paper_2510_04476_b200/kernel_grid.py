@@ -1,7 +1,8 @@
 """Latency grid of the block's kernels, after the paper's kernel study (Appendix D.1): d_model 2048, latent
 head size 64 or 128, sequence lengths 512 ... 16384, forward causal and non-causal, forward + backward
 non-causal, for CCGQA (C = 4, four query heads per kv head) and for the same kernels configured as GQA
-(no compression, four query heads per kv head, latent transforms off) and as MHA.
+(no compression, four query heads per kv head, latent transforms off), as MHA, and as MLA (Section 2.1 of the paper,
+Eq. 3-6: E / d_h heads, half of each head RoPE with one shared RoPE key, KV latent E / 4, query latent E / 2; forward only).
 
     python -m paper_2510_04476_b200.kernel_grid [--tokens 32768] [--steps 5] [--head-dims 64,128]
     python -m paper_2510_04476_b200.kernel_grid --sweep          # context x compression sweep, forward and backward
@@ -29,7 +30,40 @@ def shapes_for(dh: int, S: int, tokens: int):
     ccgqa = synth.Shape(f"grid_ccgqa_d{dh}_S{S}", B, S, E, h // 4, max(1, h // 16), dh, seed=seed)
     gqa = synth.Shape(f"grid_gqa_d{dh}_S{S}", B, S, E, h, h // 4, dh, flags=0, seed=seed)
     mha = synth.Shape(f"grid_mha_d{dh}_S{S}", B, S, E, h, h, dh, flags=0, seed=seed)
-    return {"ccgqa": ccgqa, "gqa": gqa, "mha": mha}
+    return {"ccgqa": ccgqa, "gqa": gqa, "mha": mha, "mla": synth.mla_like(mha)}
+
+
+def time_mla(m: synth.MlaShape, steps: int, device: int):
+    """ms of the MLA baseline's forward, causal and non-causal (block, attention kernel)."""
+    res = {}
+    dev = {k: v.cuda(device).contiguous() for k, v in synth.make_mla_inputs(m).items()}
+    out = torch.empty_like(dev["x"])
+    dims = (m.d_nope, m.d_rope, m.d_ckv, m.d_cq)
+    for causal in (1, 0):
+        cca = CCA(m.d_model, m.n_heads, m.n_heads, m.head_dim, causal=causal, flags=0, device=device)
+        for _ in range(3):
+            cca.mla_forward(dims, dev, dev["x"], out)
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in ev:
+            a.record(); b.record()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(steps):
+            cca.set_attention_events(*ev[i])
+            cca.mla_forward(dims, dev, dev["x"], out)
+        e1.record()
+        torch.cuda.synchronize()
+        cca.set_attention_events(None, None)
+        key = "causal" if causal else "noncausal"
+        res[f"fwd_{key}_ms"] = e0.elapsed_time(e1) / steps
+        res[f"attn_fwd_{key}_ms"] = sum(a.elapsed_time(b) for a, b in ev) / steps
+        st = cca.last_status()
+        cca.close()
+        if st != 0:
+            raise RuntimeError(f"device status {st} at {m.name}")
+    return res
 
 
 def time_shape(sh: synth.Shape, steps: int, device: int):
@@ -149,13 +183,14 @@ def main(argv=None):
         for S in [int(v) for v in a.seq_lens.split(",")]:
             rec = {"head_dim": dh, "S": S, "B": max(1, a.tokens // S)}
             for name, sh in shapes_for(dh, S, a.tokens).items():
-                r = time_shape(sh, a.steps, a.device)
+                r = time_mla(sh, a.steps, a.device) if name == "mla" else time_shape(sh, a.steps, a.device)
                 rec[name] = r
-                print(json.dumps({"method": name, "head_dim": dh, "S": S, "B": sh.B, "heads": [sh.n_q_heads, sh.n_kv_heads],
+                heads = [sh.n_heads, sh.n_heads] if name == "mla" else [sh.n_q_heads, sh.n_kv_heads]
+                print(json.dumps({"method": name, "head_dim": dh, "S": S, "B": sh.B, "heads": heads,
                                   **{k: round(v, 4) for k, v in r.items()}}), flush=True)
             rows.append(rec)
     cols = ["fwd_causal_ms", "fwd_noncausal_ms", "fwd_bwd_noncausal_ms"]
-    print("\n| d_h | S | B | " + " | ".join(f"{c[:-3]}: CCGQA / GQA / MHA (ms), MHA/CCGQA" for c in cols) + " |")
+    print("\n| d_h | S | B | " + " | ".join(f"{c[:-3]}: CCGQA / GQA / MLA / MHA (ms), MHA/CCGQA" for c in cols) + " |")
     print("|---|---|---|" + "---|" * len(cols))
     for r in rows:
         cells = []
@@ -164,7 +199,8 @@ def main(argv=None):
                 cells.append("-")
                 continue
             v = [r[m][c] for m in ("ccgqa", "gqa", "mha")]
-            cells.append(f"{v[0]:.3f} / {v[1]:.3f} / {v[2]:.3f}, {v[2] / v[0]:.2f}x")
+            mla = f"{r['mla'][c]:.3f}" if c in r["mla"] else "-"
+            cells.append(f"{v[0]:.3f} / {v[1]:.3f} / {mla} / {v[2]:.3f}, {v[2] / v[0]:.2f}x")
         print(f"| {r['head_dim']} | {r['S']} | {r['B']} | " + " | ".join(cells) + " |")
     return 0
 

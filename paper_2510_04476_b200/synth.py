@@ -112,3 +112,56 @@ def make_inputs(shape: Shape, want_dout: bool = True) -> Dict[str, torch.Tensor]
     if want_dout:
         t["d_out"] = normal((shape.B, shape.S, E), 1.0)
     return t
+
+
+@dataclasses.dataclass(frozen=True)
+class MlaShape:
+    """Multi-Latent Attention (the paper's Section 2.1) as a baseline: E, heads, per-head part sizes, latent widths."""
+    name: str
+    B: int
+    S: int
+    d_model: int
+    n_heads: int
+    d_nope: int
+    d_rope: int
+    d_ckv: int
+    d_cq: int
+    causal: int = 1
+    rope_base: float = 10000.0
+    seed: int = 0
+
+    @property
+    def head_dim(self) -> int:
+        return self.d_nope + self.d_rope
+
+
+def mla_like(shape: Shape) -> MlaShape:
+    """The MLA baseline of equal d_model and head size: E / d_h heads, half of each query / key head position-free
+    and half RoPE (one RoPE key part shared by all heads), value heads of size d_h, KV latent E / 4, query latent
+    E / 2.  The paper gives no MLA dimensions for its kernel study; these keep the attention FLOPs at MHA's, as
+    its text describes."""
+    dh = shape.head_dim
+    return MlaShape(shape.name + "_mla", shape.B, shape.S, shape.d_model, shape.d_model // dh, dh // 2, dh // 2,
+                    shape.d_model // 4, shape.d_model // 2, causal=shape.causal, seed=shape.seed)
+
+
+def make_mla_inputs(m: MlaShape) -> Dict[str, torch.Tensor]:
+    """x ~ N(0,1), every projection ~ N(0,0.02), drawn in the order x, w_dq, w_dkv, w_uq, w_uqr, w_uk, w_uv, w_kr,
+    w_o and rounded to bf16."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(m.seed)
+    E, nh, dh = m.d_model, m.n_heads, m.head_dim
+
+    def normal(size, std):
+        return (torch.randn(size, generator=g, dtype=torch.float32) * std).to(torch.bfloat16)
+
+    t = {"x": normal((m.B, m.S, E), 1.0)}
+    t["w_dq"] = normal((m.d_cq, E), 0.02)
+    t["w_dkv"] = normal((m.d_ckv, E), 0.02)
+    t["w_uq"] = normal((nh * m.d_nope, m.d_cq), 0.02)
+    t["w_uqr"] = normal((nh * m.d_rope, m.d_cq), 0.02)
+    t["w_uk"] = normal((nh * m.d_nope, m.d_ckv), 0.02)
+    t["w_uv"] = normal((nh * dh, m.d_ckv), 0.02)
+    t["w_kr"] = normal((m.d_rope, E), 0.02)
+    t["w_o"] = normal((E, nh * dh), 0.02)
+    return t
