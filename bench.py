@@ -92,7 +92,7 @@ def stage_table(sh, backward):
             ("d_o = d_out W_o", "bwd_begin", "bwd_do", "tensor", 2 * T * E * Lq),
             ("d_W_o = d_out^T o", "bwd_do", "bwd_dwo", "tensor", 2 * T * E * Lq),
             ("delta = rowsum(dO o O)", "bwd_dwo", "bwd_delta", "hbm", 4 * T * Lq + 2 * T * Lq + 4 * T * sh.n_q_heads),
-            ("latent attention backward (dK/dV and dQ kernels)", "bwd_delta", "bwd_attn", "tensor", 2.5 * attn),
+            ("latent attention backward", "bwd_delta", "bwd_attn", "tensor", 2.5 * attn),
             ("norm / RoPE adjoint, d_temp", "bwd_attn", "bwd_norm", "hbm", 2 * (4 * T * L) + 2 * T * L + 4 * T * H),
             ("conv2 adjoint, d_conv1_w", "bwd_norm", "bwd_conv2", "hbm", 4 * T * L + 4 * T * L + 4 * T * L),
             ("conv1 and q-k-mean adjoint, d_conv0_w", "bwd_conv2", "bwd_conv1", "hbm", 3 * (4 * T * L) + 2 * T * L),
@@ -401,7 +401,7 @@ def run_ours(args, rank, world, local_rank):
                 "ms_per_step": e2e_ms},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor",
-                     "kernel": "latent attention backward (dQ and dK/dV kernels)" if backward else "latent attention forward",
+                     "kernel": "latent attention backward" if backward else "latent attention forward",
                      "achieved": attn_tflops, "peak": peak,
                      "unit": "TFLOP/s", "frac": attn_tflops / peak, "peak_kind": peak_kind,
                      "frac_of_nominal_2250": attn_tflops / NOMINAL_BF16_TFLOPS, "ms_per_launch": attn_ms,

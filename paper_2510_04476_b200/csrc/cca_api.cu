@@ -86,7 +86,7 @@ Layout make_layout(const cca_config& c, int64_t B, int64_t S) {
   l.dlat = take(T * (L + Lk) * 2);
   l.dy1 = take(T * L * 4);
   l.u_s = l.u_dp = l.u_p = l.u_ds = l.u_dy1s = off;
-  l.u_rows = 1024;
+  l.u_rows = 2048;
   l.u_ld = align_up((size_t)S, 128);
   if (c.head_dim > 128) {
     l.u_s = take((size_t)l.u_rows * l.u_ld * 4);

@@ -10,11 +10,11 @@ from tests.util import check_close
 pytestmark = pytest.mark.gpu
 
 
-def run(m, impl=1):
+def run(m, impl=1, scale=4.0):
     from paper_2510_04476_b200.binding import CCA
     t = synth.make_mla_inputs(m)
     for n in ("w_uq", "w_uqr", "w_uk", "w_uv", "w_kr"):        # larger logits and outputs than the N(0, 0.02) recipe gives:
-        t[n] = (t[n].float() * 4).to(torch.bfloat16)           # peaked rows, outputs well above the absolute tolerance
+        t[n] = (t[n].float() * scale).to(torch.bfloat16)       # peaked rows, outputs well above the absolute tolerance
     cfg = M.MlaConfig(m.d_model, m.n_heads, m.d_nope, m.d_rope, m.head_dim, m.d_ckv, m.d_cq, m.causal, m.rope_base)
     out_ref, I = M.forward(cfg, t, t["x"])
     dev = {k: v.cuda().contiguous() for k, v in t.items()}
@@ -43,7 +43,7 @@ def test_mla_forward_matches_oracle(m, impl):
 
 
 def test_mla_baseline_of_the_kernel_grid_shape():
-    run(synth.mla_like(synth.Shape("grid", 1, 2048, 2048, 4, 1, 128, seed=3)))
+    run(synth.mla_like(synth.Shape("grid", 1, 2048, 2048, 4, 1, 128, seed=3)), scale=1.0)     # the grid's own recipe
 
 
 def test_mla_argument_checks():

@@ -334,9 +334,9 @@ def test_head_size_256_forward_backward(sh, impl):
 
 
 def test_head_size_256_backward_over_several_query_chunks():
-    """The adjoint at head size 256 walks the queries in chunks of 1024 rows and accumulates dK, dV over the chunks and
-    over the query heads of a group: two sequences of 2500 tokens, 4 query heads on 2 kv heads."""
-    run_case(S_("dh256_chunks", 2, 2500, 2048, 4, 2, 256), 1)
+    """The adjoint at head size 256 walks the queries in chunks of 2048 rows and accumulates dK, dV over the chunks and
+    over the query heads of a group: two sequences of 4500 tokens, 4 query heads on 2 kv heads."""
+    run_case(S_("dh256_chunks", 2, 4500, 2048, 4, 2, 256), 1)
 
 
 def test_head_size_256_at_16k_sampled_rows():
