@@ -27,8 +27,10 @@ using namespace tc;
 namespace {
 
 constexpr int FB_COMPUTE_WARPS = 16;
-constexpr int FB_TMA_WARP = FB_COMPUTE_WARPS, FB_MMA_WARP = FB_COMPUTE_WARPS + 1, FB_RED_WARP = FB_COMPUTE_WARPS + 2;
-constexpr int FB_THREADS = 32 * (FB_COMPUTE_WARPS + 3);
+// warp 16: lane 0 issues the TMA loads, lane 1 the dQ reductions (two independent loops of one warp: a third service
+// warp would cost every thread 16 registers); warp 17 issues the MMAs
+constexpr int FB_TMA_WARP = FB_COMPUTE_WARPS, FB_MMA_WARP = FB_COMPUTE_WARPS + 1;
+constexpr int FB_THREADS = 32 * (FB_COMPUTE_WARPS + 2);
 constexpr float FB_LOG2E = 1.4426950408889634f;
 constexpr int DH = 64;
 
@@ -167,6 +169,22 @@ tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         tma_load_3d(dst, &tmQ, hi * DH, m0, b, &qdo_full[st]);
         tma_load_3d(dst + SM::HALF_TILE, &tmDO, hi * DH, m0, b, &qdo_full[st]);
       }
+    } else if (lane == 1) {
+      // ---------------------------------------------------------------- dQ reductions into memory
+      unsigned char* stg = smem + SM::DQ_OFF;
+      for (int it = 0; it < n_it; ++it) {
+        if (!mbar_wait(stg_full, it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_CORR); goto done; }
+        const int hi = hj * p.g + it / n_q, m0 = (i0 + it % n_q) * 128;
+#pragma unroll
+        for (int c = 0; c < DH / 32; ++c)
+          asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+                       ::"l"(&tmDQ), "r"(hi * DH + c * 32), "r"(m0), "r"(b), "r"(smem_u32(stg + c * 16384))
+                       : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        mbar_arrive(stg_free);
+      }
+      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
   } else if (warp == FB_MMA_WARP) {
     const bool leader = elect_one();
@@ -245,24 +263,6 @@ tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       }
     }
     if (leader) mma_commit(acc_done);
-  } else if (warp == FB_RED_WARP) {
-    // ------------------------------------------------------------------ dQ reductions into memory
-    if (lane == 0) {
-      unsigned char* stg = smem + SM::DQ_OFF;
-      for (int it = 0; it < n_it; ++it) {
-        if (!mbar_wait(stg_full, it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_CORR); goto done; }
-        const int hi = hj * p.g + it / n_q, m0 = (i0 + it % n_q) * 128;
-#pragma unroll
-        for (int c = 0; c < DH / 32; ++c)
-          asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
-                       ::"l"(&tmDQ), "r"(hi * DH + c * 32), "r"(m0), "r"(b), "r"(smem_u32(stg + c * 16384))
-                       : "memory");
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        mbar_arrive(stg_free);
-      }
-      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-    }
   } else {
     // ------------------------------------------------------------------ compute, thread = key
     const int gsel = warp >> 3;                        // sub-tile (queries [64 gsel, 64 gsel + 64) of every query tile)

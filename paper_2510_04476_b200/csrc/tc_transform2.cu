@@ -12,9 +12,9 @@
 // on: the shared-memory descriptor's start address moves down by m rows of 128 bytes, the 128-byte swizzle being a
 // function of the address.  No thread touches an operand.
 //
-//   warp 8   TMA: the head's NT weight tiles when the head changes, one operand tile per unit (ring of stages)
-//   warp 9   MMA issue: acc = sum_m A_m W_m^T into one of two TMEM accumulators (128 tokens x d_h, fp32)
-//   warps 0-7  epilogue, thread = token, two groups of four warps that take every other unit: adds the q-k-mean term
+//   TMA warp   the head's NT weight tiles when the head changes, one operand tile per unit (ring of stages)
+//   MMA warp   acc = sum_m A_m W_m^T into one of NG TMEM accumulators (128 tokens x d_h, fp32)
+//   4 NG warps epilogue, thread = token, NG groups of four warps that take every NG-th unit: adds the q-k-mean term
 //            of Eq. 9 in fp32 from the fp32 latent, L2 norm * sqrt(d_h) (* exp(temp)), RoPE from the table, bf16
 //            store; the norm scale is kept for the backward.  A thread needs 128 bytes of its own token's row at a
 //            time (32 fp32 channels, or 16 (cos, sin) pairs); fetched by the thread itself that would be one memory
@@ -29,9 +29,18 @@ using namespace tc;
 
 namespace {
 
-constexpr int T2_EPI_THREADS = 256;
-constexpr int T2_TMA_WARP = 8, T2_MMA_WARP = 9;
-constexpr int T2_THREADS = 320;
+// Epilogue groups of four warps (one per TMEM lane quarter), each with a TMEM accumulator of its own, taking every
+// NG-th unit: the epilogue is a latency chain (TMA box -> shared memory -> TMEM round trip), so what matters is how many
+// units are in flight.  Four groups at head size 64 (4 x 64 TMEM columns), three at 128 (3 x 128; shared memory for the
+// boxes' slots and the register file set the limit).
+template <int DH, int NT>
+struct T2Groups {
+  static constexpr int NG = DH == 64 ? 4 : (NT <= 3 ? 3 : 2);
+  static constexpr int EPI_WARPS = 4 * NG;
+  static constexpr int TMA_WARP = EPI_WARPS, MMA_WARP = EPI_WARPS + 1;
+  static constexpr int THREADS = 32 * (EPI_WARPS + 2);
+  static constexpr int TMEM_COLS = NG * DH > 256 ? 512 : 256;      // a power of two
+};
 enum : unsigned { F_CONV1 = 1, F_CONV2 = 2, F_QK_MEAN = 4, F_QK_NORM = 16, F_ROPE = 32 };
 
 template <int DH, int NT>
@@ -43,9 +52,10 @@ struct T2Smem {
   static constexpr int W_BYTES = NT * WT;
   static constexpr int BUDGET = 232448 - 512;            // 227 KB minus barriers
   // per epilogue warp: slots for boxes of 32 rows x 128 bytes, as many as fit beside one operand tile (2..4)
-  static constexpr int NSLOT_FIT = (BUDGET - W_BYTES - A_BYTES) / (8 * 4096);
-  static constexpr int NSLOT = NSLOT_FIT > 4 ? 4 : NSLOT_FIT;
-  static constexpr int SLOT_BYTES = 8 * NSLOT * 4096;
+  static constexpr int EPI_WARPS = T2Groups<DH, NT>::EPI_WARPS;
+  static constexpr int NSLOT_FIT = (BUDGET - W_BYTES - A_BYTES) / (EPI_WARPS * 4096);
+  static constexpr int NSLOT = NSLOT_FIT > 3 ? 3 : NSLOT_FIT;
+  static constexpr int SLOT_BYTES = EPI_WARPS * NSLOT * 4096;
   static constexpr int STAGES_FIT = (BUDGET - W_BYTES - SLOT_BYTES) / A_BYTES;
   static constexpr int STAGES = STAGES_FIT > 2 ? 2 : STAGES_FIT;   // one is enough: the contraction of a unit is short
   static_assert(NSLOT >= 2, "box slots do not fit");
@@ -88,11 +98,12 @@ TC_DEVINL Unit unit_of(const T2Params& p, int u) {
 }
 
 template <int DH, int NT>
-__global__ void __launch_bounds__(T2_THREADS, 1)
+__global__ void __launch_bounds__(T2Groups<DH, NT>::THREADS, 1)
 tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                      const __grid_constant__ CUtensorMap tmF, const __grid_constant__ CUtensorMap tmR, const T2Params p) {
   using SM = T2Smem<DH, NT>;
-  constexpr int ST = SM::STAGES;
+  using GR = T2Groups<DH, NT>;
+  constexpr int ST = SM::STAGES, NG = GR::NG;
   extern __shared__ __align__(1024) unsigned char smem[];
   if (smem_u32(smem) & 1023u) {       // the swizzled tiles need it; nothing has been set up yet, so just report
     if (threadIdx.x == 0) atomicCAS(p.status, 0, ST_BAD_SMEM_ALIGNMENT);
@@ -103,10 +114,10 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   uint64_t* a_empty = bars + ST;           // [ST] MMA -> TMA (commit)
   uint64_t* w_full = bars + 2 * ST;        // TMA -> MMA: the head's weight tiles
   uint64_t* w_empty = w_full + 1;          // MMA -> TMA: every contraction with the previous head's weights is done
-  uint64_t* acc_full = w_empty + 1;        // [2] MMA -> epilogue group (commit)
-  uint64_t* acc_empty = acc_full + 2;      // [2] epilogue group -> MMA (128 arrivals)
-  uint64_t* slot_full = acc_empty + 2;     // [8 warps][NSLOT] TMA -> the warp's threads
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(slot_full + 8 * SM::NSLOT);
+  uint64_t* acc_full = w_empty + 1;        // [NG] MMA -> epilogue group (commit)
+  uint64_t* acc_empty = acc_full + NG;     // [NG] epilogue group -> MMA (128 arrivals)
+  uint64_t* slot_full = acc_empty + NG;    // [epilogue warps][NSLOT] TMA -> the warp's threads
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(slot_full + GR::EPI_WARPS * SM::NSLOT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const CcaDims& d = p.d;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -128,11 +139,11 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
     mbar_init(w_full, 1);
     mbar_init(w_empty, 1);
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < NG; ++s) {
       mbar_init(&acc_full[s], 1);
       mbar_init(&acc_empty[s], 128);
     }
-    for (int s = 0; s < 8 * SM::NSLOT; ++s) mbar_init(&slot_full[s], 1);
+    for (int s = 0; s < GR::EPI_WARPS * SM::NSLOT; ++s) mbar_init(&slot_full[s], 1);
     wait_ctl_init(abort_flag, p.status);
     fence_barrier_init();
     prefetch_tmap(&tmA);
@@ -140,8 +151,8 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     prefetch_tmap(&tmF);
     prefetch_tmap(&tmR);
   }
-  if (warp == T2_MMA_WARP) {
-    tmem_alloc(tmem_slot, 2 * DH);
+  if (warp == GR::MMA_WARP) {
+    tmem_alloc(tmem_slot, GR::TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -149,7 +160,7 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == T2_TMA_WARP) {
+  if (warp == GR::TMA_WARP) {
     // ------------------------------------------------------------------ TMA
     if (lane == 0) {
       int cur_head = -1, wk = 0, it = 0;
@@ -175,7 +186,7 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                       &a_full[stage]);
       }
     }
-  } else if (warp == T2_MMA_WARP) {
+  } else if (warp == GR::MMA_WARP) {
     // ------------------------------------------------------------------ MMA issue (whole warp walks, one lane issues)
     const bool leader = elect_one();
     const uint32_t idesc = idesc_bf16(DH, 0, 0);
@@ -192,8 +203,8 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         cur_head = un.h;
         ++wk;
       }
-      const int buf = it & 1, stage = it % ST;
-      if (!wait_all(&acc_empty[buf], ((it >> 1) & 1) ^ 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
+      const int buf = it % NG, stage = it % ST;
+      if (!wait_all(&acc_empty[buf], ((it / NG) & 1) ^ 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
       if (!wait_all(&a_full[stage], (it / ST) & 1)) { fail(abort_flag, p.status, ST_TIMEOUT_MMA); goto done; }
       tc_fence_after();
       if (leader) {
@@ -216,7 +227,7 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     // ------------------------------------------------------------------ epilogue, thread = token
     constexpr int HALF = DH / 2;
     constexpr int NS = SM::NSLOT;
-    const int grp = warp >> 2;                              // units with (it & 1) == grp, accumulator grp
+    const int grp = warp >> 2;                              // units with it % NG == grp, accumulator grp
     const int rho = (warp & 3) * 32 + lane;
     const uint32_t acc = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + grp * DH;
     const bool use_mean = (d.flags & F_QK_MEAN) != 0, use_rope = (d.flags & F_ROPE) != 0;
@@ -252,7 +263,7 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     Boxes pbx = pu < u_end ? boxes_of(pu) : Boxes{0, 0, 0, 0, 0, 0, 0};
     auto issue_next = [&]() {
       while (pu < u_end && pn >= pbx.n_box) {               // next unit of this group (units without boxes are skipped)
-        pu += 2;
+        pu += NG;
         pn = 0;
         if (pu < u_end) pbx = boxes_of(pu);
       }
@@ -273,7 +284,7 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     };
     for (int i = 0; i < NS; ++i) issue_next();
     int it = grp;
-    for (int u = u_begin + grp; u < u_end; u += 2, it += 2) {
+    for (int u = u_begin + grp; u < u_end; u += NG, it += NG) {
       const Unit un = unit_of(p, u);
       const bool is_q = un.h < d.hq;
       const int hj = is_q ? un.h / d.g : un.h - d.hq;
@@ -298,7 +309,7 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         if (lane == 0) fence_proxy_async();
         issue_next();
       };
-      if (!mbar_wait(&acc_full[grp], (it >> 1) & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
+      if (!mbar_wait(&acc_full[grp], (it / NG) & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
       tc_fence_after();
       // pass 1: pre-norm latent = conv output + mean term (Eq. 9), its squared norm; kept in the accumulator
       float ss = 0.f;
@@ -342,53 +353,54 @@ tc_transform2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       // pass 2: scale, rotate the pairs (c, c + d_h/2), store
       bf16* dst = is_q ? p.q + tok * d.Lq + un.h * DH : p.k + tok * d.Lk + hj * DH;
 #pragma unroll 1
-      for (int c = 0; c < HALF / 16; ++c) {
-        uint32_t ra[16], rb[16];
-        tmem_ld16(acc + c * 16, ra);
-        tmem_ld16(acc + HALF + c * 16, rb);
-        float4 cs[8];
-        if (use_rope) {
-          const int n = n_mean + c;
-          if (!wait_box(n)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
-          const unsigned char* src = my_slots + ((nb + n) % NS) * 4096;
+      for (int c = 0; c < HALF / 16; ++c) {              // one table box = 16 pairs; handled as two halves of 8 pairs
+        if (use_rope && !wait_box(n_mean + c)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
+        const unsigned char* src = my_slots + ((nb + n_mean + c) % NS) * 4096;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) cs[i] = *reinterpret_cast<const float4*>(src + ch_off[i]);   // (cos, sin) x 2
-        }
-        tmem_ld_wait();
-        float lo[16], hi[16];
-        if (use_rope) {
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t ra[8], rb[8];
+          tmem_ld8(acc + c * 16 + hf * 8, ra);
+          tmem_ld8(acc + HALF + c * 16 + hf * 8, rb);
+          float4 cs[4];
+          if (use_rope) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const float a0 = __uint_as_float(ra[2 * i]) * sc, b0 = __uint_as_float(rb[2 * i]) * sc;
-            const float a1 = __uint_as_float(ra[2 * i + 1]) * sc, b1 = __uint_as_float(rb[2 * i + 1]) * sc;
-            lo[2 * i] = a0 * cs[i].x - b0 * cs[i].y;
-            hi[2 * i] = b0 * cs[i].x + a0 * cs[i].y;
-            lo[2 * i + 1] = a1 * cs[i].z - b1 * cs[i].w;
-            hi[2 * i + 1] = b1 * cs[i].z + a1 * cs[i].w;
+            for (int i = 0; i < 4; ++i) cs[i] = *reinterpret_cast<const float4*>(src + ch_off[hf * 4 + i]);   // (cos, sin) x 2
           }
-          asm volatile("" ::"f"(lo[0]), "f"(hi[15]) : "memory");
-          release_box();
-        } else {
+          tmem_ld_wait();
+          float lo[8], hi[8];
+          if (use_rope) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            lo[i] = __uint_as_float(ra[i]) * sc;
-            hi[i] = __uint_as_float(rb[i]) * sc;
+            for (int i = 0; i < 4; ++i) {
+              const float a0 = __uint_as_float(ra[2 * i]) * sc, b0 = __uint_as_float(rb[2 * i]) * sc;
+              const float a1 = __uint_as_float(ra[2 * i + 1]) * sc, b1 = __uint_as_float(rb[2 * i + 1]) * sc;
+              lo[2 * i] = a0 * cs[i].x - b0 * cs[i].y;
+              hi[2 * i] = b0 * cs[i].x + a0 * cs[i].y;
+              lo[2 * i + 1] = a1 * cs[i].z - b1 * cs[i].w;
+              hi[2 * i + 1] = b1 * cs[i].z + a1 * cs[i].w;
+            }
+            if (hf == 1) {
+              asm volatile("" ::"f"(lo[0]), "f"(hi[7]) : "memory");
+              release_box();
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              lo[i] = __uint_as_float(ra[i]) * sc;
+              hi[i] = __uint_as_float(rb[i]) * sc;
+            }
           }
-        }
-        if (valid) {
-#pragma unroll
-          for (int v = 0; v < 2; ++v) {
+          if (valid) {
             uint4 w;
-            w.x = pack_bf16(lo[8 * v + 0], lo[8 * v + 1]);
-            w.y = pack_bf16(lo[8 * v + 2], lo[8 * v + 3]);
-            w.z = pack_bf16(lo[8 * v + 4], lo[8 * v + 5]);
-            w.w = pack_bf16(lo[8 * v + 6], lo[8 * v + 7]);
-            reinterpret_cast<uint4*>(dst + c * 16)[v] = w;
-            w.x = pack_bf16(hi[8 * v + 0], hi[8 * v + 1]);
-            w.y = pack_bf16(hi[8 * v + 2], hi[8 * v + 3]);
-            w.z = pack_bf16(hi[8 * v + 4], hi[8 * v + 5]);
-            w.w = pack_bf16(hi[8 * v + 6], hi[8 * v + 7]);
-            reinterpret_cast<uint4*>(dst + HALF + c * 16)[v] = w;
+            w.x = pack_bf16(lo[0], lo[1]);
+            w.y = pack_bf16(lo[2], lo[3]);
+            w.z = pack_bf16(lo[4], lo[5]);
+            w.w = pack_bf16(lo[6], lo[7]);
+            reinterpret_cast<uint4*>(dst + c * 16)[hf] = w;
+            w.x = pack_bf16(hi[0], hi[1]);
+            w.y = pack_bf16(hi[2], hi[3]);
+            w.z = pack_bf16(hi[4], hi[5]);
+            w.w = pack_bf16(hi[6], hi[7]);
+            reinterpret_cast<uint4*>(dst + HALF + c * 16)[hf] = w;
           }
         }
       }
@@ -407,9 +419,9 @@ done:
     while (clock64() - c0 < 2000000) {}
     __syncthreads();
   }
-  if (warp == T2_MMA_WARP) {
+  if (warp == GR::MMA_WARP) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 2 * DH);
+    tmem_dealloc(tmem_base, GR::TMEM_COLS);
   }
 }
 
@@ -469,7 +481,7 @@ int launch_t2(TcState* s, const CcaDims& d, const bf16* qk0b, const bf16* wc, co
       return 1;
   }
   const int grid = p0.total_units < s->sm_count ? p0.total_units : s->sm_count;
-  tc_transform2_kernel<DH, NT><<<grid, T2_THREADS, SM::TOTAL, st>>>(tmA, tmW, tmF, tmR, p0);
+  tc_transform2_kernel<DH, NT><<<grid, T2Groups<DH, NT>::THREADS, SM::TOTAL, st>>>(tmA, tmW, tmF, tmR, p0);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 0 : -(int)e;
 }
