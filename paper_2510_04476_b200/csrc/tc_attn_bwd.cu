@@ -15,6 +15,7 @@
 //
 // Both: warps 0-15 compute (four column groups x four TMEM lane quarters), warp 16 TMA loads, warp 17 issues
 // the MMAs (warp-uniform loop, one elected lane).  P and dS are bf16 MMA operands, everything else fp32.
+#include <type_traits>
 #include "tc_kernels.cuh"
 #include "tc_ptx.cuh"
 #include "tc_state.cuh"
@@ -118,7 +119,7 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   using SM = DqSmem<DH>;
   constexpr int KS = SM::K_STAGES;
   extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  unsigned char* smem = smem_align1024(smem_dyn);
   unsigned char* sQ = smem;
   unsigned char* sDO = sQ + SM::TILE;
   unsigned char* sK = sDO + SM::TILE;                 // [KS]: K_j lives from S(j) (issued a tile ahead) to dQ(j)
@@ -274,6 +275,10 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       tmem_ld_wait();
       tc_fence_before();
       mbar_arrive(dp_free);                            // the dP buffer may be overwritten
+      // masking is a compile-time variant of the whole tile's arithmetic: a branch per pair would end the instruction
+      // scheduler's window sixteen times per tile
+      auto tile_math = [&](auto mask_c) {
+      constexpr bool MASK = decltype(mask_c)::value;
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
         uint32_t pk[8];
@@ -282,7 +287,7 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           const int e = hf * 16 + 2 * c;
           const uint64_t x = fma2(pack2u(sv[e], sv[e + 1]), scale2, nl2);
           uint64_t ex = (c & 3) < POLY ? exp2_pair<true>(x) : exp2_pair<false>(x);
-          if (need_mask) {
+          if (MASK) {
             uint32_t a, bb;
             unpack2u(ex, a, bb);
             if (k0 + e > lim) a = 0u;
@@ -294,6 +299,8 @@ tc_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         // dS (bf16 pairs) over columns this thread has read: keys 32 part + [0,32) -> columns 32 part + [0,16)
         tmem_st8(s_t + hf * 8, pk);
       }
+      };
+      if (need_mask) tile_math(std::true_type{}); else tile_math(std::false_type{});
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(ds_full);
@@ -342,7 +349,7 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   using SM = BwdSmem<DH>;
   constexpr int NST = SM::STAGES;
   extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  unsigned char* smem = smem_align1024(smem_dyn);
   unsigned char* sK = smem + SM::FIX_OFF;
   unsigned char* sV = sK + SM::TILE;
   unsigned char* sRing = smem + SM::RING_OFF;         // [NST] stages of (Q half-tile, dO half-tile): 64 queries each
@@ -526,6 +533,8 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       tc_fence_after();
       const ulonglong2* nlv = reinterpret_cast<const ulonglong2*>(gstat + stb * 256 + qoff);        // pairs of -lse2
       const ulonglong2* ndv = reinterpret_cast<const ulonglong2*>(gstat + stb * 256 + 128 + qoff);  // pairs of -delta
+      auto tile_math = [&](auto diag_c) {
+      constexpr bool DIAG = decltype(diag_c)::value;
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
         uint32_t sv[16], dv[16], pk[8], dk_[8];
@@ -539,7 +548,7 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           uint64_t e1 = fma2(pack2u(sv[4 * c + 2], sv[4 * c + 3]), scale2, nl.y);
           e0 = (2 * c & 3) < POLY ? exp2_pair<true>(e0) : exp2_pair<false>(e0);
           e1 = ((2 * c + 1) & 3) < POLY ? exp2_pair<true>(e1) : exp2_pair<false>(e1);
-          if (diag) {
+          if (DIAG) {
             const int q0 = m0 + qoff + hf * 16 + 4 * c;      // query of the first of the four
             uint32_t a0, a1, a2, a3;
             unpack2u(e0, a0, a1);
@@ -559,6 +568,8 @@ tc_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tmem_st8(s_t + hf * 8, pk);                    // P^T over S^T columns this thread has read
         tmem_st8(dp_t + hf * 8, dk_);                  // dS^T over dP^T columns this thread has read
       }
+      };
+      if (diag) tile_math(std::true_type{}); else tile_math(std::false_type{});
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(&pds_full[gsel]);

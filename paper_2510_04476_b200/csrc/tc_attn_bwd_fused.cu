@@ -8,16 +8,22 @@
 // One CTA = 128 keys of one (sequence, kv head); it walks the g query heads of the group and, for each, the query
 // tiles that see these keys (thread = key, transposed tiles S^T = K Q^T, dP^T = V dO^T as in the dK/dV kernel), so
 // that dV += P^T dO and dK += dS^T Q accumulate in TMEM over the whole walk with P^T and dS^T as TMEM operands.
+// Two groups of four compute warps; a group owns the 64-query sub-tile of its TMEM buffer and a thread all 64 scores
+// of its key there (16 at a time, the next 16 and their column statistics in flight meanwhile).  A group's loop is a
+// chain  scores ready -> arithmetic -> P^T, dS^T written -> the tensor core's dV / dK and next S^T / dP^T -> ...;  the
+// two groups' chains interleave, and everything that is not on the chain (the dQ hand-over) runs while the tensor
+// core works.
 // The compute warps also leave dS^T as bf16 in shared memory ([key][query], 128-byte swizzle): read with the queries
 // as the M dimension it is the A operand of   dQ_tile = dS K   (M = 128 queries, N = d_h, K = 128 keys; the resident
 // K tile read along its rows is the B operand).  A query tile's dQ gets such a contribution from every key tile it
 // sees, i.e. from different CTAs: the compute warps copy the finished tile from TMEM to a shared-memory stage and a
-// reduce warp adds it into the zeroed fp32 dq with TMA reductions (cp.reduce.async.bulk.tensor, whole 128-byte lines;
-// rows past the end of the sequence are clipped by the tensor map).  The sum order of dq therefore varies from run to
-// run (fp32 rounding only).
+// lane of the TMA warp adds it into the zeroed fp32 dq with TMA reductions (cp.reduce.async.bulk.tensor, whole 128-byte
+// lines; rows past the end of the sequence are clipped by the tensor map).  The sum order of dq therefore varies from
+// run to run (fp32 rounding only).
 //
 // TMEM columns: S^T two 64-query buffers [0,128), dP^T likewise [128,256), dV [256,320), dK [320,384),
 // dQ two buffers [384,448) [448,512).
+#include <type_traits>
 #include "tc_kernels.cuh"
 #include "tc_ptx.cuh"
 #include "tc_state.cuh"
@@ -26,7 +32,7 @@ using namespace tc;
 
 namespace {
 
-constexpr int FB_COMPUTE_WARPS = 16;
+constexpr int FB_COMPUTE_WARPS = 8;
 // warp 16: lane 0 issues the TMA loads, lane 1 the dQ reductions (two independent loops of one warp: a third service
 // warp would cost every thread 16 registers); warp 17 issues the MMAs
 constexpr int FB_TMA_WARP = FB_COMPUTE_WARPS, FB_MMA_WARP = FB_COMPUTE_WARPS + 1;
@@ -87,7 +93,7 @@ tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   using SM = FbSmem;
   constexpr int NST = SM::STAGES;
   extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  unsigned char* smem = smem_align1024(smem_dyn);
   unsigned char* sK = smem + SM::FIX_OFF;
   unsigned char* sV = sK + SM::TILE;
   unsigned char* sRing = smem + SM::RING_OFF;         // [NST] stages of (Q half-tile, dO half-tile): 64 queries each
@@ -128,8 +134,8 @@ tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sdp_full[i], 1);
-      mbar_init(&pds_full[i], 256);
-      mbar_init(&stat_ready[i], 256);
+      mbar_init(&pds_full[i], 128);
+      mbar_init(&stat_ready[i], 128);
       mbar_init(&dq_full[i], 1);
       mbar_init(&dq_empty[i], 32 * FB_COMPUTE_WARPS);
       mbar_init(&ds_free[i], 1);
@@ -265,56 +271,62 @@ tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     if (leader) mma_commit(acc_done);
   } else {
     // ------------------------------------------------------------------ compute, thread = key
-    const int gsel = warp >> 3;                        // sub-tile (queries [64 gsel, 64 gsel + 64) of every query tile)
-    const int part = (warp >> 2) & 1;                  // which 32 of the sub-tile's 64 queries
+    // Two groups of four warps; group gsel owns the sub-tile of queries [64 gsel, 64 gsel + 64) of every query tile (TMEM
+    // buffer gsel) and a thread all 64 of its key's scores there, in quarters of 16 with the next quarter's TMEM loads
+    // in flight during the arithmetic (few warps with many independent chains each, instead of many short ones).
+    const int gsel = warp >> 2;
     const int row = (warp & 3) * 32 + lane;
-    const int ct = threadIdx.x & 255;
+    const int ct = threadIdx.x & 127;
     const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
     const int tk = n0 + row;
     const float c_scale = rsqrtf((float)DH) * FB_LOG2E;
     const float q_scale = rsqrtf((float)DH);
-    float* gstat = stat + gsel * 512;
-    auto fetch_stat = [&](int it) -> float {
+    float* gstat = stat + gsel * 512;                  // [2 buffers][-lse2 | -delta][128 queries]
+    auto fetch_stat = [&](int it, float& nl, float& nd) {
       const int hi = hj * p.g + it / n_q, m0 = (i0 + it % n_q) * 128;
-      const int tq = m0 + (ct & 127);
+      const int tq = m0 + ct;
       const long long idx = ((long long)b * p.hq + hi) * p.S + tq;
-      if (ct < 128) return tq < p.S ? -p.lse[idx] * FB_LOG2E : -INFINITY;
-      return tq < p.S ? -p.delta[idx] : 0.f;
+      nl = tq < p.S ? -p.lse[idx] * FB_LOG2E : -INFINITY;
+      nd = tq < p.S ? -p.delta[idx] : 0.f;
     };
-    // hands the finished dQ of iteration `it` (its TMEM buffer) to the reduce warp: thread = query row, 16 channels,
-    // written into the fp32 stage (rows of 128 bytes, 128-byte swizzle, two 32-channel boxes)
-    unsigned char* stg_row = smem + SM::DQ_OFF + ((warp >> 2) >> 1) * 16384 + row * 128;
-    const int stg_ch = ((warp >> 2) & 1) * 4;
-    auto flush_dq = [&](int it) -> bool {
+    // hands the finished dQ of iteration `it` (its TMEM buffer) to the reduction lane: thread = query row, 32 channels,
+    // written into the fp32 stage (rows of 128 bytes, 128-byte swizzle; box gsel = channels [32 gsel, 32 gsel + 32))
+    unsigned char* stg_row = smem + SM::DQ_OFF + gsel * 16384 + row * 128;
+    // The finished dQ of iteration `it` goes from its TMEM buffer to the fp32 stage: flush_load (wait for the contraction,
+    // issue the load) and, after a tcgen05.wait::ld, flush_store (release the buffer, wait for the stage, write it, hand it
+    // to the reduction lane).
+    auto flush_load = [&](int it, uint32_t (&t)[32]) -> bool {
       const int buf = it & 1;
       if (!mbar_wait(&dq_full[buf], (it >> 1) & 1, abort_flag)) return false;
       tc_fence_after();
-      uint32_t t[16];
-      tmem_ld16(tmem_base + lane_sel + 384 + buf * 64 + (warp >> 2) * 16, t);
-      tmem_ld_wait();
+      tmem_ld32(tmem_base + lane_sel + 384 + buf * 64 + gsel * 32, t);
+      return true;
+    };
+    auto flush_store = [&](int it, const uint32_t (&t)[32]) -> bool {
       tc_fence_before();
-      mbar_arrive(&dq_empty[buf]);
+      mbar_arrive(&dq_empty[it & 1]);
       if (!mbar_wait(stg_free, (it & 1) ^ 1, abort_flag)) return false;     // the previous tile has left the stage
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
-        *reinterpret_cast<float4*>(stg_row + (((stg_ch + i) ^ (row & 7)) << 4)) =
+      for (int i = 0; i < 8; ++i)
+        *reinterpret_cast<float4*>(stg_row + ((i ^ (row & 7)) << 4)) =
             make_float4(__uint_as_float(t[4 * i]) * q_scale, __uint_as_float(t[4 * i + 1]) * q_scale,
                         __uint_as_float(t[4 * i + 2]) * q_scale, __uint_as_float(t[4 * i + 3]) * q_scale);
       fence_proxy_async();
       mbar_arrive(stg_full);
       return true;
     };
-    float next_stat = n_it > 0 ? fetch_stat(0) : 0.f;
+    float next_nl = 0.f, next_nd = 0.f;
+    if (n_it > 0) fetch_stat(0, next_nl, next_nd);
     const uint64_t scale2 = pack2f(c_scale, c_scale);
-    const uint32_t s_t = tmem_base + lane_sel + gsel * 64 + part * 32;
-    const uint32_t dp_t = tmem_base + lane_sel + 128 + gsel * 64 + part * 32;
-    const int qoff = gsel * 64 + part * 32;            // first query (within the tile) of this thread's columns
-    // this thread's 64 bytes of a dS^T row: box gsel, row `row`, 16-byte chunks 4 part + [0,4) (swizzled)
-    unsigned char* ds_row = sDS + gsel * 16384 + row * 128;
+    const uint32_t s_t = tmem_base + lane_sel + gsel * 64;
+    const uint32_t dp_t = tmem_base + lane_sel + 128 + gsel * 64;
+    const int qoff = gsel * 64;                        // first query (within the tile) of this thread's columns
+    unsigned char* ds_row = sDS + gsel * 16384 + row * 128;      // this thread's 128-byte row of dS^T, box gsel
     for (int it = 0; it < n_it; ++it) {
       const int stb = it & 1;
-      gstat[stb * 256 + ct] = next_stat;
-      if (it + 1 < n_it) next_stat = fetch_stat(it + 1);
+      gstat[stb * 256 + ct] = next_nl;
+      gstat[stb * 256 + 128 + ct] = next_nd;
+      if (it + 1 < n_it) fetch_stat(it + 1, next_nl, next_nd);
       mbar_arrive(&stat_ready[gsel]);
       if (!mbar_wait(&stat_ready[gsel], it & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
       const int m0 = (i0 + it % n_q) * 128;
@@ -325,20 +337,43 @@ tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       tc_fence_after();
       const ulonglong2* nlv = reinterpret_cast<const ulonglong2*>(gstat + stb * 256 + qoff);
       const ulonglong2* ndv = reinterpret_cast<const ulonglong2*>(gstat + stb * 256 + 128 + qoff);
+      unsigned char* dsb = ds_row + stb * SM::DS_TILE;
+      // the whole tile's arithmetic in one basic block: the diagonal tile's masking is a compile-time variant, not a branch
+      // per group of four scores (a branch there ends the scheduler's window)
+      auto tile_math = [&](auto diag_c) {
+      constexpr bool DIAG = decltype(diag_c)::value;
+      uint32_t sv[2][16], dv[2][16];
+      ulonglong2 nlq[2][4], ndq[2][4];                 // this quarter's and the next one's column statistics
+      tmem_ld16(s_t, sv[0]);
+      tmem_ld16(dp_t, dv[0]);
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        uint32_t sv[16], dv[16], pk[8], dk_[8];
-        tmem_ld16(s_t + hf * 16, sv);
-        tmem_ld16(dp_t + hf * 16, dv);
+      for (int c = 0; c < 4; ++c) {
+        nlq[0][c] = nlv[c];
+        ndq[0][c] = ndv[c];
+      }
+#pragma unroll
+      for (int hf = 0; hf < 4; ++hf) {
+        uint32_t pk[8], dk_[8];
         tmem_ld_wait();
+        if (hf < 3) {
+          tmem_ld16(s_t + (hf + 1) * 16, sv[(hf + 1) & 1]);
+          tmem_ld16(dp_t + (hf + 1) * 16, dv[(hf + 1) & 1]);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            nlq[(hf + 1) & 1][c] = nlv[(hf + 1) * 4 + c];
+            ndq[(hf + 1) & 1][c] = ndv[(hf + 1) * 4 + c];
+          }
+        }
+        const uint32_t(&sq)[16] = sv[hf & 1];
+        const uint32_t(&dq_)[16] = dv[hf & 1];
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          const ulonglong2 nl = nlv[hf * 4 + c], nd = ndv[hf * 4 + c];
-          uint64_t e0 = fma2(pack2u(sv[4 * c + 0], sv[4 * c + 1]), scale2, nl.x);
-          uint64_t e1 = fma2(pack2u(sv[4 * c + 2], sv[4 * c + 3]), scale2, nl.y);
+          const ulonglong2 nl = nlq[hf & 1][c], nd = ndq[hf & 1][c];
+          uint64_t e0 = fma2(pack2u(sq[4 * c + 0], sq[4 * c + 1]), scale2, nl.x);
+          uint64_t e1 = fma2(pack2u(sq[4 * c + 2], sq[4 * c + 3]), scale2, nl.y);
           e0 = (2 * c & 3) < POLY ? exp2_pair<true>(e0) : exp2_pair<false>(e0);
           e1 = ((2 * c + 1) & 3) < POLY ? exp2_pair<true>(e1) : exp2_pair<false>(e1);
-          if (diag) {
+          if (DIAG) {
             const int q0 = m0 + qoff + hf * 16 + 4 * c;
             uint32_t a0, a1, a2, a3;
             unpack2u(e0, a0, a1);
@@ -352,44 +387,56 @@ tc_attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           }
           pk[2 * c] = cvt_bf16x2(e0);
           pk[2 * c + 1] = cvt_bf16x2(e1);
-          dk_[2 * c] = cvt_bf16x2(mul2(e0, add2(pack2u(dv[4 * c + 0], dv[4 * c + 1]), nd.x)));
-          dk_[2 * c + 1] = cvt_bf16x2(mul2(e1, add2(pack2u(dv[4 * c + 2], dv[4 * c + 3]), nd.y)));
+          dk_[2 * c] = cvt_bf16x2(mul2(e0, add2(pack2u(dq_[4 * c + 0], dq_[4 * c + 1]), nd.x)));
+          dk_[2 * c + 1] = cvt_bf16x2(mul2(e1, add2(pack2u(dq_[4 * c + 2], dq_[4 * c + 3]), nd.y)));
         }
-        tmem_st8(s_t + hf * 8, pk);                    // P^T over S^T columns this thread has read
-        tmem_st8(dp_t + hf * 8, dk_);                  // dS^T over dP^T columns this thread has read
-        // the same dS^T values for the dQ contraction: queries qoff + 16 hf + [0,16) of row `row`
-        unsigned char* dsb = ds_row + stb * SM::DS_TILE;
-        const int ch = part * 4 + hf * 2;
-        *reinterpret_cast<uint4*>(dsb + (((ch) ^ (row & 7)) << 4)) = make_uint4(dk_[0], dk_[1], dk_[2], dk_[3]);
-        *reinterpret_cast<uint4*>(dsb + (((ch + 1) ^ (row & 7)) << 4)) = make_uint4(dk_[4], dk_[5], dk_[6], dk_[7]);
+        // 16 queries = k-step hf of the dV / dK contractions: 8 columns at (hf >> 1) * 32 + (hf & 1) * 8, all of them
+        // columns this thread has already read
+        tmem_st8(s_t + (hf >> 1) * 32 + (hf & 1) * 8, pk);
+        tmem_st8(dp_t + (hf >> 1) * 32 + (hf & 1) * 8, dk_);
+        // the same dS^T values for the dQ contraction: 16-byte chunks 2 hf, 2 hf + 1 of the row (swizzled)
+        *reinterpret_cast<uint4*>(dsb + (((2 * hf) ^ (row & 7)) << 4)) = make_uint4(dk_[0], dk_[1], dk_[2], dk_[3]);
+        *reinterpret_cast<uint4*>(dsb + (((2 * hf + 1) ^ (row & 7)) << 4)) = make_uint4(dk_[4], dk_[5], dk_[6], dk_[7]);
       }
+      };
+      if (diag) tile_math(std::true_type{}); else tile_math(std::false_type{});
       tmem_st_wait();
       tc_fence_before();
       fence_proxy_async();                             // shared-memory writes -> visible to the tensor core
       mbar_arrive(&pds_full[gsel]);
-      if (it >= 1 && !flush_dq(it - 1)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+      // the previous tile's dQ leaves while the tensor core works on this sub-tile's contractions
+      if (it >= 1) {
+        uint32_t t[32];
+        bool ok = flush_load(it - 1, t);
+        tmem_ld_wait();
+        if (ok) ok = flush_store(it - 1, t);
+        if (!ok) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
+      }
     }
-    if (n_it > 0 && !flush_dq(n_it - 1)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
+    if (n_it > 0) {
+      uint32_t t[32];
+      bool ok = flush_load(n_it - 1, t);
+      tmem_ld_wait();
+      if (ok) ok = flush_store(n_it - 1, t);
+      if (!ok) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
+    }
     if (!mbar_wait(acc_done, 0, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
     tc_fence_after();
     {
-#pragma unroll 1
-      for (int c = 0; c < 1; ++c) {
-        uint32_t t[16], u[16];
-        const int col = (gsel * 2 + part) * (DH / 4);
-        tmem_ld16(tmem_base + lane_sel + 256 + col, t);
-        tmem_ld16(tmem_base + lane_sel + 320 + col, u);
-        tmem_ld_wait();
-        if (tk < p.S) {
-          const long long off = ((long long)b * p.S + tk) * p.Lk + hj * DH + col;
+      uint32_t t[32], u[32];
+      const int col = gsel * 32;
+      tmem_ld32(tmem_base + lane_sel + 256 + col, t);
+      tmem_ld32(tmem_base + lane_sel + 320 + col, u);
+      tmem_ld_wait();
+      if (tk < p.S) {
+        const long long off = ((long long)b * p.S + tk) * p.Lk + hj * DH + col;
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            reinterpret_cast<float4*>(p.dv + off)[i] = make_float4(__uint_as_float(t[4 * i]), __uint_as_float(t[4 * i + 1]),
-                                                                    __uint_as_float(t[4 * i + 2]), __uint_as_float(t[4 * i + 3]));
-            reinterpret_cast<float4*>(p.dk + off)[i] =
-                make_float4(__uint_as_float(u[4 * i]) * q_scale, __uint_as_float(u[4 * i + 1]) * q_scale,
-                            __uint_as_float(u[4 * i + 2]) * q_scale, __uint_as_float(u[4 * i + 3]) * q_scale);
-          }
+        for (int i = 0; i < 8; ++i) {
+          reinterpret_cast<float4*>(p.dv + off)[i] = make_float4(__uint_as_float(t[4 * i]), __uint_as_float(t[4 * i + 1]),
+                                                                  __uint_as_float(t[4 * i + 2]), __uint_as_float(t[4 * i + 3]));
+          reinterpret_cast<float4*>(p.dk + off)[i] =
+              make_float4(__uint_as_float(u[4 * i]) * q_scale, __uint_as_float(u[4 * i + 1]) * q_scale,
+                          __uint_as_float(u[4 * i + 2]) * q_scale, __uint_as_float(u[4 * i + 3]) * q_scale);
         }
       }
     }
@@ -457,8 +504,9 @@ int tc_attn_bwd_fused(TcState* s, const CcaDims& d, const bf16* q, const bf16* k
   p.lse = lse; p.delta = delta; p.dq = dq; p.dk = dk; p.dv = dv;
   p.n_tiles = (d.S + 127) / 128;
   p.status = d_status;
-  // two of every four exponential pairs on the FMA pipe measured best here (0.599 ms against 0.615 with one or none)
-  const int poly = s->attn_poly_bwd < 0 ? 2 : s->attn_poly_bwd;
+  // all exponentials on the transcendental unit measured best here (0.482 ms; 0.488 / 0.500 with one / two of every four
+  // pairs on the FMA pipe)
+  const int poly = s->attn_poly_bwd < 0 ? 0 : s->attn_poly_bwd;
   if (poly == 0) return launch_fused<0>(s, d, tmQh, tmK, tmV, tmDOh, tmDQ, p, st);
   if (poly == 1) return launch_fused<1>(s, d, tmQh, tmK, tmV, tmDOh, tmDQ, p, st);
   return launch_fused<2>(s, d, tmQh, tmK, tmV, tmDOh, tmDQ, p, st);

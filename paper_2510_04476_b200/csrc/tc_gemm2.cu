@@ -99,7 +99,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   using SM = G2Smem<BN>;
   constexpr int G2_BN = BN, G2_STAGES = SM::STAGES;
   extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  unsigned char* smem = smem_align1024(smem_dyn);
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFFSET);   // used in the leader CTA
   uint64_t* empty_bar = full_bar + G2_STAGES;                                 // one set per CTA
   uint64_t* acc_full = empty_bar + G2_STAGES;                                 // [2], one set per CTA

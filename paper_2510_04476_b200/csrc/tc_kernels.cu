@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, TcGemmParams p) {
   using SM = GemmSmem<BN>;
   extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  unsigned char* smem = smem_align1024(smem_dyn);
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFFSET);
   uint64_t* empty_bar = full_bar + GEMM_STAGES;
   uint64_t* acc_full = empty_bar + GEMM_STAGES;     // [2]

@@ -29,6 +29,10 @@ TC_DEVINL void wait_ctl_init(volatile int* abort_flag, const int* status) {
 }
 
 TC_DEVINL uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// First 1024-byte boundary at or after `base` (128-byte-swizzled tiles need it), by pointer arithmetic on the shared array
+// itself: a round trip through an integer would hide the address space from the compiler, which then emits generic
+// loads and stores for every access below it.
+TC_DEVINL unsigned char* smem_align1024(unsigned char* base) { return base + ((1024u - (smem_u32(base) & 1023u)) & 1023u); }
 
 TC_DEVINL void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));

@@ -80,7 +80,7 @@ template <int DH, int KC>
 __global__ void __launch_bounds__(TR_THREADS, 1) tc_transform_fwd_kernel(const TrParams p) {
   using SM = TrSmem<DH, KC>;
   extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  unsigned char* smem = smem_align1024(smem_dyn);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFF);
   uint64_t* a_full = bars;           // producers -> MMA   (128 arrivals)
   uint64_t* a_empty = bars + 1;      // MMA -> producers   (commit)
