@@ -266,21 +266,20 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const int tq = m0 + row;
         if (!mbar_wait(&s_full[s], j & 1, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_SOFTMAX); goto done; }
         tc_fence_after();
+        // this thread's 32 scores, loaded once: one trip to tensor memory per tile
+        uint32_t v[32];
+        tmem_ld32(s_tmem, v);
+        tmem_ld_wait();
         const int k0 = j * BKV + part * 32;            // first key of this thread's columns
         const bool need_mask = (p.causal && j * BKV + BKV - 1 > m0) || (j * BKV + BKV > p.S);
         const int lim = p.causal ? min(tq, p.S - 1) : p.S - 1;       // last visible key
         float m_use = m_run[s];
         if (!fixed) {
-          // first pass over this thread's 32 scores for the row maximum (they are read again below)
+          // first pass for the row maximum
           float mx = -INFINITY;
-          {
-            uint32_t v[32];
-            tmem_ld32(s_tmem, v);
-            tmem_ld_wait();
 #pragma unroll
-            for (int c = 0; c < 32; ++c)
-              if (!need_mask || k0 + c <= lim) mx = fmaxf(mx, __uint_as_float(v[c]));
-          }
+          for (int c = 0; c < 32; ++c)
+            if (!need_mask || k0 + c <= lim) mx = fmaxf(mx, __uint_as_float(v[c]));
           // the rest of the row belongs to three other threads: exchange through shared memory
           xch[part * 128 + row] = mx;
           sync_softmax();
@@ -313,21 +312,19 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         // chunk the MMA warp may start on those keys.
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
-          uint32_t v[16], pk[8];
-          tmem_ld16(s_tmem + hf * 16, v);
-          tmem_ld_wait();
+          uint32_t pk[8];
           if (need_mask) {
 #pragma unroll
             for (int c = 0; c < 16; ++c)
-              if (k0 + hf * 16 + c > lim) v[c] = 0xff800000u;        // -inf
+              if (k0 + hf * 16 + c > lim) v[hf * 16 + c] = 0xff800000u;        // -inf
 #pragma unroll
-            for (int c = 0; c < 2; ++c) exp8<0, false>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
+            for (int c = 0; c < 2; ++c) exp8<0, false>(&v[hf * 16 + 8 * c], scale2, negm2, sum2, &pk[4 * c]);
           } else if (fixed) {
 #pragma unroll
-            for (int c = 0; c < 2; ++c) exp8<POLY, false>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
+            for (int c = 0; c < 2; ++c) exp8<POLY, false>(&v[hf * 16 + 8 * c], scale2, negm2, sum2, &pk[4 * c]);
           } else {
 #pragma unroll
-            for (int c = 0; c < 2; ++c) exp8<POLY, true>(&v[8 * c], scale2, negm2, sum2, &pk[4 * c]);
+            for (int c = 0; c < 2; ++c) exp8<POLY, true>(&v[hf * 16 + 8 * c], scale2, negm2, sum2, &pk[4 * c]);
           }
           tmem_st8(s_tmem + hf * 8, pk);
           tmem_st_wait();
