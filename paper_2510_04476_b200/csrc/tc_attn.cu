@@ -10,6 +10,9 @@
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+DH) O1 [384,384+DH).  The bf16 probabilities P
 // overwrite the first 16 of every 32 columns of their S tile and feed the P V MMA directly from TMEM.
+// At d_h = 64 the columns behind each O tile are free, and the row sums of P are taken there by the tensor
+// core as well (L0 [320,336) L1 [448,464): P times a block of ones, beside every P V step), which takes three
+// of the seven instructions per score pair off the softmax threads.
 // Softmax: with L2-normalised q and k (Eq. 11) every logit is bounded by sqrt(d_h) * beta, so that bound
 // serves as a fixed row maximum: no max pass, no rescale of O (the kernel falls back to the online form,
 // with a lazy rescale when the running maximum grows by more than 2^8, if the latents are not normalised
@@ -41,9 +44,11 @@ struct AttnSmem {
   static constexpr int KV_OFF = 2 * TILE_BYTES;
   static constexpr int BAR_OFF = KV_OFF + NSLOT * TILE_BYTES;
   static constexpr int XCH_OFF = BAR_OFF + 256;              // float [2 tiles][2 halves][128 rows]: max / sum exchange
+  static constexpr int ONES_OFF = (XCH_OFF + 2048 + 1023) / 1024 * 1024;    // 2 KB of bf16 ones (row sums by MMA)
+  static constexpr int USED = DH == 64 ? ONES_OFF + 2048 : XCH_OFF + 2048;
   // no slack for alignment: the kernel checks that its dynamic shared memory starts on a 1024-byte boundary.
   // At least 120 KB so that two CTAs (each wanting all 512 TMEM columns) never share an SM.
-  static constexpr int TOTAL = (XCH_OFF + 2048) > 122880 ? (XCH_OFF + 2048) : 122880;
+  static constexpr int TOTAL = USED > 122880 ? USED : 122880;
 };
 
 // K-major operand tile [128 rows][DH] stored as DH/64 swizzled boxes of [128][64]: descriptor of the
@@ -57,13 +62,15 @@ TC_DEVINL uint64_t kmajor_desc(uint32_t tile_addr, int kk) {
 TC_DEVINL uint64_t v_desc(uint32_t tile_addr, int kk) { return smem_desc_sw128(tile_addr + kk * 2048, 16384, 1024); }
 
 
-template <int DH, int POLY>
+// POLY8: of every 8 score pairs, how many take the polynomial exponential.
+template <int DH, int POLY8>
 __global__ void __launch_bounds__(AT_THREADS, 1)
 tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, AttnParams p) {
   using SM = AttnSmem<DH>;
   constexpr int NBOX = DH / 64;
   constexpr int NS = SM::NSLOT;
+  constexpr bool MSUM = DH == 64;       // row sums of P by the tensor core
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
   unsigned char* smem = smem_dyn;
   if (smem_u32(smem) & 1023u) {       // the swizzled tiles need it; nothing has been set up yet, so just report
@@ -101,8 +108,8 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     for (int i = 0; i < 2; ++i) {
       mbar_init(&q_full[i], 1);
       mbar_init(&s_full[i], 1);
-      mbar_init(&p_full[2 * i], 512);
-      mbar_init(&p_full[2 * i + 1], 512);
+      mbar_init(&p_full[2 * i], AT_SOFTMAX_WARPS);         // one arrival per softmax warp
+      mbar_init(&p_full[2 * i + 1], AT_SOFTMAX_WARPS);
       mbar_init(&o_done[i], 1);
     }
     for (int i = 0; i < NS; ++i) {
@@ -118,6 +125,11 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   if (warp == AT_MMA_WARP) {
     tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
+  }
+  if (MSUM && warp < AT_SOFTMAX_WARPS) {
+    // 16 "channels" of ones for the row-sum MMA: any operand layout reads ones from this block
+    reinterpret_cast<uint32_t*>(smem + SM::ONES_OFF)[threadIdx.x] = 0x3F803F80u;
+    fence_proxy_async();
   }
   tc_fence_before();
   __syncthreads();
@@ -155,6 +167,8 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const bool leader = elect_one();
       const uint32_t idesc_s = idesc_bf16(BKV, 0, 0);
       const uint32_t idesc_o = idesc_bf16(DH, 0, 1);
+      const uint32_t idesc_l = idesc_bf16(16, 0, 0);
+      const uint32_t ones_lo = (smem_u32(smem + SM::ONES_OFF) >> 4) | (1u << 16);
       // descriptor words: low = address >> 4 | leading offset << 16, high = stride offset, version, swizzle
       const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
       const uint32_t q_lo = (smem_u32(smem + SM::Q_OFF) >> 4) | (1u << 16);
@@ -184,6 +198,9 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             const int kk = 2 * i + hf;
             mma_ts_w(tmem_base + 256 + s * 128, tmem_base + s * 128 + (kk >> 1) * 32 + (kk & 1) * 8, va + kk * (2048 >> 4),
                      desc_hi, idesc_o, (j | hf | i) != 0);
+            if (MSUM)
+              mma_ts_w(tmem_base + 256 + s * 128 + DH, tmem_base + s * 128 + (kk >> 1) * 32 + (kk & 1) * 8, ones_lo, desc_hi,
+                       idesc_l, (j | hf | i) != 0);
           }
         }
       };
@@ -292,6 +309,14 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             // rescale this thread's quarter of the running output (rare)
             const float alpha = grow ? exp2f(m_run[s] - m_use) : 1.f;
             l_run[s] *= alpha;
+            if (MSUM && part == 0) {          // the row sum lives beside O: only its first column is read at the end
+              uint32_t t[8];
+              tmem_ld8(o_tmem + DH, t);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 8; ++i) t[i] = __float_as_uint(__uint_as_float(t[i]) * alpha);
+              tmem_st8(o_tmem + DH, t);
+            }
 #pragma unroll 1
             for (int c = 0; c < DH / 64; ++c) {
               uint32_t t[16];
@@ -318,20 +343,19 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             for (int c = 0; c < 16; ++c)
               if (k0 + hf * 16 + c > lim) v[hf * 16 + c] = 0xff800000u;        // -inf
 #pragma unroll
-            for (int c = 0; c < 2; ++c) exp8<0, false>(&v[hf * 16 + 8 * c], scale2, negm2, sum2, &pk[4 * c]);
+            exp16<0, false, !MSUM>(&v[hf * 16], scale2, negm2, sum2, pk);
           } else if (fixed) {
-#pragma unroll
-            for (int c = 0; c < 2; ++c) exp8<POLY, false>(&v[hf * 16 + 8 * c], scale2, negm2, sum2, &pk[4 * c]);
+            exp16<POLY8, false, !MSUM>(&v[hf * 16], scale2, negm2, sum2, pk);
           } else {
-#pragma unroll
-            for (int c = 0; c < 2; ++c) exp8<POLY, true>(&v[hf * 16 + 8 * c], scale2, negm2, sum2, &pk[4 * c]);
+            exp16<POLY8, true, !MSUM>(&v[hf * 16], scale2, negm2, sum2, pk);
           }
           tmem_st8(s_tmem + hf * 8, pk);
           tmem_st_wait();
           tc_fence_before();
-          mbar_arrive(&p_full[2 * s + hf]);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&p_full[2 * s + hf]);
         }
-        {
+        if (!MSUM) {
           uint32_t a, b2;
           unpack2u(sum2, a, b2);
           l_run[s] += __uint_as_float(a) + __uint_as_float(b2);
@@ -343,13 +367,22 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       if (n_s[s] == 0) continue;
       const uint32_t o_tmem = tmem_base + lane_sel + 256 + s * 128;
       const int tq = blk * 256 + s * BQ + row;
-      // total of the four parts of the row
-      sync_softmax();
-      xch[part * 128 + row] = l_run[s];
-      sync_softmax();
-      const float l_tot = (xch[row] + xch[128 + row]) + (xch[256 + row] + xch[384 + row]);
+      float l_tot;
+      if (!MSUM) {
+        // total of the four parts of the row
+        sync_softmax();
+        xch[part * 128 + row] = l_run[s];
+        sync_softmax();
+        l_tot = (xch[row] + xch[128 + row]) + (xch[256 + row] + xch[384 + row]);
+      }
       if (!mbar_wait(&o_done[s], 0, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
       tc_fence_after();
+      if (MSUM) {
+        uint32_t t;
+        tmem_ld1(o_tmem + DH, t);
+        tmem_ld_wait();
+        l_tot = __uint_as_float(t);
+      }
       const float inv_l = 1.f / l_tot;
       const long long row_g = (long long)b * p.S + tq;
 #pragma unroll 1
@@ -400,17 +433,17 @@ done:
 }  // namespace
 
 namespace {
-template <int DH, int POLY>
+template <int DH, int POLY8>
 int launch_attn(TcState* s, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnParams& p,
                 unsigned grid, cudaStream_t st) {
   static bool attr_set[TC_MAX_DEVICES] = {};
   if (!attr_set[s->device]) {
-    cudaError_t e = cudaFuncSetAttribute(tc_attn_fwd_kernel<DH, POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(tc_attn_fwd_kernel<DH, POLY8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          AttnSmem<DH>::TOTAL);
     if (e != cudaSuccess) return -(int)e;
     attr_set[s->device] = true;
   }
-  tc_attn_fwd_kernel<DH, POLY><<<grid, AT_THREADS, AttnSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, p);
+  tc_attn_fwd_kernel<DH, POLY8><<<grid, AT_THREADS, AttnSmem<DH>::TOTAL, st>>>(tmQ, tmK, tmV, p);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 0 : -(int)e;
 }
@@ -437,18 +470,20 @@ int tc_attn_fwd(TcState* s, const CcaDims& d, const bf16* q, const bf16* k, cons
   p.status = d_status;
   const long long grid = (long long)p.n_blocks * d.B * d.hq;
   if (grid > 0x7fffffffLL) return 1;
-  // at d_h = 128 the packed polynomial only moves the bottleneck to the half-rate heavy FMA pipe
-  const int knob = s->attn_poly < 0 ? (d.dh == 128 ? 0 : 1) : s->attn_poly;
+  // The knob counts eighths of the score pairs that take the polynomial (bit 3: ignore the norm bound).  At d_h = 128
+  // the exponential unit and the tensor pipe need the same time and the packed FMA pipe is no faster; at d_h = 64,
+  // with the row sums on the tensor core, two of eight measured best (1.256 ms against 1.308 with none and 1.280
+  // with three at 4 x 16384 tokens, 8 / 2 heads).
+  const int knob = s->attn_poly < 0 ? (d.dh == 128 ? 0 : 2) : s->attn_poly;
   p.temp = (knob & 8) ? nullptr : temp;
   const int poly = knob & 7;
   if (d.dh == 128) {
     if (poly == 0) return launch_attn<128, 0>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
-    if (poly == 1) return launch_attn<128, 1>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
-    if (poly == 3) return launch_attn<128, 3>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
-    return launch_attn<128, 2>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
+    if (poly <= 2) return launch_attn<128, 2>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
+    return launch_attn<128, 4>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
   }
   if (poly == 0) return launch_attn<64, 0>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
-  if (poly == 1) return launch_attn<64, 1>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
+  if (poly <= 2) return launch_attn<64, 2>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
   if (poly == 3) return launch_attn<64, 3>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
-  return launch_attn<64, 2>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
+  return launch_attn<64, 4>(s, tmQ, tmK, tmV, p, (unsigned)grid, st);
 }

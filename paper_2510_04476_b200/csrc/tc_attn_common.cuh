@@ -58,4 +58,32 @@ TC_DEVINL void exp8(const uint32_t* v, uint64_t scale2, uint64_t negm2, uint64_t
   }
 }
 
+// The same for 16 consecutive scores -> 8 packed pairs, POLY8 of the 8 pairs through the polynomial.  SUM = false
+// leaves the row sum to the caller (the tensor core adds the rounded probabilities against a column of ones).
+template <int POLY8, bool CLAMP, bool SUM>
+TC_DEVINL void exp16(const uint32_t* v, uint64_t scale2, uint64_t negm2, uint64_t& sum2, uint32_t* out) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    uint64_t x = fma2(pack2u(v[2 * i], v[2 * i + 1]), scale2, negm2);
+    uint64_t e;
+    if (i < POLY8) {
+      if (CLAMP) {
+        uint32_t a, b;
+        unpack2u(x, a, b);
+        x = pack2f(fmaxf(__uint_as_float(a), -120.f), fmaxf(__uint_as_float(b), -120.f));
+      }
+      e = exp2_poly2(x);
+    } else {
+      uint32_t a, b;
+      unpack2u(x, a, b);
+      e = pack2f(ex2f(__uint_as_float(a)), ex2f(__uint_as_float(b)));
+    }
+    uint32_t a, b;
+    unpack2u(e, a, b);
+    const uint32_t w = pack_bf16(__uint_as_float(a), __uint_as_float(b));
+    out[i] = w;
+    if (SUM) sum2 = add2(sum2, pack2u(w << 16, w & 0xffff0000u));
+  }
+}
+
 }  // namespace tc

@@ -22,7 +22,7 @@ struct TcState {
   bool attn_attr_set[2];
   int attn_poly_bwd;      // the same share in the backward kernels
   int attn_bwd_fused;     // head size 64: the one-kernel attention adjoint (0: the dQ and dK/dV kernels)
-  int attn_poly;          // of every 4 score pairs, how many take the polynomial exp2 (0..3)
+  int attn_poly;          // forward: of every 8 score pairs, how many take the polynomial exp2 (-1: per head size)
 };
 
 // bf16 tensor maps with 128-byte swizzle.  2-D: dim0 (contiguous) extent d0, dim1 extent d1, row pitch ld
