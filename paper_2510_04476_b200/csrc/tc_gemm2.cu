@@ -9,7 +9,12 @@
 //
 //   warp 0      : TMA producer, in both CTAs (transaction bytes are counted on the leader CTA's barrier)
 //   warp 1      : TMEM owner in both CTAs; in the leader CTA it issues the MMAs for the pair
-//   warps 2..5  : epilogue, each CTA drains its own 128 accumulator rows from its own TMEM
+//   warps 2..5  : epilogue, each CTA drains its own 128 accumulator rows from its own TMEM.  A thread holds one row of
+//                 the accumulator (TMEM lane = row), so stored as they are the 32 lanes of a warp would write 16 bytes
+//                 each into 32 different rows: 32 partial-sector requests per instruction, which bounded the GEMMs with
+//                 a short k loop.  Each warp therefore turns its 32 x 32 block through a private 4 KB shared-memory
+//                 stage (swizzled, conflict-free both ways) and stores whole 128-byte (fp32) or 64-byte (bf16) row
+//                 segments, 4 or 8 rows per instruction.
 #include <cstdio>
 
 #include "tc_kernels.cuh"
@@ -45,7 +50,9 @@ struct G2Smem {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = BN == 256 ? 6 : 7;
   static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-  static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;
+  static constexpr int EPI_OFFSET = BAR_OFFSET + 256;        // four epilogue warps x 4 KB
+  static constexpr int TOTAL = EPI_OFFSET + 4 * 4096 + 1024;
+  static_assert(TOTAL <= 232448, "shared memory");
 };
 
 TC_DEVINL void fail(volatile int* abort_flag, int* status, int code) {
@@ -210,6 +217,58 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     }
   } else {
     const int q = warp & 3;                       // TMEM lane quarter this warp may access
+    unsigned char* stg = smem + SM::EPI_OFFSET + (warp - 2) * 4096;
+    // fp32 block: rows of 128 bytes, 16-byte chunk i of row r at chunk i ^ (r & 7)
+    auto stage_f32 = [&](const uint32_t (&r)[32]) {
+      __syncwarp();                               // the previous block has been read out
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        *reinterpret_cast<uint4*>(stg + lane * 128 + ((i ^ (lane & 7)) << 4)) = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+      __syncwarp();
+    };
+    // 4 rows x 128 bytes per instruction: lane -> row 4 i + lane / 8, chunk lane % 8
+    auto flush_f32 = [&](float* col0, long long ld, int m_first) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int rr = 4 * i + (lane >> 3), ch = lane & 7;
+        const uint4 v = *reinterpret_cast<const uint4*>(stg + rr * 128 + ((ch ^ (rr & 7)) << 4));
+        if (m_first + rr < p.M) *reinterpret_cast<uint4*>(col0 + (long long)(m_first + rr) * ld + ch * 4) = v;
+      }
+    };
+    // bf16 block: rows of 64 bytes, chunk i of row r at chunk i ^ ((r >> 1) & 3)
+    auto stage_bf16 = [&](const uint32_t (&r)[32]) {
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(r[8 * i + 0]), __uint_as_float(r[8 * i + 1]));
+        v.y = pack_bf16(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]));
+        v.z = pack_bf16(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]));
+        v.w = pack_bf16(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7]));
+        *reinterpret_cast<uint4*>(stg + lane * 64 + ((i ^ ((lane >> 1) & 3)) << 4)) = v;
+      }
+      __syncwarp();
+    };
+    // 8 rows x 64 bytes per instruction: lane -> row 8 i + lane / 4, chunk lane % 4.  value = true: the value columns of
+    // the fused down-projection, stored `late` rows further down inside the same sequence (value shift), a zero row at
+    // each sequence start.
+    auto flush_bf16 = [&](bf16* col0, long long ld, int m_first, bool value, int late) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int rr = 8 * i + (lane >> 2), ch = lane & 3;
+        const uint4 v = *reinterpret_cast<const uint4*>(stg + rr * 64 + ((ch ^ ((rr >> 1) & 3)) << 4));
+        const int mm = m_first + rr;
+        if (mm < p.M) {
+          if (!value) {
+            *reinterpret_cast<uint4*>(col0 + (long long)mm * ld + ch * 8) = v;
+          } else {
+            const int t = (mm + p.row0) % p.seq_len;
+            if (!late || t + 1 < p.seq_len) *reinterpret_cast<uint4*>(col0 + (long long)(mm + late) * ld + ch * 8) = v;
+            if (late && t == 0) *reinterpret_cast<uint4*>(col0 + (long long)mm * ld + ch * 8) = make_uint4(0u, 0u, 0u, 0u);   // x_{-1} = 0
+          }
+        }
+      }
+    };
     int it = 0;
     for (int tile = pair; tile < num_tiles; tile += n_pairs, ++it) {
       const int as = it & 1;
@@ -219,77 +278,45 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       if (!mbar_wait(&acc_full[as], aphase, abort_flag)) { fail(abort_flag, p.status, ST_TIMEOUT_EPI); goto done; }
       tc_fence_after();
       const int m = m0 + q * 32 + lane;
+      const int m_base = m0 + q * 32;               // first row of this warp's block
 #pragma unroll 1
       for (int c = 0; c < G2_BN / 32; ++c) {
         uint32_t r[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + as * G2_BN + c * 32, r);
         tmem_ld_wait();
         const int n = n0 + c * 32;
+        if (n >= p.N) continue;                     // (warp-uniform)
+        const bool whole = n + 32 <= p.N;
         if (p.split_L > 0) {
           // fused down-projection: latent columns in fp32, value columns in bf16 (second half one token later)
-          if (m < p.M && n < p.N) {
-            if (n < p.split_L) {
-              float* dst = p.out_f32 + (long long)m * p.ldc + n;
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                reinterpret_cast<uint4*>(dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
-              if (p.out_lat_bf16) {            // the operand copy the latent-transform kernel loads by TMA
-                bf16* dlb = p.out_lat_bf16 + (long long)m * p.split_L + n;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  uint4 v;
-                  v.x = pack_bf16(__uint_as_float(r[8 * i + 0]), __uint_as_float(r[8 * i + 1]));
-                  v.y = pack_bf16(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]));
-                  v.z = pack_bf16(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]));
-                  v.w = pack_bf16(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7]));
-                  reinterpret_cast<uint4*>(dlb)[i] = v;
-                }
-              }
-            } else {
-              const int vc = n - p.split_L;
-              const bool late = p.split_shift && vc >= p.split_Lk / 2;
-              const int t = (m + p.row0) % p.seq_len;
-              bf16* dst = p.out_bf16 + (long long)(m + (late ? 1 : 0)) * p.split_Lk + vc;
-              if (!late || t + 1 < p.seq_len) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  uint4 v;
-                  v.x = pack_bf16(__uint_as_float(r[8 * i + 0]), __uint_as_float(r[8 * i + 1]));
-                  v.y = pack_bf16(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]));
-                  v.z = pack_bf16(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]));
-                  v.w = pack_bf16(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7]));
-                  reinterpret_cast<uint4*>(dst)[i] = v;
-                }
-              }
-              if (late && t == 0) {                     // x_{-1} = 0
-                bf16* z = p.out_bf16 + (long long)m * p.split_Lk + vc;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(z)[i] = make_uint4(0u, 0u, 0u, 0u);
-              }
+          if (n < p.split_L) {
+            stage_f32(r);
+            flush_f32(p.out_f32 + n, p.ldc, m_base);
+            if (p.out_lat_bf16) {                   // the operand copy the latent-transform kernel loads by TMA
+              stage_bf16(r);
+              flush_bf16(p.out_lat_bf16 + n, p.split_L, m_base, false, 0);
             }
+          } else {
+            const int vc = n - p.split_L;
+            stage_bf16(r);
+            flush_bf16(p.out_bf16 + vc, p.split_Lk, m_base, true, (p.split_shift && vc >= p.split_Lk / 2) ? 1 : 0);
           }
-        } else if (m < p.M && n < p.N) {
+        } else if (p.out_bf16 && p.vec_ok && whole) {
+          stage_bf16(r);
+          flush_bf16(p.out_bf16 + n, p.ldc, m_base, false, 0);
+        } else if (p.out_f32 && p.splits == 1 && p.vec_ok && whole) {
+          stage_f32(r);
+          flush_f32(p.out_f32 + n, p.ldc, m_base);
+        } else if (m < p.M) {
           if (p.out_bf16) {
             bf16* dst = p.out_bf16 + (long long)m * p.ldc + n;
-            if (p.vec_ok && n + 32 <= p.N) {
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                uint4 v;
-                v.x = pack_bf16(__uint_as_float(r[8 * i + 0]), __uint_as_float(r[8 * i + 1]));
-                v.y = pack_bf16(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]));
-                v.z = pack_bf16(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]));
-                v.w = pack_bf16(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7]));
-                reinterpret_cast<uint4*>(dst)[i] = v;
-              }
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (n + i < p.N) dst[i] = __float2bfloat16(__uint_as_float(r[i]));
-            }
+            for (int i = 0; i < 32; ++i)
+              if (n + i < p.N) dst[i] = __float2bfloat16(__uint_as_float(r[i]));
           } else {
             float* dst = p.out_f32 + (long long)m * p.ldc + n;
             if (p.splits > 1) {
-              if (p.vec_ok && n + 32 <= p.N) {
+              if (p.vec_ok && whole) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4 * i), "f"(__uint_as_float(r[4 * i])),
@@ -301,10 +328,6 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 for (int i = 0; i < 32; ++i)
                   if (n + i < p.N) atomicAdd(dst + i, __uint_as_float(r[i]));
               }
-            } else if (p.vec_ok && n + 32 <= p.N) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                reinterpret_cast<uint4*>(dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
             } else {
 #pragma unroll
               for (int i = 0; i < 32; ++i)
