@@ -384,33 +384,31 @@ tc_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         l_tot = __uint_as_float(t);
       }
       const float inv_l = 1.f / l_tot;
-      const long long row_g = (long long)b * p.S + tq;
-#pragma unroll 1
-      for (int c = 0; c < DH / 64; ++c) {
-        uint32_t t[16];
-        const int col = part * (DH / 4) + c * 16;
-        tmem_ld16(o_tmem + col, t);
-        tmem_ld_wait();
-        if (tq < p.S) {
-          bf16* dst = p.o + row_g * p.Lq + hi * DH + col;
+      // The warp's block of O: 32 rows x d_h / 4 columns.  Stored through a shared-memory stage in the tile's own Q
+      // buffer (free: every S MMA of the tile finished before its last P V), whole row segments per instruction.
+      constexpr int CW = DH / 4;                             // columns per warp
+      constexpr int RB = CW * 2;                             // bytes of a bf16 row segment (64 or 32)
+      unsigned char* stg = smem + SM::Q_OFF + s * SM::TILE_BYTES + warp * (32 * RB);
+      const int row0 = blk * 256 + s * BQ + (warp & 3) * 32;         // first query row of the block
+      const int rows_ok = p.S - row0;
+      const long long e0 = ((long long)b * p.S + row0) * p.Lq + hi * DH + part * CW;   // element offset of the block
+      uint32_t t[CW];
+      if (DH == 128) tmem_ld32(o_tmem + part * CW, reinterpret_cast<uint32_t(&)[32]>(t[0]));
+      else tmem_ld16(o_tmem + part * CW, reinterpret_cast<uint32_t(&)[16]>(t[0]));
+      tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 2; ++i) {
-            uint4 w;
-            w.x = pack_bf16(__uint_as_float(t[8 * i + 0]) * inv_l, __uint_as_float(t[8 * i + 1]) * inv_l);
-            w.y = pack_bf16(__uint_as_float(t[8 * i + 2]) * inv_l, __uint_as_float(t[8 * i + 3]) * inv_l);
-            w.z = pack_bf16(__uint_as_float(t[8 * i + 4]) * inv_l, __uint_as_float(t[8 * i + 5]) * inv_l);
-            w.w = pack_bf16(__uint_as_float(t[8 * i + 6]) * inv_l, __uint_as_float(t[8 * i + 7]) * inv_l);
-            reinterpret_cast<uint4*>(dst)[i] = w;
-          }
-          if (p.o32) {
-            float* d32 = p.o32 + row_g * p.Lq + hi * DH + col;
+      for (int i = 0; i < CW; ++i) t[i] = __float_as_uint(__uint_as_float(t[i]) * inv_l);
+      {
+        uint32_t w[CW / 2];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-              reinterpret_cast<float4*>(d32)[i] =
-                  make_float4(__uint_as_float(t[4 * i]) * inv_l, __uint_as_float(t[4 * i + 1]) * inv_l,
-                              __uint_as_float(t[4 * i + 2]) * inv_l, __uint_as_float(t[4 * i + 3]) * inv_l);
-          }
-        }
+        for (int i = 0; i < CW / 2; ++i) w[i] = pack_bf16(__uint_as_float(t[2 * i]), __uint_as_float(t[2 * i + 1]));
+        warp_store_rows<RB>(stg, w, reinterpret_cast<unsigned char*>(p.o + e0), (long long)p.Lq * 2, rows_ok);
+      }
+      if (p.o32) {                                            // the fp32 copy for the backward, in two halves
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+          warp_store_rows<RB>(stg, &t[h * (CW / 2)], reinterpret_cast<unsigned char*>(p.o32 + e0 + h * (CW / 2)),
+                              (long long)p.Lq * 4, rows_ok);
       }
       if (part == 0 && tq < p.S) p.lse[((long long)b * p.hq + hi) * p.S + tq] = (m_run[s] + log2f(l_tot)) * LN2_F;
     }

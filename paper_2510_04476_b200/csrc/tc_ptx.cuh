@@ -284,4 +284,30 @@ TC_DEVINL uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// ---- row blocks held one row per lane -> coalesced global stores ------------------------------------------
+// A warp holds a block of 32 rows x RB bytes, lane = row (the layout tensor memory hands out).  Stored as it is, one
+// instruction would write 16 bytes into each of 32 rows: 32 partial-sector requests.  The block goes through a private
+// shared-memory stage of 32 x RB bytes instead (16-byte chunks swizzled so that neither direction has bank conflicts) and
+// leaves as whole row segments, 512 / RB rows per instruction.  RB = 32, 64 or 128; w = the lane's RB / 4 words;
+// g_row0 = address of the block's first row segment (16-byte aligned, like ld_bytes); rows from n_rows on are not stored.
+template <int RB>
+TC_DEVINL void warp_store_rows(unsigned char* stg, const uint32_t* w, unsigned char* g_row0, long long ld_bytes, int n_rows) {
+  constexpr int CH = RB / 16;                      // chunks per row: 2, 4, 8
+  constexpr int RPI = 32 / CH;                     // rows per instruction: 16, 8, 4
+  const int lane = threadIdx.x & 31;
+  // chunk c of row r sits at chunk c ^ f(r): f takes CH different values over rows that share a 128-byte line phase
+  auto f = [](int r) -> int { return RB == 128 ? (r & 7) : RB == 64 ? ((r >> 1) & 3) : ((r >> 2) & 1); };
+  __syncwarp();                                    // the previous block has been read out
+#pragma unroll
+  for (int c = 0; c < CH; ++c)
+    *reinterpret_cast<uint4*>(stg + lane * RB + ((c ^ f(lane)) << 4)) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < CH; ++i) {
+    const int r = RPI * i + lane / CH, c = lane % CH;
+    const uint4 v = *reinterpret_cast<const uint4*>(stg + r * RB + ((c ^ f(r)) << 4));
+    if (r < n_rows) *reinterpret_cast<uint4*>(g_row0 + (long long)r * ld_bytes + c * 16) = v;
+  }
+}
+
 }  // namespace tc
