@@ -467,6 +467,7 @@ int tc_gemm_pair(TcState* s, const GemmArgs& g, int* d_status, cudaStream_t st) 
     return ((tiles + s->pair_clusters - 1) / s->pair_clusters) * bn;
   };
   // (an MN-major B half of 96 columns would not be a whole number of 64-column swizzle chunks)
-  if (!b_mn && cost(192) < cost(256)) return launch_pair<192>(s, g, p, a_mn, b_mn, lda, ldb, st);
+  const bool narrow = s->gemm_bn == 192 ? true : s->gemm_bn == 256 ? false : cost(192) < cost(256);
+  if (!b_mn && narrow) return launch_pair<192>(s, g, p, a_mn, b_mn, lda, ldb, st);
   return launch_pair<256>(s, g, p, a_mn, b_mn, lda, ldb, st);
 }

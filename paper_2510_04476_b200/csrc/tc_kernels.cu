@@ -284,6 +284,8 @@ TcState* tc_create(int sm_count) {
   s->pair_clusters = -1;
   s->use_pairs = 1;
   if (const char* e = getenv("CCA_GEMM_PAIRS")) s->use_pairs = atoi(e);
+  s->gemm_bn = 0;
+  if (const char* e = getenv("CCA_GEMM_BN")) s->gemm_bn = atoi(e);
   s->attn_attr_set[0] = s->attn_attr_set[1] = false;
   s->attn_poly = -1;      // -1: per head size (0 at d_h = 128, 2 of 8 at d_h = 64)
   if (const char* e = getenv("CCA_ATTN_POLY")) s->attn_poly = atoi(e);

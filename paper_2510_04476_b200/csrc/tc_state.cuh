@@ -19,6 +19,7 @@ struct TcState {
   bool attr_set_128, attr_set_256;
   int pair_clusters;      // co-resident CTA pairs of the pair GEMM (-1: not asked yet, 0: unavailable)
   int use_pairs;          // 0 disables the pair GEMM
+  int gemm_bn;            // tile width of the pair GEMM: 0 = chosen per shape, 192 or 256 = forced
   bool attn_attr_set[2];
   int attn_poly_bwd;      // the same share in the backward kernels
   int attn_bwd_fused;     // head size 64: the one-kernel attention adjoint (0: the dQ and dK/dV kernels)
