@@ -42,7 +42,9 @@ struct TbSmem {
   static constexpr int G_OFF = KC * TILE;
   static constexpr int W_OFF = 2 * KC * TILE;
   static constexpr int BAR_OFF = W_OFF + KC * BT;
-  static constexpr int TOTAL = BAR_OFF + 128 + 1024;
+  static constexpr int STG_OFF = BAR_OFF + 128;      // four epilogue warps x 4 KB: row blocks on their way to memory
+  static constexpr int TOTAL = STG_OFF + 4 * 4096 + 1024;
+  static_assert(TOTAL <= 232448, "shared memory");
   static constexpr int NGRP = DH == 128 ? KC : (KC + 1) / 2;          // weight-gradient accumulators
   static constexpr int GRP_COLS = DH == 128 ? 128 : 64;
   static constexpr int DW_COL = 2 * DH;                               // after the two d_y1 buffers
@@ -293,12 +295,10 @@ __global__ void __launch_bounds__(TB_THREADS, 1) tc_transform_bwd_kernel(const T
         uint32_t r[32];
         tmem_ld32(acc + c * 32, r);
         tmem_ld_wait();
-        if (t < d.S) {
-          float* dst = p.dy1 + ((long long)b * d.S + t) * d.L + h * DH + c * 32;
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            reinterpret_cast<uint4*>(dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
-        }
+        // the warp's 32 tokens x 32 channels leave as whole 128-byte row segments, four rows per instruction
+        warp_store_rows<128>(smem + SM::STG_OFF + warp * 4096, r,
+                             reinterpret_cast<unsigned char*>(p.dy1 + ((long long)b * d.S + t0 + warp * 32) * d.L + h * DH + c * 32),
+                             (long long)d.L * 4, d.S - (t0 + warp * 32));
       }
       if (last_of_head) {
         // accumulator rows: d_h = 128: lane = i of tap gp; d_h = 64: lanes 0-63 = tap 2gp, lanes 64-127 = tap 2gp+1
